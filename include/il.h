@@ -1,0 +1,132 @@
+/*
+ * il.h — C ABI of the interlocking-backpropagation training-step library (CUDA, sm_100a).
+ *
+ * One il_model is a decoder-only Transformer language model cut into K contiguous
+ * components ("modules", Sec. 3 of the paper: f = f_cK o ... o f_c1), each of
+ * `layers_per_component` pre-LN blocks, with an auxiliary LM head h_ck (LayerNorm + untied
+ * linear map to the vocabulary) after every component and the local loss
+ *     L_ck(x, y) = L(h_ck(f_ck o ... o f_c1 (x)), y)            (Sec. 3, unnumbered equations)
+ * with L the mean next-token cross-entropy.  One training step is
+ *     il_set_batch -> il_forward_component(0..K-1) -> il_aux_head_loss(0..K-1)
+ *                  -> il_backward_nwise -> il_adamw_step
+ * where il_backward_nwise applies the n-wise rule (Sec. 3, Fig. 2): the gradient of head h
+ * flows through component h and across n-1 component boundaries and then stops; the
+ * contributions of all heads crossing a component are summed.  n = 1 is local learning,
+ * n = K is ordinary backpropagation of the sum of the K head losses.
+ *
+ * Conventions
+ *  - Every call returns il_status.  Nothing throws, aborts or exits across this boundary.
+ *    On an error other than IL_ERR_CUDA the model stays usable and outputs are untouched.
+ *  - The library owns all device memory it obtains (through il_options.alloc when given,
+ *    cudaMalloc otherwise) and every string it returns.  The caller owns every buffer it
+ *    passes; "host" pointers are ordinary host memory, "device" pointers are CUDA device
+ *    memory on the model's device.  Inputs are copied before the call returns unless the
+ *    call is documented as asynchronous on device pointers.
+ *  - Components, heads and tensors are 0-based.  Matrices are row-major [out, in].
+ *  - Work is issued on K CUDA streams (component k on stream k); calls return once the
+ *    work is enqueued unless stated otherwise.  One host thread per model.
+ *  - Arithmetic: bf16 tensor-core operands, fp32 accumulation, fp32 residual stream,
+ *    fp32 master weights, gradients and optimiser state.
+ */
+#ifndef IL_H_
+#define IL_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct il_model il_model;
+
+typedef enum {
+  IL_OK = 0,
+  IL_ERR_INVALID_ARG = 1, /* bad shape, NULL pointer, index out of range, n outside [1,K]          */
+  IL_ERR_STATE = 2,       /* call order violated (e.g. backward before all K forwards + losses)     */
+  IL_ERR_OOM = 3,         /* the allocator returned NULL                                            */
+  IL_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed; see il_last_error                   */
+  IL_ERR_TIMEOUT = 5,     /* a bounded device-side wait expired (kernel returned early)             */
+  IL_ERR_NONFINITE = 6    /* reserved                                                               */
+} il_status;
+
+typedef struct {
+  int device;                       /* CUDA device ordinal                                           */
+  int max_batch, max_seq;           /* activation arena is sized for max_batch*max_seq tokens;       */
+                                    /* wpe has max_seq rows                                          */
+  void* (*alloc)(size_t bytes, void* ctx);  /* device allocator hook (256-byte aligned); NULL => cudaMalloc */
+  void (*free_)(void* p, void* ctx);
+  void* alloc_ctx;
+  void** streams;                   /* K cudaStream_t owned by the caller; NULL => library-created   */
+  int n_streams;
+  int use_bias;                     /* reserved, must be 1 (GPT-2 style biases)                      */
+  float ln_eps;                     /* <= 0 => 1e-5                                                  */
+} il_options;
+
+/* Build a model: K components x layers_per_component blocks, d_model, n_heads, d_ff, vocab, and the
+ * n of the n-wise rule (Sec. 3: N in [1, number of modules]).  Requires d_model % n_heads == 0,
+ * head dim in {32, 64, 80, 128}, d_model % 8 == 0, d_ff % 8 == 0.  opt must be non-NULL with
+ * max_batch, max_seq > 0.  Parameters start at zero (LayerNorm gains at one); set them with
+ * il_set_param. */
+il_status il_create(int K, int layers_per_component, int d_model, int n_heads, int d_ff, int vocab,
+                    int n, const il_options* opt, il_model** out);
+il_status il_destroy(il_model* m);
+/* Change n (1..K) between steps. */
+il_status il_set_n(il_model* m, int n);
+
+/* Parameter registry.  Order and names: "wte" [V,d], "wpe" [max_seq,d] (component 0: the first
+ * module holds the input projection, App. B.3), then per component k and layer l
+ * "c{k}.l{l}.{ln1.g,ln1.b,attn.wqkv,attn.bqkv,attn.wo,attn.bo,ln2.g,ln2.b,mlp.w1,mlp.b1,mlp.w2,mlp.b2}",
+ * then per head "head{k}.{ln.g,ln.b,w}".  Host fp32 buffers; `count` must equal the tensor size.
+ * These calls synchronise the device. */
+int il_num_tensors(const il_model* m);
+il_status il_tensor_info(const il_model* m, int idx, const char** name, int* component, int* is_head,
+                         int* rank, long long shape[2]);
+il_status il_set_param(il_model* m, int idx, const float* host, size_t count);
+il_status il_get_param(il_model* m, int idx, float* host, size_t count);
+il_status il_get_grad(il_model* m, int idx, float* host, size_t count); /* after il_backward_nwise */
+il_status il_get_opt_state(il_model* m, int idx, float* m_host, float* v_host, long long* step);
+il_status il_set_opt_state(il_model* m, int idx, const float* m_host, const float* v_host, long long step);
+
+/* One step.  tokens/targets: B*T int32 ids in [0, vocab), HOST pointers when on_device == 0
+ * (copied with cudaMemcpyAsync before the call returns control; the caller may reuse the buffers
+ * after il_sync or any synchronising call), DEVICE pointers when on_device != 0.  Ids outside
+ * [0, vocab) are clamped on the device, never dereferenced out of bounds. */
+il_status il_set_batch(il_model* m, const int* tokens, const int* targets, int B, int T, int on_device);
+/* Forward of component k (Sec. 3: a_k = f_ck(a_{k-1}); k = 0 also performs the embedding lookup).
+ * Must be called for k = 0..K-1 in order. */
+il_status il_forward_component(il_model* m, int k);
+/* Auxiliary head k: LayerNorm, vocabulary projection and mean cross-entropy, with the logits
+ * consumed tile by tile (never stored).  Needs il_forward_component(k).  loss_host != NULL makes the
+ * call wait for this head and return its loss; NULL leaves it asynchronous. */
+il_status il_aux_head_loss(il_model* m, int k, float* loss_host);
+/* All K losses of the current step (waits for them). */
+il_status il_get_losses(il_model* m, float* losses_host);
+/* n-wise backward (Sec. 3, Fig. 2): for every head, back-propagation through the head and through
+ * the n components below it, a stop at each window's lowest component input, contributions of
+ * overlapping heads summed.  Overwrites all gradients.  Needs all K forwards and head losses. */
+il_status il_backward_nwise(il_model* m);
+/* AdamW (decoupled weight decay on rank-2 tensors; weight_decay = 0 is the paper's Adam,
+ * App. B.3: beta1 0.9, beta2 0.98, eps 1e-9).  Needs il_backward_nwise.  Increments the step. */
+il_status il_adamw_step(il_model* m, float lr, float beta1, float beta2, float eps, float weight_decay);
+/* Wait for all enqueued work; reports device-side timeouts as IL_ERR_TIMEOUT. */
+il_status il_sync(il_model* m);
+/* Boundary activation a_k, k = 0..K (a_0 = embeddings), fp32 [B*T, d] to host; synchronises. */
+il_status il_get_boundary(il_model* m, int k, float* host, size_t count);
+/* Bytes of device memory obtained so far, and kernels launched since creation. */
+il_status il_stats(const il_model* m, long long* device_bytes, long long* kernel_launches);
+/* Device time of the GEMM kernels launched since the last reset, measured with CUDA events on
+ * their own streams when profiling is switched on (adds event records; off by default). */
+il_status il_profile(il_model* m, int enable);
+il_status il_profile_read(il_model* m, double* gemm_ms, long long* gemm_launches, double* gemm_flops);
+/* Host-only helper (no device needed): the gradient streams component k carries under the n-wise rule
+ * (Sec. 3, Fig. 2).  Head h stops at the input of component max(h-n+1, 0); the heads crossing component
+ * k are grouped by that level.  Writes the distinct levels, descending, to terms[0..*count) (terms may be
+ * NULL; it needs room for min(n, K) ints).  *count is the number of stacked backward passes of k. */
+il_status il_nwise_streams(int K, int n, int k, int* terms, int* count);
+const char* il_last_error(const il_model* m); /* library-owned, valid until the next call on m */
+const char* il_status_string(il_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* IL_H_ */

@@ -1,0 +1,78 @@
+/*
+ * il_ops.h — operator-level entry points of the same library (CUDA, sm_100a).
+ *
+ * These expose the individual kernels that il.h's training step is built from, so that each can be
+ * checked and profiled in isolation.  Every pointer is a DEVICE pointer on the current device, every
+ * call is asynchronous on `stream` (a cudaStream_t passed as void*; NULL = the default stream), nothing
+ * is allocated or freed unless stated, and the return value is an il_status (see il.h).  Arguments are
+ * validated on the host; a failed validation returns IL_ERR_INVALID_ARG before anything is launched.
+ */
+#ifndef IL_OPS_H_
+#define IL_OPS_H_
+
+#include "il.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Dense contraction C[M,N] = A[M,K] * B[N,K]^T on the tensor cores (bf16 operands, fp32 accumulate),
+ * used for every projection of the Transformer blocks (forward, dgrad, wgrad) and for the auxiliary
+ * heads' vocabulary projection (Sec. 3: h_ck; Sec. 4.3: GPT-2-like blocks).
+ * Operand storage: mn_major = 0: row-major [rows, K] (contraction index contiguous);
+ *                  mn_major = 1: row-major [K, rows] (the operand's own index contiguous).
+ * Supported combinations (a_mn, b_mn): (0,0) forward, (0,1) dgrad, (1,1) wgrad.
+ * Leading dimensions in elements, multiples of 8; pointers 16-byte aligned.
+ * Epilogues (the `epilogue` field):
+ *   0 C(bf16) = acc + bias                         1 C(bf16) = pre, C2(bf16) = gelu_tanh(pre), pre = acc + bias
+ *   2 C(f32) = resid(f32) + acc + bias             3 C(bf16) = acc * gelu_tanh'(aux[row % aux_rows, col])
+ *   4 C(f32) = acc (+ C when accumulate != 0)
+ *   5 per-(row, 256-column tile) softmax partials: part_max, part_sum [M, part_ld] at tile index
+ *     col0/256 + tile, and tgt_logit[row] = acc[row, targets[row] - col0] when that column is in range
+ *   6 C(bf16) = (exp(acc - lse[row]) - [col + col0 == targets[row]]) * scale
+ * (0,1) supports epilogues 0, 3, 4; (1,1) supports 4; (0,0) supports all. */
+typedef struct {
+  int M, N, K;
+  const void* A; int lda; int a_mn_major;
+  const void* B; int ldb; int b_mn_major;
+  int epilogue;
+  void* C; int ldc;
+  void* C2;
+  const float* bias;
+  const float* resid;
+  const void* aux; int ld_aux; int aux_rows;
+  int accumulate;
+  const int* targets;
+  float* part_max; float* part_sum; int part_ld;
+  float* tgt_logit;
+  const float* lse;
+  float scale;
+  int col0;
+} il_gemm_desc;
+
+/* err_word: device word (unsigned) the kernel sets non-zero if one of its bounded waits expired. */
+il_status il_op_gemm(const il_gemm_desc* desc, unsigned* err_word, void* stream);
+
+/* Causal multi-head self-attention of the Transformer blocks on packed qkv [B*T, 3*H*dh] bf16
+ * (Q | K | V; head h at columns h*dh): o [B*T, H*dh] bf16, lse [B, H, T] fp32.  dh in {32,64,80,128}. */
+il_status il_op_attention_fwd(const void* qkv, void* o, float* lse, int B, int T, int H, int dh, void* stream);
+/* Its backward.  NB gradient batches may share the saved forward of B sequences (gradient batch b uses
+ * sequence b % B): dout [NB*T, H*dh] bf16 -> dqkv [NB*T, 3*H*dh] bf16.  delta: scratch [NB*H*T] fp32. */
+il_status il_op_attention_bwd(const void* qkv, const void* o, const float* lse, const void* dout, void* dqkv,
+                              float* delta, int NB, int B, int T, int H, int dh, void* stream);
+
+/* LayerNorm over the last axis (biased variance, eps inside the square root): y bf16 [rows, d],
+ * mean/rstd fp32 [rows].  d % 8 == 0. */
+il_status il_op_layernorm_fwd(const float* x, const float* gamma, const float* beta, void* y, float* mean,
+                              float* rstd, int rows, int d, float eps, void* stream);
+/* LayerNorm backward: dx[row,:] = (resid ? resid[row,:] : 0) + dLN(dy[row,:]) with x/mean/rstd indexed by
+ * row % x_rows; dgamma/dbeta (accumulated atomically, zeroed by the caller) over the first x_rows rows.
+ * dy is bf16 unless dy_is_f32.  dx_bf16 may be NULL. */
+il_status il_op_layernorm_bwd(const void* dy, int dy_is_f32, const float* x, const float* mean, const float* rstd,
+                              const float* gamma, const float* resid, float* dx, void* dx_bf16, float* dgamma,
+                              float* dbeta, int rows, int x_rows, int d, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* IL_OPS_H_ */

@@ -1,0 +1,419 @@
+// HBM-bound kernels of the training step: embedding, LayerNorm forward/backward, column reductions for
+// bias and LayerNorm parameter gradients, gradient-stream sums, softmax-partial merge, AdamW.
+// All of them use 16-byte (or 8-byte for bf16x4) coalesced accesses and warp-shuffle reductions.
+#include "common.cuh"
+#include "kernels.h"
+
+namespace il {
+
+static inline int ceil_div(long long a, long long b) { return (int)((a + b - 1) / b); }
+
+// ---------------------------------------------------------------------------------------------
+// Embedding
+// ---------------------------------------------------------------------------------------------
+__global__ void embed_fwd_kernel(const int* __restrict__ tok, const float* __restrict__ wte,
+                                 const float* __restrict__ wpe, float* __restrict__ x, int ntok, int T, int d, int V) {
+  const int d4 = d >> 2;
+  const size_t total = (size_t)ntok * d4;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    const int row = (int)(i / d4);
+    const int c = (int)(i % d4);
+    int t = tok[row];
+    t = t < 0 ? 0 : (t >= V ? V - 1 : t);
+    const float4 a = __ldg(reinterpret_cast<const float4*>(wte + (size_t)t * d) + c);
+    const float4 b = __ldg(reinterpret_cast<const float4*>(wpe + (size_t)(row % T) * d) + c);
+    reinterpret_cast<float4*>(x + (size_t)row * d)[c] = make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w);
+  }
+}
+
+cudaError_t embed_fwd(const int* tok, const float* wte, const float* wpe, float* x, int ntok, int T, int d, int V,
+                      cudaStream_t s) {
+  const size_t total = (size_t)ntok * (d / 4);
+  int blocks = ceil_div(total, 256);
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  embed_fwd_kernel<<<blocks, 256, 0, s>>>(tok, wte, wpe, x, ntok, T, d, V);
+  return cudaGetLastError();
+}
+
+__global__ void embed_bwd_wte_kernel(const int* __restrict__ tok, const float* __restrict__ dx,
+                                     float* __restrict__ dwte, int ntok, int d, int V) {
+  const size_t total = (size_t)ntok * d;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    const int row = (int)(i / d);
+    const int c = (int)(i % d);
+    int t = tok[row];
+    t = t < 0 ? 0 : (t >= V ? V - 1 : t);
+    atomicAdd(dwte + (size_t)t * d + c, dx[i]);
+  }
+}
+__global__ void embed_bwd_wpe_kernel(const float* __restrict__ dx, float* __restrict__ dwpe, int B, int T, int d) {
+  const int d4 = d >> 2;
+  const size_t total = (size_t)T * d4;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int b = 0; b < B; ++b) {
+      const float4 v = reinterpret_cast<const float4*>(dx + (size_t)b * T * d)[i];
+      acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    reinterpret_cast<float4*>(dwpe)[i] = acc;
+  }
+}
+
+cudaError_t embed_bwd(const int* tok, const float* dx, float* dwte, float* dwpe, int ntok, int T, int d, int V,
+                      cudaStream_t s) {
+  int blocks = ceil_div((size_t)ntok * d, 256);
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  embed_bwd_wte_kernel<<<blocks, 256, 0, s>>>(tok, dx, dwte, ntok, d, V);
+  int blocks2 = ceil_div((size_t)T * (d / 4), 256);
+  embed_bwd_wpe_kernel<<<blocks2, 256, 0, s>>>(dx, dwpe, ntok / T, T, d);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// LayerNorm forward: one warp per row
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) layernorm_fwd_kernel(const float* __restrict__ x, const float* __restrict__ gamma,
+                                                            const float* __restrict__ beta, bf16* __restrict__ y,
+                                                            float* __restrict__ mean, float* __restrict__ rstd,
+                                                            int rows, int d, float eps) {
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (row >= rows) return;
+  const float4* xr = reinterpret_cast<const float4*>(x + (size_t)row * d);
+  const int d4 = d >> 2;
+  float s = 0.f;
+  for (int c = lane; c < d4; c += 32) {
+    const float4 v = xr[c];
+    s += (v.x + v.y) + (v.z + v.w);
+  }
+  const float mu = warp_sum(s) / d;
+  float q = 0.f;
+  for (int c = lane; c < d4; c += 32) {
+    const float4 v = xr[c];
+    const float a = v.x - mu, b = v.y - mu, cc = v.z - mu, e = v.w - mu;
+    q += (a * a + b * b) + (cc * cc + e * e);
+  }
+  const float rs = rsqrtf(warp_sum(q) / d + eps);
+  if (lane == 0) { mean[row] = mu; rstd[row] = rs; }
+  uint2* yr = reinterpret_cast<uint2*>(y + (size_t)row * d);
+  for (int c = lane; c < d4; c += 32) {
+    const float4 v = xr[c];
+    const float4 g = __ldg(reinterpret_cast<const float4*>(gamma) + c);
+    const float4 b = __ldg(reinterpret_cast<const float4*>(beta) + c);
+    uint2 o;
+    o.x = pack_bf16x2((v.x - mu) * rs * g.x + b.x, (v.y - mu) * rs * g.y + b.y);
+    o.y = pack_bf16x2((v.z - mu) * rs * g.z + b.z, (v.w - mu) * rs * g.w + b.w);
+    yr[c] = o;
+  }
+}
+
+cudaError_t layernorm_fwd(const float* x, const float* gamma, const float* beta, bf16* y, float* mean, float* rstd,
+                          int rows, int d, float eps, cudaStream_t s) {
+  layernorm_fwd_kernel<<<ceil_div(rows, 8), 256, 0, s>>>(x, gamma, beta, y, mean, rstd, rows, d, eps);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// LayerNorm backward, row part: one warp per row
+// ---------------------------------------------------------------------------------------------
+template <bool DY_F32>
+__device__ __forceinline__ float4 load_dy4(const void* dy, size_t row, int d, int c4) {
+  if constexpr (DY_F32) {
+    return reinterpret_cast<const float4*>(reinterpret_cast<const float*>(dy) + row * d)[c4];
+  } else {
+    const uint2 u = reinterpret_cast<const uint2*>(reinterpret_cast<const bf16*>(dy) + row * d)[c4];
+    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u.x));
+    const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u.y));
+    return make_float4(a.x, a.y, b.x, b.y);
+  }
+}
+
+template <bool DY_F32>
+__global__ void __launch_bounds__(256) layernorm_bwd_rows_kernel(const void* __restrict__ dy, const float* __restrict__ x,
+                                                                 const float* __restrict__ mean,
+                                                                 const float* __restrict__ rstd,
+                                                                 const float* __restrict__ gamma, const float* resid,
+                                                                 float* dx_out, bf16* __restrict__ dx_bf16, int rows,
+                                                                 int x_rows, int d) {
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (row >= rows) return;
+  const int xrow = row % x_rows;
+  const float mu = mean[xrow], rs = rstd[xrow];
+  const float4* xr = reinterpret_cast<const float4*>(x + (size_t)xrow * d);
+  const int d4 = d >> 2;
+  float s1 = 0.f, s2 = 0.f;
+  for (int c = lane; c < d4; c += 32) {
+    const float4 g = __ldg(reinterpret_cast<const float4*>(gamma) + c);
+    const float4 dv = load_dy4<DY_F32>(dy, (size_t)row, d, c);
+    const float4 xv = xr[c];
+    const float a0 = dv.x * g.x, a1 = dv.y * g.y, a2 = dv.z * g.z, a3 = dv.w * g.w;
+    s1 += (a0 + a1) + (a2 + a3);
+    s2 += (a0 * (xv.x - mu) + a1 * (xv.y - mu)) + (a2 * (xv.z - mu) + a3 * (xv.w - mu));
+  }
+  const float m1 = warp_sum(s1) / d;
+  const float m2 = warp_sum(s2) * rs / d;   // mean of dxhat * xhat
+  const float4* rr = resid ? reinterpret_cast<const float4*>(resid + (size_t)row * d) : nullptr;
+  float4* outr = reinterpret_cast<float4*>(dx_out + (size_t)row * d);
+  uint2* outb = dx_bf16 ? reinterpret_cast<uint2*>(dx_bf16 + (size_t)row * d) : nullptr;
+  for (int c = lane; c < d4; c += 32) {
+    const float4 g = __ldg(reinterpret_cast<const float4*>(gamma) + c);
+    const float4 dv = load_dy4<DY_F32>(dy, (size_t)row, d, c);
+    const float4 xv = xr[c];
+    float4 o;
+    o.x = (dv.x * g.x - m1 - (xv.x - mu) * rs * m2) * rs;
+    o.y = (dv.y * g.y - m1 - (xv.y - mu) * rs * m2) * rs;
+    o.z = (dv.z * g.z - m1 - (xv.z - mu) * rs * m2) * rs;
+    o.w = (dv.w * g.w - m1 - (xv.w - mu) * rs * m2) * rs;
+    if (rr) {
+      const float4 r = rr[c];
+      o.x += r.x; o.y += r.y; o.z += r.z; o.w += r.w;
+    }
+    outr[c] = o;
+    if (outb) {
+      uint2 b;
+      b.x = pack_bf16x2(o.x, o.y);
+      b.y = pack_bf16x2(o.z, o.w);
+      outb[c] = b;
+    }
+  }
+}
+
+cudaError_t layernorm_bwd_rows(const void* dy, int dy_is_f32, const float* x, const float* mean, const float* rstd,
+                               const float* gamma, const float* resid, float* dx_out, bf16* dx_bf16, int rows, int x_rows,
+                               int d, cudaStream_t s) {
+  if (dy_is_f32)
+    layernorm_bwd_rows_kernel<true><<<ceil_div(rows, 8), 256, 0, s>>>(dy, x, mean, rstd, gamma, resid, dx_out, dx_bf16,
+                                                                       rows, x_rows, d);
+  else
+    layernorm_bwd_rows_kernel<false><<<ceil_div(rows, 8), 256, 0, s>>>(dy, x, mean, rstd, gamma, resid, dx_out, dx_bf16,
+                                                                        rows, x_rows, d);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Column reductions.  Block = 32 lanes x 8 warps; a lane owns 4 consecutive columns, a block 128 columns;
+// the rows are split over gridDim.y; partial sums are combined through shared memory and one atomicAdd
+// per column per block.
+// ---------------------------------------------------------------------------------------------
+template <bool DY_F32>
+__global__ void __launch_bounds__(256) layernorm_bwd_params_kernel(const void* __restrict__ dy, const float* __restrict__ x,
+                                                                   const float* __restrict__ mean,
+                                                                   const float* __restrict__ rstd,
+                                                                   float* __restrict__ dgamma, float* __restrict__ dbeta,
+                                                                   int rows, int d, int rows_per_block) {
+  __shared__ float4 sg[8][32], sb[8][32];
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int c4 = blockIdx.x * 32 + lane;       // float4 column index
+  const bool col_ok = c4 * 4 < d;
+  const int r0 = blockIdx.y * rows_per_block;
+  const int r1 = min(rows, r0 + rows_per_block);
+  float4 ag = make_float4(0.f, 0.f, 0.f, 0.f), ab = ag;
+  if (col_ok) {
+    for (int r = r0 + w; r < r1; r += 8) {
+      const float mu = mean[r], rs = rstd[r];
+      const float4 dv = load_dy4<DY_F32>(dy, (size_t)r, d, c4);
+      const float4 xv = reinterpret_cast<const float4*>(x + (size_t)r * d)[c4];
+      ag.x += dv.x * (xv.x - mu) * rs; ag.y += dv.y * (xv.y - mu) * rs;
+      ag.z += dv.z * (xv.z - mu) * rs; ag.w += dv.w * (xv.w - mu) * rs;
+      ab.x += dv.x; ab.y += dv.y; ab.z += dv.z; ab.w += dv.w;
+    }
+  }
+  sg[w][lane] = ag;
+  sb[w][lane] = ab;
+  __syncthreads();
+  if (w == 0 && col_ok) {
+    for (int i = 1; i < 8; ++i) {
+      const float4 g = sg[i][lane], b = sb[i][lane];
+      ag.x += g.x; ag.y += g.y; ag.z += g.z; ag.w += g.w;
+      ab.x += b.x; ab.y += b.y; ab.z += b.z; ab.w += b.w;
+    }
+    float* pg = dgamma + c4 * 4;
+    float* pb = dbeta + c4 * 4;
+    atomicAdd(pg, ag.x); atomicAdd(pg + 1, ag.y); atomicAdd(pg + 2, ag.z); atomicAdd(pg + 3, ag.w);
+    atomicAdd(pb, ab.x); atomicAdd(pb + 1, ab.y); atomicAdd(pb + 2, ab.z); atomicAdd(pb + 3, ab.w);
+  }
+}
+
+static inline void colreduce_grid(int rows, int cols_per_block, int cols, dim3* grid, int* rows_per_block) {
+  const int bx = ceil_div(cols, cols_per_block);
+  int by = ceil_div(148 * 4, bx);
+  if (by > ceil_div(rows, 8)) by = ceil_div(rows, 8);
+  if (by < 1) by = 1;
+  *rows_per_block = ceil_div(rows, by);
+  by = ceil_div(rows, *rows_per_block);
+  *grid = dim3(bx, by, 1);
+}
+
+cudaError_t layernorm_bwd_params(const void* dy, int dy_is_f32, const float* x, const float* mean, const float* rstd,
+                                 float* dgamma, float* dbeta, int rows, int d, cudaStream_t s) {
+  dim3 grid;
+  int rpb;
+  colreduce_grid(rows, 128, d, &grid, &rpb);
+  if (dy_is_f32)
+    layernorm_bwd_params_kernel<true><<<grid, 256, 0, s>>>(dy, x, mean, rstd, dgamma, dbeta, rows, d, rpb);
+  else
+    layernorm_bwd_params_kernel<false><<<grid, 256, 0, s>>>(dy, x, mean, rstd, dgamma, dbeta, rows, d, rpb);
+  return cudaGetLastError();
+}
+
+template <bool IN_F32>
+__global__ void __launch_bounds__(256) colsum_kernel(const void* __restrict__ y, int ld, float* __restrict__ out, int rows,
+                                                     int cols, int rows_per_block) {
+  __shared__ float4 sm[8][32];
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int c4 = blockIdx.x * 32 + lane;
+  const bool col_ok = c4 * 4 < cols;
+  const int r0 = blockIdx.y * rows_per_block;
+  const int r1 = min(rows, r0 + rows_per_block);
+  float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (col_ok) {
+    for (int r = r0 + w; r < r1; r += 8) {
+      const float4 v = load_dy4<IN_F32>(y, (size_t)r, ld, c4);
+      a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+    }
+  }
+  sm[w][lane] = a;
+  __syncthreads();
+  if (w == 0 && col_ok) {
+    for (int i = 1; i < 8; ++i) {
+      const float4 v = sm[i][lane];
+      a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+    }
+    float* po = out + c4 * 4;
+    atomicAdd(po, a.x); atomicAdd(po + 1, a.y); atomicAdd(po + 2, a.z); atomicAdd(po + 3, a.w);
+  }
+}
+
+cudaError_t colsum_bf16(const bf16* y, int ld, float* out, int rows, int cols, cudaStream_t s) {
+  dim3 grid;
+  int rpb;
+  colreduce_grid(rows, 128, cols, &grid, &rpb);
+  colsum_kernel<false><<<grid, 256, 0, s>>>(y, ld, out, rows, cols, rpb);
+  return cudaGetLastError();
+}
+cudaError_t colsum_f32(const float* y, int ld, float* out, int rows, int cols, cudaStream_t s) {
+  dim3 grid;
+  int rpb;
+  colreduce_grid(rows, 128, cols, &grid, &rpb);
+  colsum_kernel<true><<<grid, 256, 0, s>>>(y, ld, out, rows, cols, rpb);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Elementwise
+// ---------------------------------------------------------------------------------------------
+__global__ void add_convert_kernel(const float4* __restrict__ a, const float4* __restrict__ b, float4* out_f32,
+                                   uint2* __restrict__ out_bf16, size_t n4) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+    float4 v = a[i];
+    if (b) {
+      const float4 w = b[i];
+      v.x += w.x; v.y += w.y; v.z += w.z; v.w += w.w;
+    }
+    if (out_f32) out_f32[i] = v;
+    if (out_bf16) {
+      uint2 o;
+      o.x = pack_bf16x2(v.x, v.y);
+      o.y = pack_bf16x2(v.z, v.w);
+      out_bf16[i] = o;
+    }
+  }
+}
+
+cudaError_t add_convert(const float* a, const float* b, float* out_f32, bf16* out_bf16, size_t n, cudaStream_t s) {
+  const size_t n4 = n / 4;
+  int blocks = ceil_div(n4, 256);
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks < 1) blocks = 1;
+  add_convert_kernel<<<blocks, 256, 0, s>>>(reinterpret_cast<const float4*>(a), reinterpret_cast<const float4*>(b),
+                                            reinterpret_cast<float4*>(out_f32), reinterpret_cast<uint2*>(out_bf16), n4);
+  return cudaGetLastError();
+}
+
+cudaError_t f32_to_bf16(const float* in, bf16* out, size_t n, cudaStream_t s) {
+  return add_convert(in, nullptr, nullptr, out, n, s);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Merge of the per-tile softmax partials and the mean cross-entropy: one warp per row
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) lse_finalize_kernel(const float* __restrict__ pm, const float* __restrict__ ps,
+                                                           int part_ld, int ntiles, const float* __restrict__ tgt_logit,
+                                                           float* __restrict__ lse, float* loss_out, int rows,
+                                                           float inv_rows) {
+  __shared__ float sm[8];
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int row = blockIdx.x * 8 + w;
+  float contrib = 0.f;
+  if (row < rows) {
+    float m = -INFINITY;
+    for (int t = lane; t < ntiles; t += 32) m = fmaxf(m, pm[(size_t)row * part_ld + t]);
+    m = warp_max(m);
+    float sum = 0.f;
+    for (int t = lane; t < ntiles; t += 32) {
+      const float tm = pm[(size_t)row * part_ld + t];
+      if (tm > -INFINITY) sum += ps[(size_t)row * part_ld + t] * __expf(tm - m);
+    }
+    sum = warp_sum(sum);
+    const float l = m + logf(sum);
+    if (lane == 0) {
+      lse[row] = l;
+      contrib = l - tgt_logit[row];
+    }
+  }
+  if (lane == 0) sm[w] = contrib;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float t = 0.f;
+    for (int i = 0; i < 8; ++i) t += sm[i];
+    atomicAdd(loss_out, t * inv_rows);
+  }
+}
+
+cudaError_t lse_finalize(const float* part_max, const float* part_sum, int part_ld, int ntiles, const float* tgt_logit,
+                         float* lse, float* loss_out, int rows, cudaStream_t s) {
+  lse_finalize_kernel<<<ceil_div(rows, 8), 256, 0, s>>>(part_max, part_sum, part_ld, ntiles, tgt_logit, lse, loss_out,
+                                                         rows, 1.0f / rows);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// AdamW: 16 bytes/param read (p, m, v, g), 12 written (p, m, v) + 2 (bf16 shadow) = 30 B/param
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) adamw_kernel(float4* __restrict__ p, float4* __restrict__ m, float4* __restrict__ v,
+                                                    const float4* __restrict__ g, uint2* __restrict__ pb, size_t n4,
+                                                    size_t n4_decay, float lr, float b1, float b2, float eps, float wd,
+                                                    float ibc1, float ibc2) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+    const float w = i < n4_decay ? wd : 0.f;
+    float4 pv = p[i], mv = m[i], vv = v[i];
+    const float4 gv = g[i];
+#define IL_ADAM1(F)                                                        \
+  mv.F = b1 * mv.F + (1.f - b1) * gv.F;                                    \
+  vv.F = b2 * vv.F + (1.f - b2) * gv.F * gv.F;                             \
+  pv.F = pv.F - lr * ((mv.F * ibc1) / (sqrtf(vv.F * ibc2) + eps) + w * pv.F);
+    IL_ADAM1(x) IL_ADAM1(y) IL_ADAM1(z) IL_ADAM1(w)
+#undef IL_ADAM1
+    p[i] = pv; m[i] = mv; v[i] = vv;
+    uint2 o;
+    o.x = pack_bf16x2(pv.x, pv.y);
+    o.y = pack_bf16x2(pv.z, pv.w);
+    pb[i] = o;
+  }
+}
+
+cudaError_t adamw(float* p, float* m, float* v, const float* g, bf16* p_bf16, size_t n, size_t n_decay, float lr,
+                  float beta1, float beta2, float eps, float wd, float bc1, float bc2, cudaStream_t s) {
+  const size_t n4 = n / 4;
+  if (n4 == 0) return cudaSuccess;
+  int blocks = ceil_div(n4, 256);
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  adamw_kernel<<<blocks, 256, 0, s>>>(reinterpret_cast<float4*>(p), reinterpret_cast<float4*>(m),
+                                      reinterpret_cast<float4*>(v), reinterpret_cast<const float4*>(g),
+                                      reinterpret_cast<uint2*>(p_bf16), n4, n_decay / 4, lr, beta1, beta2, eps, wd,
+                                      1.0f / bc1, 1.0f / bc2);
+  return cudaGetLastError();
+}
+
+}  // namespace il

@@ -1,0 +1,57 @@
+// Host-side interface of the tcgen05 GEMM: C[M,N] = A[M,K] * B[N,K]^T with bf16 operands, fp32
+// accumulation in tensor memory, operands staged by TMA, and a fused epilogue.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace il {
+
+enum GemmEpilogue : int {
+  EPI_BF16 = 0,        // C(bf16) = acc + bias
+  EPI_BF16_GELU = 1,   // C(bf16) = pre = acc + bias ; C2(bf16) = gelu(pre)
+  EPI_F32_RESID = 2,   // C(f32)  = resid(f32) + acc + bias        (C may alias resid)
+  EPI_BF16_DGELU = 3,  // C(bf16) = acc * gelu'(aux[row % aux_rows, col])
+  EPI_F32 = 4,         // C(f32)  = acc (+ C if accumulate)
+  EPI_LSE = 5,         // online-softmax partials per (row, column tile) + logit of the target column
+  EPI_DZ = 6,          // C(bf16) = (exp(acc - lse[row]) - [col + col0 == target[row]]) * scale
+  EPI_COUNT = 7
+};
+
+// Operand storage.  "K-major": the contraction index is contiguous (row-major [rows, K]).
+// "MN-major": the row index of the operand is contiguous (memory is row-major [K, rows]).
+struct GemmOperand {
+  const void* ptr;   // bf16, 16-byte aligned
+  int ld;            // leading dimension in elements (multiple of 8)
+  int mn_major;      // 0 = K-major, 1 = MN-major
+};
+
+struct GemmArgs {
+  int M, N, K;
+  GemmOperand A, B;
+  int epilogue;
+  void* C;            // [M, ldc]
+  int ldc;
+  void* C2;           // EPI_BF16_GELU: activated output, same ld as C
+  const float* bias;  // [N] or NULL
+  const float* resid; // EPI_F32_RESID: [M, ldc] fp32
+  const void* aux;    // EPI_BF16_DGELU: bf16 [aux_rows, ld_aux]
+  int ld_aux, aux_rows;
+  int accumulate;     // EPI_F32
+  // EPI_LSE / EPI_DZ (vocabulary chunk starting at column col0 of the full vocabulary)
+  const int* targets; // [M]
+  float* part_max;    // [M, part_ld]  written at column (col0 / 256 + column tile)
+  float* part_sum;    // [M, part_ld]
+  int part_ld;
+  float* tgt_logit;   // [M]
+  const float* lse;   // [M]
+  float scale;        // EPI_DZ: 1 / Ntok
+  int col0;
+};
+
+// Enqueue one GEMM on `stream`.  `err_word` is a device word set non-zero when a bounded wait in
+// the kernel expired.  Returns a cudaError_t (argument errors are reported as cudaErrorInvalidValue).
+cudaError_t gemm_launch(const GemmArgs& a, unsigned* err_word, int num_sms, cudaStream_t stream);
+// One-time per-process setup (driver entry point for tensor-map encoding, smem opt-in).
+cudaError_t gemm_init();
+
+}  // namespace il

@@ -1,0 +1,58 @@
+// Host-side launchers of the non-GEMM kernels (HBM-bound elementwise / normalisation / reduction
+// kernels and the attention kernels).  All pointers are device pointers; all launches are asynchronous
+// on `stream` and return cudaGetLastError().
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+namespace il {
+
+// a_0[i,:] = wte[clamp(tok[i]),:] + wpe[i % T,:]  (fp32 residual stream)
+cudaError_t embed_fwd(const int* tok, const float* wte, const float* wpe, float* x, int ntok, int T, int d, int V,
+                      cudaStream_t s);
+// dwte[tok[i],:] += dx[i,:] (atomic), dwpe[t,:] = sum_b dx[b*T+t,:];  dwte must be zeroed by the caller.
+cudaError_t embed_bwd(const int* tok, const float* dx, float* dwte, float* dwpe, int ntok, int T, int d, int V,
+                      cudaStream_t s);
+
+// y(bf16) = gamma * (x - mean) * rstd + beta per row; mean/rstd saved in fp32.
+cudaError_t layernorm_fwd(const float* x, const float* gamma, const float* beta, __nv_bfloat16* y, float* mean,
+                          float* rstd, int rows, int d, float eps, cudaStream_t s);
+// Row part of the LayerNorm backward.  dy is bf16 or fp32 [rows, d]; x/mean/rstd have x_rows rows and are
+// indexed by (row % x_rows) so that several stacked gradient streams can share one saved activation.
+//   dx_out[row,:] = (resid ? resid[row,:] : 0) + LNbwd(dy[row,:]);   dx_bf16 (optional) = bf16 copy.
+cudaError_t layernorm_bwd_rows(const void* dy, int dy_is_f32, const float* x, const float* mean, const float* rstd,
+                               const float* gamma, const float* resid, float* dx_out, __nv_bfloat16* dx_bf16,
+                               int rows, int x_rows, int d, cudaStream_t s);
+// Column reductions over the first `rows` rows: dgamma[c] += sum_r dy[r,c]*xhat[r,c], dbeta[c] += sum_r dy[r,c].
+// Outputs are accumulated atomically and must be zeroed by the caller.
+cudaError_t layernorm_bwd_params(const void* dy, int dy_is_f32, const float* x, const float* mean, const float* rstd,
+                                 float* dgamma, float* dbeta, int rows, int d, cudaStream_t s);
+// out[c] += sum_r y[r,c] for bf16 y [rows, ld] (bias gradients).  out zeroed by the caller.
+cudaError_t colsum_bf16(const __nv_bfloat16* y, int ld, float* out, int rows, int cols, cudaStream_t s);
+// out[c] += sum_r y[r,c] for fp32 y.
+cudaError_t colsum_f32(const float* y, int ld, float* out, int rows, int cols, cudaStream_t s);
+
+// out_f32 = a + (b ? b : 0); out_bf16 (optional) = bf16 copy.   n elements (multiple of 4).
+cudaError_t add_convert(const float* a, const float* b, float* out_f32, __nv_bfloat16* out_bf16, size_t n,
+                        cudaStream_t s);
+cudaError_t f32_to_bf16(const float* in, __nv_bfloat16* out, size_t n, cudaStream_t s);
+
+// Merge per-tile online-softmax partials: lse[r] = log sum_t exp(pm[r,t]) * ps[r,t];
+// loss_out += (1/rows) * sum_r (lse[r] - tgt_logit[r])   (loss_out zeroed by the caller).
+cudaError_t lse_finalize(const float* part_max, const float* part_sum, int part_ld, int ntiles, const float* tgt_logit,
+                         float* lse, float* loss_out, int rows, cudaStream_t s);
+
+// AdamW over a flat range: the first n_decay elements get decoupled weight decay.  Writes the bf16 shadow.
+cudaError_t adamw(float* p, float* m, float* v, const float* g, __nv_bfloat16* p_bf16, size_t n, size_t n_decay,
+                  float lr, float beta1, float beta2, float eps, float wd, float bc1, float bc2, cudaStream_t s);
+
+// Causal attention on packed qkv [B*T, 3d] (Q | K | V, head h at columns h*dh).  dh in {32, 64, 80, 128}.
+//   o [B*T, d] bf16, lse [B, H, T] fp32 (natural log of the softmax denominator, scores scaled by 1/sqrt(dh)).
+cudaError_t attention_fwd(const __nv_bfloat16* qkv, __nv_bfloat16* o, float* lse, int B, int T, int H, int dh,
+                          cudaStream_t s);
+// Backward.  NB batches of gradients share one saved forward of B sequences: gradient batch b uses saved
+// sequence (b % B).  dqkv [NB*T, 3d] bf16; delta is scratch [NB, H, T] fp32.
+cudaError_t attention_bwd(const __nv_bfloat16* qkv, const __nv_bfloat16* o, const float* lse, const __nv_bfloat16* dout,
+                          __nv_bfloat16* dqkv, float* delta, int NB, int B, int T, int H, int dh, cudaStream_t s);
+
+}  // namespace il

@@ -1,0 +1,946 @@
+// C ABI and host runtime of the n-wise training step: parameter registry, activation arena, one CUDA
+// stream per component with event dependencies, and the bookkeeping of the gradient streams of the
+// n-wise rule (Sec. 3, Fig. 2 of the paper).
+//
+// Gradient streams.  Head h (0-based) back-propagates through components h, h-1, ..., term(h) with
+// term(h) = max(h-n+1, 0) and is dropped at the input of component term(h).  Back-propagation is linear
+// in the incoming gradient, so component k does not carry one tensor per head but one per distinct
+// termination level among the heads crossing it, as cumulative sums
+//     U_j = sum of the gradients of heads h crossing k with term(h) <= t_j,   t_0 > t_1 > ...
+// U_0 is the sum over all crossing heads: the parameter gradients of component k come from U_0 alone (one
+// wgrad per matrix), and the U_j are stacked along the token axis so that each dgrad GEMM / attention
+// backward / LayerNorm backward of the component runs once on s_k * Ntok rows.  At the boundary below,
+// the stream that terminates is dropped, the own head's gradient is added to every remaining stream.
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <new>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "../../include/il.h"
+#include "../../include/il_ops.h"
+#include "common.cuh"
+#include "gemm.h"
+#include "kernels.h"
+
+using namespace il;
+
+namespace {
+
+constexpr int VOCAB_CHUNK = 4096;   // columns of dZ held at once in the head backward (bf16, stays near L2)
+
+struct TensorRec {
+  std::string name;
+  int component, is_head, rank;
+  long long shape[2];
+  size_t off, count;
+};
+
+struct LayerOff { size_t ln1g, ln1b, wqkv, bqkv, wo, bo, ln2g, ln2b, w1, b1, w2, b2; };
+struct HeadOff { size_t lng, lnb, w; };
+
+struct LayerActs {
+  bf16 *ln1, *qkv, *attn_o, *ln2, *hpre, *hact;
+  float *mean1, *rstd1, *lse, *x_mid, *mean2, *rstd2, *x_out;
+};
+
+struct CompScratch {     // backward scratch of one component, rows = s_cap * ntok_max
+  float* dx; bf16* dxb; bf16* dbig; bf16* dln; bf16* dattn; bf16* dqkv; float* delta;
+};
+struct HeadScratch {
+  bf16* u; float *mean, *rstd, *pmax, *psum, *tgt_logit, *lse, *du, *ghead; bf16* dz;
+};
+
+struct ProfRec { cudaEvent_t a, b; double flops; };
+
+}  // namespace
+
+struct il_model {
+  int K, Lc, d, H, F, V, n, dh;
+  int device, num_sms;
+  int max_batch, max_seq, ntok_max;
+  float ln_eps;
+  il_options opt;
+  bool own_streams;
+  std::vector<cudaStream_t> streams;
+  std::vector<cudaEvent_t> ev_fwd, ev_bwd, ev_join;
+  cudaEvent_t ev_batch;
+  // parameters
+  std::vector<TensorRec> tensors;
+  std::vector<LayerOff> layer_off;   // K*Lc
+  std::vector<HeadOff> head_off;     // K
+  size_t off_wte, off_wpe;
+  std::vector<size_t> comp_begin, comp_mat_end, comp_end;   // flat ranges per component
+  size_t total;
+  float *P, *G, *M1, *M2;
+  bf16* Pb;
+  long long step;
+  // activations
+  std::vector<float*> a;             // K+1 boundaries; a[k+1] aliases the last layer's x_out
+  std::vector<LayerActs> acts;       // K*Lc
+  std::vector<CompScratch> cs;
+  std::vector<HeadScratch> hs;
+  int s_cap;
+  int *tokens, *targets;
+  float* losses;                     // device [K]
+  unsigned* err_word;
+  int part_ld;
+  // step state
+  int B, T, ntok;
+  bool batch_set, bwd_done;
+  std::vector<char> fwd_done, loss_done;
+  // allocations
+  std::vector<void*> allocs;
+  long long bytes, launches;
+  // profiling
+  bool prof;
+  std::vector<ProfRec> prof_recs;
+  std::vector<cudaEvent_t> prof_pool;
+  std::string err;
+};
+
+namespace {
+
+il_status fail(il_model* m, il_status s, const char* fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  if (m) m->err = buf;
+  return s;
+}
+
+#define IL_CUDA(m, call)                                                                            \
+  do {                                                                                              \
+    cudaError_t e__ = (call);                                                                       \
+    if (e__ != cudaSuccess)                                                                         \
+      return fail(m, IL_ERR_CUDA, "%s failed: %s (%s:%d)", #call, cudaGetErrorString(e__), __FILE__, __LINE__); \
+  } while (0)
+#define IL_TRY(call)                      \
+  do {                                    \
+    il_status s__ = (call);               \
+    if (s__ != IL_OK) return s__;         \
+  } while (0)
+
+il_status dev_alloc(il_model* m, void** out, size_t bytes) {
+  bytes = (bytes + 255) & ~size_t(255);
+  if (bytes == 0) bytes = 256;
+  void* p = nullptr;
+  if (m->opt.alloc) {
+    p = m->opt.alloc(bytes, m->opt.alloc_ctx);
+  } else {
+    if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); p = nullptr; }
+  }
+  if (!p) return fail(m, IL_ERR_OOM, "device allocation of %zu bytes failed", bytes);
+  if ((uintptr_t)p % 256) return fail(m, IL_ERR_INVALID_ARG, "allocator returned a pointer that is not 256-byte aligned");
+  m->allocs.push_back(p);
+  m->bytes += (long long)bytes;
+  *out = p;
+  return IL_OK;
+}
+template <typename T>
+il_status dev_alloc_t(il_model* m, T** out, size_t count) {
+  void* p;
+  IL_TRY(dev_alloc(m, &p, count * sizeof(T)));
+  *out = reinterpret_cast<T*>(p);
+  return IL_OK;
+}
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// termination level of head h under the n-wise rule
+inline int term_of(int h, int n) { return h - n + 1 > 0 ? h - n + 1 : 0; }
+// distinct termination levels of the heads crossing component k, descending
+std::vector<int> terms_of(int k, int K, int n) {
+  std::vector<int> t;
+  const int hi = k + n - 1 < K - 1 ? k + n - 1 : K - 1;
+  for (int h = hi; h >= k; --h) {
+    const int th = term_of(h, n);
+    if (t.empty() || t.back() != th) t.push_back(th);
+  }
+  return t;
+}
+int s_cap_for(int K, int n) {
+  size_t s = 1;
+  for (int k = 0; k < K; ++k) s = std::max(s, terms_of(k, K, n).size());
+  return (int)s;
+}
+
+il_status gemm(il_model* m, int k, const GemmArgs& g) {
+  cudaStream_t st = m->streams[k];
+  ProfRec rec{};
+  if (m->prof) {
+    for (int i = 0; i < 2; ++i) {
+      cudaEvent_t e;
+      if (!m->prof_pool.empty()) { e = m->prof_pool.back(); m->prof_pool.pop_back(); }
+      else IL_CUDA(m, cudaEventCreate(&e));
+      (i == 0 ? rec.a : rec.b) = e;
+    }
+    rec.flops = 2.0 * g.M * g.N * (double)g.K;
+    IL_CUDA(m, cudaEventRecord(rec.a, st));
+  }
+  cudaError_t e = gemm_launch(g, m->err_word, m->num_sms, st);
+  if (e != cudaSuccess)
+    return fail(m, e == cudaErrorInvalidValue ? IL_ERR_INVALID_ARG : IL_ERR_CUDA, "gemm launch (M=%d N=%d K=%d epi=%d): %s",
+                g.M, g.N, g.K, g.epilogue, cudaGetErrorString(e));
+  if (m->prof) {
+    IL_CUDA(m, cudaEventRecord(rec.b, st));
+    m->prof_recs.push_back(rec);
+  }
+  m->launches++;
+  return IL_OK;
+}
+
+GemmArgs gemm_args(int M, int N, int K, const void* A, int lda, int a_mn, const void* B, int ldb, int b_mn, int epi,
+                   void* C, int ldc) {
+  GemmArgs g;
+  memset(&g, 0, sizeof g);
+  g.M = M; g.N = N; g.K = K;
+  g.A = {A, lda, a_mn};
+  g.B = {B, ldb, b_mn};
+  g.epilogue = epi;
+  g.C = C; g.ldc = ldc;
+  return g;
+}
+
+#define IL_K(m, call)                                                                                   \
+  do {                                                                                                  \
+    cudaError_t e__ = (call);                                                                           \
+    if (e__ != cudaSuccess) return fail(m, IL_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e__));      \
+    (m)->launches++;                                                                                    \
+  } while (0)
+
+il_status alloc_scratch(il_model* m, int s_cap) {
+  // grow-only: backward scratch for s_cap stacked gradient streams per component
+  if (s_cap <= m->s_cap) return IL_OK;
+  const size_t R = (size_t)s_cap * m->ntok_max;
+  const int d = m->d, F = m->F;
+  m->cs.assign(m->K, CompScratch{});
+  for (int k = 0; k < m->K; ++k) {
+    CompScratch& c = m->cs[k];
+    IL_TRY(dev_alloc_t(m, &c.dx, R * d));
+    IL_TRY(dev_alloc_t(m, &c.dxb, R * d));
+    IL_TRY(dev_alloc_t(m, &c.dbig, R * F));
+    IL_TRY(dev_alloc_t(m, &c.dln, R * d));
+    IL_TRY(dev_alloc_t(m, &c.dattn, R * d));
+    IL_TRY(dev_alloc_t(m, &c.dqkv, R * 3 * d));
+    IL_TRY(dev_alloc_t(m, &c.delta, R * m->H));
+  }
+  m->s_cap = s_cap;
+  return IL_OK;
+}
+
+il_status join_all(il_model* m) {
+  // stream 0 waits for every other stream, then everyone waits for stream 0
+  for (int k = 1; k < m->K; ++k) {
+    IL_CUDA(m, cudaEventRecord(m->ev_join[k], m->streams[k]));
+    IL_CUDA(m, cudaStreamWaitEvent(m->streams[0], m->ev_join[k], 0));
+  }
+  return IL_OK;
+}
+
+il_status check_model(const il_model* m) { return m ? IL_OK : IL_ERR_INVALID_ARG; }
+
+}  // namespace
+
+// =================================================================================================
+// creation / destruction
+// =================================================================================================
+extern "C" il_status il_create(int K, int Lc, int d, int H, int F, int V, int n, const il_options* opt, il_model** out) {
+  if (!out) return IL_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!opt || K < 1 || Lc < 1 || d < 8 || H < 1 || F < 8 || V < 2 || n < 1 || n > K) return IL_ERR_INVALID_ARG;
+  if (d % H || d % 8 || F % 8 || opt->max_batch < 1 || opt->max_seq < 1) return IL_ERR_INVALID_ARG;
+  const int dh = d / H;
+  if (!(dh == 32 || dh == 64 || dh == 80 || dh == 128)) return IL_ERR_INVALID_ARG;
+  if (opt->streams && opt->n_streams < K) return IL_ERR_INVALID_ARG;
+  if ((opt->alloc == nullptr) != (opt->free_ == nullptr)) return IL_ERR_INVALID_ARG;
+
+  il_model* m = new (std::nothrow) il_model();
+  if (!m) return IL_ERR_OOM;
+  m->K = K; m->Lc = Lc; m->d = d; m->H = H; m->F = F; m->V = V; m->n = n; m->dh = dh;
+  m->opt = *opt;
+  m->device = opt->device;
+  m->max_batch = opt->max_batch; m->max_seq = opt->max_seq;
+  m->ntok_max = opt->max_batch * opt->max_seq;
+  m->ln_eps = opt->ln_eps > 0 ? opt->ln_eps : 1e-5f;
+  m->step = 0; m->bytes = 0; m->launches = 0; m->s_cap = 0;
+  m->prof = false; m->batch_set = false; m->bwd_done = false;
+  m->B = m->T = m->ntok = 0;
+  m->P = m->G = m->M1 = m->M2 = nullptr; m->Pb = nullptr;
+  *out = m;   // returned even on failure below so that il_last_error/il_destroy work
+
+  auto bail = [&](il_status s) { return s; };
+  {
+    cudaError_t e = cudaSetDevice(m->device);
+    if (e != cudaSuccess) return bail(fail(m, IL_ERR_CUDA, "cudaSetDevice(%d): %s", m->device, cudaGetErrorString(e)));
+    cudaDeviceProp prop;
+    e = cudaGetDeviceProperties(&prop, m->device);
+    if (e != cudaSuccess) return bail(fail(m, IL_ERR_CUDA, "cudaGetDeviceProperties: %s", cudaGetErrorString(e)));
+    if (prop.major != 10) return bail(fail(m, IL_ERR_CUDA, "device %d is sm_%d%d; this library is built for sm_100a only", m->device, prop.major, prop.minor));
+    m->num_sms = prop.multiProcessorCount;
+    e = gemm_init();
+    if (e != cudaSuccess) return bail(fail(m, IL_ERR_CUDA, "gemm_init: %s", cudaGetErrorString(e)));
+  }
+
+  // ---- parameter registry and flat layout (per component: matrices first, then vectors)
+  auto add = [&](const std::string& name, int comp, int is_head, int rank, long long s0, long long s1) {
+    TensorRec t;
+    t.name = name; t.component = comp; t.is_head = is_head; t.rank = rank;
+    t.shape[0] = s0; t.shape[1] = rank == 2 ? s1 : 1;
+    t.count = (size_t)s0 * (rank == 2 ? s1 : 1);
+    t.off = 0;
+    m->tensors.push_back(t);
+    return (int)m->tensors.size() - 1;
+  };
+  add("wte", 0, 0, 2, V, d);
+  add("wpe", 0, 0, 2, m->max_seq, d);
+  const char* lnames[12] = {"ln1.g", "ln1.b", "attn.wqkv", "attn.bqkv", "attn.wo", "attn.bo",
+                            "ln2.g", "ln2.b", "mlp.w1", "mlp.b1", "mlp.w2", "mlp.b2"};
+  for (int k = 0; k < K; ++k)
+    for (int l = 0; l < Lc; ++l) {
+      char pre[64];
+      snprintf(pre, sizeof pre, "c%d.l%d.", k, l);
+      const long long s0[12] = {d, d, 3LL * d, 3LL * d, d, d, d, d, F, F, d, d};
+      const long long s1[12] = {0, 0, d, 0, d, 0, 0, 0, d, 0, F, 0};
+      for (int i = 0; i < 12; ++i) add(std::string(pre) + lnames[i], k, 0, s1[i] ? 2 : 1, s0[i], s1[i]);
+    }
+  for (int k = 0; k < K; ++k) {
+    char pre[64];
+    snprintf(pre, sizeof pre, "head%d.", k);
+    add(std::string(pre) + "ln.g", k, 1, 1, d, 0);
+    add(std::string(pre) + "ln.b", k, 1, 1, d, 0);
+    add(std::string(pre) + "w", k, 1, 2, V, d);
+  }
+  size_t cur = 0;
+  m->comp_begin.resize(K); m->comp_mat_end.resize(K); m->comp_end.resize(K);
+  for (int k = 0; k < K; ++k) {
+    m->comp_begin[k] = cur;
+    for (int pass = 0; pass < 2; ++pass) {       // pass 0: rank-2 (decayed), pass 1: rank-1
+      for (auto& t : m->tensors)
+        if (t.component == k && (t.rank == 2) == (pass == 0)) {
+          t.off = cur;
+          cur = align_up(cur + t.count, 64);
+        }
+      if (pass == 0) m->comp_mat_end[k] = cur;
+    }
+    m->comp_end[k] = cur;
+  }
+  m->total = cur;
+  m->layer_off.resize((size_t)K * Lc);
+  m->head_off.resize(K);
+  {
+    size_t i = 0;
+    m->off_wte = m->tensors[i++].off;
+    m->off_wpe = m->tensors[i++].off;
+    for (int kl = 0; kl < K * Lc; ++kl) {
+      LayerOff& o = m->layer_off[kl];
+      o.ln1g = m->tensors[i++].off; o.ln1b = m->tensors[i++].off; o.wqkv = m->tensors[i++].off;
+      o.bqkv = m->tensors[i++].off; o.wo = m->tensors[i++].off; o.bo = m->tensors[i++].off;
+      o.ln2g = m->tensors[i++].off; o.ln2b = m->tensors[i++].off; o.w1 = m->tensors[i++].off;
+      o.b1 = m->tensors[i++].off; o.w2 = m->tensors[i++].off; o.b2 = m->tensors[i++].off;
+    }
+    for (int k = 0; k < K; ++k) {
+      HeadOff& o = m->head_off[k];
+      o.lng = m->tensors[i++].off; o.lnb = m->tensors[i++].off; o.w = m->tensors[i++].off;
+    }
+  }
+
+  // ---- streams and events
+  m->own_streams = (opt->streams == nullptr);
+  m->streams.resize(K);
+  for (int k = 0; k < K; ++k) {
+    if (m->own_streams) {
+      cudaError_t e = cudaStreamCreateWithFlags(&m->streams[k], cudaStreamNonBlocking);
+      if (e != cudaSuccess) { m->streams.resize(k); return bail(fail(m, IL_ERR_CUDA, "cudaStreamCreate: %s", cudaGetErrorString(e))); }
+    } else {
+      m->streams[k] = reinterpret_cast<cudaStream_t>(opt->streams[k]);
+    }
+  }
+  auto mk_events = [&](std::vector<cudaEvent_t>& v) -> il_status {
+    v.resize(K);
+    for (int k = 0; k < K; ++k) {
+      cudaError_t e = cudaEventCreateWithFlags(&v[k], cudaEventDisableTiming);
+      if (e != cudaSuccess) { v.resize(k); return fail(m, IL_ERR_CUDA, "cudaEventCreate: %s", cudaGetErrorString(e)); }
+    }
+    return IL_OK;
+  };
+  IL_TRY(mk_events(m->ev_fwd));
+  IL_TRY(mk_events(m->ev_bwd));
+  IL_TRY(mk_events(m->ev_join));
+  IL_CUDA(m, cudaEventCreateWithFlags(&m->ev_batch, cudaEventDisableTiming));
+
+  // ---- parameter, gradient and optimiser storage
+  IL_TRY(dev_alloc_t(m, &m->P, m->total));
+  IL_TRY(dev_alloc_t(m, &m->G, m->total));
+  IL_TRY(dev_alloc_t(m, &m->M1, m->total));
+  IL_TRY(dev_alloc_t(m, &m->M2, m->total));
+  IL_TRY(dev_alloc_t(m, &m->Pb, m->total));
+  IL_CUDA(m, cudaMemset(m->P, 0, m->total * 4));
+  IL_CUDA(m, cudaMemset(m->G, 0, m->total * 4));
+  IL_CUDA(m, cudaMemset(m->M1, 0, m->total * 4));
+  IL_CUDA(m, cudaMemset(m->M2, 0, m->total * 4));
+  IL_CUDA(m, cudaMemset(m->Pb, 0, m->total * 2));
+  {  // LayerNorm gains start at one
+    std::vector<float> ones(d, 1.0f);
+    for (auto& t : m->tensors)
+      if (t.name.size() >= 2 && t.name.compare(t.name.size() - 2, 2, ".g") == 0) {
+        IL_CUDA(m, cudaMemcpy(m->P + t.off, ones.data(), d * 4, cudaMemcpyHostToDevice));
+      }
+    IL_K(m, f32_to_bf16(m->P, m->Pb, m->total, m->streams[0]));
+    IL_CUDA(m, cudaStreamSynchronize(m->streams[0]));
+  }
+
+  // ---- activations
+  const size_t N = m->ntok_max;
+  m->a.assign(K + 1, nullptr);
+  IL_TRY(dev_alloc_t(m, &m->a[0], N * d));
+  m->acts.resize((size_t)K * Lc);
+  for (int k = 0; k < K; ++k)
+    for (int l = 0; l < Lc; ++l) {
+      LayerActs& A = m->acts[(size_t)k * Lc + l];
+      IL_TRY(dev_alloc_t(m, &A.ln1, N * d));
+      IL_TRY(dev_alloc_t(m, &A.qkv, N * 3 * d));
+      IL_TRY(dev_alloc_t(m, &A.attn_o, N * d));
+      IL_TRY(dev_alloc_t(m, &A.ln2, N * d));
+      IL_TRY(dev_alloc_t(m, &A.hpre, N * F));
+      IL_TRY(dev_alloc_t(m, &A.hact, N * F));
+      IL_TRY(dev_alloc_t(m, &A.mean1, N));
+      IL_TRY(dev_alloc_t(m, &A.rstd1, N));
+      IL_TRY(dev_alloc_t(m, &A.mean2, N));
+      IL_TRY(dev_alloc_t(m, &A.rstd2, N));
+      IL_TRY(dev_alloc_t(m, &A.lse, N * H));
+      IL_TRY(dev_alloc_t(m, &A.x_mid, N * d));
+      IL_TRY(dev_alloc_t(m, &A.x_out, N * d));
+      if (l == Lc - 1) m->a[k + 1] = A.x_out;
+    }
+  m->part_ld = (V + 255) / 256;
+  m->hs.assign(K, HeadScratch{});
+  for (int k = 0; k < K; ++k) {
+    HeadScratch& h = m->hs[k];
+    IL_TRY(dev_alloc_t(m, &h.u, N * d));
+    IL_TRY(dev_alloc_t(m, &h.mean, N));
+    IL_TRY(dev_alloc_t(m, &h.rstd, N));
+    IL_TRY(dev_alloc_t(m, &h.pmax, N * m->part_ld));
+    IL_TRY(dev_alloc_t(m, &h.psum, N * m->part_ld));
+    IL_TRY(dev_alloc_t(m, &h.tgt_logit, N));
+    IL_TRY(dev_alloc_t(m, &h.lse, N));
+    IL_TRY(dev_alloc_t(m, &h.du, N * d));
+    IL_TRY(dev_alloc_t(m, &h.ghead, N * d));
+    IL_TRY(dev_alloc_t(m, &h.dz, N * (size_t)VOCAB_CHUNK));
+  }
+  IL_TRY(alloc_scratch(m, s_cap_for(K, n)));
+  IL_TRY(dev_alloc_t(m, &m->tokens, N));
+  IL_TRY(dev_alloc_t(m, &m->targets, N));
+  IL_TRY(dev_alloc_t(m, &m->losses, (size_t)K));
+  IL_TRY(dev_alloc_t(m, &m->err_word, (size_t)1));
+  IL_CUDA(m, cudaMemset(m->err_word, 0, 4));
+  IL_CUDA(m, cudaMemset(m->losses, 0, K * 4));
+  m->fwd_done.assign(K, 0);
+  m->loss_done.assign(K, 0);
+  IL_CUDA(m, cudaDeviceSynchronize());
+  return IL_OK;
+}
+
+extern "C" il_status il_destroy(il_model* m) {
+  if (!m) return IL_ERR_INVALID_ARG;
+  cudaSetDevice(m->device);
+  cudaDeviceSynchronize();
+  for (void* p : m->allocs) {
+    if (m->opt.free_) m->opt.free_(p, m->opt.alloc_ctx);
+    else cudaFree(p);
+  }
+  for (auto e : m->ev_fwd) cudaEventDestroy(e);
+  for (auto e : m->ev_bwd) cudaEventDestroy(e);
+  for (auto e : m->ev_join) cudaEventDestroy(e);
+  if (m->ev_batch) cudaEventDestroy(m->ev_batch);
+  for (auto e : m->prof_pool) cudaEventDestroy(e);
+  for (auto& r : m->prof_recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+  if (m->own_streams)
+    for (auto s : m->streams) cudaStreamDestroy(s);
+  delete m;
+  return IL_OK;
+}
+
+extern "C" il_status il_set_n(il_model* m, int n) {
+  IL_TRY(check_model(m));
+  if (n < 1 || n > m->K) return fail(m, IL_ERR_INVALID_ARG, "n=%d outside [1, %d]", n, m->K);
+  IL_CUDA(m, cudaSetDevice(m->device));
+  IL_CUDA(m, cudaDeviceSynchronize());
+  IL_TRY(alloc_scratch(m, s_cap_for(m->K, n)));
+  m->n = n;
+  return IL_OK;
+}
+
+// =================================================================================================
+// registry
+// =================================================================================================
+extern "C" int il_num_tensors(const il_model* m) { return m ? (int)m->tensors.size() : -1; }
+
+extern "C" il_status il_tensor_info(const il_model* m, int idx, const char** name, int* component, int* is_head, int* rank,
+                                    long long shape[2]) {
+  if (!m || idx < 0 || idx >= (int)m->tensors.size()) return IL_ERR_INVALID_ARG;
+  const TensorRec& t = m->tensors[idx];
+  if (name) *name = t.name.c_str();
+  if (component) *component = t.component;
+  if (is_head) *is_head = t.is_head;
+  if (rank) *rank = t.rank;
+  if (shape) { shape[0] = t.shape[0]; shape[1] = t.shape[1]; }
+  return IL_OK;
+}
+
+static il_status tensor_io(il_model* m, int idx, size_t count, const TensorRec** t) {
+  IL_TRY(check_model(m));
+  if (idx < 0 || idx >= (int)m->tensors.size()) return fail(m, IL_ERR_INVALID_ARG, "tensor index %d out of range", idx);
+  *t = &m->tensors[idx];
+  if (count != (*t)->count) return fail(m, IL_ERR_INVALID_ARG, "tensor %s has %zu elements, got %zu", (*t)->name.c_str(), (*t)->count, count);
+  IL_CUDA(m, cudaSetDevice(m->device));
+  IL_CUDA(m, cudaDeviceSynchronize());
+  return IL_OK;
+}
+
+extern "C" il_status il_set_param(il_model* m, int idx, const float* host, size_t count) {
+  const TensorRec* t;
+  if (!host) return IL_ERR_INVALID_ARG;
+  IL_TRY(tensor_io(m, idx, count, &t));
+  IL_CUDA(m, cudaMemcpy(m->P + t->off, host, count * 4, cudaMemcpyHostToDevice));
+  IL_K(m, f32_to_bf16(m->P + t->off, m->Pb + t->off, align_up(count, 4), m->streams[0]));
+  IL_CUDA(m, cudaStreamSynchronize(m->streams[0]));
+  return IL_OK;
+}
+extern "C" il_status il_get_param(il_model* m, int idx, float* host, size_t count) {
+  const TensorRec* t;
+  if (!host) return IL_ERR_INVALID_ARG;
+  IL_TRY(tensor_io(m, idx, count, &t));
+  IL_CUDA(m, cudaMemcpy(host, m->P + t->off, count * 4, cudaMemcpyDeviceToHost));
+  return IL_OK;
+}
+extern "C" il_status il_get_grad(il_model* m, int idx, float* host, size_t count) {
+  const TensorRec* t;
+  if (!host) return IL_ERR_INVALID_ARG;
+  IL_TRY(tensor_io(m, idx, count, &t));
+  if (!m->bwd_done) return fail(m, IL_ERR_STATE, "il_get_grad before il_backward_nwise");
+  IL_CUDA(m, cudaMemcpy(host, m->G + t->off, count * 4, cudaMemcpyDeviceToHost));
+  return IL_OK;
+}
+extern "C" il_status il_get_opt_state(il_model* m, int idx, float* mh, float* vh, long long* step) {
+  IL_TRY(check_model(m));
+  if (idx < 0 || idx >= (int)m->tensors.size()) return fail(m, IL_ERR_INVALID_ARG, "tensor index %d out of range", idx);
+  const TensorRec* t;
+  IL_TRY(tensor_io(m, idx, m->tensors[idx].count, &t));
+  if (mh) IL_CUDA(m, cudaMemcpy(mh, m->M1 + t->off, t->count * 4, cudaMemcpyDeviceToHost));
+  if (vh) IL_CUDA(m, cudaMemcpy(vh, m->M2 + t->off, t->count * 4, cudaMemcpyDeviceToHost));
+  if (step) *step = m->step;
+  return IL_OK;
+}
+extern "C" il_status il_set_opt_state(il_model* m, int idx, const float* mh, const float* vh, long long step) {
+  IL_TRY(check_model(m));
+  if (idx < 0 || idx >= (int)m->tensors.size()) return fail(m, IL_ERR_INVALID_ARG, "tensor index %d out of range", idx);
+  if (step < 0) return fail(m, IL_ERR_INVALID_ARG, "negative step");
+  const TensorRec* t;
+  IL_TRY(tensor_io(m, idx, m->tensors[idx].count, &t));
+  if (mh) IL_CUDA(m, cudaMemcpy(m->M1 + t->off, mh, t->count * 4, cudaMemcpyHostToDevice));
+  if (vh) IL_CUDA(m, cudaMemcpy(m->M2 + t->off, vh, t->count * 4, cudaMemcpyHostToDevice));
+  m->step = step;
+  return IL_OK;
+}
+
+// =================================================================================================
+// the step
+// =================================================================================================
+extern "C" il_status il_set_batch(il_model* m, const int* tokens, const int* targets, int B, int T, int on_device) {
+  IL_TRY(check_model(m));
+  if (!tokens || !targets) return fail(m, IL_ERR_INVALID_ARG, "NULL tokens/targets");
+  if (B < 1 || T < 1 || B > m->max_batch || T > m->max_seq || (size_t)B * T > (size_t)m->ntok_max)
+    return fail(m, IL_ERR_INVALID_ARG, "batch %dx%d exceeds max_batch=%d, max_seq=%d", B, T, m->max_batch, m->max_seq);
+  IL_CUDA(m, cudaSetDevice(m->device));
+  // every stream's previous work must be finished before buffers of the last step are overwritten
+  IL_TRY(join_all(m));
+  cudaStream_t s0 = m->streams[0];
+  const size_t bytes = (size_t)B * T * sizeof(int);
+  const cudaMemcpyKind kind = on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
+  IL_CUDA(m, cudaMemcpyAsync(m->tokens, tokens, bytes, kind, s0));
+  IL_CUDA(m, cudaMemcpyAsync(m->targets, targets, bytes, kind, s0));
+  IL_CUDA(m, cudaMemsetAsync(m->losses, 0, m->K * sizeof(float), s0));
+  IL_CUDA(m, cudaEventRecord(m->ev_batch, s0));
+  for (int k = 1; k < m->K; ++k) IL_CUDA(m, cudaStreamWaitEvent(m->streams[k], m->ev_batch, 0));
+  m->B = B; m->T = T; m->ntok = B * T;
+  m->batch_set = true;
+  m->bwd_done = false;
+  std::fill(m->fwd_done.begin(), m->fwd_done.end(), 0);
+  std::fill(m->loss_done.begin(), m->loss_done.end(), 0);
+  return IL_OK;
+}
+
+extern "C" il_status il_forward_component(il_model* m, int k) {
+  IL_TRY(check_model(m));
+  if (k < 0 || k >= m->K) return fail(m, IL_ERR_INVALID_ARG, "component %d out of range", k);
+  if (!m->batch_set) return fail(m, IL_ERR_STATE, "il_forward_component before il_set_batch");
+  if (k > 0 && !m->fwd_done[k - 1]) return fail(m, IL_ERR_STATE, "component %d forward needs component %d first", k, k - 1);
+  if (m->fwd_done[k]) return fail(m, IL_ERR_STATE, "component %d already forwarded in this step", k);
+  IL_CUDA(m, cudaSetDevice(m->device));
+  cudaStream_t st = m->streams[k];
+  const int N = m->ntok, d = m->d, F = m->F;
+  if (k == 0) {
+    IL_K(m, embed_fwd(m->tokens, m->P + m->off_wte, m->P + m->off_wpe, m->a[0], N, m->T, d, m->V, st));
+  } else {
+    IL_CUDA(m, cudaStreamWaitEvent(st, m->ev_fwd[k - 1], 0));
+  }
+  const float* x_in = m->a[k];
+  for (int l = 0; l < m->Lc; ++l) {
+    const LayerOff& o = m->layer_off[(size_t)k * m->Lc + l];
+    LayerActs& A = m->acts[(size_t)k * m->Lc + l];
+    IL_K(m, layernorm_fwd(x_in, m->P + o.ln1g, m->P + o.ln1b, A.ln1, A.mean1, A.rstd1, N, d, m->ln_eps, st));
+    {
+      GemmArgs g = gemm_args(N, 3 * d, d, A.ln1, d, 0, m->Pb + o.wqkv, d, 0, EPI_BF16, A.qkv, 3 * d);
+      g.bias = m->P + o.bqkv;
+      IL_TRY(gemm(m, k, g));
+    }
+    IL_K(m, attention_fwd(A.qkv, A.attn_o, A.lse, m->B, m->T, m->H, m->dh, st));
+    {
+      GemmArgs g = gemm_args(N, d, d, A.attn_o, d, 0, m->Pb + o.wo, d, 0, EPI_F32_RESID, A.x_mid, d);
+      g.bias = m->P + o.bo;
+      g.resid = x_in;
+      IL_TRY(gemm(m, k, g));
+    }
+    IL_K(m, layernorm_fwd(A.x_mid, m->P + o.ln2g, m->P + o.ln2b, A.ln2, A.mean2, A.rstd2, N, d, m->ln_eps, st));
+    {
+      GemmArgs g = gemm_args(N, F, d, A.ln2, d, 0, m->Pb + o.w1, d, 0, EPI_BF16_GELU, A.hpre, F);
+      g.C2 = A.hact;
+      g.bias = m->P + o.b1;
+      IL_TRY(gemm(m, k, g));
+    }
+    {
+      GemmArgs g = gemm_args(N, d, F, A.hact, F, 0, m->Pb + o.w2, F, 0, EPI_F32_RESID, A.x_out, d);
+      g.bias = m->P + o.b2;
+      g.resid = A.x_mid;
+      IL_TRY(gemm(m, k, g));
+    }
+    x_in = A.x_out;
+  }
+  IL_CUDA(m, cudaEventRecord(m->ev_fwd[k], st));
+  m->fwd_done[k] = 1;
+  return IL_OK;
+}
+
+extern "C" il_status il_aux_head_loss(il_model* m, int k, float* loss_host) {
+  IL_TRY(check_model(m));
+  if (k < 0 || k >= m->K) return fail(m, IL_ERR_INVALID_ARG, "head %d out of range", k);
+  if (!m->batch_set || !m->fwd_done[k]) return fail(m, IL_ERR_STATE, "il_aux_head_loss(%d) needs il_forward_component(%d)", k, k);
+  IL_CUDA(m, cudaSetDevice(m->device));
+  cudaStream_t st = m->streams[k];
+  if (!m->loss_done[k]) {
+    const int N = m->ntok, d = m->d, V = m->V;
+    const HeadOff& o = m->head_off[k];
+    HeadScratch& h = m->hs[k];
+    IL_K(m, layernorm_fwd(m->a[k + 1], m->P + o.lng, m->P + o.lnb, h.u, h.mean, h.rstd, N, d, m->ln_eps, st));
+    GemmArgs g = gemm_args(N, V, d, h.u, d, 0, m->Pb + o.w, d, 0, EPI_LSE, nullptr, 0);
+    g.targets = m->targets;
+    g.part_max = h.pmax; g.part_sum = h.psum; g.part_ld = m->part_ld;
+    g.tgt_logit = h.tgt_logit;
+    g.col0 = 0;
+    IL_TRY(gemm(m, k, g));
+    IL_K(m, lse_finalize(h.pmax, h.psum, m->part_ld, m->part_ld, h.tgt_logit, h.lse, m->losses + k, N, st));
+    m->loss_done[k] = 1;
+  }
+  if (loss_host) {
+    IL_CUDA(m, cudaMemcpyAsync(loss_host, m->losses + k, sizeof(float), cudaMemcpyDeviceToHost, st));
+    IL_CUDA(m, cudaStreamSynchronize(st));
+  }
+  return IL_OK;
+}
+
+extern "C" il_status il_get_losses(il_model* m, float* losses_host) {
+  IL_TRY(check_model(m));
+  if (!losses_host) return fail(m, IL_ERR_INVALID_ARG, "NULL output");
+  for (int k = 0; k < m->K; ++k)
+    if (!m->loss_done[k]) return fail(m, IL_ERR_STATE, "head %d has no loss in this step", k);
+  IL_CUDA(m, cudaSetDevice(m->device));
+  for (int k = 0; k < m->K; ++k) IL_CUDA(m, cudaStreamSynchronize(m->streams[k]));
+  IL_CUDA(m, cudaMemcpy(losses_host, m->losses, m->K * sizeof(float), cudaMemcpyDeviceToHost));
+  return IL_OK;
+}
+
+namespace {
+
+// Head k backward on stream k: dZ chunk by chunk over the vocabulary -> dW_h, dU; LayerNorm backward -> ghead.
+il_status head_backward(il_model* m, int k) {
+  cudaStream_t st = m->streams[k];
+  const int N = m->ntok, d = m->d, V = m->V;
+  const HeadOff& o = m->head_off[k];
+  HeadScratch& h = m->hs[k];
+  for (int v0 = 0; v0 < V; v0 += VOCAB_CHUNK) {
+    const int nv = V - v0 < VOCAB_CHUNK ? V - v0 : VOCAB_CHUNK;
+    const bf16* Wc = m->Pb + o.w + (size_t)v0 * d;
+    {  // logits of the chunk recomputed, turned into dZ = (softmax - onehot) / Ntok in the epilogue
+      GemmArgs g = gemm_args(N, nv, d, h.u, d, 0, Wc, d, 0, EPI_DZ, h.dz, VOCAB_CHUNK);
+      g.targets = m->targets;
+      g.lse = h.lse;
+      g.scale = 1.0f / (float)N;
+      g.col0 = v0;
+      IL_TRY(gemm(m, k, g));
+    }
+    {  // dU += dZ_chunk * W_chunk
+      GemmArgs g = gemm_args(N, d, nv, h.dz, VOCAB_CHUNK, 0, Wc, d, 1, EPI_F32, h.du, d);
+      g.accumulate = v0 > 0;
+      IL_TRY(gemm(m, k, g));
+    }
+    {  // dW_chunk = dZ_chunk^T * U
+      GemmArgs g = gemm_args(nv, d, N, h.dz, VOCAB_CHUNK, 1, h.u, d, 1, EPI_F32, m->G + o.w + (size_t)v0 * d, d);
+      IL_TRY(gemm(m, k, g));
+    }
+  }
+  IL_K(m, layernorm_bwd_params(h.du, 1, m->a[k + 1], h.mean, h.rstd, m->G + o.lng, m->G + o.lnb, N, d, st));
+  IL_K(m, layernorm_bwd_rows(h.du, 1, m->a[k + 1], h.mean, h.rstd, m->P + o.lng, nullptr, h.ghead, nullptr, N, N, d, st));
+  return IL_OK;
+}
+
+// Component k backward on stream k for s stacked gradient streams already placed in cs[k].dx / dxb.
+il_status component_backward(il_model* m, int k, int s) {
+  cudaStream_t st = m->streams[k];
+  const int N = m->ntok, d = m->d, F = m->F;
+  const int R = s * N;
+  CompScratch& c = m->cs[k];
+  for (int l = m->Lc - 1; l >= 0; --l) {
+    const LayerOff& o = m->layer_off[(size_t)k * m->Lc + l];
+    LayerActs& A = m->acts[(size_t)k * m->Lc + l];
+    const float* x_in = (l == 0) ? m->a[k] : m->acts[(size_t)k * m->Lc + l - 1].x_out;
+    // ---- MLP: x_out = x_mid + W2 gelu(W1 ln2 + b1) + b2
+    IL_K(m, colsum_f32(c.dx, d, m->G + o.b2, N, d, st));
+    IL_TRY(gemm(m, k, gemm_args(d, F, N, c.dxb, d, 1, A.hact, F, 1, EPI_F32, m->G + o.w2, F)));
+    {
+      GemmArgs g = gemm_args(R, F, d, c.dxb, d, 0, m->Pb + o.w2, F, 1, EPI_BF16_DGELU, c.dbig, F);
+      g.aux = A.hpre; g.ld_aux = F; g.aux_rows = N;
+      IL_TRY(gemm(m, k, g));
+    }
+    IL_K(m, colsum_bf16(c.dbig, F, m->G + o.b1, N, F, st));
+    IL_TRY(gemm(m, k, gemm_args(F, d, N, c.dbig, F, 1, A.ln2, d, 1, EPI_F32, m->G + o.w1, d)));
+    IL_TRY(gemm(m, k, gemm_args(R, d, F, c.dbig, F, 0, m->Pb + o.w1, d, 1, EPI_BF16, c.dln, d)));
+    IL_K(m, layernorm_bwd_params(c.dln, 0, A.x_mid, A.mean2, A.rstd2, m->G + o.ln2g, m->G + o.ln2b, N, d, st));
+    IL_K(m, layernorm_bwd_rows(c.dln, 0, A.x_mid, A.mean2, A.rstd2, m->P + o.ln2g, c.dx, c.dx, c.dxb, R, N, d, st));
+    // ---- attention: x_mid = x_in + Wo attn(Wqkv ln1 + bqkv) + bo
+    IL_K(m, colsum_f32(c.dx, d, m->G + o.bo, N, d, st));
+    IL_TRY(gemm(m, k, gemm_args(d, d, N, c.dxb, d, 1, A.attn_o, d, 1, EPI_F32, m->G + o.wo, d)));
+    IL_TRY(gemm(m, k, gemm_args(R, d, d, c.dxb, d, 0, m->Pb + o.wo, d, 1, EPI_BF16, c.dattn, d)));
+    IL_K(m, attention_bwd(A.qkv, A.attn_o, A.lse, c.dattn, c.dqkv, c.delta, s * m->B, m->B, m->T, m->H, m->dh, st));
+    m->launches += 2;
+    IL_K(m, colsum_bf16(c.dqkv, 3 * d, m->G + o.bqkv, N, 3 * d, st));
+    IL_TRY(gemm(m, k, gemm_args(3 * d, d, N, c.dqkv, 3 * d, 1, A.ln1, d, 1, EPI_F32, m->G + o.wqkv, d)));
+    IL_TRY(gemm(m, k, gemm_args(R, d, 3 * d, c.dqkv, 3 * d, 0, m->Pb + o.wqkv, d, 1, EPI_BF16, c.dln, d)));
+    IL_K(m, layernorm_bwd_params(c.dln, 0, x_in, A.mean1, A.rstd1, m->G + o.ln1g, m->G + o.ln1b, N, d, st));
+    IL_K(m, layernorm_bwd_rows(c.dln, 0, x_in, A.mean1, A.rstd1, m->P + o.ln1g, c.dx, c.dx, c.dxb, R, N, d, st));
+  }
+  return IL_OK;
+}
+
+}  // namespace
+
+extern "C" il_status il_backward_nwise(il_model* m) {
+  IL_TRY(check_model(m));
+  if (!m->batch_set) return fail(m, IL_ERR_STATE, "il_backward_nwise before il_set_batch");
+  for (int k = 0; k < m->K; ++k)
+    if (!m->fwd_done[k] || !m->loss_done[k])
+      return fail(m, IL_ERR_STATE, "il_backward_nwise needs all %d forwards and head losses (component %d missing)", m->K, k);
+  if (m->bwd_done) return fail(m, IL_ERR_STATE, "il_backward_nwise already called in this step");
+  IL_CUDA(m, cudaSetDevice(m->device));
+  const int K = m->K, n = m->n, N = m->ntok, d = m->d;
+  const size_t slice = (size_t)N * d;
+
+  // every head's own backward is independent of the others: enqueue all of them first
+  for (int k = 0; k < K; ++k) {
+    cudaStream_t st = m->streams[k];
+    IL_CUDA(m, cudaMemsetAsync(m->G + m->comp_mat_end[k], 0, (m->comp_end[k] - m->comp_mat_end[k]) * 4, st));
+    if (k == 0) {
+      const size_t emb = (size_t)m->V * d;
+      IL_CUDA(m, cudaMemsetAsync(m->G + m->off_wte, 0, emb * 4, st));
+      IL_CUDA(m, cudaMemsetAsync(m->G + m->off_wpe, 0, (size_t)m->max_seq * d * 4, st));
+    }
+    IL_TRY(head_backward(m, k));
+  }
+  // components from the top down; component k needs the pass-down of component k+1 when any stream crosses
+  std::vector<int> above;   // termination levels of the streams of component k+1
+  for (int k = K - 1; k >= 0; --k) {
+    cudaStream_t st = m->streams[k];
+    const std::vector<int> terms = terms_of(k, K, n);
+    const int s = (int)terms.size();
+    bool needs_above = false;
+    for (int j = 0; j < s; ++j) {
+      int src = -1;
+      for (size_t q = 0; q < above.size(); ++q)
+        if (above[q] == terms[j]) src = (int)q;
+      if (src >= 0 && !needs_above) {
+        IL_CUDA(m, cudaStreamWaitEvent(st, m->ev_bwd[k + 1], 0));
+        needs_above = true;
+      }
+      const float* passed = src >= 0 ? m->cs[k + 1].dx + (size_t)src * slice : nullptr;
+      IL_K(m, add_convert(m->hs[k].ghead, passed, m->cs[k].dx + (size_t)j * slice, m->cs[k].dxb + (size_t)j * slice, slice, st));
+    }
+    IL_TRY(component_backward(m, k, s));
+    if (k == 0) {
+      IL_K(m, embed_bwd(m->tokens, m->cs[0].dx, m->G + m->off_wte, m->G + m->off_wpe, N, m->T, d, m->V, st));
+      m->launches++;
+    }
+    IL_CUDA(m, cudaEventRecord(m->ev_bwd[k], st));
+    above = terms;
+  }
+  m->bwd_done = true;
+  return IL_OK;
+}
+
+extern "C" il_status il_adamw_step(il_model* m, float lr, float beta1, float beta2, float eps, float wd) {
+  IL_TRY(check_model(m));
+  if (!m->bwd_done || !m->batch_set) return fail(m, IL_ERR_STATE, "il_adamw_step needs il_backward_nwise of the current step");
+  if (!(beta1 >= 0 && beta1 < 1 && beta2 >= 0 && beta2 < 1 && eps >= 0)) return fail(m, IL_ERR_INVALID_ARG, "bad AdamW hyper-parameters");
+  IL_CUDA(m, cudaSetDevice(m->device));
+  m->step += 1;
+  const double bc1 = 1.0 - pow((double)beta1, (double)m->step);
+  const double bc2 = 1.0 - pow((double)beta2, (double)m->step);
+  // Parameters, gradients and bf16 shadows of component k (its head and, for k = 0, the embeddings included)
+  // are read and written by stream k only, so each component updates on its own stream as soon as its
+  // gradients are final (the last backward pass through a module triggers its update, App. C).
+  for (int k = 0; k < m->K; ++k) {
+    const size_t b = m->comp_begin[k], e = m->comp_end[k], me = m->comp_mat_end[k];
+    IL_K(m, adamw(m->P + b, m->M1 + b, m->M2 + b, m->G + b, m->Pb + b, e - b, me - b, lr, beta1, beta2, eps, wd, (float)bc1,
+                  (float)bc2, m->streams[k]));
+  }
+  m->batch_set = false;   // a new batch is required for the next step
+  return IL_OK;
+}
+
+extern "C" il_status il_sync(il_model* m) {
+  IL_TRY(check_model(m));
+  IL_CUDA(m, cudaSetDevice(m->device));
+  for (int k = 0; k < m->K; ++k) IL_CUDA(m, cudaStreamSynchronize(m->streams[k]));
+  unsigned w = 0;
+  IL_CUDA(m, cudaMemcpy(&w, m->err_word, 4, cudaMemcpyDeviceToHost));
+  if (w) {
+    IL_CUDA(m, cudaMemset(m->err_word, 0, 4));
+    return fail(m, IL_ERR_TIMEOUT, "a bounded device-side wait expired (code %u)", w);
+  }
+  return IL_OK;
+}
+
+extern "C" il_status il_get_boundary(il_model* m, int k, float* host, size_t count) {
+  IL_TRY(check_model(m));
+  if (k < 0 || k > m->K || !host) return fail(m, IL_ERR_INVALID_ARG, "boundary %d out of range", k);
+  if (!m->batch_set || (k > 0 && !m->fwd_done[k - 1]) || (k == 0 && !m->fwd_done[0])) return fail(m, IL_ERR_STATE, "boundary %d not computed in this step", k);
+  if (count != (size_t)m->ntok * m->d) return fail(m, IL_ERR_INVALID_ARG, "boundary has %zu elements, got %zu", (size_t)m->ntok * m->d, count);
+  IL_CUDA(m, cudaSetDevice(m->device));
+  IL_CUDA(m, cudaDeviceSynchronize());
+  IL_CUDA(m, cudaMemcpy(host, m->a[k], count * 4, cudaMemcpyDeviceToHost));
+  return IL_OK;
+}
+
+extern "C" il_status il_stats(const il_model* m, long long* device_bytes, long long* kernel_launches) {
+  if (!m) return IL_ERR_INVALID_ARG;
+  if (device_bytes) *device_bytes = m->bytes;
+  if (kernel_launches) *kernel_launches = m->launches;
+  return IL_OK;
+}
+
+extern "C" il_status il_profile(il_model* m, int enable) {
+  IL_TRY(check_model(m));
+  IL_CUDA(m, cudaSetDevice(m->device));
+  IL_CUDA(m, cudaDeviceSynchronize());
+  for (auto& r : m->prof_recs) { m->prof_pool.push_back(r.a); m->prof_pool.push_back(r.b); }
+  m->prof_recs.clear();
+  m->prof = enable != 0;
+  return IL_OK;
+}
+
+extern "C" il_status il_profile_read(il_model* m, double* gemm_ms, long long* gemm_launches, double* gemm_flops) {
+  IL_TRY(check_model(m));
+  IL_CUDA(m, cudaSetDevice(m->device));
+  IL_CUDA(m, cudaDeviceSynchronize());
+  double ms = 0, fl = 0;
+  for (auto& r : m->prof_recs) {
+    float t = 0;
+    IL_CUDA(m, cudaEventElapsedTime(&t, r.a, r.b));
+    ms += t;
+    fl += r.flops;
+  }
+  if (gemm_ms) *gemm_ms = ms;
+  if (gemm_launches) *gemm_launches = (long long)m->prof_recs.size();
+  if (gemm_flops) *gemm_flops = fl;
+  for (auto& r : m->prof_recs) { m->prof_pool.push_back(r.a); m->prof_pool.push_back(r.b); }
+  m->prof_recs.clear();
+  return IL_OK;
+}
+
+extern "C" il_status il_nwise_streams(int K, int n, int k, int* terms, int* count) {
+  if (K < 1 || n < 1 || n > K || k < 0 || k >= K || !count) return IL_ERR_INVALID_ARG;
+  const std::vector<int> t = terms_of(k, K, n);
+  *count = (int)t.size();
+  if (terms)
+    for (size_t i = 0; i < t.size(); ++i) terms[i] = t[i];
+  return IL_OK;
+}
+
+extern "C" const char* il_last_error(const il_model* m) { return m ? m->err.c_str() : "null model"; }
+
+extern "C" const char* il_status_string(il_status s) {
+  switch (s) {
+    case IL_OK: return "IL_OK";
+    case IL_ERR_INVALID_ARG: return "IL_ERR_INVALID_ARG";
+    case IL_ERR_STATE: return "IL_ERR_STATE";
+    case IL_ERR_OOM: return "IL_ERR_OOM";
+    case IL_ERR_CUDA: return "IL_ERR_CUDA";
+    case IL_ERR_TIMEOUT: return "IL_ERR_TIMEOUT";
+    case IL_ERR_NONFINITE: return "IL_ERR_NONFINITE";
+  }
+  return "unknown";
+}
+
+// =================================================================================================
+// operator-level entry points
+// =================================================================================================
+static il_status op_status(cudaError_t e) {
+  if (e == cudaSuccess) return IL_OK;
+  return e == cudaErrorInvalidValue ? IL_ERR_INVALID_ARG : IL_ERR_CUDA;
+}
+
+extern "C" il_status il_op_gemm(const il_gemm_desc* q, unsigned* err_word, void* stream) {
+  if (!q || !err_word) return IL_ERR_INVALID_ARG;
+  GemmArgs g = gemm_args(q->M, q->N, q->K, q->A, q->lda, q->a_mn_major, q->B, q->ldb, q->b_mn_major, q->epilogue, q->C, q->ldc);
+  g.C2 = q->C2; g.bias = q->bias; g.resid = q->resid; g.aux = q->aux; g.ld_aux = q->ld_aux; g.aux_rows = q->aux_rows;
+  g.accumulate = q->accumulate; g.targets = q->targets; g.part_max = q->part_max; g.part_sum = q->part_sum;
+  g.part_ld = q->part_ld; g.tgt_logit = q->tgt_logit; g.lse = q->lse; g.scale = q->scale; g.col0 = q->col0;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return IL_ERR_CUDA;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return IL_ERR_CUDA;
+  return op_status(gemm_launch(g, err_word, sms, reinterpret_cast<cudaStream_t>(stream)));
+}
+
+extern "C" il_status il_op_attention_fwd(const void* qkv, void* o, float* lse, int B, int T, int H, int dh, void* stream) {
+  if (!qkv || !o || !lse || B < 1 || T < 1 || H < 1) return IL_ERR_INVALID_ARG;
+  return op_status(attention_fwd((const bf16*)qkv, (bf16*)o, lse, B, T, H, dh, reinterpret_cast<cudaStream_t>(stream)));
+}
+
+extern "C" il_status il_op_attention_bwd(const void* qkv, const void* o, const float* lse, const void* dout, void* dqkv,
+                                         float* delta, int NB, int B, int T, int H, int dh, void* stream) {
+  if (!qkv || !o || !lse || !dout || !dqkv || !delta || B < 1 || NB < 1 || T < 1 || H < 1) return IL_ERR_INVALID_ARG;
+  return op_status(attention_bwd((const bf16*)qkv, (const bf16*)o, lse, (const bf16*)dout, (bf16*)dqkv, delta, NB, B, T, H, dh,
+                                 reinterpret_cast<cudaStream_t>(stream)));
+}
+
+extern "C" il_status il_op_layernorm_fwd(const float* x, const float* gamma, const float* beta, void* y, float* mean,
+                                         float* rstd, int rows, int d, float eps, void* stream) {
+  if (!x || !gamma || !beta || !y || !mean || !rstd || rows < 1 || d < 8 || d % 8) return IL_ERR_INVALID_ARG;
+  return op_status(layernorm_fwd(x, gamma, beta, (bf16*)y, mean, rstd, rows, d, eps, reinterpret_cast<cudaStream_t>(stream)));
+}
+
+extern "C" il_status il_op_layernorm_bwd(const void* dy, int dy_is_f32, const float* x, const float* mean, const float* rstd,
+                                         const float* gamma, const float* resid, float* dx, void* dx_bf16, float* dgamma,
+                                         float* dbeta, int rows, int x_rows, int d, void* stream) {
+  if (!dy || !x || !mean || !rstd || !gamma || !dx || rows < 1 || x_rows < 1 || d < 8 || d % 8) return IL_ERR_INVALID_ARG;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (dgamma && dbeta) {
+    cudaError_t e = layernorm_bwd_params(dy, dy_is_f32, x, mean, rstd, dgamma, dbeta, x_rows < rows ? x_rows : rows, d, st);
+    if (e != cudaSuccess) return op_status(e);
+  }
+  return op_status(layernorm_bwd_rows(dy, dy_is_f32, x, mean, rstd, gamma, resid, dx, (bf16*)dx_bf16, rows, x_rows, d, st));
+}
