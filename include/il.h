@@ -99,6 +99,9 @@ il_status il_forward_component(il_model* m, int k);
  * consumed tile by tile (never stored).  Needs il_forward_component(k).  loss_host != NULL makes the
  * call wait for this head and return its loss; NULL leaves it asynchronous. */
 il_status il_aux_head_loss(il_model* m, int k, float* loss_host);
+/* Per-token negative log-likelihood of head k for the current step, fp32 [B*T] to host (their mean is
+ * the head's loss).  Needs il_aux_head_loss(k); waits for it. */
+il_status il_get_token_losses(il_model* m, int k, float* host, size_t count);
 /* All K losses of the current step (waits for them). */
 il_status il_get_losses(il_model* m, float* losses_host);
 /* n-wise backward (Sec. 3, Fig. 2): for every head, back-propagation through the head and through

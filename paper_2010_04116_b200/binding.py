@@ -76,6 +76,7 @@ def lib() -> C.CDLL:
         "il_get_losses": [vp, C.POINTER(f)], "il_backward_nwise": [vp],
         "il_adamw_step": [vp, f, f, f, f, f], "il_sync": [vp],
         "il_get_boundary": [vp, i, vp, sz],
+        "il_get_token_losses": [vp, i, vp, sz],
         "il_stats": [vp, C.POINTER(C.c_longlong), C.POINTER(C.c_longlong)],
         "il_profile": [vp, i],
         "il_profile_read": [vp, C.POINTER(C.c_double), C.POINTER(C.c_longlong), C.POINTER(C.c_double)],
@@ -262,6 +263,11 @@ class Model:
         out = (C.c_float * self.K)()
         self._ck(self.L.il_get_losses(self._h, out))
         return np.array(list(out), dtype=np.float32)
+
+    def get_token_losses(self, k: int, ntok: int) -> np.ndarray:
+        out = np.empty(ntok, dtype=np.float32)
+        self._ck(self.L.il_get_token_losses(self._h, k, out.ctypes.data, out.size))
+        return out
 
     def backward_nwise(self):
         self._ck(self.L.il_backward_nwise(self._h))

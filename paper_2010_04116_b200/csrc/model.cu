@@ -245,6 +245,13 @@ il_status join_all(il_model* m) {
 
 il_status check_model(const il_model* m) { return m ? IL_OK : IL_ERR_INVALID_ARG; }
 
+// Stream-ordered copy on stream 0 followed by a wait: the data is in place when this returns.
+il_status copy_sync(il_model* m, void* dst, const void* src, size_t bytes, cudaMemcpyKind kind) {
+  IL_CUDA(m, cudaMemcpyAsync(dst, src, bytes, kind, m->streams[0]));
+  IL_CUDA(m, cudaStreamSynchronize(m->streams[0]));
+  return IL_OK;
+}
+
 }  // namespace
 
 // =================================================================================================
@@ -380,19 +387,23 @@ extern "C" il_status il_create(int K, int Lc, int d, int H, int F, int V, int n,
   IL_TRY(dev_alloc_t(m, &m->M1, m->total));
   IL_TRY(dev_alloc_t(m, &m->M2, m->total));
   IL_TRY(dev_alloc_t(m, &m->Pb, m->total));
-  IL_CUDA(m, cudaMemset(m->P, 0, m->total * 4));
-  IL_CUDA(m, cudaMemset(m->G, 0, m->total * 4));
-  IL_CUDA(m, cudaMemset(m->M1, 0, m->total * 4));
-  IL_CUDA(m, cudaMemset(m->M2, 0, m->total * 4));
-  IL_CUDA(m, cudaMemset(m->Pb, 0, m->total * 2));
+  // All host<->device copies of the library are stream-ordered on stream 0 (a synchronous cudaMemcpy from
+  // pageable memory may return before its DMA has landed, and the legacy stream does not order against
+  // the non-blocking streams used here).
+  cudaStream_t s0 = m->streams[0];
+  IL_CUDA(m, cudaMemsetAsync(m->P, 0, m->total * 4, s0));
+  IL_CUDA(m, cudaMemsetAsync(m->G, 0, m->total * 4, s0));
+  IL_CUDA(m, cudaMemsetAsync(m->M1, 0, m->total * 4, s0));
+  IL_CUDA(m, cudaMemsetAsync(m->M2, 0, m->total * 4, s0));
+  IL_CUDA(m, cudaMemsetAsync(m->Pb, 0, m->total * 2, s0));
   {  // LayerNorm gains start at one
     std::vector<float> ones(d, 1.0f);
     for (auto& t : m->tensors)
       if (t.name.size() >= 2 && t.name.compare(t.name.size() - 2, 2, ".g") == 0) {
-        IL_CUDA(m, cudaMemcpy(m->P + t.off, ones.data(), d * 4, cudaMemcpyHostToDevice));
+        IL_CUDA(m, cudaMemcpyAsync(m->P + t.off, ones.data(), d * 4, cudaMemcpyHostToDevice, s0));
       }
-    IL_K(m, f32_to_bf16(m->P, m->Pb, m->total, m->streams[0]));
-    IL_CUDA(m, cudaStreamSynchronize(m->streams[0]));
+    IL_K(m, f32_to_bf16(m->P, m->Pb, m->total, s0));
+    IL_CUDA(m, cudaStreamSynchronize(s0));
   }
 
   // ---- activations
@@ -438,8 +449,8 @@ extern "C" il_status il_create(int K, int Lc, int d, int H, int F, int V, int n,
   IL_TRY(dev_alloc_t(m, &m->targets, N));
   IL_TRY(dev_alloc_t(m, &m->losses, (size_t)K));
   IL_TRY(dev_alloc_t(m, &m->err_word, (size_t)1));
-  IL_CUDA(m, cudaMemset(m->err_word, 0, 4));
-  IL_CUDA(m, cudaMemset(m->losses, 0, K * 4));
+  IL_CUDA(m, cudaMemsetAsync(m->err_word, 0, 4, s0));
+  IL_CUDA(m, cudaMemsetAsync(m->losses, 0, K * 4, s0));
   m->fwd_done.assign(K, 0);
   m->loss_done.assign(K, 0);
   IL_CUDA(m, cudaDeviceSynchronize());
@@ -507,7 +518,7 @@ extern "C" il_status il_set_param(il_model* m, int idx, const float* host, size_
   const TensorRec* t;
   if (!host) return IL_ERR_INVALID_ARG;
   IL_TRY(tensor_io(m, idx, count, &t));
-  IL_CUDA(m, cudaMemcpy(m->P + t->off, host, count * 4, cudaMemcpyHostToDevice));
+  IL_CUDA(m, cudaMemcpyAsync(m->P + t->off, host, count * 4, cudaMemcpyHostToDevice, m->streams[0]));
   IL_K(m, f32_to_bf16(m->P + t->off, m->Pb + t->off, align_up(count, 4), m->streams[0]));
   IL_CUDA(m, cudaStreamSynchronize(m->streams[0]));
   return IL_OK;
@@ -516,7 +527,7 @@ extern "C" il_status il_get_param(il_model* m, int idx, float* host, size_t coun
   const TensorRec* t;
   if (!host) return IL_ERR_INVALID_ARG;
   IL_TRY(tensor_io(m, idx, count, &t));
-  IL_CUDA(m, cudaMemcpy(host, m->P + t->off, count * 4, cudaMemcpyDeviceToHost));
+  IL_TRY(copy_sync(m, host, m->P + t->off, count * 4, cudaMemcpyDeviceToHost));
   return IL_OK;
 }
 extern "C" il_status il_get_grad(il_model* m, int idx, float* host, size_t count) {
@@ -524,7 +535,7 @@ extern "C" il_status il_get_grad(il_model* m, int idx, float* host, size_t count
   if (!host) return IL_ERR_INVALID_ARG;
   IL_TRY(tensor_io(m, idx, count, &t));
   if (!m->bwd_done) return fail(m, IL_ERR_STATE, "il_get_grad before il_backward_nwise");
-  IL_CUDA(m, cudaMemcpy(host, m->G + t->off, count * 4, cudaMemcpyDeviceToHost));
+  IL_TRY(copy_sync(m, host, m->G + t->off, count * 4, cudaMemcpyDeviceToHost));
   return IL_OK;
 }
 extern "C" il_status il_get_opt_state(il_model* m, int idx, float* mh, float* vh, long long* step) {
@@ -532,8 +543,8 @@ extern "C" il_status il_get_opt_state(il_model* m, int idx, float* mh, float* vh
   if (idx < 0 || idx >= (int)m->tensors.size()) return fail(m, IL_ERR_INVALID_ARG, "tensor index %d out of range", idx);
   const TensorRec* t;
   IL_TRY(tensor_io(m, idx, m->tensors[idx].count, &t));
-  if (mh) IL_CUDA(m, cudaMemcpy(mh, m->M1 + t->off, t->count * 4, cudaMemcpyDeviceToHost));
-  if (vh) IL_CUDA(m, cudaMemcpy(vh, m->M2 + t->off, t->count * 4, cudaMemcpyDeviceToHost));
+  if (mh) IL_TRY(copy_sync(m, mh, m->M1 + t->off, t->count * 4, cudaMemcpyDeviceToHost));
+  if (vh) IL_TRY(copy_sync(m, vh, m->M2 + t->off, t->count * 4, cudaMemcpyDeviceToHost));
   if (step) *step = m->step;
   return IL_OK;
 }
@@ -543,8 +554,8 @@ extern "C" il_status il_set_opt_state(il_model* m, int idx, const float* mh, con
   if (step < 0) return fail(m, IL_ERR_INVALID_ARG, "negative step");
   const TensorRec* t;
   IL_TRY(tensor_io(m, idx, m->tensors[idx].count, &t));
-  if (mh) IL_CUDA(m, cudaMemcpy(m->M1 + t->off, mh, t->count * 4, cudaMemcpyHostToDevice));
-  if (vh) IL_CUDA(m, cudaMemcpy(m->M2 + t->off, vh, t->count * 4, cudaMemcpyHostToDevice));
+  if (mh) IL_TRY(copy_sync(m, m->M1 + t->off, mh, t->count * 4, cudaMemcpyHostToDevice));
+  if (vh) IL_TRY(copy_sync(m, m->M2 + t->off, vh, t->count * 4, cudaMemcpyHostToDevice));
   m->step = step;
   return IL_OK;
 }
@@ -654,6 +665,21 @@ extern "C" il_status il_aux_head_loss(il_model* m, int k, float* loss_host) {
   return IL_OK;
 }
 
+extern "C" il_status il_get_token_losses(il_model* m, int k, float* host, size_t count) {
+  IL_TRY(check_model(m));
+  if (k < 0 || k >= m->K || !host) return fail(m, IL_ERR_INVALID_ARG, "head %d out of range or NULL output", k);
+  if (!m->batch_set || !m->loss_done[k]) return fail(m, IL_ERR_STATE, "head %d has no loss in this step", k);
+  if (count != (size_t)m->ntok) return fail(m, IL_ERR_INVALID_ARG, "expected %d values, got %zu", m->ntok, count);
+  IL_CUDA(m, cudaSetDevice(m->device));
+  IL_CUDA(m, cudaStreamSynchronize(m->streams[k]));
+  std::vector<float> tl(count);
+  IL_CUDA(m, cudaMemcpyAsync(host, m->hs[k].lse, count * 4, cudaMemcpyDeviceToHost, m->streams[k]));
+  IL_CUDA(m, cudaMemcpyAsync(tl.data(), m->hs[k].tgt_logit, count * 4, cudaMemcpyDeviceToHost, m->streams[k]));
+  IL_CUDA(m, cudaStreamSynchronize(m->streams[k]));
+  for (size_t i = 0; i < count; ++i) host[i] -= tl[i];
+  return IL_OK;
+}
+
 extern "C" il_status il_get_losses(il_model* m, float* losses_host) {
   IL_TRY(check_model(m));
   if (!losses_host) return fail(m, IL_ERR_INVALID_ARG, "NULL output");
@@ -661,7 +687,7 @@ extern "C" il_status il_get_losses(il_model* m, float* losses_host) {
     if (!m->loss_done[k]) return fail(m, IL_ERR_STATE, "head %d has no loss in this step", k);
   IL_CUDA(m, cudaSetDevice(m->device));
   for (int k = 0; k < m->K; ++k) IL_CUDA(m, cudaStreamSynchronize(m->streams[k]));
-  IL_CUDA(m, cudaMemcpy(losses_host, m->losses, m->K * sizeof(float), cudaMemcpyDeviceToHost));
+  IL_TRY(copy_sync(m, losses_host, m->losses, m->K * sizeof(float), cudaMemcpyDeviceToHost));
   return IL_OK;
 }
 
@@ -816,9 +842,10 @@ extern "C" il_status il_sync(il_model* m) {
   IL_CUDA(m, cudaSetDevice(m->device));
   for (int k = 0; k < m->K; ++k) IL_CUDA(m, cudaStreamSynchronize(m->streams[k]));
   unsigned w = 0;
-  IL_CUDA(m, cudaMemcpy(&w, m->err_word, 4, cudaMemcpyDeviceToHost));
+  IL_TRY(copy_sync(m, &w, m->err_word, 4, cudaMemcpyDeviceToHost));
   if (w) {
-    IL_CUDA(m, cudaMemset(m->err_word, 0, 4));
+    IL_CUDA(m, cudaMemsetAsync(m->err_word, 0, 4, m->streams[0]));
+    IL_CUDA(m, cudaStreamSynchronize(m->streams[0]));
     return fail(m, IL_ERR_TIMEOUT, "a bounded device-side wait expired (code %u)", w);
   }
   return IL_OK;
@@ -831,7 +858,7 @@ extern "C" il_status il_get_boundary(il_model* m, int k, float* host, size_t cou
   if (count != (size_t)m->ntok * m->d) return fail(m, IL_ERR_INVALID_ARG, "boundary has %zu elements, got %zu", (size_t)m->ntok * m->d, count);
   IL_CUDA(m, cudaSetDevice(m->device));
   IL_CUDA(m, cudaDeviceSynchronize());
-  IL_CUDA(m, cudaMemcpy(host, m->a[k], count * 4, cudaMemcpyDeviceToHost));
+  IL_TRY(copy_sync(m, host, m->a[k], count * 4, cudaMemcpyDeviceToHost));
   return IL_OK;
 }
 

@@ -90,8 +90,8 @@ def test_head_dim_80():
 
 
 def test_one_wise_locality_on_device():
-    """n = 1: changing head 1 leaves every gradient of component 0 and head 0 bit-identical... up to the
-    atomics' summation order, so compare within a tight tolerance instead of bit-exactly."""
+    """n = 1: changing head 1 leaves every gradient of component 0 and head 0 unchanged (up to the
+    summation order of the atomic column reductions, hence a tight tolerance rather than bit equality)."""
     w = wl.CONFIGS["cfg1"]
     P = wl.draw_params(w)
     tok, tgt = wl.draw_tokens(w)
@@ -109,7 +109,8 @@ def test_one_wise_locality_on_device():
         for nme in m.names:
             g1 = m.get_grad(nme)
             if nme.startswith("c0.") or nme.startswith("head0.") or nme in ("wte", "wpe"):
-                assert np.allclose(g0[nme], g1, rtol=1e-4, atol=1e-9), nme
+                den = max(np.linalg.norm(g0[nme]), 1e-30)
+                assert np.linalg.norm(g0[nme] - g1) / den < 1e-5, nme
         assert not np.allclose(g0["c1.l0.mlp.w1"], m.get_grad("c1.l0.mlp.w1"))
     finally:
         m.close()
