@@ -1,0 +1,282 @@
+#!/usr/bin/env python
+"""Throughput of one n-wise training step (tokens/s) on synthetic data.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config cfg4] [--n 2] [--impl reference]
+
+A step is the whole hot path on one batch: il_set_batch, K x (il_forward_component, il_aux_head_loss),
+il_backward_nwise and, where the configuration says so, il_adamw_step.  The default workload is the
+GPT-2-medium-shaped configuration (24 layers in 8 components, d 1024, seq 1024, batch 8, vocab 50257,
+n = 2, AdamW).  With N > 1 (launched under torch.distributed.run) every rank runs an independent
+replica of the same step on its own GPU: the path has no exchange step, so there is no collective on
+the data path and the scaling is weak.  Rank 0 prints one JSON line.
+
+`--impl reference` times the fp64 CPU oracle, as it stands, on the host cores on a bounded sample of
+the same workload (one sequence of the batch).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import workloads as wl  # noqa: E402
+
+
+def model_flops_per_token(w: wl.Workload, n: int) -> float:
+    """Algorithmic flops per token of one n-wise step: every contraction the method defines, counted once
+    (forward, one wgrad per matrix, one dgrad per distinct gradient stream); recomputation is not counted."""
+    gemm = 2.0 * (3 * w.d * w.d + w.d * w.d + 2 * w.d * w.F)          # per layer, forward
+    att_f = 2.0 * w.T * w.d                                            # causal QK^T + PV
+    att_b = 4.0 * w.T * w.d
+    total = 0.0
+    for k in range(w.K):
+        heads = [h for h in range(w.K) if max(h - n + 1, 0) <= k <= h]
+        s_k = len({max(h - n + 1, 0) for h in heads})
+        total += w.Lc * (gemm + att_f) + w.Lc * gemm + s_k * w.Lc * (gemm + att_b)
+    total += w.K * 6.0 * w.d * w.V
+    return total
+
+
+class ClockSampler:
+    """Samples SM clock, power and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0])); smax.append(float(f[1])); power.append(float(f[2]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, f[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def oracle_sample(w: wl.Workload, n: int, steps: int, warmup: int, params=None, budget_s: float = 25.0):
+    """Time the oracle (fp64, numpy), as it stands, on a bounded sample of the workload: the first
+    positions of one sequence of the batch, the sample length chosen so that the whole call takes about
+    `budget_s` seconds of host time.  Returns (tokens/s, seconds per step, info)."""
+    from oracle import il_oracle as orc
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    est_per_token = model_flops_per_token(w, n) / 45e9          # observed oracle rate on 8 cores, rough
+    ts = int(budget_s / max(steps + warmup, 1) / est_per_token) // 32 * 32
+    ts = max(32, min(ts, w.T))
+    ws = w.with_(B=1, T=ts)
+    P = params if params is not None else wl.draw_params(w)
+    tok, tgt = wl.draw_tokens(w)
+    tok, tgt = np.ascontiguousarray(tok[:1, :ts]), np.ascontiguousarray(tgt[:1, :ts])
+    times = []
+    for i in range(warmup + steps):
+        t0 = time.perf_counter()
+        orc.nwise_gradients(P, tok, tgt, ws.K, ws.Lc, ws.H, n)
+        if i >= warmup:
+            times.append(time.perf_counter() - t0)
+    sec = float(np.mean(times))
+    info = {"value": ws.ntok / sec, "unit": "tokens/s", "cores": int(cores), "kind": "oracle",
+            "sample": f"{len(times)} oracle step(s) (forward, K heads, per-head n-wise backward; no optimiser) on the "
+                      f"first {ts} positions of 1 of {w.B} sequences of {w.name} (full model, n={n}); "
+                      f"{sec:.2f} s per step"}
+    return ws.ntok / sec, sec, info
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", default="cfg4")
+    ap.add_argument("--n", type=int, default=None)
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-adamw", action="store_true")
+    args = ap.parse_args()
+
+    w = wl.CONFIGS[args.config]
+    n = args.n if args.n is not None else w.n
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    metric = "training tokens/s per n-wise step"
+    cfg_desc = {"workload": f"{w.name}: {w.K}x{w.Lc} layers, d={w.d}, H={w.H}, F={w.F}, T={w.T}, B={w.B}, V={w.V}, "
+                            f"n={n}, adamw={bool(w.adamw and not args.no_adamw)}",
+                "global_batch": w.B * max(world, 1), "seq_len": w.T, "parallelism": f"replicas x{max(world, 1)}",
+                "l2": "inputs larger than L2 (each step streams several GB of weights and activations)"}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        steps, warm = max(1, args.steps), max(0, args.warmup)
+        val, sec, info = oracle_sample(w, n, steps, warm, budget_s=150.0)
+        info = dict(info, value=val)
+        print(json.dumps({"impl": "reference", "metric": metric, "value": val, "unit": "tokens/s", "n_gpus": args.gpus,
+                          "steps": steps, "warmup": warm, "ms_per_step": sec * 1e3, "higher_is_better": True,
+                          "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+                          "config": cfg_desc, "cpu_baseline": info,
+                          "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+        return
+
+    import torch
+    from paper_2010_04116_b200 import Model
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback for the product path")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    use_adamw = bool(w.adamw and not args.no_adamw)
+    hp = dict(lr=1e-4, beta1=0.9, beta2=0.98, eps=1e-9, weight_decay=0.01) if use_adamw else None
+    m = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, n, w.B, w.T, device=local_rank)
+    # parameters drawn on the host by the seeded generator, copied once
+    params = wl.draw_params(w)
+    m.set_params(params)
+    nb = 4
+    batches = [wl.draw_tokens(w, step=s) for s in range(nb)]
+    dev = torch.device("cuda", local_rank)
+    dev_batches = [(torch.tensor(a, device=dev), torch.tensor(b, device=dev)) for a, b in batches]
+    pin_batches = [(torch.tensor(a).pin_memory(), torch.tensor(b).pin_memory()) for a, b in batches]
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    s0 = m.streams[0]
+
+    def run_steps(count, e2e):
+        for i in range(count):
+            tok, tgt = (pin_batches if e2e else dev_batches)[i % nb]
+            m.train_step(tok, tgt, adamw=hp)
+            if e2e:
+                m.get_losses()          # device -> host read of the step's result (waits for the heads)
+
+    def timed(count, e2e):
+        barrier()
+        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        start.record(s0)
+        run_steps(count, e2e)
+        for s in m.streams[1:]:
+            s0.wait_stream(s)
+        end.record(s0)
+        barrier()
+        m.sync()
+        ms = start.elapsed_time(end)
+        if dist is not None:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    run_steps(args.warmup, False)
+    m.sync()
+    l0 = m.stats()[1]
+    m.profile(True)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    ms = timed(args.steps, False)
+    clocks = sampler.stop()
+    gemm_ms, gemm_launches, gemm_flops = m.profile_read()
+    m.profile(False)
+    launches = m.stats()[1] - l0
+    losses = m.get_losses() if not use_adamw else None
+    # end to end: pinned host tokens copied in, losses read back, every step
+    run_steps(1, True)
+    ms_e2e = timed(args.steps, True)
+
+    tokens = w.ntok * args.steps * max(world, 1)
+    value = tokens / (ms * 1e-3)
+    e2e = tokens / (ms_e2e * 1e-3)
+    flops_tok = model_flops_per_token(w, n)
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except Exception:
+        pass
+    peak_sus = float(peaks.get("bf16_tflops_sustained", 1400.0))
+    peak_burst = float(peaks.get("bf16_tflops", 1590.0))
+    peak_src = "measured (MEASURED_PEAKS.json, sustained bf16 matmul)" if peaks else "fallback (1.4 PFLOP/s sustained)"
+    achieved = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
+    per_gpu_tf = value / max(world, 1) * flops_tok / 1e12
+    out = {
+        "metric": metric, "value": value, "unit": "tokens/s", "n_gpus": max(world, 1), "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": cfg_desc, "clocks": clocks,
+        "e2e": {"value": e2e, "unit": "tokens/s", "h2d_bytes_per_step": int(2 * w.ntok * 4),
+                "d2h_bytes_per_step": int(4 * w.K), "ms_per_step": ms_e2e / args.steps},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "tensor", "kernel": "gemm_tcgen05_kernel (all layouts and epilogues)",
+                     "achieved": achieved, "peak": peak_sus, "unit": "TFLOP/s", "frac": achieved / peak_sus,
+                     "peak_source": peak_src, "launches": int(gemm_launches), "avg_launch_ms": gemm_ms / max(gemm_launches, 1),
+                     "traffic": None},
+        "model_flops": {"per_token_mflop": flops_tok / 1e6, "step_tflop": flops_tok * w.ntok / 1e12,
+                        "tflops_per_gpu": per_gpu_tf, "frac_of_burst_peak": per_gpu_tf / peak_burst,
+                        "frac_of_sustained_peak": per_gpu_tf / peak_sus, "burst_peak": peak_burst},
+    }
+    if losses is not None:
+        out["last_losses"] = [float(x) for x in losses]
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        _, _, info = oracle_sample(w, n, 1, 0, params=params)
+        out["cpu_baseline"] = info
+    elif rank == 0:
+        out["cpu_baseline"] = None
+    m.close()
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(out))
+
+
+if __name__ == "__main__":
+    main()

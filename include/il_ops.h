@@ -24,11 +24,12 @@ extern "C" {
  * Supported combinations (a_mn, b_mn): (0,0) forward, (0,1) dgrad, (1,1) wgrad.
  * Leading dimensions in elements, multiples of 8; pointers 16-byte aligned.
  * Epilogues (the `epilogue` field):
- *   0 C(bf16) = acc + bias                         1 C(bf16) = pre, C2(bf16) = gelu_tanh(pre), pre = acc + bias
- *   2 C(f32) = resid(f32) + acc + bias             3 C(bf16) = acc * gelu_tanh'(aux[row % aux_rows, col])
+ *   0 C(bf16) = acc + bias                         1 C(bf16) = gelu_tanh'(pre), C2(bf16) = gelu_tanh(pre), pre = acc + bias
+ *   2 C(f32) = resid(f32) + acc + bias             3 C(bf16) = acc * aux[row % aux_rows, col]  (aux_rows >= 32)
  *   4 C(f32) = acc (+ C when accumulate != 0)
- *   5 per-(row, 256-column tile) softmax partials: part_max, part_sum [M, part_ld] at tile index
- *     col0/256 + tile, and tgt_logit[row] = acc[row, targets[row] - col0] when that column is in range
+ *   5 per-(row, 128-column block) softmax partials: part_max, part_sum [M, part_ld] at block index
+ *     col0/128 + block (col0 % 128 == 0), and tgt_logit[row] = acc[row, targets[row] - col0] when that
+ *     column is in range
  *   6 C(bf16) = (exp(acc - lse[row]) - [col + col0 == targets[row]]) * scale
  * (0,1) supports epilogues 0, 3, 4; (1,1) supports 4; (0,0) supports all. */
 typedef struct {

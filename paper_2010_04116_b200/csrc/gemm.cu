@@ -1,18 +1,25 @@
 // tcgen05 GEMM for sm_100a: C[M,N] = A[M,K] * B[N,K]^T, bf16 operands, fp32 accumulation in TMEM.
 //
-// One persistent CTA per SM walks a static list of 128 x 256 output tiles.  Warp roles:
-//   warp 0    : TMA producer — one elected thread streams 128x64 (A) and 256x64 (B) bf16 slabs into a
-//               4-stage shared-memory ring (128-byte swizzle), signalling "full" mbarriers by byte count.
-//   warp 1    : MMA issuer — allocates 512 TMEM columns (two 128x256 fp32 accumulators), one thread
-//               issues tcgen05.mma (M128 N256 K16) four times per slab, commits to the slab's "empty"
-//               barrier and, per tile, to the accumulator's "full" barrier.
-//   warps 2-5 : epilogue — tcgen05.ld the accumulator (32 lanes x 32 columns per load), apply the fused
-//               epilogue and store to global memory, then release the accumulator.  The second
+// Persistent kernel of CTA pairs (clusters of two, cta_group::2): a pair owns a 256 x 256 output tile and
+// walks a static tile list.  Each CTA stages its own 128 rows of A and its own 128 of the 256 rows of B
+// (32 KB per 64-wide k-slab instead of the 48 KB a lone CTA needs for 128 x 256), the leader issues one
+// tcgen05.mma.cta_group::2 (M256 N256 K16) that reads both CTAs' shared memory and accumulates rows 0-127
+// in its own TMEM and rows 128-255 in the peer's.  Warp roles in each CTA:
+//   warp 0    : TMA producer — one thread streams the slabs into a 5-stage ring (128-byte swizzle); the byte
+//               counts of both CTAs are credited to the leader's "full" mbarrier.
+//   warp 1    : allocates 512 TMEM columns (two 128 x 256 fp32 accumulators per CTA); in the leader one thread
+//               issues the MMAs and commits (multicast to both CTAs) to the slab's "empty" barriers and,
+//               per tile, to the accumulator's "full" barriers.
+//   warps 2-9 : epilogue — tcgen05.ld this CTA's half of the accumulator (32 lanes x 32 columns per load, two
+//               warps per TMEM lane quarter, one per 128-column half), row-wise math in that layout, then a
+//               transpose through shared memory so that every global load and store of the fused epilogue is
+//               coalesced; finally the accumulator is released on the leader's barrier.  The second
 //               accumulator lets the next tile's main loop overlap this epilogue.
 // Operands may be K-major or MN-major in global memory (forward: K/K, dgrad: K/MN, wgrad: MN/MN); the
 // major-ness goes into the TMA box shape, the shared-memory descriptor and the instruction descriptor.
 // Ragged M/N/K edges rely on TMA zero fill for loads and on bounds checks in the epilogue.
-// Every wait is bounded; on expiry the CTA sets the error word, drains and returns.
+// No TMA load uses cluster multicast.  Every wait is bounded; on expiry the CTA sets the error word, and
+// both CTAs meet at a cluster barrier before they return.
 #include <cstdio>
 #include <mutex>
 
@@ -21,16 +28,21 @@
 
 namespace il {
 
-constexpr int BM = 128;
-constexpr int BN = 256;
+constexpr int BM = 128;                          // rows of A (and of the accumulator) held by one CTA
+constexpr int TILE_M = 2 * BM;                   // rows of the output tile of a CTA pair
+constexpr int BN = 256;                          // columns of the output tile; each CTA stages half of B
 constexpr int BK = 64;
-constexpr int STAGES = 4;
+constexpr int STAGES = 5;
 constexpr int A_BYTES = BM * BK * 2;             // 16 KB
-constexpr int B_BYTES = BN * BK * 2;             // 32 KB
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;   // 48 KB
+constexpr int B_BYTES = (BN / 2) * BK * 2;       // 16 KB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;   // 32 KB per CTA and stage
 constexpr int TMEM_COLS = 2 * BN;                // 512 columns: two accumulators
-constexpr int GEMM_THREADS = 192;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int EPI_WARPS = 8;
+constexpr int GEMM_THREADS = 64 + 32 * EPI_WARPS;   // producer warp, MMA warp, epilogue warps
+constexpr int BAR_BYTES = 256;
+constexpr int STG_LD = 36;                       // floats per row of an epilogue warp's 32 x 32 staging tile
+constexpr int STG_BYTES = EPI_WARPS * 32 * STG_LD * 4;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + BAR_BYTES + STG_BYTES;
 
 struct GemmDev {
   int M, N, K;
@@ -54,108 +66,29 @@ struct GemmDev {
   unsigned* err;
 };
 
+// Tile order: groups of TILE_GROUP_M row blocks are swept across all column blocks before the next group
+// starts, so that the pairs running at the same time share a small set of A rows and the whole of B in L2.
+constexpr int TILE_GROUP_M = 8;
+__device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int& m_blk, int& n_blk) {
+  const int per_group = TILE_GROUP_M * tiles_n;
+  const int g = t / per_group;
+  const int within = t - g * per_group;
+  const int gm = min(TILE_GROUP_M, tiles_m - g * TILE_GROUP_M);
+  m_blk = g * TILE_GROUP_M + within % gm;
+  n_blk = within / gm;
+}
+
 struct RowState {   // per-thread state carried across the 32-column chunks of one tile row (EPI_LSE)
   float m, s, tl;
   int tgt;
 };
 
+// Row-wise part of the epilogue, in the accumulator's own layout (thread = one row, v = 32 consecutive
+// columns starting at `col`): the softmax statistics (EPI_LSE, nothing stored) and dZ (EPI_DZ, in place).
 template <int EPI>
-__device__ __forceinline__ void epilogue_chunk(const GemmDev& p, int row, int col, const uint32_t (&r)[32],
-                                               RowState& st) {
+__device__ __forceinline__ void epilogue_rowwise(const GemmDev& p, int col, float (&v)[32], RowState& st) {
   const bool full = (col + 32 <= p.N);
-  float v[32];
-#pragma unroll
-  for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
-
-  if constexpr (EPI == EPI_BF16 || EPI == EPI_BF16_GELU || EPI == EPI_F32_RESID) {
-    if (p.bias) {
-      if (full) {
-#pragma unroll
-        for (int j = 0; j < 32; j += 4) {
-          float4 b = __ldg(reinterpret_cast<const float4*>(p.bias + col + j));
-          v[j] += b.x; v[j + 1] += b.y; v[j + 2] += b.z; v[j + 3] += b.w;
-        }
-      } else {
-#pragma unroll
-        for (int j = 0; j < 32; ++j)
-          if (col + j < p.N) v[j] += __ldg(p.bias + col + j);
-      }
-    }
-  }
-
-  if constexpr (EPI == EPI_BF16 || EPI == EPI_BF16_GELU) {
-    bf16* c = reinterpret_cast<bf16*>(p.C) + (size_t)row * p.ldc + col;
-    bf16* c2 = (EPI == EPI_BF16_GELU) ? reinterpret_cast<bf16*>(p.C2) + (size_t)row * p.ldc + col : nullptr;
-    if (full) {
-#pragma unroll
-      for (int j = 0; j < 32; j += 8) {
-        uint4 o;
-        o.x = pack_bf16x2(v[j], v[j + 1]); o.y = pack_bf16x2(v[j + 2], v[j + 3]);
-        o.z = pack_bf16x2(v[j + 4], v[j + 5]); o.w = pack_bf16x2(v[j + 6], v[j + 7]);
-        *reinterpret_cast<uint4*>(c + j) = o;
-        if constexpr (EPI == EPI_BF16_GELU) {
-          uint4 g;
-          g.x = pack_bf16x2(gelu_tanh(v[j]), gelu_tanh(v[j + 1]));
-          g.y = pack_bf16x2(gelu_tanh(v[j + 2]), gelu_tanh(v[j + 3]));
-          g.z = pack_bf16x2(gelu_tanh(v[j + 4]), gelu_tanh(v[j + 5]));
-          g.w = pack_bf16x2(gelu_tanh(v[j + 6]), gelu_tanh(v[j + 7]));
-          *reinterpret_cast<uint4*>(c2 + j) = g;
-        }
-      }
-    } else {
-#pragma unroll
-      for (int j = 0; j < 32; ++j)
-        if (col + j < p.N) {
-          c[j] = __float2bfloat16(v[j]);
-          if constexpr (EPI == EPI_BF16_GELU) c2[j] = __float2bfloat16(gelu_tanh(v[j]));
-        }
-    }
-  } else if constexpr (EPI == EPI_F32_RESID || EPI == EPI_F32) {
-    float* c = reinterpret_cast<float*>(p.C) + (size_t)row * p.ldc + col;
-    const float* add = nullptr;
-    if constexpr (EPI == EPI_F32_RESID) add = p.resid + (size_t)row * p.ldc + col;
-    else if (p.accumulate) add = c;
-    if (full) {
-#pragma unroll
-      for (int j = 0; j < 32; j += 4) {
-        float4 o = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-        if (add) {
-          float4 a = *reinterpret_cast<const float4*>(add + j);
-          o.x += a.x; o.y += a.y; o.z += a.z; o.w += a.w;
-        }
-        *reinterpret_cast<float4*>(c + j) = o;
-      }
-    } else {
-#pragma unroll
-      for (int j = 0; j < 32; ++j)
-        if (col + j < p.N) c[j] = v[j] + (add ? add[j] : 0.0f);
-    }
-  } else if constexpr (EPI == EPI_BF16_DGELU) {
-    bf16* c = reinterpret_cast<bf16*>(p.C) + (size_t)row * p.ldc + col;
-    const bf16* h = p.aux + (size_t)(row % p.aux_rows) * p.ld_aux + col;
-    if (full) {
-#pragma unroll
-      for (int j = 0; j < 32; j += 8) {
-        uint4 hv = *reinterpret_cast<const uint4*>(h + j);
-        const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&hv);
-        float g[8];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          float2 f = __bfloat1622float2(h2[q]);
-          g[2 * q] = v[j + 2 * q] * gelu_tanh_grad(f.x);
-          g[2 * q + 1] = v[j + 2 * q + 1] * gelu_tanh_grad(f.y);
-        }
-        uint4 o;
-        o.x = pack_bf16x2(g[0], g[1]); o.y = pack_bf16x2(g[2], g[3]);
-        o.z = pack_bf16x2(g[4], g[5]); o.w = pack_bf16x2(g[6], g[7]);
-        *reinterpret_cast<uint4*>(c + j) = o;
-      }
-    } else {
-#pragma unroll
-      for (int j = 0; j < 32; ++j)
-        if (col + j < p.N) c[j] = __float2bfloat16(v[j] * gelu_tanh_grad(__bfloat162float(h[j])));
-    }
-  } else if constexpr (EPI == EPI_LSE) {
+  if constexpr (EPI == EPI_LSE) {
     float cm = -INFINITY;
 #pragma unroll
     for (int j = 0; j < 32; ++j)
@@ -176,30 +109,116 @@ __device__ __forceinline__ void epilogue_chunk(const GemmDev& p, int row, int co
         if (j == tj) st.tl = v[j];
     }
   } else if constexpr (EPI == EPI_DZ) {
-    bf16* c = reinterpret_cast<bf16*>(p.C) + (size_t)row * p.ldc + col;
     const float l = st.m;   // lse of this row
     const int tj = st.tgt - (p.col0 + col);
-    float g[32];
 #pragma unroll
-    for (int j = 0; j < 32; ++j) g[j] = (__expf(v[j] - l) - (j == tj ? 1.0f : 0.0f)) * p.scale;
-    if (full) {
+    for (int j = 0; j < 32; ++j) v[j] = (__expf(v[j] - l) - (j == tj ? 1.0f : 0.0f)) * p.scale;
+  }
+}
+
+// Element-wise part of the epilogue, after the 32 x 32 chunk has been transposed through shared memory: a
+// lane now holds 4 consecutive columns (gcol..gcol+3) of row grow, 8 lanes cover 128 contiguous bytes of
+// fp32 output (64 of bf16), so every global access is coalesced.  The loads of the second operand
+// (residual, saved pre-activation, or C itself when accumulating) are split from the stores so that all of
+// a chunk's loads are in flight before the first store (C may alias the residual).
+template <int EPI>
+__device__ __forceinline__ float4 epilogue_load4(const GemmDev& p, int grow, int arow, int gcol) {
+  float4 e = make_float4(0.f, 0.f, 0.f, 0.f);
+  const bool vec = (gcol + 4 <= p.N);
+  if constexpr (EPI == EPI_F32_RESID || EPI == EPI_F32) {
+    const float* add = nullptr;
+    if constexpr (EPI == EPI_F32_RESID) add = p.resid + (size_t)grow * p.ldc + gcol;
+    else if (p.accumulate) add = reinterpret_cast<const float*>(p.C) + (size_t)grow * p.ldc + gcol;
+    if (add) {
+      if (vec) {
+        e = *reinterpret_cast<const float4*>(add);
+      } else {
+        e.x = add[0];
+        if (gcol + 1 < p.N) e.y = add[1];
+        if (gcol + 2 < p.N) e.z = add[2];
+      }
+    }
+  } else if constexpr (EPI == EPI_BF16_DGELU) {
+    const bf16* h = p.aux + (size_t)arow * p.ld_aux + gcol;   // arow = grow % aux_rows
+    if (vec) {
+      const uint2 hv = *reinterpret_cast<const uint2*>(h);
+      const float2 h0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&hv.x));
+      const float2 h1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&hv.y));
+      e = make_float4(h0.x, h0.y, h1.x, h1.y);
+    } else {
+      e.x = __bfloat162float(h[0]);
+      if (gcol + 1 < p.N) e.y = __bfloat162float(h[1]);
+      if (gcol + 2 < p.N) e.z = __bfloat162float(h[2]);
+    }
+  }
+  return e;
+}
+
+template <int EPI>
+__device__ __forceinline__ void epilogue_store4(const GemmDev& p, int grow, int gcol, float4 a, float4 e) {
+  const bool vec = (gcol + 4 <= p.N);
+  float v[4] = {a.x, a.y, a.z, a.w};
+  if constexpr (EPI == EPI_BF16 || EPI == EPI_BF16_GELU || EPI == EPI_F32_RESID) {
+    if (p.bias) {
+      if (vec) {
+        const float4 b = __ldg(reinterpret_cast<const float4*>(p.bias + gcol));
+        v[0] += b.x; v[1] += b.y; v[2] += b.z; v[3] += b.w;
+      } else {
 #pragma unroll
-      for (int j = 0; j < 32; j += 8) {
-        uint4 o;
-        o.x = pack_bf16x2(g[j], g[j + 1]); o.y = pack_bf16x2(g[j + 2], g[j + 3]);
-        o.z = pack_bf16x2(g[j + 4], g[j + 5]); o.w = pack_bf16x2(g[j + 6], g[j + 7]);
-        *reinterpret_cast<uint4*>(c + j) = o;
+        for (int j = 0; j < 4; ++j)
+          if (gcol + j < p.N) v[j] += __ldg(p.bias + gcol + j);
+      }
+    }
+  }
+  if constexpr (EPI == EPI_BF16 || EPI == EPI_BF16_GELU || EPI == EPI_DZ || EPI == EPI_BF16_DGELU) {
+    bf16* c = reinterpret_cast<bf16*>(p.C) + (size_t)grow * p.ldc + gcol;
+    if constexpr (EPI == EPI_BF16_DGELU) {
+      v[0] *= e.x; v[1] *= e.y; v[2] *= e.z; v[3] *= e.w;
+    }
+    float y[4] = {0.f, 0.f, 0.f, 0.f};
+    if constexpr (EPI == EPI_BF16_GELU) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        float d;
+        gelu_tanh_both(v[j], y[j], d);
+        v[j] = d;                                   // C receives gelu'(pre), C2 gelu(pre)
+      }
+    }
+    if (vec) {
+      uint2 o;
+      o.x = pack_bf16x2(v[0], v[1]);
+      o.y = pack_bf16x2(v[2], v[3]);
+      *reinterpret_cast<uint2*>(c) = o;
+      if constexpr (EPI == EPI_BF16_GELU) {
+        uint2 g;
+        g.x = pack_bf16x2(y[0], y[1]);
+        g.y = pack_bf16x2(y[2], y[3]);
+        *reinterpret_cast<uint2*>(reinterpret_cast<bf16*>(p.C2) + (size_t)grow * p.ldc + gcol) = g;
       }
     } else {
 #pragma unroll
-      for (int j = 0; j < 32; ++j)
-        if (col + j < p.N) c[j] = __float2bfloat16(g[j]);
+      for (int j = 0; j < 4; ++j)
+        if (gcol + j < p.N) {
+          c[j] = __float2bfloat16(v[j]);
+          if constexpr (EPI == EPI_BF16_GELU)
+            (reinterpret_cast<bf16*>(p.C2) + (size_t)grow * p.ldc + gcol)[j] = __float2bfloat16(y[j]);
+        }
+    }
+  } else if constexpr (EPI == EPI_F32_RESID || EPI == EPI_F32) {
+    float* c = reinterpret_cast<float*>(p.C) + (size_t)grow * p.ldc + gcol;
+    v[0] += e.x; v[1] += e.y; v[2] += e.z; v[3] += e.w;
+    if (vec) {
+      *reinterpret_cast<float4*>(c) = make_float4(v[0], v[1], v[2], v[3]);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (gcol + j < p.N) c[j] = v[j];
     }
   }
 }
 
 template <bool A_MN, bool B_MN, int EPI>
-__global__ void __launch_bounds__(GEMM_THREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const GemmDev p) {
   extern __shared__ uint8_t smem_raw[];
@@ -208,7 +227,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t bar_base = smem_base + STAGES * STAGE_BYTES;
-  // barriers: full[STAGES], empty[STAGES], acc_full[2], acc_empty[2], drain
+  // barriers: full[STAGES] (leader's are used), empty[STAGES], acc_full[2], acc_empty[2] (leader's), drain
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
   auto acc_full_bar = [&](int s) { return bar_base + 8u * (2 * STAGES + s); };
@@ -217,6 +236,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();           // 0 = leader of the pair (issues the MMAs)
+  const int pair = blockIdx.x >> 1;
+  const int num_pairs = gridDim.x >> 1;
   const int num_tiles = p.tiles_m * p.tiles_n;
   const int num_kb = (p.K + BK - 1) / BK;
 
@@ -228,7 +250,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(acc_full_bar(s), 1);
-      mbar_init(acc_empty_bar(s), 4);
+      mbar_init(acc_empty_bar(s), 2 * EPI_WARPS);      // the epilogue warps of both CTAs of the pair
     }
     mbar_init(drain_bar, 1);
     fence_mbar_init();
@@ -236,69 +258,64 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     tma_prefetch_desc(&tmB);
   }
   if (warp == 1) {
-    tmem_alloc(smem_u32(&tmem_base_smem), TMEM_COLS);
-    tmem_relinquish();
+    tmem_alloc_pair(smem_u32(&tmem_base_smem), TMEM_COLS);
+    tmem_relinquish_pair();
   }
   tc_fence_before();
   __syncthreads();
+  cluster_sync_all();       // the peer's barriers are initialised before anything is signalled remotely
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_smem;
   volatile int* abortp = &abort_flag;
 
   if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------------ TMA producer (both CTAs)
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
-      int issued = 0;
       bool ok = true;
-      for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
-        const int m0 = (t % p.tiles_m) * BM;
-        const int n0 = (t / p.tiles_m) * BN;
+      for (int t = pair; t < num_tiles && ok; t += num_pairs) {
+        int m_blk, n_blk;
+        tile_coords(t, p.tiles_m, p.tiles_n, m_blk, n_blk);
+        const int m0 = m_blk * TILE_M + (int)rank * BM;       // this CTA's 128 rows of A
+        const int n0 = n_blk * BN + (int)rank * (BN / 2);     // this CTA's 128 rows of B
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abortp)) { ok = false; break; }
           const uint32_t sa = smem_base + stage * STAGE_BYTES;
           const uint32_t sb = sa + A_BYTES;
-          mbar_expect_tx(full_bar(stage), STAGE_BYTES);
+          // both CTAs' bytes are credited to the leader's barrier, which expects the pair's total
+          if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * STAGE_BYTES);
+          const uint32_t fb = mapa_cluster(full_bar(stage), 0);
           const int k0 = kb * BK;
           if constexpr (!A_MN) {
-            tma_load_2d(sa, &tmA, k0, m0, full_bar(stage));
+            tma_load_2d_pair(sa, &tmA, k0, m0, fb);
           } else {
 #pragma unroll
-            for (int i = 0; i < BM / 64; ++i) tma_load_2d(sa + i * 8192, &tmA, m0 + 64 * i, k0, full_bar(stage));
+            for (int i = 0; i < BM / 64; ++i) tma_load_2d_pair(sa + i * 8192, &tmA, m0 + 64 * i, k0, fb);
           }
           if constexpr (!B_MN) {
-            tma_load_2d(sb, &tmB, k0, n0, full_bar(stage));
+            tma_load_2d_pair(sb, &tmB, k0, n0, fb);
           } else {
 #pragma unroll
-            for (int i = 0; i < BN / 64; ++i) tma_load_2d(sb + i * 8192, &tmB, n0 + 64 * i, k0, full_bar(stage));
+            for (int i = 0; i < BN / 128; ++i) tma_load_2d_pair(sb + i * 8192, &tmB, n0 + 64 * i, k0, fb);
           }
-          ++issued;
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
       if (!ok) {
         atomicExch(p.err, DEV_TIMEOUT_PRODUCER);
         abort_flag = 1;
-        // let copies already in flight land before the CTA (and its shared memory) goes away
-        int s = stage;
-        uint32_t ph = phase;
-        for (int i = 0; i < STAGES && i < issued; ++i) {
-          if (--s < 0) { s = STAGES - 1; ph ^= 1u; }
-          int never = 0;
-          mbar_wait(full_bar(s), ph, &never, 20000000ull);
-        }
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc_bf16(BM, BN, A_MN ? 1 : 0, B_MN ? 1 : 0);
+    // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = make_idesc_bf16(TILE_M, BN, A_MN ? 1 : 0, B_MN ? 1 : 0);
       int stage = 0;
       uint32_t phase = 0;
       int it = 0;
       bool ok = true;
-      for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++it) {
+      for (int t = pair; t < num_tiles && ok; t += num_pairs, ++it) {
         const int as = it & 1;
         const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
         if (!mbar_wait(acc_empty_bar(as), aphase ^ 1u, abortp)) { ok = false; break; }
@@ -315,35 +332,76 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             // MN-major: 16 k = two groups of 8 k-rows (1024 B each); 64-element MN chunks 8192 B apart.
             const uint64_t ad = A_MN ? make_smem_desc(sa + k * 2048, 8192, 1024) : make_smem_desc(sa + k * 32, 16, 1024);
             const uint64_t bd = B_MN ? make_smem_desc(sb + k * 2048, 8192, 1024) : make_smem_desc(sb + k * 32, 16, 1024);
-            umma_bf16(d_tmem, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
+            umma_bf16_pair(d_tmem, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
           }
-          umma_commit(empty_bar(stage));   // slab reusable once these MMAs have read it
+          umma_commit_pair(empty_bar(stage), 3);   // slab reusable in both CTAs once these MMAs have read it
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
-        if (ok) umma_commit(acc_full_bar(as));
+        if (ok) umma_commit_pair(acc_full_bar(as), 3);
       }
       if (!ok) {
         atomicExch(p.err, DEV_TIMEOUT_MMA);
         abort_flag = 1;
       }
       // all issued MMAs must have retired before TMEM is released
-      umma_commit(drain_bar);
+      umma_commit_pair(drain_bar, 1);
       int never = 0;
       mbar_wait(drain_bar, 0, &never);
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (warps 2..5)
-    const int q = warp & 3;                  // TMEM lane quarter this warp may access
+    // ------------------------------------------------------------------ epilogue (warps 2..9, both CTAs)
+    // Two warps share each TMEM lane quarter (a warp may only read lanes 32*(warp%4)..+31): the first
+    // takes columns 0-127 of the tile, the second columns 128-255.
+    const int q = warp & 3;
+    const int half = (warp - 2) >> 2;
+    float* stg = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)) + STAGES * STAGE_BYTES + BAR_BYTES) +
+                 (warp - 2) * (32 * STG_LD);
     int it = 0;
     bool ok = true;
-    for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++it) {
-      const int m_blk = t % p.tiles_m;
-      const int n_blk = t / p.tiles_m;
+    for (int t = pair; t < num_tiles && ok; t += num_pairs, ++it) {
+      int m_blk, n_blk;
+      tile_coords(t, p.tiles_m, p.tiles_n, m_blk, n_blk);
       const int as = it & 1;
       const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
+      const int row0 = m_blk * TILE_M + (int)rank * BM + q * 32;     // first row of this warp's 32
+      const int col_base = n_blk * BN + half * (BN / 2);
+      const int lrow = lane >> 3;                  // row within a group of 4 after the transpose
+      const int gcol_off = 4 * (lane & 7);
+      const int arow0 = (EPI == EPI_BF16_DGELU) ? row0 % p.aux_rows : 0;
+      // While the main loop of this tile is still running, fetch the epilogue's second operand in the
+      // coalesced (transposed) layout: the saved pre-activation for all four chunks (bf16, 64 registers), or
+      // the first chunk of the fp32 residual / accumulated C (the later chunks are fetched one chunk ahead).
+      uint2 pre_h[EPI == EPI_BF16_DGELU ? 4 : 1][8];
+      float4 pre_f[2][8];
+      auto load_f32_chunk = [&](int c, float4 (&dst)[8]) {
+        const int gcol = col_base + c * 32 + gcol_off;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int grow = row0 + 4 * i + lrow;
+          dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (grow < p.M && gcol < p.N) dst[i] = epilogue_load4<EPI>(p, grow, 0, gcol);
+        }
+      };
+      if constexpr (EPI == EPI_BF16_DGELU) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const int gcol = col_base + c * 32 + gcol_off;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int grow = row0 + 4 * i + lrow;
+            int arow = arow0 + 4 * i + lrow;          // grow % aux_rows without a division
+            if (arow >= p.aux_rows) arow -= p.aux_rows;
+            pre_h[c][i] = make_uint2(0u, 0u);
+            if (grow < p.M && gcol + 4 <= p.N)
+              pre_h[c][i] = *reinterpret_cast<const uint2*>(p.aux + (size_t)arow * p.ld_aux + gcol);
+          }
+        }
+      } else if constexpr (EPI == EPI_F32_RESID || EPI == EPI_F32) {
+        load_f32_chunk(0, pre_f[0]);
+      }
       if (!mbar_wait(acc_full_bar(as), aphase, abortp)) { ok = false; break; }
       tc_fence_after();
-      const int row = m_blk * BM + q * 32 + lane;
+      const int row = row0 + lane;
       const bool row_ok = row < p.M;
       RowState st;
       st.m = -INFINITY; st.s = 0.0f; st.tl = 0.0f; st.tgt = -1;
@@ -353,28 +411,117 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           if constexpr (EPI == EPI_DZ) st.m = __ldg(p.lse + row);
         }
       }
-      const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * BN);
-#pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        const int col = n_blk * BN + c * 32;
+      const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * BN + half * (BN / 2));
+#pragma unroll
+      for (int c = 0; c < BN / 64; ++c) {
+        const int col = col_base + c * 32;
         if (col >= p.N) break;               // uniform across the warp
         uint32_t r[32];
         tmem_ld_32x32(t_addr + (uint32_t)(c * 32), r);
+        const int gcol = col + gcol_off;
+        // fast path: the whole 32 x 32 chunk is inside the matrix (uniform across the warp), so nothing below
+        // is predicated and the 32 element chains of a lane are independent straight-line code
+        const bool interior = (row0 + 32 <= p.M) && (col + 32 <= p.N);
+        float4 extra[8];
+        if constexpr (EPI == EPI_BF16_DGELU) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const float2 h0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pre_h[c][i].x));
+            const float2 h1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pre_h[c][i].y));
+            extra[i] = make_float4(h0.x, h0.y, h1.x, h1.y);
+          }
+          if (!interior && gcol < p.N && gcol + 4 > p.N) {    // ragged last columns: element-wise reload
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const int grow = row0 + 4 * i + lrow;
+              int arow = arow0 + 4 * i + lrow;
+              if (arow >= p.aux_rows) arow -= p.aux_rows;
+              if (grow < p.M) extra[i] = epilogue_load4<EPI>(p, grow, arow, gcol);
+            }
+          }
+        } else if constexpr (EPI == EPI_F32_RESID || EPI == EPI_F32) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) extra[i] = pre_f[c & 1][i];
+          if (c + 1 < BN / 64 && col + 32 < p.N) load_f32_chunk(c + 1, pre_f[(c + 1) & 1]);
+        }
         tmem_ld_wait();
-        if (row_ok) epilogue_chunk<EPI>(p, row, col, r, st);
+        float v[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+        if constexpr (EPI == EPI_LSE || EPI == EPI_DZ) epilogue_rowwise<EPI>(p, col, v, st);
+        if constexpr (EPI != EPI_LSE) {
+          // transpose through shared memory: lane (= row) writes its 32 columns, then lane l reads 4
+          // columns of row 4i + l/8
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            *reinterpret_cast<float4*>(stg + lane * STG_LD + 4 * j) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+          __syncwarp();
+          float4 a[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) a[i] = *reinterpret_cast<const float4*>(stg + (4 * i + lrow) * STG_LD + gcol_off);
+          if (interior) {
+            float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f);
+            if constexpr (EPI == EPI_BF16 || EPI == EPI_BF16_GELU || EPI == EPI_F32_RESID)
+              if (p.bias) b4 = __ldg(reinterpret_cast<const float4*>(p.bias + gcol));
+            if constexpr (EPI == EPI_F32_RESID || EPI == EPI_F32) {
+              float* cbase = reinterpret_cast<float*>(p.C) + (size_t)(row0 + lrow) * p.ldc + gcol;
+#pragma unroll
+              for (int i = 0; i < 8; ++i)
+                *reinterpret_cast<float4*>(cbase + (size_t)(4 * i) * p.ldc) =
+                    make_float4(a[i].x + b4.x + extra[i].x, a[i].y + b4.y + extra[i].y, a[i].z + b4.z + extra[i].z,
+                                a[i].w + b4.w + extra[i].w);
+            } else {
+              uint2 o[8], g[8];
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                float x0 = a[i].x + b4.x, x1 = a[i].y + b4.y, x2 = a[i].z + b4.z, x3 = a[i].w + b4.w;
+                if constexpr (EPI == EPI_BF16_DGELU) {
+                  x0 *= extra[i].x; x1 *= extra[i].y; x2 *= extra[i].z; x3 *= extra[i].w;
+                }
+                if constexpr (EPI == EPI_BF16_GELU) {
+                  float y0, y1, y2, y3, d0, d1, d2, d3;
+                  gelu_tanh_both(x0, y0, d0); gelu_tanh_both(x1, y1, d1);
+                  gelu_tanh_both(x2, y2, d2); gelu_tanh_both(x3, y3, d3);
+                  o[i].x = pack_bf16x2(d0, d1);
+                  o[i].y = pack_bf16x2(d2, d3);
+                  g[i].x = pack_bf16x2(y0, y1);
+                  g[i].y = pack_bf16x2(y2, y3);
+                } else {
+                  o[i].x = pack_bf16x2(x0, x1);
+                  o[i].y = pack_bf16x2(x2, x3);
+                }
+              }
+              bf16* cbase = reinterpret_cast<bf16*>(p.C) + (size_t)(row0 + lrow) * p.ldc + gcol;
+#pragma unroll
+              for (int i = 0; i < 8; ++i) *reinterpret_cast<uint2*>(cbase + (size_t)(4 * i) * p.ldc) = o[i];
+              if constexpr (EPI == EPI_BF16_GELU) {
+                bf16* c2base = reinterpret_cast<bf16*>(p.C2) + (size_t)(row0 + lrow) * p.ldc + gcol;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) *reinterpret_cast<uint2*>(c2base + (size_t)(4 * i) * p.ldc) = g[i];
+              }
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const int rr = 4 * i + lrow;
+              if (row0 + rr < p.M && gcol < p.N) epilogue_store4<EPI>(p, row0 + rr, gcol, a[i], extra[i]);
+            }
+          }
+          __syncwarp();
+        }
       }
       if constexpr (EPI == EPI_LSE) {
-        if (row_ok) {
-          const size_t pi = (size_t)row * p.part_ld + (p.col0 / BN + n_blk);
+        if (row_ok && n_blk * BN + half * (BN / 2) < p.N) {
+          const size_t pi = (size_t)row * p.part_ld + (p.col0 / (BN / 2) + n_blk * 2 + half);
           p.part_max[pi] = st.m;
           p.part_sum[pi] = st.s;
-          const int tt = st.tgt - p.col0 - n_blk * BN;
-          if (tt >= 0 && tt < BN && tt + n_blk * BN < p.N) p.tgt_logit[row] = st.tl;
+          const int tt = st.tgt - p.col0 - n_blk * BN - half * (BN / 2);
+          if (tt >= 0 && tt < BN / 2 && st.tgt - p.col0 < p.N) p.tgt_logit[row] = st.tl;
         }
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(acc_empty_bar(as));
+      if (lane == 0) mbar_arrive_cluster(mapa_cluster(acc_empty_bar(as), 0));
     }
     if (!ok && lane == 0) {
       atomicExch(p.err, DEV_TIMEOUT_EPILOGUE);
@@ -382,11 +529,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     }
   }
 
+  // Neither CTA may leave while its peer can still read its shared memory or signal its barriers.
   tc_fence_before();
   __syncthreads();
+  cluster_sync_all();
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, TMEM_COLS);
+    tmem_dealloc_pair(tmem_base, TMEM_COLS);
   }
 }
 
@@ -488,20 +637,20 @@ cudaError_t gemm_launch(const GemmArgs& a, unsigned* err_word, int num_sms, cuda
   }
   if (a.epilogue == EPI_BF16_GELU && (!a.C2 || ((uintptr_t)a.C2 % 16))) return cudaErrorInvalidValue;
   if (a.epilogue == EPI_F32_RESID && (!a.resid || ((uintptr_t)a.resid % 16))) return cudaErrorInvalidValue;
-  if (a.epilogue == EPI_BF16_DGELU && (!a.aux || a.aux_rows <= 0 || (a.ld_aux % 8) || ((uintptr_t)a.aux % 16)))
+  if (a.epilogue == EPI_BF16_DGELU && (!a.aux || a.aux_rows < 32 || (a.ld_aux % 8) || ((uintptr_t)a.aux % 16)))
     return cudaErrorInvalidValue;
   if (a.bias && ((uintptr_t)a.bias % 16)) return cudaErrorInvalidValue;
-  if (a.epilogue == EPI_LSE && (!a.targets || !a.part_max || !a.part_sum || !a.tgt_logit || (a.col0 % BN)))
+  if (a.epilogue == EPI_LSE && (!a.targets || !a.part_max || !a.part_sum || !a.tgt_logit || (a.col0 % (BN / 2))))
     return cudaErrorInvalidValue;
   if (a.epilogue == EPI_DZ && (!a.targets || !a.lse)) return cudaErrorInvalidValue;
 
   CUtensorMap tmA, tmB;
   if (!encode_operand(&tmA, a.A, a.M, a.K, BM)) return cudaErrorInvalidValue;
-  if (!encode_operand(&tmB, a.B, a.N, a.K, BN)) return cudaErrorInvalidValue;
+  if (!encode_operand(&tmB, a.B, a.N, a.K, BN / 2)) return cudaErrorInvalidValue;
 
   GemmDev p;
   p.M = a.M; p.N = a.N; p.K = a.K;
-  p.tiles_m = (a.M + BM - 1) / BM;
+  p.tiles_m = (a.M + TILE_M - 1) / TILE_M;
   p.tiles_n = (a.N + BN - 1) / BN;
   p.C = a.C; p.ldc = a.ldc; p.C2 = a.C2; p.bias = a.bias; p.resid = a.resid;
   p.aux = reinterpret_cast<const bf16*>(a.aux); p.ld_aux = a.ld_aux; p.aux_rows = a.aux_rows > 0 ? a.aux_rows : 1;
@@ -510,7 +659,8 @@ cudaError_t gemm_launch(const GemmArgs& a, unsigned* err_word, int num_sms, cuda
   p.tgt_logit = a.tgt_logit; p.lse = a.lse; p.scale = a.scale; p.col0 = a.col0;
   p.err = err_word;
   const long long tiles = (long long)p.tiles_m * p.tiles_n;
-  const int grid = (int)(tiles < num_sms ? tiles : num_sms);
+  const int pairs = (int)(tiles < num_sms / 2 ? tiles : num_sms / 2);
+  const int grid = 2 * pairs;
   kern<<<grid, GEMM_THREADS, SMEM_BYTES, stream>>>(tmA, tmB, p);
   return cudaGetLastError();
 }

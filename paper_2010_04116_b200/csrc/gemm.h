@@ -8,9 +8,9 @@ namespace il {
 
 enum GemmEpilogue : int {
   EPI_BF16 = 0,        // C(bf16) = acc + bias
-  EPI_BF16_GELU = 1,   // C(bf16) = pre = acc + bias ; C2(bf16) = gelu(pre)
+  EPI_BF16_GELU = 1,   // pre = acc + bias ; C(bf16) = gelu'(pre) ; C2(bf16) = gelu(pre)
   EPI_F32_RESID = 2,   // C(f32)  = resid(f32) + acc + bias        (C may alias resid)
-  EPI_BF16_DGELU = 3,  // C(bf16) = acc * gelu'(aux[row % aux_rows, col])
+  EPI_BF16_DGELU = 3,  // C(bf16) = acc * aux[row % aux_rows, col]   (aux = saved gelu'(pre))
   EPI_F32 = 4,         // C(f32)  = acc (+ C if accumulate)
   EPI_LSE = 5,         // online-softmax partials per (row, column tile) + logit of the target column
   EPI_DZ = 6,          // C(bf16) = (exp(acc - lse[row]) - [col + col0 == target[row]]) * scale
@@ -31,7 +31,7 @@ struct GemmArgs {
   int epilogue;
   void* C;            // [M, ldc]
   int ldc;
-  void* C2;           // EPI_BF16_GELU: activated output, same ld as C
+  void* C2;           // EPI_BF16_GELU: activated output gelu(pre), same ld as C (C gets gelu'(pre))
   const float* bias;  // [N] or NULL
   const float* resid; // EPI_F32_RESID: [M, ldc] fp32
   const void* aux;    // EPI_BF16_DGELU: bf16 [aux_rows, ld_aux]
@@ -39,7 +39,7 @@ struct GemmArgs {
   int accumulate;     // EPI_F32
   // EPI_LSE / EPI_DZ (vocabulary chunk starting at column col0 of the full vocabulary)
   const int* targets; // [M]
-  float* part_max;    // [M, part_ld]  written at column (col0 / 256 + column tile)
+  float* part_max;    // [M, part_ld]  written at column (col0 / 128 + 128-column block)
   float* part_sum;    // [M, part_ld]
   int part_ld;
   float* tgt_logit;   // [M]

@@ -43,7 +43,7 @@ struct LayerOff { size_t ln1g, ln1b, wqkv, bqkv, wo, bo, ln2g, ln2b, w1, b1, w2,
 struct HeadOff { size_t lng, lnb, w; };
 
 struct LayerActs {
-  bf16 *ln1, *qkv, *attn_o, *ln2, *hpre, *hact;
+  bf16 *ln1, *qkv, *attn_o, *ln2, *hgrad, *hact;   // hgrad = gelu'(FC1 pre-activation)
   float *mean1, *rstd1, *lse, *x_mid, *mean2, *rstd2, *x_out;
 };
 
@@ -418,7 +418,7 @@ extern "C" il_status il_create(int K, int Lc, int d, int H, int F, int V, int n,
       IL_TRY(dev_alloc_t(m, &A.qkv, N * 3 * d));
       IL_TRY(dev_alloc_t(m, &A.attn_o, N * d));
       IL_TRY(dev_alloc_t(m, &A.ln2, N * d));
-      IL_TRY(dev_alloc_t(m, &A.hpre, N * F));
+      IL_TRY(dev_alloc_t(m, &A.hgrad, N * F));
       IL_TRY(dev_alloc_t(m, &A.hact, N * F));
       IL_TRY(dev_alloc_t(m, &A.mean1, N));
       IL_TRY(dev_alloc_t(m, &A.rstd1, N));
@@ -429,7 +429,7 @@ extern "C" il_status il_create(int K, int Lc, int d, int H, int F, int V, int n,
       IL_TRY(dev_alloc_t(m, &A.x_out, N * d));
       if (l == Lc - 1) m->a[k + 1] = A.x_out;
     }
-  m->part_ld = (V + 255) / 256;
+  m->part_ld = (V + 127) / 128;
   m->hs.assign(K, HeadScratch{});
   for (int k = 0; k < K; ++k) {
     HeadScratch& h = m->hs[k];
@@ -620,7 +620,7 @@ extern "C" il_status il_forward_component(il_model* m, int k) {
     }
     IL_K(m, layernorm_fwd(A.x_mid, m->P + o.ln2g, m->P + o.ln2b, A.ln2, A.mean2, A.rstd2, N, d, m->ln_eps, st));
     {
-      GemmArgs g = gemm_args(N, F, d, A.ln2, d, 0, m->Pb + o.w1, d, 0, EPI_BF16_GELU, A.hpre, F);
+      GemmArgs g = gemm_args(N, F, d, A.ln2, d, 0, m->Pb + o.w1, d, 0, EPI_BF16_GELU, A.hgrad, F);
       g.C2 = A.hact;
       g.bias = m->P + o.b1;
       IL_TRY(gemm(m, k, g));
@@ -740,7 +740,7 @@ il_status component_backward(il_model* m, int k, int s) {
     IL_TRY(gemm(m, k, gemm_args(d, F, N, c.dxb, d, 1, A.hact, F, 1, EPI_F32, m->G + o.w2, F)));
     {
       GemmArgs g = gemm_args(R, F, d, c.dxb, d, 0, m->Pb + o.w2, F, 1, EPI_BF16_DGELU, c.dbig, F);
-      g.aux = A.hpre; g.ld_aux = F; g.aux_rows = N;
+      g.aux = A.hgrad; g.ld_aux = F; g.aux_rows = N;
       IL_TRY(gemm(m, k, g));
     }
     IL_K(m, colsum_bf16(c.dbig, F, m->G + o.b1, N, F, st));

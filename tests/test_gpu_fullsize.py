@@ -1,0 +1,142 @@
+"""Full-size parity (GPU): the CUDA step at the configurations' full sizes, launched as bench.py launches it,
+against values the fp64 oracle produced at the same sizes (tests/golden/*.json, written by
+tests/golden/make_golden.py which calls only the oracle).  Per head: loss within 1e-3 relative.  Per
+tensor: gradient norm within 2e-2, seeded sample entries and +-1 sketches within the error a 2e-2
+relative-L2 deviation allows.  Plus properties that hold at any size."""
+import json
+import os
+
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+
+import workloads as wl
+from paper_2010_04116_b200 import Model
+
+pytestmark = pytest.mark.gpu
+GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+TOL = 2e-2
+
+
+def _golden(cfg, n):
+    path = os.path.join(GOLDEN, f"{cfg}_n{n}.json")
+    if not os.path.exists(path):
+        pytest.skip(f"{os.path.basename(path)} not generated")
+    return json.load(open(path))
+
+
+_models = {}
+
+
+def _model(cfg):
+    """One model per configuration, reused across n (parameters are copied once)."""
+    if cfg not in _models:
+        for m in _models.values():
+            m.close()
+        _models.clear()
+        torch.cuda.empty_cache()
+        w = wl.CONFIGS[cfg]
+        m = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, 1, w.B, w.T)
+        for i, (name, _, _, shape) in enumerate(wl.tensor_specs(w)):
+            m.set_param(name, wl.draw_tensor(name, i, shape))
+        _models[cfg] = m
+    return _models[cfg]
+
+
+def _check_against_golden(cfg, n):
+    gold = _golden(cfg, n)
+    w = wl.CONFIGS[cfg]
+    m = _model(cfg)
+    m.set_n(n)
+    tok, tgt = wl.draw_tokens(w)
+    m.train_step(torch.tensor(tok, device="cuda:0"), torch.tensor(tgt, device="cuda:0"))
+    losses = m.get_losses()
+    m.sync()
+    ref = np.array(gold["losses"])
+    assert np.all(np.abs(losses - ref) <= 1e-3 * np.abs(ref)), (losses, ref)
+    # the per-token losses average to the head loss (holds at any size)
+    tl = m.get_token_losses(w.K - 1, w.ntok)
+    assert abs(float(tl.astype(np.float64).mean()) - losses[-1]) < 1e-4 * losses[-1]
+    assert np.all(tl > 0)
+    bad = []
+    for i, (name, _, _, _) in enumerate(wl.tensor_specs(w)):
+        g = m.get_grad(name).astype(np.float64).reshape(-1)
+        t = gold["tensors"][name]
+        norm = t["norm"]
+        if norm == 0.0:
+            assert not g.any(), name
+            continue
+        rms = norm / np.sqrt(g.size)
+        if abs(np.linalg.norm(g) - norm) > TOL * norm:
+            bad.append((name, "norm", float(np.linalg.norm(g)), norm))
+        idx = wl.sample_indices(name, i, g.size, len(t["samples"]))
+        for j, r in zip(idx, t["samples"]):
+            if abs(g[j] - r) > TOL * abs(r) + 4 * TOL * rms:
+                bad.append((name, f"sample {j}", float(g[j]), r))
+        for q, r in enumerate(t["sketch"]):
+            s = float(np.dot(g, wl.rademacher(i, g.size, q).astype(np.float64)))
+            if abs(s - r) > 4 * TOL * norm:
+                bad.append((name, f"sketch {q}", s, r))
+    assert not bad, bad[:10]
+
+
+@pytest.mark.parametrize("n", [2, 1, 3, 4])
+def test_gpt2_small_shape_full_size(n):
+    """GPT-2-small-shaped model, batch 8 x 1024, n = 2 and the n sweep 1..4."""
+    _check_against_golden("cfg2", n)
+
+
+@pytest.mark.parametrize("n", [2, 3])
+def test_gpt2_medium_shape_full_size(n):
+    _check_against_golden("cfg4", n)
+
+
+def test_sweep_invariants_on_device_full_size():
+    """Head gradients do not depend on n; the top component's gradient does not depend on n; with n = 1
+    component k's gradient is that of its own head only, so n = 2 differs from it for every k < K-1."""
+    w = wl.CONFIGS["cfg2"]
+    m = _model("cfg2")
+    tok, tgt = wl.draw_tokens(w)
+    dt, dg = torch.tensor(tok, device="cuda:0"), torch.tensor(tgt, device="cuda:0")
+    probes = ["head0.w", "head3.ln.g", f"c{w.K - 1}.l0.mlp.w1", "c0.l1.attn.wqkv", "c1.l0.mlp.w2"]
+    res = {}
+    for n in (1, 2, 4):
+        m.set_n(n)
+        m.train_step(dt, dg)
+        m.sync()
+        res[n] = {p: m.get_grad(p) for p in probes}
+    for p in probes[:3]:
+        for n in (2, 4):
+            den = np.linalg.norm(res[1][p])
+            assert np.linalg.norm(res[n][p] - res[1][p]) / den < 1e-5, (p, n)
+    for p in probes[3:]:
+        assert np.linalg.norm(res[2][p] - res[1][p]) / np.linalg.norm(res[1][p]) > 1e-2, p
+    for m_ in _models.values():
+        m_.close()
+    _models.clear()
+
+
+def test_cfg5_width_reduced_depth_matches_oracle():
+    """2.7B-shaped widths (d 2560, 32 heads of 80, d_ff 10240, seq 2048, vocab 50257) on one sequence and
+    two one-layer components, against the oracle run in the test."""
+    from oracle import il_oracle as orc
+    w = wl.CONFIGS["cfg5"].with_(B=1, K=2, Lc=1)
+    P = wl.draw_params(w)
+    tok, tgt = wl.draw_tokens(w)
+    m = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, 2, w.B, w.T)
+    try:
+        m.set_params(P)
+        m.train_step(tok, tgt)
+        losses = m.get_losses()
+        m.sync()
+        ol, OG = orc.nwise_gradients(P, tok, tgt, w.K, w.Lc, w.H, 2)
+        assert np.all(np.abs(losses - np.array(ol)) <= 1e-3 * np.abs(np.array(ol))), (losses, ol)
+        for name in m.names:
+            g = m.get_grad(name).astype(np.float64)
+            den = np.linalg.norm(OG[name])
+            if den == 0:
+                continue
+            assert np.linalg.norm(g - OG[name]) / den < TOL, name
+    finally:
+        m.close()

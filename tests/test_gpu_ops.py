@@ -79,7 +79,7 @@ def test_gemm_epilogues_forward():
     # 0: bf16 out + bias
     C0 = torch.zeros((M, N), dtype=torch.bfloat16, device=DEV)
     il.op_gemm(M, N, K, At, K, 0, Bt, K, 0, 0, err, C_=C0, ldc=N, bias=bt)
-    # 1: pre + gelu
+    # 1: gelu'(pre) and gelu(pre)
     C1 = torch.zeros((M, N), dtype=torch.bfloat16, device=DEV)
     C2 = torch.zeros((M, N), dtype=torch.bfloat16, device=DEV)
     il.op_gemm(M, N, K, At, K, 0, Bt, K, 0, 1, err, C_=C1, ldc=N, C2=C2, bias=bt)
@@ -90,14 +90,14 @@ def test_gemm_epilogues_forward():
     torch.cuda.synchronize()
     assert int(err.item()) == 0
     assert _rel(C0.float().cpu().numpy(), pre) < 3e-3
-    assert _rel(C1.float().cpu().numpy(), pre) < 3e-3
+    assert _rel(C1.float().cpu().numpy(), orc.gelu_grad(pre)) < 3e-3
     assert _rel(C2.float().cpu().numpy(), orc.gelu(pre)) < 3e-3
     assert _rel(R.cpu().numpy(), R0 + pre) < 1e-6
 
 
-def test_gemm_dgelu_epilogue_with_stacked_rows():
+def test_gemm_multiply_epilogue_with_stacked_rows():
     rng = np.random.default_rng(6)
-    rows, s, N, K = 200, 2, 264, 128          # 2 stacked gradient streams share one saved pre-activation
+    rows, s, N, K = 200, 2, 264, 128          # 2 stacked gradient streams share one saved gelu'
     M = rows * s
     At, Ae = _bf16(rng.standard_normal((M, K)))
     Wt, We = _bf16(rng.standard_normal((K, N)) * 0.3)      # dgrad: B stored [K, N] (MN-major)
@@ -107,7 +107,7 @@ def test_gemm_dgelu_epilogue_with_stacked_rows():
     il.op_gemm(M, N, K, At, K, 0, Wt, N, 1, 3, err, C_=Ct, ldc=N, aux=Ht, ld_aux=N, aux_rows=rows)
     torch.cuda.synchronize()
     assert int(err.item()) == 0
-    ref = (Ae @ We) * orc.gelu_grad(np.tile(He, (s, 1)))
+    ref = (Ae @ We) * np.tile(He, (s, 1))
     assert _rel(Ct.float().cpu().numpy(), ref) < 3e-3
 
 
@@ -121,7 +121,7 @@ def test_gemm_softmax_epilogues(V):
     tgt = rng.integers(0, V, size=M).astype(np.int32)
     tgt[0], tgt[1] = 0, V - 1
     tt = torch.tensor(tgt, device=DEV)
-    ntiles = (V + 255) // 256
+    ntiles = (V + 127) // 128
     pm = torch.zeros((M, ntiles), dtype=torch.float32, device=DEV)
     ps = torch.zeros((M, ntiles), dtype=torch.float32, device=DEV)
     tl = torch.zeros(M, dtype=torch.float32, device=DEV)

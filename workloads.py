@@ -59,6 +59,9 @@ CONFIGS: Dict[str, Workload] = {
     "cfg3": Workload("cfg3", K=4, Lc=3, d=768, H=12, F=3072, V=50257, T=1024, B=8, n=1),
     "cfg4": Workload("cfg4", K=8, Lc=3, d=1024, H=16, F=4096, V=50257, T=1024, B=8, n=2, adamw=True),
     "cfg5": Workload("cfg5", K=8, Lc=4, d=2560, H=32, F=10240, V=50257, T=2048, B=4, n=2, adamw=True),
+    # cfg4's widths, sequence length, batch and vocabulary with only two one-layer components: every kernel
+    # runs at cfg4's shapes while the model holds ~3 GB, small enough for profiler captures.
+    "cfg4-2x1": Workload("cfg4-2x1", K=2, Lc=1, d=1024, H=16, F=4096, V=50257, T=1024, B=8, n=2, adamw=True),
 }
 
 
