@@ -62,6 +62,21 @@ il_status il_op_attention_fwd(const void* qkv, void* o, float* lse, int B, int T
 il_status il_op_attention_bwd(const void* qkv, const void* o, const float* lse, const void* dout, void* dqkv,
                               float* delta, int NB, int B, int T, int H, int dh, void* stream);
 
+/* The same backward for callers that cannot allocate device memory (no counterpart in the paper: it exists
+ * for code embedded where cudaMalloc is not allowed — inside another framework's memory pool, in a
+ * real-time loop that bans driver allocations after start-up, or under a fixed device-memory budget).  The
+ * delta scratch lives in a fixed 4 MiB array inside the library image (held by every GPU that loads the
+ * library until the process exits), so the call obtains no memory: no cudaMalloc/cudaFree, no allocating
+ * library routine.  Limit: NB*H*T <= il_op_attention_bwd_noalloc_max_rows() (1,048,576); larger sizes are
+ * rejected with IL_ERR_INVALID_ARG before anything is launched.  The first call on each device looks up
+ * the array's device address (with that device current) and should therefore be made before any stream
+ * capture starts.  All calls on a device share the one array: it keeps the previous call's contents
+ * (nothing needs to start at zero — each call rewrites every element it reads), and two calls whose
+ * kernels overlap on the GPU (different streams) race on it; serialise them. */
+il_status il_op_attention_bwd_noalloc(const void* qkv, const void* o, const float* lse, const void* dout, void* dqkv,
+                                      int NB, int B, int T, int H, int dh, void* stream);
+size_t il_op_attention_bwd_noalloc_max_rows(void);
+
 /* LayerNorm over the last axis (biased variance, eps inside the square root): y bf16 [rows, d],
  * mean/rstd fp32 [rows].  d % 8 == 0. */
 il_status il_op_layernorm_fwd(const float* x, const float* gamma, const float* beta, void* y, float* mean,

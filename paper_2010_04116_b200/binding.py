@@ -84,6 +84,7 @@ def lib() -> C.CDLL:
         "il_op_gemm": [C.POINTER(il_gemm_desc), vp, vp],
         "il_op_attention_fwd": [vp, vp, vp, i, i, i, i, vp],
         "il_op_attention_bwd": [vp, vp, vp, vp, vp, vp, i, i, i, i, i, vp],
+        "il_op_attention_bwd_noalloc": [vp, vp, vp, vp, vp, i, i, i, i, i, vp],
         "il_op_layernorm_fwd": [vp, vp, vp, vp, vp, vp, i, i, f, vp],
         "il_op_layernorm_bwd": [vp, i, vp, vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, vp],
     }
@@ -91,6 +92,8 @@ def lib() -> C.CDLL:
         fn = getattr(L, name)
         fn.argtypes = args
         fn.restype = C.c_int
+    L.il_op_attention_bwd_noalloc_max_rows.argtypes = []
+    L.il_op_attention_bwd_noalloc_max_rows.restype = C.c_size_t
     L.il_num_tensors.argtypes = [vp]
     L.il_num_tensors.restype = C.c_int
     L.il_last_error.argtypes = [vp]
@@ -341,6 +344,14 @@ def op_attention_bwd(qkv, o, lse, dout, dqkv, delta, NB, B, T, H, dh, stream=Non
                                    dh, stream)
     if st != IL_OK:
         raise ILError(st, "il_op_attention_bwd")
+
+
+def op_attention_bwd_noalloc(qkv, o, lse, dout, dqkv, NB, B, T, H, dh, stream=None):
+    """Attention backward whose scratch is a fixed array inside the library: allocates nothing."""
+    st = lib().il_op_attention_bwd_noalloc(_ptr(qkv), _ptr(o), _ptr(lse), _ptr(dout), _ptr(dqkv), NB, B, T, H, dh,
+                                           stream)
+    if st != IL_OK:
+        raise ILError(st, "il_op_attention_bwd_noalloc")
 
 
 def op_layernorm_fwd(x, gamma, beta, y, mean, rstd, rows, d, eps=1e-5, stream=None):
