@@ -421,7 +421,7 @@ static cudaError_t fwd_launch(const bf16* qkv, bf16* o, float* lse, int B, int T
   return cudaGetLastError();
 }
 
-cudaError_t attention_fwd(const bf16* qkv, bf16* o, float* lse, int B, int T, int H, int dh, cudaStream_t s) {
+cudaError_t attention_fwd_legacy(const bf16* qkv, bf16* o, float* lse, int B, int T, int H, int dh, cudaStream_t s) {
   switch (dh) {
     case 32: return fwd_launch<32>(qkv, o, lse, B, T, H, s);
     case 64: return fwd_launch<64>(qkv, o, lse, B, T, H, s);
@@ -449,7 +449,7 @@ static cudaError_t bwd_launch(const bf16* qkv, const bf16* o, const float* lse, 
   return cudaGetLastError();
 }
 
-cudaError_t attention_bwd(const bf16* qkv, const bf16* o, const float* lse, const bf16* dout, bf16* dqkv, float* delta,
+cudaError_t attention_bwd_legacy(const bf16* qkv, const bf16* o, const float* lse, const bf16* dout, bf16* dqkv, float* delta,
                           int NB, int B, int T, int H, int dh, cudaStream_t s) {
   switch (dh) {
     case 32: return bwd_launch<32>(qkv, o, lse, dout, dqkv, delta, NB, B, T, H, s);

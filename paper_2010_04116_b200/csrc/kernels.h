@@ -48,11 +48,13 @@ cudaError_t adamw(float* p, float* m, float* v, const float* g, __nv_bfloat16* p
 
 // Causal attention on packed qkv [B*T, 3d] (Q | K | V, head h at columns h*dh).  dh in {32, 64, 80, 128}.
 //   o [B*T, d] bf16, lse [B, H, T] fp32 (natural log of the softmax denominator, scores scaled by 1/sqrt(dh)).
+// err (may be NULL): device word set non-zero if a bounded wait in the kernel expired.
 cudaError_t attention_fwd(const __nv_bfloat16* qkv, __nv_bfloat16* o, float* lse, int B, int T, int H, int dh,
-                          cudaStream_t s);
+                          unsigned* err, cudaStream_t s);
 // Backward.  NB batches of gradients share one saved forward of B sequences: gradient batch b uses saved
 // sequence (b % B).  dqkv [NB*T, 3d] bf16; delta is scratch [NB, H, T] fp32.
 cudaError_t attention_bwd(const __nv_bfloat16* qkv, const __nv_bfloat16* o, const float* lse, const __nv_bfloat16* dout,
-                          __nv_bfloat16* dqkv, float* delta, int NB, int B, int T, int H, int dh, cudaStream_t s);
+                          __nv_bfloat16* dqkv, float* delta, int NB, int B, int T, int H, int dh, unsigned* err,
+                          cudaStream_t s);
 
 }  // namespace il

@@ -611,7 +611,7 @@ extern "C" il_status il_forward_component(il_model* m, int k) {
       g.bias = m->P + o.bqkv;
       IL_TRY(gemm(m, k, g));
     }
-    IL_K(m, attention_fwd(A.qkv, A.attn_o, A.lse, m->B, m->T, m->H, m->dh, st));
+    IL_K(m, attention_fwd(A.qkv, A.attn_o, A.lse, m->B, m->T, m->H, m->dh, m->err_word, st));
     {
       GemmArgs g = gemm_args(N, d, d, A.attn_o, d, 0, m->Pb + o.wo, d, 0, EPI_F32_RESID, A.x_mid, d);
       g.bias = m->P + o.bo;
@@ -752,7 +752,7 @@ il_status component_backward(il_model* m, int k, int s) {
     IL_K(m, colsum_f32(c.dx, d, m->G + o.bo, N, d, st));
     IL_TRY(gemm(m, k, gemm_args(d, d, N, c.dxb, d, 1, A.attn_o, d, 1, EPI_F32, m->G + o.wo, d)));
     IL_TRY(gemm(m, k, gemm_args(R, d, d, c.dxb, d, 0, m->Pb + o.wo, d, 1, EPI_BF16, c.dattn, d)));
-    IL_K(m, attention_bwd(A.qkv, A.attn_o, A.lse, c.dattn, c.dqkv, c.delta, s * m->B, m->B, m->T, m->H, m->dh, st));
+    IL_K(m, attention_bwd(A.qkv, A.attn_o, A.lse, c.dattn, c.dqkv, c.delta, s * m->B, m->B, m->T, m->H, m->dh, m->err_word, st));
     m->launches += 2;
     IL_K(m, colsum_bf16(c.dqkv, 3 * d, m->G + o.bqkv, N, 3 * d, st));
     IL_TRY(gemm(m, k, gemm_args(3 * d, d, N, c.dqkv, 3 * d, 1, A.ln1, d, 1, EPI_F32, m->G + o.wqkv, d)));
@@ -944,14 +944,14 @@ extern "C" il_status il_op_gemm(const il_gemm_desc* q, unsigned* err_word, void*
 
 extern "C" il_status il_op_attention_fwd(const void* qkv, void* o, float* lse, int B, int T, int H, int dh, void* stream) {
   if (!qkv || !o || !lse || B < 1 || T < 1 || H < 1) return IL_ERR_INVALID_ARG;
-  return op_status(attention_fwd((const bf16*)qkv, (bf16*)o, lse, B, T, H, dh, reinterpret_cast<cudaStream_t>(stream)));
+  return op_status(attention_fwd((const bf16*)qkv, (bf16*)o, lse, B, T, H, dh, nullptr, reinterpret_cast<cudaStream_t>(stream)));
 }
 
 extern "C" il_status il_op_attention_bwd(const void* qkv, const void* o, const float* lse, const void* dout, void* dqkv,
                                          float* delta, int NB, int B, int T, int H, int dh, void* stream) {
   if (!qkv || !o || !lse || !dout || !dqkv || !delta || B < 1 || NB < 1 || T < 1 || H < 1) return IL_ERR_INVALID_ARG;
   return op_status(attention_bwd((const bf16*)qkv, (const bf16*)o, lse, (const bf16*)dout, (bf16*)dqkv, delta, NB, B, T, H, dh,
-                                 reinterpret_cast<cudaStream_t>(stream)));
+                                 nullptr, reinterpret_cast<cudaStream_t>(stream)));
 }
 
 extern "C" il_status il_op_layernorm_fwd(const float* x, const float* gamma, const float* beta, void* y, float* mean,
