@@ -1,463 +1,837 @@
-// Causal self-attention forward and backward on packed qkv [B*T, 3d] (softmax(Q K^T / sqrt(dh)) V).
+// Causal self-attention forward on the tcgen05 tensor cores (sm_100a).
 //
-// Blockwise online-softmax formulation: the T x T score matrix is never stored.  One CTA owns a block of
-// 64 query rows (forward, dQ) or 64 key rows (dK/dV) of one (sequence, head) and sweeps the other index in
-// blocks of 64; each of its 4 warps owns 16 rows.  Contractions run on the tensor cores through
-// mma.sync m16n8k16 (bf16 in, fp32 accumulate) with ldmatrix-fed fragments; softmax statistics are fp32.
-// Backward recomputes the probabilities from the saved per-row log-sum-exp and uses
-// delta_i = sum_c dO_ic O_ic (= sum_j P_ij dP_ij).
+// One CTA owns 128 query rows of one (sequence, head) and sweeps the keys in blocks of 64.  Q, K and V
+// tiles come in by TMA from the packed qkv tensor viewed as a 4-D tensor (column within head, head slot,
+// position, sequence) so that head selection, the ragged last rows of a sequence and head dimensions
+// that are not a multiple of 64 are all handled by the tensor map's bounds (zero fill).  Per key block:
+//   S = Q K^T        tcgen05.mma (M128 N64, both operands K-major in shared memory) -> TMEM columns [0, 64)
+//   softmax          thread r owns query row r: tcgen05.ld its 64 scores, running max / sum in registers
+//                    (no cross-lane reduction), P = exp2(...) rounded to bf16 and written to shared memory in
+//                    the K-major 128-byte-swizzled layout the next MMA expects
+//   O += P V         tcgen05.mma (M128 N=dh, A = P K-major, B = V MN-major), accumulated in TMEM columns
+//                    [64, 64+dh).  The reference maximum of a row is raised only when a block exceeds it by a
+//                    factor 2^8, so the accumulator is rescaled (tcgen05.ld / st) rarely.
+// A CTA runs these phases one after the other; several CTAs are resident per SM (128 threads, 64-112 KB of
+// shared memory, 128-256 TMEM columns each), which is what overlaps one CTA's softmax with another's MMAs.
+// The T x T score matrix is never stored.  Every wait is bounded.
 #include "common.cuh"
 #include "kernels.h"
+#include "tma.h"
 
 namespace il {
 
-constexpr int AT_BLK = 64;        // rows per CTA tile and per sweep step
-constexpr int AT_THREADS = 128;
-#define LOG2E_F 1.4426950408889634f
+namespace {
 
-__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
-}
-__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
-}
-__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
-  const int sz = valid ? 16 : 0;
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
-}
-__device__ __forceinline__ void cp_async_wait_all() {
-  asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
-}
+constexpr int TQ = 128;     // query rows per CTA
+constexpr int TK = 64;      // keys per sweep step
+#define IL_LOG2E 1.4426950408889634f
 
-// Copy a [64, DH] bf16 tile (row stride ld elements, rows >= rows_valid zero-filled) into padded smem.
 template <int DH>
-__device__ __forceinline__ void load_tile(bf16* dst, const bf16* src, int ld, int row0, int rows_valid) {
-  constexpr int LD = DH + 8;
-  constexpr int CH = DH / 8;
-  for (int i = threadIdx.x; i < AT_BLK * CH; i += AT_THREADS) {
-    const int r = i / CH, c = i % CH;
-    const bool ok = (row0 + r) < rows_valid;
-    const bf16* g = src + (size_t)(ok ? row0 + r : 0) * ld + c * 8;
-    cp_async16(smem_u32(dst + r * LD + c * 8), g, ok);
-  }
-}
+struct FwdCfg {
+  static constexpr int NCH = (DH + 63) / 64;            // 64-column chunks of the head dimension
+  static constexpr int Q_BYTES = NCH * TQ * 128;
+  static constexpr int KV_BYTES = NCH * TK * 128;
+  static constexpr int P_BYTES = TQ * 128;
+  static constexpr int TCOLS = (64 + DH <= 128) ? 128 : 256;   // 64 score columns + the O accumulator
+  static constexpr int SMEM = Q_BYTES + 4 * KV_BYTES + P_BYTES + 1024 + 64;
+};
 
-// A-operand fragment (16 rows x 16 k) from row-major smem [rows][LD]
-template <int LD>
-__device__ __forceinline__ void load_a(const bf16* s, int row0, int k0, uint32_t (&a)[4]) {
-  const int lane = threadIdx.x & 31;
-  const int r = row0 + (lane & 7) + 8 * ((lane >> 3) & 1);
-  const int c = k0 + 8 * (lane >> 4);
-  ldsm_x4(smem_u32(s + r * LD + c), a[0], a[1], a[2], a[3]);
-}
-// B-operand fragments for two adjacent n-tiles (16 n x 16 k) where smem holds [n][k] (k contiguous)
-template <int LD>
-__device__ __forceinline__ void load_b_nk(const bf16* s, int n0, int k0, uint32_t (&b)[4]) {
-  const int lane = threadIdx.x & 31;
-  const int r = n0 + (lane & 7) + 8 * (lane >> 4);
-  const int c = k0 + 8 * ((lane >> 3) & 1);
-  ldsm_x4(smem_u32(s + r * LD + c), b[0], b[1], b[2], b[3]);
-}
-// B-operand fragments for two adjacent n-tiles where smem holds [k][n] (n contiguous): transposing load
-template <int LD>
-__device__ __forceinline__ void load_b_kn(const bf16* s, int k0, int n0, uint32_t (&b)[4]) {
-  const int lane = threadIdx.x & 31;
-  const int r = k0 + (lane & 7) + 8 * ((lane >> 3) & 1);
-  const int c = n0 + 8 * (lane >> 4);
-  ldsm_x4_t(smem_u32(s + r * LD + c), b[0], b[1], b[2], b[3]);
-}
-
-// acc[8 n-tiles] (16 x 64) = A[16 x DH] (smem rows a_row0..) * Bs[64 x DH]^T
 template <int DH>
-__device__ __forceinline__ void mm_16x64_nk(float (&acc)[8][4], const bf16* sA, int a_row0, const bf16* sB) {
-  constexpr int LD = DH + 8;
-#pragma unroll
-  for (int j = 0; j < 8; ++j)
-#pragma unroll
-    for (int e = 0; e < 4; ++e) acc[j][e] = 0.f;
-#pragma unroll
-  for (int ks = 0; ks < DH / 16; ++ks) {
-    uint32_t a[4];
-    load_a<LD>(sA, a_row0, ks * 16, a);
-#pragma unroll
-    for (int np = 0; np < 4; ++np) {
-      uint32_t b[4];
-      load_b_nk<LD>(sB, np * 16, ks * 16, b);
-      mma_bf16(acc[2 * np], a, b[0], b[1]);
-      mma_bf16(acc[2 * np + 1], a, b[2], b[3]);
-    }
-  }
-}
+__global__ void __launch_bounds__(128) attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ,
+                                                          const __grid_constant__ CUtensorMap tmKV, bf16* __restrict__ o,
+                                                          float* __restrict__ lse, int T, int H, float scale, unsigned* err) {
+  using C = FwdCfg<DH>;
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ int abort_flag;
+  __shared__ uint32_t tmem_base_smem;
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t sQ = base;
+  const uint32_t sK0 = sQ + C::Q_BYTES;                       // two K stages, then two V stages
+  const uint32_t sV0 = sK0 + 2 * C::KV_BYTES;
+  const uint32_t sP = sV0 + 2 * C::KV_BYTES;
+  const uint32_t bars = sP + C::P_BYTES;
+  const uint32_t bar_q = bars, bar_kv0 = bars + 8, bar_s = bars + 24, bar_o = bars + 32, bar_drain = bars + 40;
+  uint8_t* sP_gen = smem_raw + (sP - smem_u32(smem_raw));
 
-// out[DH/8 n-tiles] (16 x DH) += P[16 x 64] (register fragments) * Bs[64 x DH]   (Bs row-major [k][n])
-template <int DH>
-__device__ __forceinline__ void mm_acc_p(float (&out)[DH / 8][4], const uint32_t (&p)[4][4], const bf16* sB) {
-  constexpr int LD = DH + 8;
-#pragma unroll
-  for (int kk = 0; kk < 4; ++kk) {
-#pragma unroll
-    for (int dp = 0; dp < DH / 16; ++dp) {
-      uint32_t b[4];
-      load_b_kn<LD>(sB, kk * 16, dp * 16, b);
-      mma_bf16(out[2 * dp], p[kk], b[0], b[1]);
-      mma_bf16(out[2 * dp + 1], p[kk], b[2], b[3]);
-    }
-  }
-}
-
-__device__ __forceinline__ void pack_p(const float (&s)[8][4], uint32_t (&p)[4][4]) {
-#pragma unroll
-  for (int kk = 0; kk < 4; ++kk) {
-    p[kk][0] = pack_bf16x2(s[2 * kk][0], s[2 * kk][1]);
-    p[kk][1] = pack_bf16x2(s[2 * kk][2], s[2 * kk][3]);
-    p[kk][2] = pack_bf16x2(s[2 * kk + 1][0], s[2 * kk + 1][1]);
-    p[kk][3] = pack_bf16x2(s[2 * kk + 1][2], s[2 * kk + 1][3]);
-  }
-}
-
-// ---------------------------------------------------------------------------------------------
-// Forward
-// ---------------------------------------------------------------------------------------------
-template <int DH>
-__global__ void __launch_bounds__(AT_THREADS) attn_fwd_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ o,
-                                                              float* __restrict__ lse, int T, int H, float scale) {
-  constexpr int LD = DH + 8;
-  extern __shared__ __align__(16) uint8_t at_smem[];
-  bf16* sQ = reinterpret_cast<bf16*>(at_smem);
-  bf16* sK = sQ + AT_BLK * LD;
-  bf16* sV = sK + AT_BLK * LD;
-  const int qt = gridDim.x - 1 - blockIdx.x;      // longest sweeps first
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int qb = gridDim.x - 1 - blockIdx.x;                  // longest sweeps first
   const int b = blockIdx.y / H, h = blockIdx.y % H;
   const int d = H * DH;
-  const int ld = 3 * d;
-  const bf16* qb = qkv + (size_t)b * T * ld + h * DH;
-  const bf16* kb = qb + d;
-  const bf16* vb = qb + 2 * d;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int g = lane >> 2, t4 = lane & 3;
-  const float c = scale * LOG2E_F;
+  const int row = qb * TQ + tid;                              // query position of this thread
+  int nkv = (qb * TQ + TQ + TK - 1) / TK;
+  const int nkv_all = (T + TK - 1) / TK;
+  if (nkv > nkv_all) nkv = nkv_all;
 
-  load_tile<DH>(sQ, qb, ld, qt * AT_BLK, T);
-  float oacc[DH / 8][4];
-#pragma unroll
-  for (int j = 0; j < DH / 8; ++j)
-#pragma unroll
-    for (int e = 0; e < 4; ++e) oacc[j][e] = 0.f;
-  float mrow[2] = {-INFINITY, -INFINITY};
-  float lrow[2] = {0.f, 0.f};
+  if (tid == 0) {
+    abort_flag = 0;
+    mbar_init(bar_q, 1);
+    mbar_init(bar_kv0, 1);
+    mbar_init(bar_kv0 + 8, 1);
+    mbar_init(bar_s, 1);
+    mbar_init(bar_o, 1);
+    mbar_init(bar_drain, 1);
+    fence_mbar_init();
+    tma_prefetch_desc(&tmQ);
+    tma_prefetch_desc(&tmKV);
+  }
+  if (warp == 0) {
+    tmem_alloc(smem_u32(&tmem_base_smem), C::TCOLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_smem;                  // scores at columns [0, 64), O at [64, 64 + dh)
+  const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
+  volatile int* abortp = &abort_flag;
+  constexpr uint32_t idesc_s = make_idesc_bf16(TQ, TK, 0, 0);
+  constexpr uint32_t idesc_o = make_idesc_bf16(TQ, DH, 0, 1);
+  int fail = 0;
 
-  for (int kt = 0; kt <= qt; ++kt) {
-    __syncthreads();   // previous sweep step has finished reading sK/sV
-    load_tile<DH>(sK, kb, ld, kt * AT_BLK, T);
-    load_tile<DH>(sV, vb, ld, kt * AT_BLK, T);
-    cp_async_wait_all();
-    __syncthreads();
-    float s[8][4];
-    mm_16x64_nk<DH>(s, sQ, warp * 16, sK);
-    if (kt == qt) {
+  auto load_kv = [&](int j) {
+    const int st = j & 1;
+    mbar_expect_tx(bar_kv0 + 8 * st, 2 * C::KV_BYTES);
 #pragma unroll
-      for (int j = 0; j < 8; ++j)
+    for (int c = 0; c < C::NCH; ++c) {
+      tma_load_4d(sK0 + st * C::KV_BYTES + c * (TK * 128), &tmKV, c * 64, H + h, j * TK, b, bar_kv0 + 8 * st);
+      tma_load_4d(sV0 + st * C::KV_BYTES + c * (TK * 128), &tmKV, c * 64, 2 * H + h, j * TK, b, bar_kv0 + 8 * st);
+    }
+  };
+  if (tid == 0) {
+    mbar_expect_tx(bar_q, C::Q_BYTES);
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int key = j * 8 + 2 * t4 + (e & 1);
-          const int qry = warp * 16 + g + 8 * (e >> 1);
-          if (key > qry) s[j][e] = -INFINITY;
+    for (int c = 0; c < C::NCH; ++c) tma_load_4d(sQ + c * (TQ * 128), &tmQ, c * 64, h, qb * TQ, b, bar_q);
+    load_kv(0);
+    if (nkv > 1) load_kv(1);
+  }
+
+  const float c2 = scale * IL_LOG2E;
+  // Running statistics of this thread's row.  m is the reference maximum the exponentials are taken against; it
+  // is only raised when a block's maximum exceeds it by more than 8 (in log2 units), so that the accumulator in
+  // TMEM rarely needs rescaling; l and O stay consistent with whatever m is, and O / l is exact either way.
+  float m = -INFINITY, l = 0.f;
+  const float slack = 8.0f / c2;
+
+  for (int j = 0; j < nkv; ++j) {
+    const int st = j & 1;
+    const uint32_t ph = (uint32_t)j & 1u;
+    if (tid == 0) {
+      bool ok = true;
+      if (j == 0) ok = mbar_wait(bar_q, 0, abortp);
+      ok = ok && mbar_wait(bar_kv0 + 8 * st, (uint32_t)(j >> 1) & 1u, abortp);
+      if (!ok) { fail = 1; abort_flag = 1; }
+      tc_fence_after();
+#pragma unroll
+      for (int ks = 0; ks < DH / 16; ++ks) {
+        const uint64_t ad = make_smem_desc(sQ + (ks >> 2) * (TQ * 128) + (ks & 3) * 32, 16, 1024);
+        const uint64_t bd = make_smem_desc(sK0 + st * C::KV_BYTES + (ks >> 2) * (TK * 128) + (ks & 3) * 32, 16, 1024);
+        umma_bf16(tmem_base, ad, bd, idesc_s, ks ? 1u : 0u);
+      }
+      umma_commit(bar_s);
+    }
+    if (!mbar_wait(bar_s, ph, abortp)) { fail = 1; abort_flag = 1; }
+    tc_fence_after();
+    // ---- softmax of this thread's row over the 64 keys of the block
+    uint32_t r0[32], r1[32];
+    tmem_ld_32x32(t_lane, r0);
+    tmem_ld_32x32(t_lane + 32, r1);
+    tmem_ld_wait();
+    float s[64];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) { s[i] = __uint_as_float(r0[i]); s[32 + i] = __uint_as_float(r1[i]); }
+    if (j * TK + TK - 1 > qb * TQ) {              // block touches the diagonal: mask keys after the query
+#pragma unroll
+      for (int i = 0; i < 64; ++i)
+        if (j * TK + i > row) s[i] = -INFINITY;
+    }
+    float mx4[4] = {s[0], s[1], s[2], s[3]};
+#pragma unroll
+    for (int i = 4; i < 64; i += 4) {
+      mx4[0] = fmaxf(mx4[0], s[i]); mx4[1] = fmaxf(mx4[1], s[i + 1]);
+      mx4[2] = fmaxf(mx4[2], s[i + 2]); mx4[3] = fmaxf(mx4[3], s[i + 3]);
+    }
+    const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+    // the previous block's P V must have landed before P's buffer is overwritten or O is rescaled
+    if (j > 0) {
+      if (!mbar_wait(bar_o, (uint32_t)(j - 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
+      tc_fence_after();
+      if (tid == 0 && j + 1 < nkv) load_kv(j + 1);            // both MMAs that read that stage have completed
+    }
+    if (__any_sync(0xffffffffu, mx > m + slack)) {            // warp-uniform: raise the reference maximum
+      const float mn = fmaxf(m, mx);
+      const float alpha = ex2_fast((m - mn) * c2);            // 0 on the first block (m = -inf)
+      l *= alpha;
+      m = mn;
+      if (j > 0) {
+#pragma unroll
+        for (int c0 = 0; c0 < DH; c0 += 32) {
+          if (c0 + 32 <= DH) {
+            uint32_t r[32];
+            tmem_ld_32x32(t_lane + 64 + c0, r);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+            tmem_st_32x32(t_lane + 64 + c0, r);
+          } else {
+            uint32_t r[16];
+            tmem_ld_32x16(t_lane + 64 + c0, r);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+            tmem_st_32x16(t_lane + 64 + c0, r);
+          }
         }
-    }
-    float mx[2] = {-INFINITY, -INFINITY};
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      mx[0] = fmaxf(mx[0], fmaxf(s[j][0], s[j][1]));
-      mx[1] = fmaxf(mx[1], fmaxf(s[j][2], s[j][3]));
-    }
-#pragma unroll
-    for (int r = 0; r < 2; ++r) {
-      mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
-      mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
-    }
-    float alpha[2], mc[2];
-#pragma unroll
-    for (int r = 0; r < 2; ++r) {
-      const float mn = fmaxf(mrow[r], mx[r]);      // finite: key 0 is always visible
-      alpha[r] = exp2f((mrow[r] - mn) * c);
-      mrow[r] = mn;
-      mc[r] = mn * c;
-      lrow[r] *= alpha[r];
-    }
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      s[j][0] = exp2f(s[j][0] * c - mc[0]);
-      s[j][1] = exp2f(s[j][1] * c - mc[0]);
-      s[j][2] = exp2f(s[j][2] * c - mc[1]);
-      s[j][3] = exp2f(s[j][3] * c - mc[1]);
-      lrow[0] += s[j][0] + s[j][1];
-      lrow[1] += s[j][2] + s[j][3];
-    }
-#pragma unroll
-    for (int j = 0; j < DH / 8; ++j) {
-      oacc[j][0] *= alpha[0]; oacc[j][1] *= alpha[0];
-      oacc[j][2] *= alpha[1]; oacc[j][3] *= alpha[1];
-    }
-    uint32_t p[4][4];
-    pack_p(s, p);
-    mm_acc_p<DH>(oacc, p, sV);
-  }
-#pragma unroll
-  for (int r = 0; r < 2; ++r) {
-    lrow[r] += __shfl_xor_sync(0xffffffffu, lrow[r], 1);
-    lrow[r] += __shfl_xor_sync(0xffffffffu, lrow[r], 2);
-  }
-#pragma unroll
-  for (int r = 0; r < 2; ++r) {
-    const int qry = qt * AT_BLK + warp * 16 + g + 8 * r;
-    if (qry < T) {
-      const float inv = 1.0f / lrow[r];
-      bf16* orow = o + ((size_t)b * T + qry) * d + h * DH;
-#pragma unroll
-      for (int j = 0; j < DH / 8; ++j)
-        *reinterpret_cast<uint32_t*>(orow + j * 8 + 2 * t4) = pack_bf16x2(oacc[j][2 * r] * inv, oacc[j][2 * r + 1] * inv);
-      if (t4 == 0) lse[((size_t)b * H + h) * T + qry] = mrow[r] * scale + logf(lrow[r]);
-    }
-  }
-}
-
-// ---------------------------------------------------------------------------------------------
-// Backward: delta, dK/dV, dQ
-// ---------------------------------------------------------------------------------------------
-// delta[nb, h, t] = sum_c dO[nb*T+t, h*dh+c] * O[(nb%B)*T+t, h*dh+c];  one warp per (row, head)
-__global__ void __launch_bounds__(256) attn_delta_kernel(const bf16* __restrict__ dout, const bf16* __restrict__ o,
-                                                         float* __restrict__ delta, int NB, int B, int T, int H, int dh) {
-  const int wid = blockIdx.x * 8 + (threadIdx.x >> 5);
-  const int lane = threadIdx.x & 31;
-  const int total = NB * T * H;
-  if (wid >= total) return;
-  const int h = wid % H;
-  const int row = wid / H;               // nb*T + t
-  const int nb = row / T, t = row % T;
-  const int d = H * dh;
-  const bf16* a = dout + (size_t)row * d + h * dh;
-  const bf16* bb = o + ((size_t)(nb % B) * T + t) * d + h * dh;
-  float s = 0.f;
-  for (int c = lane * 2; c < dh; c += 64) {
-    const float2 x = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(a + c));
-    const float2 y = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(bb + c));
-    s += x.x * y.x + x.y * y.y;
-  }
-  s = warp_sum(s);
-  if (lane == 0) delta[((size_t)nb * H + h) * T + t] = s;
-}
-
-template <int DH>
-__global__ void __launch_bounds__(AT_THREADS) attn_bwd_dkv_kernel(const bf16* __restrict__ qkv, const float* __restrict__ lse,
-                                                                  const bf16* __restrict__ dout,
-                                                                  const float* __restrict__ delta, bf16* __restrict__ dqkv,
-                                                                  int B, int T, int H, float scale) {
-  constexpr int LD = DH + 8;
-  extern __shared__ __align__(16) uint8_t at_smem[];
-  bf16* sK = reinterpret_cast<bf16*>(at_smem);
-  bf16* sV = sK + AT_BLK * LD;
-  bf16* sQ = sV + AT_BLK * LD;
-  bf16* sdO = sQ + AT_BLK * LD;
-  float* sLse = reinterpret_cast<float*>(sdO + AT_BLK * LD);
-  float* sDel = sLse + AT_BLK;
-  const int kt = blockIdx.x;
-  const int nb = blockIdx.y / H, h = blockIdx.y % H;
-  const int bs = nb % B;
-  const int d = H * DH, ld = 3 * d;
-  const bf16* qb = qkv + (size_t)bs * T * ld + h * DH;
-  const bf16* dob = dout + (size_t)nb * T * d + h * DH;
-  const float* lseb = lse + ((size_t)bs * H + h) * T;
-  const float* delb = delta + ((size_t)nb * H + h) * T;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int g = lane >> 2, t4 = lane & 3;
-  const float c = scale * LOG2E_F;
-  const int nq = (T + AT_BLK - 1) / AT_BLK;
-
-  load_tile<DH>(sK, qb + d, ld, kt * AT_BLK, T);
-  load_tile<DH>(sV, qb + 2 * d, ld, kt * AT_BLK, T);
-  float dk[DH / 8][4], dv[DH / 8][4];
-#pragma unroll
-  for (int j = 0; j < DH / 8; ++j)
-#pragma unroll
-    for (int e = 0; e < 4; ++e) { dk[j][e] = 0.f; dv[j][e] = 0.f; }
-
-  for (int qt = kt; qt < nq; ++qt) {
-    __syncthreads();
-    load_tile<DH>(sQ, qb, ld, qt * AT_BLK, T);
-    load_tile<DH>(sdO, dob, d, qt * AT_BLK, T);
-    if (threadIdx.x < AT_BLK) {
-      const int q = qt * AT_BLK + threadIdx.x;
-      sLse[threadIdx.x] = q < T ? lseb[q] * LOG2E_F : 0.f;
-      sDel[threadIdx.x] = q < T ? delb[q] : 0.f;
-    }
-    cp_async_wait_all();
-    __syncthreads();
-    // S^T (16 keys x 64 queries) and dP^T
-    float st[8][4], dpt[8][4];
-    mm_16x64_nk<DH>(st, sK, warp * 16, sQ);
-    mm_16x64_nk<DH>(dpt, sV, warp * 16, sdO);
-#pragma unroll
-    for (int j = 0; j < 8; ++j)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int key = kt * AT_BLK + warp * 16 + g + 8 * (e >> 1);
-        const int ql = j * 8 + 2 * t4 + (e & 1);
-        const int qry = qt * AT_BLK + ql;
-        const float p = (qry >= key && qry < T) ? exp2f(st[j][e] * c - sLse[ql]) : 0.f;
-        st[j][e] = p;
-        dpt[j][e] = p * (dpt[j][e] - sDel[ql]);
-      }
-    uint32_t pf[4][4];
-    pack_p(st, pf);
-    mm_acc_p<DH>(dv, pf, sdO);
-    pack_p(dpt, pf);
-    mm_acc_p<DH>(dk, pf, sQ);
-  }
-#pragma unroll
-  for (int r = 0; r < 2; ++r) {
-    const int key = kt * AT_BLK + warp * 16 + g + 8 * r;
-    if (key < T) {
-      bf16* row = dqkv + ((size_t)nb * T + key) * ld + h * DH;
-#pragma unroll
-      for (int j = 0; j < DH / 8; ++j) {
-        *reinterpret_cast<uint32_t*>(row + d + j * 8 + 2 * t4) = pack_bf16x2(dk[j][2 * r] * scale, dk[j][2 * r + 1] * scale);
-        *reinterpret_cast<uint32_t*>(row + 2 * d + j * 8 + 2 * t4) = pack_bf16x2(dv[j][2 * r], dv[j][2 * r + 1]);
+        tmem_st_wait();
       }
     }
+    const float mc = m * c2;
+    float ps4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int i = 0; i < 64; i += 4) {
+      s[i] = ex2_fast(fmaf(s[i], c2, -mc)); s[i + 1] = ex2_fast(fmaf(s[i + 1], c2, -mc));
+      s[i + 2] = ex2_fast(fmaf(s[i + 2], c2, -mc)); s[i + 3] = ex2_fast(fmaf(s[i + 3], c2, -mc));
+      ps4[0] += s[i]; ps4[1] += s[i + 1]; ps4[2] += s[i + 2]; ps4[3] += s[i + 3];
+    }
+    l += (ps4[0] + ps4[1]) + (ps4[2] + ps4[3]);
+    // P (bf16) into shared memory: row = tid, 16-byte chunk c8 lands at chunk (c8 ^ (row & 7)) of the 128-byte row
+#pragma unroll
+    for (int c8 = 0; c8 < 8; ++c8) {
+      uint4 pk;
+      pk.x = pack_bf16x2(s[8 * c8], s[8 * c8 + 1]);
+      pk.y = pack_bf16x2(s[8 * c8 + 2], s[8 * c8 + 3]);
+      pk.z = pack_bf16x2(s[8 * c8 + 4], s[8 * c8 + 5]);
+      pk.w = pack_bf16x2(s[8 * c8 + 6], s[8 * c8 + 7]);
+      *reinterpret_cast<uint4*>(sP_gen + tid * 128 + ((c8 ^ (tid & 7)) << 4)) = pk;
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    if (__syncthreads_or(fail)) { fail = 1; break; }     // uniform exit if any thread's wait expired
+    if (tid == 0) {
+      tc_fence_after();
+#pragma unroll
+      for (int ks = 0; ks < TK / 16; ++ks) {
+        const uint64_t ad = make_smem_desc(sP + ks * 32, 16, 1024);
+        const uint64_t bd = make_smem_desc(sV0 + st * C::KV_BYTES + ks * 2048, TK * 128, 1024);   // MN-major
+        umma_bf16(tmem_base + 64, ad, bd, idesc_o, (j | ks) ? 1u : 0u);                            // O accumulates in TMEM
+      }
+      umma_commit(bar_o);
+    }
+  }
+  if (!fail && nkv > 0) {
+    if (!mbar_wait(bar_o, (uint32_t)(nkv - 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
+    tc_fence_after();
+  }
+  fail = __syncthreads_or(fail);
+  if (!fail) {
+    const float inv = 1.0f / l;
+    bf16* orow = o + ((size_t)b * T + row) * d + h * DH;
+#pragma unroll
+    for (int c0 = 0; c0 < DH; c0 += 32) {
+      float v[32];
+      if (c0 + 32 <= DH) {
+        uint32_t r[32];
+        tmem_ld_32x32(t_lane + 64 + c0, r);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]) * inv;
+      } else {
+        uint32_t r[16];
+        tmem_ld_32x16(t_lane + 64 + c0, r);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]) * inv;
+      }
+      if (row < T) {
+#pragma unroll
+        for (int i = 0; i < 32 && c0 + i < DH; i += 8) {
+          uint4 pk;
+          pk.x = pack_bf16x2(v[i], v[i + 1]);
+          pk.y = pack_bf16x2(v[i + 2], v[i + 3]);
+          pk.z = pack_bf16x2(v[i + 4], v[i + 5]);
+          pk.w = pack_bf16x2(v[i + 6], v[i + 7]);
+          *reinterpret_cast<uint4*>(orow + c0 + i) = pk;
+        }
+      }
+    }
+    if (row < T) lse[((size_t)b * H + h) * T + row] = m * scale + logf(l);
+  }
+  if (tid == 0) {
+    if (fail && err) atomicExch(err, DEV_TIMEOUT_MMA);
+    umma_commit(bar_drain);                      // every MMA issued by this CTA has retired before TMEM goes
+    int never = 0;
+    mbar_wait(bar_drain, 0, &never);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, C::TCOLS);
   }
 }
 
 template <int DH>
-__global__ void __launch_bounds__(AT_THREADS) attn_bwd_dq_kernel(const bf16* __restrict__ qkv, const float* __restrict__ lse,
-                                                                 const bf16* __restrict__ dout,
-                                                                 const float* __restrict__ delta, bf16* __restrict__ dqkv,
-                                                                 int B, int T, int H, float scale) {
-  constexpr int LD = DH + 8;
-  extern __shared__ __align__(16) uint8_t at_smem[];
-  bf16* sQ = reinterpret_cast<bf16*>(at_smem);
-  bf16* sdO = sQ + AT_BLK * LD;
-  bf16* sK = sdO + AT_BLK * LD;
-  bf16* sV = sK + AT_BLK * LD;
-  const int qt = gridDim.x - 1 - blockIdx.x;
-  const int nb = blockIdx.y / H, h = blockIdx.y % H;
-  const int bs = nb % B;
-  const int d = H * DH, ld = 3 * d;
-  const bf16* qb = qkv + (size_t)bs * T * ld + h * DH;
-  const bf16* dob = dout + (size_t)nb * T * d + h * DH;
-  const float* lseb = lse + ((size_t)bs * H + h) * T;
-  const float* delb = delta + ((size_t)nb * H + h) * T;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int g = lane >> 2, t4 = lane & 3;
-  const float c = scale * LOG2E_F;
-
-  load_tile<DH>(sQ, qb, ld, qt * AT_BLK, T);
-  load_tile<DH>(sdO, dob, d, qt * AT_BLK, T);
-  float lrow[2], drow[2];
-#pragma unroll
-  for (int r = 0; r < 2; ++r) {
-    const int q = qt * AT_BLK + warp * 16 + g + 8 * r;
-    lrow[r] = q < T ? lseb[q] * LOG2E_F : 0.f;
-    drow[r] = q < T ? delb[q] : 0.f;
-  }
-  float dq[DH / 8][4];
-#pragma unroll
-  for (int j = 0; j < DH / 8; ++j)
-#pragma unroll
-    for (int e = 0; e < 4; ++e) dq[j][e] = 0.f;
-
-  for (int kt = 0; kt <= qt; ++kt) {
-    __syncthreads();
-    load_tile<DH>(sK, qb + d, ld, kt * AT_BLK, T);
-    load_tile<DH>(sV, qb + 2 * d, ld, kt * AT_BLK, T);
-    cp_async_wait_all();
-    __syncthreads();
-    float s[8][4], dp[8][4];
-    mm_16x64_nk<DH>(s, sQ, warp * 16, sK);
-    mm_16x64_nk<DH>(dp, sdO, warp * 16, sV);
-#pragma unroll
-    for (int j = 0; j < 8; ++j)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int key = kt * AT_BLK + j * 8 + 2 * t4 + (e & 1);
-        const int r = e >> 1;
-        const int qry = qt * AT_BLK + warp * 16 + g + 8 * r;
-        const float p = (key <= qry && key < T) ? exp2f(s[j][e] * c - lrow[r]) : 0.f;
-        dp[j][e] = p * (dp[j][e] - drow[r]);
-      }
-    uint32_t pf[4][4];
-    pack_p(dp, pf);
-    mm_acc_p<DH>(dq, pf, sK);
-  }
-#pragma unroll
-  for (int r = 0; r < 2; ++r) {
-    const int qry = qt * AT_BLK + warp * 16 + g + 8 * r;
-    if (qry < T) {
-      bf16* row = dqkv + ((size_t)nb * T + qry) * ld + h * DH;
-#pragma unroll
-      for (int j = 0; j < DH / 8; ++j)
-        *reinterpret_cast<uint32_t*>(row + j * 8 + 2 * t4) = pack_bf16x2(dq[j][2 * r] * scale, dq[j][2 * r + 1] * scale);
-    }
-  }
-}
-
-// ---------------------------------------------------------------------------------------------
-// Host launchers
-// ---------------------------------------------------------------------------------------------
-template <int DH>
-static cudaError_t fwd_launch(const bf16* qkv, bf16* o, float* lse, int B, int T, int H, cudaStream_t s) {
-  const int smem = 3 * AT_BLK * (DH + 8) * 2;
-  cudaError_t e = cudaFuncSetAttribute(attn_fwd_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+cudaError_t fwd_tc_launch(const bf16* qkv, bf16* o, float* lse, int B, int T, int H, unsigned* err, cudaStream_t s) {
+  using C = FwdCfg<DH>;
+  const unsigned long long d3 = 3ull * H * DH;
+  const unsigned long long dims[4] = {(unsigned long long)DH, 3ull * H, (unsigned long long)T, (unsigned long long)B};
+  const unsigned long long strides[3] = {(unsigned long long)DH * 2, d3 * 2, (unsigned long long)T * d3 * 2};
+  const unsigned boxq[4] = {64, 1, TQ, 1}, boxk[4] = {64, 1, TK, 1};
+  CUtensorMap tmQ, tmKV;
+  if (!tma_encode_bf16(&tmQ, qkv, 4, dims, strides, boxq)) return cudaErrorInvalidValue;
+  if (!tma_encode_bf16(&tmKV, qkv, 4, dims, strides, boxk)) return cudaErrorInvalidValue;
+  cudaError_t e = cudaFuncSetAttribute(attn_fwd_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
   if (e != cudaSuccess) return e;
-  dim3 grid((T + AT_BLK - 1) / AT_BLK, B * H);
-  attn_fwd_kernel<DH><<<grid, AT_THREADS, smem, s>>>(qkv, o, lse, T, H, rsqrtf((float)DH));
+  dim3 grid((T + TQ - 1) / TQ, B * H);
+  attn_fwd_tc_kernel<DH><<<grid, 128, C::SMEM, s>>>(tmQ, tmKV, o, lse, T, H, rsqrtf((float)DH), err);
   return cudaGetLastError();
 }
 
-cudaError_t attention_fwd_legacy(const bf16* qkv, bf16* o, float* lse, int B, int T, int H, int dh, cudaStream_t s) {
+
+// ------------------------------------------------------------------------------------------------
+// Backward.  Same structure as the forward: a CTA owns 128 rows (keys for dK/dV, queries for dQ), the other
+// index is swept in blocks of 64; two threads share a row (32 columns of each block each: the backward has
+// no row-wise reduction, so they never need to talk), all products run on tcgen05 and
+// — because the backward has no running maximum — every gradient accumulates in TMEM across the sweep.
+// Probabilities are recomputed from the saved log-sum-exp; delta_i = sum_c dO_ic O_ic.
+// ------------------------------------------------------------------------------------------------
+
+// 64 fp32 values -> bf16 row `tid` of a [128 x 64] K-major tile with 128-byte swizzle
+__device__ __forceinline__ void store_row_swizzled(uint8_t* tile, int tid, const float (&v)[64]) {
+#pragma unroll
+  for (int c8 = 0; c8 < 8; ++c8) {
+    uint4 pk;
+    pk.x = pack_bf16x2(v[8 * c8], v[8 * c8 + 1]);
+    pk.y = pack_bf16x2(v[8 * c8 + 2], v[8 * c8 + 3]);
+    pk.z = pack_bf16x2(v[8 * c8 + 4], v[8 * c8 + 5]);
+    pk.w = pack_bf16x2(v[8 * c8 + 6], v[8 * c8 + 7]);
+    *reinterpret_cast<uint4*>(tile + tid * 128 + ((c8 ^ (tid & 7)) << 4)) = pk;
+  }
+}
+
+// 32 fp32 values -> bf16 columns [32 hf, 32 hf + 32) of row r of the same kind of tile
+__device__ __forceinline__ void store_half_row_swizzled(uint8_t* tile, int r, int hf, const float (&v)[32]) {
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    const int c8 = 4 * hf + c;
+    uint4 pk;
+    pk.x = pack_bf16x2(v[8 * c], v[8 * c + 1]);
+    pk.y = pack_bf16x2(v[8 * c + 2], v[8 * c + 3]);
+    pk.z = pack_bf16x2(v[8 * c + 4], v[8 * c + 5]);
+    pk.w = pack_bf16x2(v[8 * c + 6], v[8 * c + 7]);
+    *reinterpret_cast<uint4*>(tile + r * 128 + ((c8 ^ (r & 7)) << 4)) = pk;
+  }
+}
+
+template <int DH>
+struct BwdCfg {
+  static constexpr int NCH = (DH + 63) / 64;
+  static constexpr int ROW_BYTES = NCH * TQ * 128;      // a 128-row operand (all chunks)
+  static constexpr int BLK_BYTES = NCH * TK * 128;      // a 64-row operand
+  static constexpr int T_BYTES = TQ * 128;              // a [128 x 64] bf16 tile written by the threads
+  // dK/dV: K, V resident; Q, dO double-buffered; P^T, dS^T; lse/delta vectors.  TMEM: S^T, dP^T, dV, dK.
+  static constexpr int SMEM_KV = 2 * ROW_BYTES + 4 * BLK_BYTES + 2 * T_BYTES + 1024 + 2 * 2 * 64 * 4 + 64;
+  static constexpr int TCOLS_KV = (128 + 2 * DH <= 256) ? 256 : 512;
+  // dQ: Q, dO resident; K, V double-buffered; dS.  TMEM: S, dP, dQ.
+  static constexpr int SMEM_Q = 2 * ROW_BYTES + 4 * BLK_BYTES + T_BYTES + 1024 + 64;
+  static constexpr int TCOLS_Q = 256;
+};
+
+template <int DH>
+__global__ void __launch_bounds__(256) attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmRow,   // qkv, 128-row box
+                                                              const __grid_constant__ CUtensorMap tmBlk,   // qkv, 64-row box
+                                                              const __grid_constant__ CUtensorMap tmdO,    // dout, 64-row box
+                                                              const float* __restrict__ lse, const float* __restrict__ delta,
+                                                              bf16* __restrict__ dqkv, int B, int T, int H, float scale,
+                                                              unsigned* err) {
+  using C = BwdCfg<DH>;
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ int abort_flag;
+  __shared__ uint32_t tmem_base_smem;
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t sK = base, sV = sK + C::ROW_BYTES;
+  const uint32_t sQ0 = sV + C::ROW_BYTES, sdO0 = sQ0 + 2 * C::BLK_BYTES;
+  const uint32_t sPT = sdO0 + 2 * C::BLK_BYTES, sdST = sPT + C::T_BYTES;
+  const uint32_t vecs = sdST + C::T_BYTES;                       // lse2[2][64], delta[2][64]
+  const uint32_t bars = vecs + 2 * 2 * 64 * 4;
+  const uint32_t bar_kv = bars, bar_q0 = bars + 8, bar_s = bars + 24, bar_acc = bars + 32, bar_drain = bars + 40;
+  uint8_t* gen = smem_raw + (base - smem_u32(smem_raw));
+  uint8_t* sPT_gen = gen + (sPT - base);
+  uint8_t* sdST_gen = gen + (sdST - base);
+  float* s_lse = reinterpret_cast<float*>(gen + (vecs - base));  // [2][64]
+  float* s_del = s_lse + 128;                                    // [2][64]
+
+  // 256 threads: thread (r, hf) owns row r = tid % 128 and columns [32 hf, 32 hf + 32) of each 64-wide block
+  const int tid = threadIdx.x, warp = tid >> 5, r = tid & 127, hf = tid >> 7;
+  const int kb = blockIdx.x;
+  const int nb = blockIdx.y / H, h = blockIdx.y % H;
+  const int bs = nb % B;
+  const int d = H * DH;
+  const int key = kb * TQ + r;
+  const int nq = (T + TK - 1) / TK;
+  const int q0 = (kb * TQ) / TK;                                 // first query block that can see these keys
+  const float* lse_b = lse + ((size_t)bs * H + h) * T;
+  const float* del_b = delta + ((size_t)nb * H + h) * T;
+
+  if (tid == 0) {
+    abort_flag = 0;
+    mbar_init(bar_kv, 1);
+    mbar_init(bar_q0, 1);
+    mbar_init(bar_q0 + 8, 1);
+    mbar_init(bar_s, 1);
+    mbar_init(bar_acc, 1);
+    mbar_init(bar_drain, 1);
+    fence_mbar_init();
+    tma_prefetch_desc(&tmRow);
+    tma_prefetch_desc(&tmBlk);
+    tma_prefetch_desc(&tmdO);
+  }
+  if (warp == 0) {
+    tmem_alloc(smem_u32(&tmem_base_smem), C::TCOLS_KV);
+    tmem_relinquish();
+  }
+  auto load_vec = [&](int j) {       // lse (in log2 units) and delta of query block j into buffer j&1
+    const int q = j * TK + (tid & 63);
+    if (tid < 64) s_lse[(j & 1) * 64 + tid] = q < T ? lse_b[q] * IL_LOG2E : 0.f;
+    else if (tid < 128) s_del[(j & 1) * 64 + (tid & 63)] = q < T ? del_b[q] : 0.f;
+  };
+  if (q0 < nq) load_vec(q0);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_smem;     // S^T [0,64), dP^T [64,128), dV [128,128+dh), dK [128+dh, 128+2dh)
+  const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+  volatile int* abortp = &abort_flag;
+  constexpr uint32_t idesc_s = make_idesc_bf16(TQ, TK, 0, 0);
+  constexpr uint32_t idesc_g = make_idesc_bf16(TQ, DH, 0, 1);
+  int fail = 0;
+
+  auto load_q = [&](int j) {
+    const int st = (j - q0) & 1;
+    mbar_expect_tx(bar_q0 + 8 * st, 2 * C::BLK_BYTES);
+#pragma unroll
+    for (int c = 0; c < C::NCH; ++c) {
+      tma_load_4d(sQ0 + st * C::BLK_BYTES + c * (TK * 128), &tmBlk, c * 64, h, j * TK, bs, bar_q0 + 8 * st);
+      tma_load_4d(sdO0 + st * C::BLK_BYTES + c * (TK * 128), &tmdO, c * 64, h, j * TK, nb, bar_q0 + 8 * st);
+    }
+  };
+  if (tid == 0) {
+    mbar_expect_tx(bar_kv, 2 * C::ROW_BYTES);
+#pragma unroll
+    for (int c = 0; c < C::NCH; ++c) {
+      tma_load_4d(sK + c * (TQ * 128), &tmRow, c * 64, H + h, kb * TQ, bs, bar_kv);
+      tma_load_4d(sV + c * (TQ * 128), &tmRow, c * 64, 2 * H + h, kb * TQ, bs, bar_kv);
+    }
+    if (q0 < nq) load_q(q0);
+    if (q0 + 1 < nq) load_q(q0 + 1);
+  }
+  const float c2 = scale * IL_LOG2E;
+
+  for (int j = q0; j < nq; ++j) {
+    const int it = j - q0;
+    const int st = it & 1;
+    if (tid == 0) {
+      bool ok = true;
+      if (it == 0) ok = mbar_wait(bar_kv, 0, abortp);
+      ok = ok && mbar_wait(bar_q0 + 8 * st, (uint32_t)(it >> 1) & 1u, abortp);
+      if (!ok) { fail = 1; abort_flag = 1; }
+      tc_fence_after();
+#pragma unroll
+      for (int ks = 0; ks < DH / 16; ++ks) {
+        const uint32_t off_a = (ks >> 2) * (TQ * 128) + (ks & 3) * 32;
+        const uint32_t off_b = st * C::BLK_BYTES + (ks >> 2) * (TK * 128) + (ks & 3) * 32;
+        umma_bf16(tmem_base, make_smem_desc(sK + off_a, 16, 1024), make_smem_desc(sQ0 + off_b, 16, 1024), idesc_s, ks ? 1u : 0u);
+        umma_bf16(tmem_base + 64, make_smem_desc(sV + off_a, 16, 1024), make_smem_desc(sdO0 + off_b, 16, 1024), idesc_s,
+                  ks ? 1u : 0u);
+      }
+      umma_commit(bar_s);
+    }
+    if (j + 1 < nq) load_vec(j + 1);               // visible after this step's barrier
+    if (!mbar_wait(bar_s, (uint32_t)it & 1u, abortp)) { fail = 1; abort_flag = 1; }
+    tc_fence_after();
+    float p[32], ds[32];
+    {
+      uint32_t r0[32], r1[32];
+      tmem_ld_32x32(t_lane + 32 * hf, r0);
+      tmem_ld_32x32(t_lane + 64 + 32 * hf, r1);
+      tmem_ld_wait();
+      const float4* lv = reinterpret_cast<const float4*>(s_lse + st * 64 + 32 * hf);
+      const float4* dv_ = reinterpret_cast<const float4*>(s_del + st * 64 + 32 * hf);
+      const bool diag = (j * TK < kb * TQ + TQ);   // some queries of this block precede some keys of this CTA
+      const bool tail = (j * TK + TK > T);
+      const int qbase = j * TK + 32 * hf;
+#pragma unroll
+      for (int i4 = 0; i4 < 8; ++i4) {
+        const float4 l4 = lv[i4], d4 = dv_[i4];
+        const float ll[4] = {l4.x, l4.y, l4.z, l4.w}, dd[4] = {d4.x, d4.y, d4.z, d4.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int i = 4 * i4 + e;
+          p[i] = ex2_fast(fmaf(__uint_as_float(r0[i]), c2, -ll[e]));
+          ds[i] = __uint_as_float(r1[i]) - dd[e];
+        }
+      }
+      if (diag || tail) {                          // uniform: only blocks on the diagonal or past the sequence end
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+          if (qbase + i < key || qbase + i >= T) p[i] = 0.f;
+      }
+#pragma unroll
+      for (int i = 0; i < 32; ++i) ds[i] *= p[i];
+    }
+    // the previous step's dV/dK products must have finished reading P^T / dS^T before they are overwritten
+    if (it > 0) {
+      if (!mbar_wait(bar_acc, (uint32_t)(it - 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
+      tc_fence_after();
+      if (tid == 0 && j + 1 < nq) load_q(j + 1);   // ... and reading that Q/dO stage
+    }
+    store_half_row_swizzled(sPT_gen, r, hf, p);
+    store_half_row_swizzled(sdST_gen, r, hf, ds);
+    fence_proxy_async();
+    tc_fence_before();
+    if (__syncthreads_or(fail)) { fail = 1; break; }
+    if (tid == 0) {
+      tc_fence_after();
+#pragma unroll
+      for (int ks = 0; ks < TK / 16; ++ks) {
+        const uint32_t off_b = st * C::BLK_BYTES + ks * 2048;                               // MN-major: 16 queries
+        umma_bf16(tmem_base + 128, make_smem_desc(sPT + ks * 32, 16, 1024), make_smem_desc(sdO0 + off_b, TK * 128, 1024),
+                  idesc_g, (it | ks) ? 1u : 0u);
+        umma_bf16(tmem_base + 128 + DH, make_smem_desc(sdST + ks * 32, 16, 1024), make_smem_desc(sQ0 + off_b, TK * 128, 1024),
+                  idesc_g, (it | ks) ? 1u : 0u);
+      }
+      umma_commit(bar_acc);
+    }
+  }
+  const int nit = nq - q0;
+  if (!fail && nit > 0) {
+    if (!mbar_wait(bar_acc, (uint32_t)(nit - 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
+    tc_fence_after();
+  }
+  fail = __syncthreads_or(fail);
+  if (!fail) {
+    bf16* rowp = dqkv + ((size_t)nb * T + key) * (3 * d) + h * DH;
+    {
+      const int which = hf;                          // first half of the threads writes dV, second half dK
+      const uint32_t tcol = t_lane + 128 + which * DH;
+      bf16* dst = rowp + (which == 0 ? 2 * d : d);
+      const float f = which == 0 ? 1.0f : scale;
+#pragma unroll
+      for (int c0 = 0; c0 < DH; c0 += 32) {
+        float v[32];
+        if (c0 + 32 <= DH) {
+          uint32_t rr[32];
+          tmem_ld_32x32(tcol + c0, rr);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = nit > 0 ? __uint_as_float(rr[i]) * f : 0.f;
+        } else {
+          uint32_t rr[16];
+          tmem_ld_32x16(tcol + c0, rr);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 16; ++i) v[i] = nit > 0 ? __uint_as_float(rr[i]) * f : 0.f;
+        }
+        if (key < T) {
+#pragma unroll
+          for (int i = 0; i < 32 && c0 + i < DH; i += 8) {
+            uint4 pk;
+            pk.x = pack_bf16x2(v[i], v[i + 1]);
+            pk.y = pack_bf16x2(v[i + 2], v[i + 3]);
+            pk.z = pack_bf16x2(v[i + 4], v[i + 5]);
+            pk.w = pack_bf16x2(v[i + 6], v[i + 7]);
+            *reinterpret_cast<uint4*>(dst + c0 + i) = pk;
+          }
+        }
+      }
+    }
+  }
+  if (tid == 0) {
+    if (fail && err) atomicExch(err, DEV_TIMEOUT_MMA);
+    umma_commit(bar_drain);
+    int never = 0;
+    mbar_wait(bar_drain, 0, &never);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, C::TCOLS_KV);
+  }
+}
+
+template <int DH>
+__global__ void __launch_bounds__(256) attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmRow,    // qkv, 128-row box
+                                                             const __grid_constant__ CUtensorMap tmBlk,    // qkv, 64-row box
+                                                             const __grid_constant__ CUtensorMap tmdO,     // dout, 128-row box
+                                                             const float* __restrict__ lse, const float* __restrict__ delta,
+                                                             bf16* __restrict__ dqkv, int B, int T, int H, float scale,
+                                                             unsigned* err) {
+  using C = BwdCfg<DH>;
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ int abort_flag;
+  __shared__ uint32_t tmem_base_smem;
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t sQ = base, sdO = sQ + C::ROW_BYTES;
+  const uint32_t sK0 = sdO + C::ROW_BYTES, sV0 = sK0 + 2 * C::BLK_BYTES;
+  const uint32_t sdS = sV0 + 2 * C::BLK_BYTES;
+  const uint32_t bars = sdS + C::T_BYTES;
+  const uint32_t bar_q = bars, bar_kv0 = bars + 8, bar_s = bars + 24, bar_acc = bars + 32, bar_drain = bars + 40;
+  uint8_t* sdS_gen = smem_raw + (sdS - smem_u32(smem_raw));
+
+  // 256 threads: thread (r, hf) owns row r = tid % 128 and columns [32 hf, 32 hf + 32) of each 64-wide block
+  const int tid = threadIdx.x, warp = tid >> 5, r = tid & 127, hf = tid >> 7;
+  const int qb = gridDim.x - 1 - blockIdx.x;
+  const int nb = blockIdx.y / H, h = blockIdx.y % H;
+  const int bs = nb % B;
+  const int d = H * DH;
+  const int row = qb * TQ + r;
+  int nkv = (qb * TQ + TQ + TK - 1) / TK;
+  const int nkv_all = (T + TK - 1) / TK;
+  if (nkv > nkv_all) nkv = nkv_all;
+
+  if (tid == 0) {
+    abort_flag = 0;
+    mbar_init(bar_q, 1);
+    mbar_init(bar_kv0, 1);
+    mbar_init(bar_kv0 + 8, 1);
+    mbar_init(bar_s, 1);
+    mbar_init(bar_acc, 1);
+    mbar_init(bar_drain, 1);
+    fence_mbar_init();
+    tma_prefetch_desc(&tmRow);
+    tma_prefetch_desc(&tmBlk);
+    tma_prefetch_desc(&tmdO);
+  }
+  if (warp == 0) {
+    tmem_alloc(smem_u32(&tmem_base_smem), C::TCOLS_Q);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_smem;     // S [0,64), dP [64,128), dQ [128,128+dh)
+  const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+  volatile int* abortp = &abort_flag;
+  constexpr uint32_t idesc_s = make_idesc_bf16(TQ, TK, 0, 0);
+  constexpr uint32_t idesc_g = make_idesc_bf16(TQ, DH, 0, 1);
+  int fail = 0;
+
+  auto load_kv = [&](int j) {
+    const int st = j & 1;
+    mbar_expect_tx(bar_kv0 + 8 * st, 2 * C::BLK_BYTES);
+#pragma unroll
+    for (int c = 0; c < C::NCH; ++c) {
+      tma_load_4d(sK0 + st * C::BLK_BYTES + c * (TK * 128), &tmBlk, c * 64, H + h, j * TK, bs, bar_kv0 + 8 * st);
+      tma_load_4d(sV0 + st * C::BLK_BYTES + c * (TK * 128), &tmBlk, c * 64, 2 * H + h, j * TK, bs, bar_kv0 + 8 * st);
+    }
+  };
+  if (tid == 0) {
+    mbar_expect_tx(bar_q, 2 * C::ROW_BYTES);
+#pragma unroll
+    for (int c = 0; c < C::NCH; ++c) {
+      tma_load_4d(sQ + c * (TQ * 128), &tmRow, c * 64, h, qb * TQ, bs, bar_q);
+      tma_load_4d(sdO + c * (TQ * 128), &tmdO, c * 64, h, qb * TQ, nb, bar_q);
+    }
+    load_kv(0);
+    if (nkv > 1) load_kv(1);
+  }
+  const float c2 = scale * IL_LOG2E;
+  const float lse2 = row < T ? lse[((size_t)bs * H + h) * T + row] * IL_LOG2E : 0.f;
+  const float del = row < T ? delta[((size_t)nb * H + h) * T + row] : 0.f;
+
+  for (int j = 0; j < nkv; ++j) {
+    const int st = j & 1;
+    if (tid == 0) {
+      bool ok = true;
+      if (j == 0) ok = mbar_wait(bar_q, 0, abortp);
+      ok = ok && mbar_wait(bar_kv0 + 8 * st, (uint32_t)(j >> 1) & 1u, abortp);
+      if (!ok) { fail = 1; abort_flag = 1; }
+      tc_fence_after();
+#pragma unroll
+      for (int ks = 0; ks < DH / 16; ++ks) {
+        const uint32_t off_a = (ks >> 2) * (TQ * 128) + (ks & 3) * 32;
+        const uint32_t off_b = st * C::BLK_BYTES + (ks >> 2) * (TK * 128) + (ks & 3) * 32;
+        umma_bf16(tmem_base, make_smem_desc(sQ + off_a, 16, 1024), make_smem_desc(sK0 + off_b, 16, 1024), idesc_s, ks ? 1u : 0u);
+        umma_bf16(tmem_base + 64, make_smem_desc(sdO + off_a, 16, 1024), make_smem_desc(sV0 + off_b, 16, 1024), idesc_s,
+                  ks ? 1u : 0u);
+      }
+      umma_commit(bar_s);
+    }
+    if (!mbar_wait(bar_s, (uint32_t)j & 1u, abortp)) { fail = 1; abort_flag = 1; }
+    tc_fence_after();
+    float ds[32];
+    {
+      uint32_t r0[32], r1[32];
+      tmem_ld_32x32(t_lane + 32 * hf, r0);
+      tmem_ld_32x32(t_lane + 64 + 32 * hf, r1);
+      tmem_ld_wait();
+      const bool diag = (j * TK + TK - 1 > qb * TQ);
+      const int kbase = j * TK + 32 * hf;
+#pragma unroll
+      for (int i = 0; i < 32; ++i) ds[i] = ex2_fast(fmaf(__uint_as_float(r0[i]), c2, -lse2));
+      if (diag) {                                  // uniform: only blocks on the diagonal
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+          if (kbase + i > row) ds[i] = 0.f;
+      }
+#pragma unroll
+      for (int i = 0; i < 32; ++i) ds[i] *= (__uint_as_float(r1[i]) - del);
+    }
+    if (j > 0) {
+      if (!mbar_wait(bar_acc, (uint32_t)(j - 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
+      tc_fence_after();
+      if (tid == 0 && j + 1 < nkv) load_kv(j + 1);
+    }
+    store_half_row_swizzled(sdS_gen, r, hf, ds);
+    fence_proxy_async();
+    tc_fence_before();
+    if (__syncthreads_or(fail)) { fail = 1; break; }
+    if (tid == 0) {
+      tc_fence_after();
+#pragma unroll
+      for (int ks = 0; ks < TK / 16; ++ks)
+        umma_bf16(tmem_base + 128, make_smem_desc(sdS + ks * 32, 16, 1024),
+                  make_smem_desc(sK0 + st * C::BLK_BYTES + ks * 2048, TK * 128, 1024), idesc_g, (j | ks) ? 1u : 0u);
+      umma_commit(bar_acc);
+    }
+  }
+  if (!fail && nkv > 0) {
+    if (!mbar_wait(bar_acc, (uint32_t)(nkv - 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
+    tc_fence_after();
+  }
+  fail = __syncthreads_or(fail);
+  if (!fail) {
+    bf16* dst = dqkv + ((size_t)nb * T + row) * (3 * d) + h * DH;
+#pragma unroll
+    for (int u = 0; u < DH / 16; ++u) {              // 16-column units, alternating between the two halves
+      if ((u & 1) != hf) continue;
+      const int c0 = u * 16;
+      float v[16];
+      {
+        uint32_t rr[16];
+        tmem_ld_32x16(t_lane + 128 + c0, rr);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(rr[i]) * scale;
+      }
+      if (row < T) {
+#pragma unroll
+        for (int i = 0; i < 16; i += 8) {
+          uint4 pk;
+          pk.x = pack_bf16x2(v[i], v[i + 1]);
+          pk.y = pack_bf16x2(v[i + 2], v[i + 3]);
+          pk.z = pack_bf16x2(v[i + 4], v[i + 5]);
+          pk.w = pack_bf16x2(v[i + 6], v[i + 7]);
+          *reinterpret_cast<uint4*>(dst + c0 + i) = pk;
+        }
+      }
+    }
+  }
+  if (tid == 0) {
+    if (fail && err) atomicExch(err, DEV_TIMEOUT_MMA);
+    umma_commit(bar_drain);
+    int never = 0;
+    mbar_wait(bar_drain, 0, &never);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, C::TCOLS_Q);
+  }
+}
+
+// delta[nb, h, t] = sum_c dO[nb*T+t, h*dh+c] * O[(nb%B)*T+t, h*dh+c].  A thread takes 8 consecutive columns
+// (16 bytes of each operand); the dh/8 threads of a (row, head) sit in one warp and combine by shuffles.
+template <int DH>
+__global__ void __launch_bounds__(256) attn_delta_tc_kernel(const bf16* __restrict__ dout, const bf16* __restrict__ o,
+                                                            float* __restrict__ delta, int NB, int B, int T, int H) {
+  constexpr int TPR = (DH == 80) ? 16 : DH / 8;      // threads per (row, head): a power of two (dh 80: 10 of 16 active)
+  const long long gid = (long long)blockIdx.x * 256 + threadIdx.x;
+  const long long item = gid / TPR;                  // (row, head) index
+  const int part = (int)(gid % TPR);
+  const long long total = (long long)NB * T * H;
+  float s = 0.f;
+  int h = 0;
+  long long row = 0;
+  if (item < total) {
+    h = (int)(item % H);
+    row = item / H;
+    const int nb = (int)(row / T), t = (int)(row % T);
+    if (part * 8 < DH) {
+      const int d = H * DH;
+      const uint4 a = *reinterpret_cast<const uint4*>(dout + (size_t)row * d + h * DH + part * 8);
+      const uint4 c = *reinterpret_cast<const uint4*>(o + ((size_t)(nb % B) * T + t) * d + h * DH + part * 8);
+      const __nv_bfloat162* a2 = reinterpret_cast<const __nv_bfloat162*>(&a);
+      const __nv_bfloat162* c2 = reinterpret_cast<const __nv_bfloat162*>(&c);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float2 x = __bfloat1622float2(a2[i]), y = __bfloat1622float2(c2[i]);
+        s += x.x * y.x + x.y * y.y;
+      }
+    }
+  }
+#pragma unroll
+  for (int off = TPR / 2; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+  if (item < total && part == 0) {
+    const int nb = (int)(row / T), t = (int)(row % T);
+    delta[((size_t)nb * H + h) * T + t] = s;
+  }
+}
+
+template <int DH>
+cudaError_t bwd_tc_launch(const bf16* qkv, const bf16* o, const float* lse, const bf16* dout, bf16* dqkv, float* delta, int NB,
+                          int B, int T, int H, unsigned* err, cudaStream_t s) {
+  using C = BwdCfg<DH>;
+  const unsigned long long d3 = 3ull * H * DH, d1 = (unsigned long long)H * DH;
+  const unsigned long long dims[4] = {(unsigned long long)DH, 3ull * H, (unsigned long long)T, (unsigned long long)B};
+  const unsigned long long strides[3] = {(unsigned long long)DH * 2, d3 * 2, (unsigned long long)T * d3 * 2};
+  const unsigned long long ddims[4] = {(unsigned long long)DH, (unsigned long long)H, (unsigned long long)T, (unsigned long long)NB};
+  const unsigned long long dstrides[3] = {(unsigned long long)DH * 2, d1 * 2, (unsigned long long)T * d1 * 2};
+  const unsigned box128[4] = {64, 1, TQ, 1}, box64[4] = {64, 1, TK, 1};
+  CUtensorMap tmRow, tmBlk, tmdO64, tmdO128;
+  if (!tma_encode_bf16(&tmRow, qkv, 4, dims, strides, box128) || !tma_encode_bf16(&tmBlk, qkv, 4, dims, strides, box64) ||
+      !tma_encode_bf16(&tmdO64, dout, 4, ddims, dstrides, box64) || !tma_encode_bf16(&tmdO128, dout, 4, ddims, dstrides, box128))
+    return cudaErrorInvalidValue;
+  cudaError_t e = cudaFuncSetAttribute(attn_bwd_dkv_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_KV);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(attn_bwd_dq_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_Q);
+  if (e != cudaSuccess) return e;
+  constexpr int TPR = (DH == 80) ? 16 : DH / 8;
+  const long long nthreads = (long long)NB * T * H * TPR;
+  attn_delta_tc_kernel<DH><<<(unsigned)((nthreads + 255) / 256), 256, 0, s>>>(dout, o, delta, NB, B, T, H);
+  dim3 grid((T + TQ - 1) / TQ, NB * H);
+  const float scale = rsqrtf((float)DH);
+  attn_bwd_dkv_tc_kernel<DH><<<grid, 256, C::SMEM_KV, s>>>(tmRow, tmBlk, tmdO64, lse, delta, dqkv, B, T, H, scale, err);
+  attn_bwd_dq_tc_kernel<DH><<<grid, 256, C::SMEM_Q, s>>>(tmRow, tmBlk, tmdO128, lse, delta, dqkv, B, T, H, scale, err);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t attention_fwd(const bf16* qkv, bf16* o, float* lse, int B, int T, int H, int dh, unsigned* err,
+                          cudaStream_t s) {
+  if (((uintptr_t)qkv % 16) || ((uintptr_t)o % 16)) return cudaErrorInvalidValue;
   switch (dh) {
-    case 32: return fwd_launch<32>(qkv, o, lse, B, T, H, s);
-    case 64: return fwd_launch<64>(qkv, o, lse, B, T, H, s);
-    case 80: return fwd_launch<80>(qkv, o, lse, B, T, H, s);
-    case 128: return fwd_launch<128>(qkv, o, lse, B, T, H, s);
+    case 32: return fwd_tc_launch<32>(qkv, o, lse, B, T, H, err, s);
+    case 64: return fwd_tc_launch<64>(qkv, o, lse, B, T, H, err, s);
+    case 80: return fwd_tc_launch<80>(qkv, o, lse, B, T, H, err, s);
+    case 128: return fwd_tc_launch<128>(qkv, o, lse, B, T, H, err, s);
   }
   return cudaErrorInvalidValue;
 }
 
-template <int DH>
-static cudaError_t bwd_launch(const bf16* qkv, const bf16* o, const float* lse, const bf16* dout, bf16* dqkv, float* delta,
-                              int NB, int B, int T, int H, cudaStream_t s) {
-  const int smem_kv = 4 * AT_BLK * (DH + 8) * 2 + 2 * AT_BLK * 4;
-  const int smem_q = 4 * AT_BLK * (DH + 8) * 2;
-  cudaError_t e = cudaFuncSetAttribute(attn_bwd_dkv_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_kv);
-  if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(attn_bwd_dq_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_q);
-  if (e != cudaSuccess) return e;
-  const int nwarps = NB * T * H;
-  attn_delta_kernel<<<(nwarps + 7) / 8, 256, 0, s>>>(dout, o, delta, NB, B, T, H, DH);
-  dim3 grid((T + AT_BLK - 1) / AT_BLK, NB * H);
-  const float scale = rsqrtf((float)DH);
-  attn_bwd_dkv_kernel<DH><<<grid, AT_THREADS, smem_kv, s>>>(qkv, lse, dout, delta, dqkv, B, T, H, scale);
-  attn_bwd_dq_kernel<DH><<<grid, AT_THREADS, smem_q, s>>>(qkv, lse, dout, delta, dqkv, B, T, H, scale);
-  return cudaGetLastError();
-}
-
-cudaError_t attention_bwd_legacy(const bf16* qkv, const bf16* o, const float* lse, const bf16* dout, bf16* dqkv, float* delta,
-                          int NB, int B, int T, int H, int dh, cudaStream_t s) {
+cudaError_t attention_bwd(const bf16* qkv, const bf16* o, const float* lse, const bf16* dout, bf16* dqkv, float* delta,
+                             int NB, int B, int T, int H, int dh, unsigned* err, cudaStream_t s) {
+  if (((uintptr_t)qkv % 16) || ((uintptr_t)dout % 16) || ((uintptr_t)dqkv % 16)) return cudaErrorInvalidValue;
   switch (dh) {
-    case 32: return bwd_launch<32>(qkv, o, lse, dout, dqkv, delta, NB, B, T, H, s);
-    case 64: return bwd_launch<64>(qkv, o, lse, dout, dqkv, delta, NB, B, T, H, s);
-    case 80: return bwd_launch<80>(qkv, o, lse, dout, dqkv, delta, NB, B, T, H, s);
-    case 128: return bwd_launch<128>(qkv, o, lse, dout, dqkv, delta, NB, B, T, H, s);
+    case 32: return bwd_tc_launch<32>(qkv, o, lse, dout, dqkv, delta, NB, B, T, H, err, s);
+    case 64: return bwd_tc_launch<64>(qkv, o, lse, dout, dqkv, delta, NB, B, T, H, err, s);
+    case 80: return bwd_tc_launch<80>(qkv, o, lse, dout, dqkv, delta, NB, B, T, H, err, s);
+    case 128: return bwd_tc_launch<128>(qkv, o, lse, dout, dqkv, delta, NB, B, T, H, err, s);
   }
   return cudaErrorInvalidValue;
 }
 
 }  // namespace il
+

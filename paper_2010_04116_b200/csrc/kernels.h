@@ -46,7 +46,8 @@ cudaError_t lse_finalize(const float* part_max, const float* part_sum, int part_
 cudaError_t adamw(float* p, float* m, float* v, const float* g, __nv_bfloat16* p_bf16, size_t n, size_t n_decay,
                   float lr, float beta1, float beta2, float eps, float wd, float bc1, float bc2, cudaStream_t s);
 
-// Causal attention on packed qkv [B*T, 3d] (Q | K | V, head h at columns h*dh).  dh in {32, 64, 80, 128}.
+// Causal attention on packed qkv [B*T, 3d] (Q | K | V, head h at columns h*dh) on the tcgen05 tensor cores.
+// dh in {32, 64, 80, 128}; pointers 16-byte aligned.
 //   o [B*T, d] bf16, lse [B, H, T] fp32 (natural log of the softmax denominator, scores scaled by 1/sqrt(dh)).
 // err (may be NULL): device word set non-zero if a bounded wait in the kernel expired.
 cudaError_t attention_fwd(const __nv_bfloat16* qkv, __nv_bfloat16* o, float* lse, int B, int T, int H, int dh,
