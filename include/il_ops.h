@@ -43,6 +43,8 @@ typedef struct {
   const float* resid;
   const void* aux; int ld_aux; int aux_rows;
   int accumulate;
+  int split_k;   /* epilogue 4 without accumulate: > 1 splits the contraction over that many work units per
+                    tile and adds the partial sums into C atomically (C must be zero on entry); 0/1 = off */
   const int* targets;
   float* part_max; float* part_sum; int part_ld;
   float* tgt_logit;

@@ -47,6 +47,7 @@ constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + BAR
 struct GemmDev {
   int M, N, K;
   int tiles_m, tiles_n;
+  int split_k, kb_per_split;     // work unit = (tile, k-range); split_k > 1 adds into C with red.add
   void* C;
   int ldc;
   void* C2;
@@ -207,7 +208,11 @@ __device__ __forceinline__ void epilogue_store4(const GemmDev& p, int grow, int 
   } else if constexpr (EPI == EPI_F32_RESID || EPI == EPI_F32) {
     float* c = reinterpret_cast<float*>(p.C) + (size_t)grow * p.ldc + gcol;
     v[0] += e.x; v[1] += e.y; v[2] += e.z; v[3] += e.w;
-    if (vec) {
+    if (EPI == EPI_F32 && p.split_k > 1) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (gcol + j < p.N) atomicAdd(c + j, v[j]);
+    } else if (vec) {
       *reinterpret_cast<float4*>(c) = make_float4(v[0], v[1], v[2], v[3]);
     } else {
 #pragma unroll
@@ -239,8 +244,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   const uint32_t rank = cluster_ctarank();           // 0 = leader of the pair (issues the MMAs)
   const int pair = blockIdx.x >> 1;
   const int num_pairs = gridDim.x >> 1;
-  const int num_tiles = p.tiles_m * p.tiles_n;
-  const int num_kb = (p.K + BK - 1) / BK;
+  const int num_tiles = p.tiles_m * p.tiles_n * p.split_k;    // work units: unit u = (tile u / split_k, k-range u % split_k)
+  const int num_kb_all = (p.K + BK - 1) / BK;
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -276,10 +281,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       bool ok = true;
       for (int t = pair; t < num_tiles && ok; t += num_pairs) {
         int m_blk, n_blk;
-        tile_coords(t, p.tiles_m, p.tiles_n, m_blk, n_blk);
+        tile_coords(t / p.split_k, p.tiles_m, p.tiles_n, m_blk, n_blk);
         const int m0 = m_blk * TILE_M + (int)rank * BM;       // this CTA's 128 rows of A
         const int n0 = n_blk * BN + (int)rank * (BN / 2);     // this CTA's 128 rows of B
-        for (int kb = 0; kb < num_kb; ++kb) {
+        const int kb0 = (t % p.split_k) * p.kb_per_split;
+        const int kb1 = min(num_kb_all, kb0 + p.kb_per_split);
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abortp)) { ok = false; break; }
           const uint32_t sa = smem_base + stage * STAGE_BYTES;
           const uint32_t sb = sa + A_BYTES;
@@ -321,7 +328,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         if (!mbar_wait(acc_empty_bar(as), aphase ^ 1u, abortp)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(as * BN);
-        for (int kb = 0; kb < num_kb; ++kb) {
+        const int kb0 = (t % p.split_k) * p.kb_per_split;
+        const int kb1 = min(num_kb_all, kb0 + p.kb_per_split);
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abortp)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_base + stage * STAGE_BYTES;
@@ -332,7 +341,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             // MN-major: 16 k = two groups of 8 k-rows (1024 B each); 64-element MN chunks 8192 B apart.
             const uint64_t ad = A_MN ? make_smem_desc(sa + k * 2048, 8192, 1024) : make_smem_desc(sa + k * 32, 16, 1024);
             const uint64_t bd = B_MN ? make_smem_desc(sb + k * 2048, 8192, 1024) : make_smem_desc(sb + k * 32, 16, 1024);
-            umma_bf16_pair(d_tmem, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
+            umma_bf16_pair(d_tmem, ad, bd, idesc, (kb > kb0 || k != 0) ? 1u : 0u);
           }
           umma_commit_pair(empty_bar(stage), 3);   // slab reusable in both CTAs once these MMAs have read it
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -360,7 +369,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     bool ok = true;
     for (int t = pair; t < num_tiles && ok; t += num_pairs, ++it) {
       int m_blk, n_blk;
-      tile_coords(t, p.tiles_m, p.tiles_n, m_blk, n_blk);
+      tile_coords(t / p.split_k, p.tiles_m, p.tiles_n, m_blk, n_blk);
       const int as = it & 1;
       const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
       const int row0 = m_blk * TILE_M + (int)rank * BM + q * 32;     // first row of this warp's 32
@@ -399,7 +408,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       } else if constexpr (EPI == EPI_F32_RESID || EPI == EPI_F32) {
         load_f32_chunk(0, pre_f[0]);
       }
-      if (!mbar_wait(acc_full_bar(as), aphase, abortp)) { ok = false; break; }
+      {   // one lane polls the barrier (keeps 255 pollers off the shared-memory pipe the main loop lives on)
+        int got = 1;
+        if (lane == 0) got = mbar_wait(acc_full_bar(as), aphase, abortp) ? 1 : 0;
+        got = __shfl_sync(0xffffffffu, got, 0);
+        if (!got) { ok = false; break; }
+      }
       tc_fence_after();
       const int row = row0 + lane;
       const bool row_ok = row < p.M;
@@ -465,11 +479,16 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
               if (p.bias) b4 = __ldg(reinterpret_cast<const float4*>(p.bias + gcol));
             if constexpr (EPI == EPI_F32_RESID || EPI == EPI_F32) {
               float* cbase = reinterpret_cast<float*>(p.C) + (size_t)(row0 + lrow) * p.ldc + gcol;
+              if (EPI == EPI_F32 && p.split_k > 1) {       // partial sums of a k-range: add into the zeroed output
 #pragma unroll
-              for (int i = 0; i < 8; ++i)
-                *reinterpret_cast<float4*>(cbase + (size_t)(4 * i) * p.ldc) =
-                    make_float4(a[i].x + b4.x + extra[i].x, a[i].y + b4.y + extra[i].y, a[i].z + b4.z + extra[i].z,
-                                a[i].w + b4.w + extra[i].w);
+                for (int i = 0; i < 8; ++i) red_add_f32x4(cbase + (size_t)(4 * i) * p.ldc, a[i]);
+              } else {
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                  *reinterpret_cast<float4*>(cbase + (size_t)(4 * i) * p.ldc) =
+                      make_float4(a[i].x + b4.x + extra[i].x, a[i].y + b4.y + extra[i].y, a[i].z + b4.z + extra[i].z,
+                                  a[i].w + b4.w + extra[i].w);
+              }
             } else {
               uint2 o[8], g[8];
 #pragma unroll
@@ -664,13 +683,23 @@ cudaError_t gemm_launch(const GemmArgs& a, unsigned* err_word, int num_sms, cuda
   p.M = a.M; p.N = a.N; p.K = a.K;
   p.tiles_m = (a.M + TILE_M - 1) / TILE_M;
   p.tiles_n = (a.N + BN - 1) / BN;
+  {
+    // Split the contraction when the tile count leaves most CTA pairs idle (fp32 outputs only; the caller
+    // zeroes C and the partial sums are added with red.global.add).
+    const int num_kb = (a.K + BK - 1) / BK;
+    int split = a.split_k > 1 ? a.split_k : 1;
+    if (a.epilogue != EPI_F32 || a.accumulate) split = 1;
+    if (split > num_kb) split = num_kb;
+    p.kb_per_split = (num_kb + split - 1) / split;
+    p.split_k = (num_kb + p.kb_per_split - 1) / p.kb_per_split;
+  }
   p.C = a.C; p.ldc = a.ldc; p.C2 = a.C2; p.bias = a.bias; p.resid = a.resid;
   p.aux = reinterpret_cast<const bf16*>(a.aux); p.ld_aux = a.ld_aux; p.aux_rows = a.aux_rows > 0 ? a.aux_rows : 1;
   p.accumulate = a.accumulate;
   p.targets = a.targets; p.part_max = a.part_max; p.part_sum = a.part_sum; p.part_ld = a.part_ld;
   p.tgt_logit = a.tgt_logit; p.lse = a.lse; p.scale = a.scale; p.col0 = a.col0;
   p.err = err_word;
-  const long long tiles = (long long)p.tiles_m * p.tiles_n;
+  const long long tiles = (long long)p.tiles_m * p.tiles_n * p.split_k;
   const int pairs = (int)(tiles < num_sms / 2 ? tiles : num_sms / 2);
   const int grid = 2 * pairs;
   kern<<<grid, GEMM_THREADS, SMEM_BYTES, stream>>>(tmA, tmB, p);

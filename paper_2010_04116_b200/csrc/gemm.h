@@ -37,6 +37,8 @@ struct GemmArgs {
   const void* aux;    // EPI_BF16_DGELU: bf16 [aux_rows, ld_aux]
   int ld_aux, aux_rows;
   int accumulate;     // EPI_F32
+  int split_k;        // EPI_F32 without accumulate: > 1 splits K over that many work units per tile; C must be
+                      // zero on entry (partial sums are added atomically).  0/1 = off
   // EPI_LSE / EPI_DZ (vocabulary chunk starting at column col0 of the full vocabulary)
   const int* targets; // [M]
   float* part_max;    // [M, part_ld]  written at column (col0 / 128 + 128-column block)

@@ -30,7 +30,9 @@ using namespace il;
 
 namespace {
 
-constexpr int VOCAB_CHUNK = 4096;   // columns of dZ held at once in the head backward (bf16, stays near L2)
+// Columns of dZ held at once in the head backward (bf16 [Ntok, chunk], L2-sized).  18 tiles of 256 columns:
+// with d_model 1024 the chunk's weight-gradient GEMM then has 72 output tiles for 74 CTA pairs.
+constexpr int VOCAB_CHUNK = 4608;
 
 struct TensorRec {
   std::string name;
@@ -213,6 +215,27 @@ GemmArgs gemm_args(int M, int N, int K, const void* A, int lda, int a_mn, const 
     if (e__ != cudaSuccess) return fail(m, IL_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e__));      \
     (m)->launches++;                                                                                    \
   } while (0)
+
+// Weight-gradient GEMM dW[M,N] = dY^T X over K tokens.  When the output has far fewer 256 x 256 tiles than the
+// GPU has CTA pairs, the token axis is split over several work units per tile (partial sums are added
+// atomically into the zeroed gradient).
+il_status wgrad(il_model* m, int k, int M, int N, int K, const bf16* dY, int ld_dy, const bf16* X, int ld_x, float* dW) {
+  const int tiles = ((M + 255) / 256) * ((N + 255) / 256);
+  const int pairs = m->num_sms / 2;
+  int best = 1;
+  double best_cost = (double)((tiles + pairs - 1) / pairs);
+  for (int s = 2; s <= 4; ++s) {
+    if (K / 64 / s < 16) break;
+    const double cost = (double)((tiles * s + pairs - 1) / pairs) / s;
+    if (cost < best_cost * 0.9) { best_cost = cost; best = s; }
+  }
+  GemmArgs g = gemm_args(M, N, K, dY, ld_dy, 1, X, ld_x, 1, EPI_F32, dW, N);
+  if (best > 1) {
+    IL_CUDA(m, cudaMemsetAsync(dW, 0, (size_t)M * N * sizeof(float), m->streams[k]));
+    g.split_k = best;
+  }
+  return gemm(m, k, g);
+}
 
 il_status alloc_scratch(il_model* m, int s_cap) {
   // grow-only: backward scratch for s_cap stacked gradient streams per component
@@ -737,25 +760,25 @@ il_status component_backward(il_model* m, int k, int s) {
     const float* x_in = (l == 0) ? m->a[k] : m->acts[(size_t)k * m->Lc + l - 1].x_out;
     // ---- MLP: x_out = x_mid + W2 gelu(W1 ln2 + b1) + b2
     IL_K(m, colsum_f32(c.dx, d, m->G + o.b2, N, d, st));
-    IL_TRY(gemm(m, k, gemm_args(d, F, N, c.dxb, d, 1, A.hact, F, 1, EPI_F32, m->G + o.w2, F)));
+    IL_TRY(wgrad(m, k, d, F, N, c.dxb, d, A.hact, F, m->G + o.w2));
     {
       GemmArgs g = gemm_args(R, F, d, c.dxb, d, 0, m->Pb + o.w2, F, 1, EPI_BF16_DGELU, c.dbig, F);
       g.aux = A.hgrad; g.ld_aux = F; g.aux_rows = N;
       IL_TRY(gemm(m, k, g));
     }
     IL_K(m, colsum_bf16(c.dbig, F, m->G + o.b1, N, F, st));
-    IL_TRY(gemm(m, k, gemm_args(F, d, N, c.dbig, F, 1, A.ln2, d, 1, EPI_F32, m->G + o.w1, d)));
+    IL_TRY(wgrad(m, k, F, d, N, c.dbig, F, A.ln2, d, m->G + o.w1));
     IL_TRY(gemm(m, k, gemm_args(R, d, F, c.dbig, F, 0, m->Pb + o.w1, d, 1, EPI_BF16, c.dln, d)));
     IL_K(m, layernorm_bwd_params(c.dln, 0, A.x_mid, A.mean2, A.rstd2, m->G + o.ln2g, m->G + o.ln2b, N, d, st));
     IL_K(m, layernorm_bwd_rows(c.dln, 0, A.x_mid, A.mean2, A.rstd2, m->P + o.ln2g, c.dx, c.dx, c.dxb, R, N, d, st));
     // ---- attention: x_mid = x_in + Wo attn(Wqkv ln1 + bqkv) + bo
     IL_K(m, colsum_f32(c.dx, d, m->G + o.bo, N, d, st));
-    IL_TRY(gemm(m, k, gemm_args(d, d, N, c.dxb, d, 1, A.attn_o, d, 1, EPI_F32, m->G + o.wo, d)));
+    IL_TRY(wgrad(m, k, d, d, N, c.dxb, d, A.attn_o, d, m->G + o.wo));
     IL_TRY(gemm(m, k, gemm_args(R, d, d, c.dxb, d, 0, m->Pb + o.wo, d, 1, EPI_BF16, c.dattn, d)));
     IL_K(m, attention_bwd(A.qkv, A.attn_o, A.lse, c.dattn, c.dqkv, c.delta, s * m->B, m->B, m->T, m->H, m->dh, m->err_word, st));
     m->launches += 2;
     IL_K(m, colsum_bf16(c.dqkv, 3 * d, m->G + o.bqkv, N, 3 * d, st));
-    IL_TRY(gemm(m, k, gemm_args(3 * d, d, N, c.dqkv, 3 * d, 1, A.ln1, d, 1, EPI_F32, m->G + o.wqkv, d)));
+    IL_TRY(wgrad(m, k, 3 * d, d, N, c.dqkv, 3 * d, A.ln1, d, m->G + o.wqkv));
     IL_TRY(gemm(m, k, gemm_args(R, d, 3 * d, c.dqkv, 3 * d, 0, m->Pb + o.wqkv, d, 1, EPI_BF16, c.dln, d)));
     IL_K(m, layernorm_bwd_params(c.dln, 0, x_in, A.mean1, A.rstd1, m->G + o.ln1g, m->G + o.ln1b, N, d, st));
     IL_K(m, layernorm_bwd_rows(c.dln, 0, x_in, A.mean1, A.rstd1, m->P + o.ln1g, c.dx, c.dx, c.dxb, R, N, d, st));
@@ -934,7 +957,7 @@ extern "C" il_status il_op_gemm(const il_gemm_desc* q, unsigned* err_word, void*
   if (!q || !err_word) return IL_ERR_INVALID_ARG;
   GemmArgs g = gemm_args(q->M, q->N, q->K, q->A, q->lda, q->a_mn_major, q->B, q->ldb, q->b_mn_major, q->epilogue, q->C, q->ldc);
   g.C2 = q->C2; g.bias = q->bias; g.resid = q->resid; g.aux = q->aux; g.ld_aux = q->ld_aux; g.aux_rows = q->aux_rows;
-  g.accumulate = q->accumulate; g.targets = q->targets; g.part_max = q->part_max; g.part_sum = q->part_sum;
+  g.accumulate = q->accumulate; g.split_k = q->split_k; g.targets = q->targets; g.part_max = q->part_max; g.part_sum = q->part_sum;
   g.part_ld = q->part_ld; g.tgt_logit = q->tgt_logit; g.lse = q->lse; g.scale = q->scale; g.col0 = q->col0;
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return IL_ERR_CUDA;

@@ -230,3 +230,19 @@ def test_layernorm_forward_backward(rows, d):
                 assert _rel(dg.cpu().numpy(), dgr) < 1e-4
                 assert _rel(db.cpu().numpy(), dbr) < 1e-4
         assert _rel(dxb.float().cpu().numpy(), got.astype(np.float64)) < 3e-3
+
+
+@pytest.mark.parametrize("split", [2, 4])
+def test_gemm_split_k_adds_partial_sums(split):
+    """wgrad layout with the contraction split over several work units per tile (atomic fp32 accumulation)."""
+    rng = np.random.default_rng(split)
+    M, N, K = 300, 264, 4096 + 72
+    At, Ae = _bf16(rng.standard_normal((K, M + 4)))          # MN-major A: memory [K, M], ld padded
+    Bt, Be = _bf16(rng.standard_normal((K, N)))
+    Ct = torch.zeros((M, N), dtype=torch.float32, device=DEV)
+    err = _err_word()
+    il.op_gemm(M, N, K, At, M + 4, 1, Bt, N, 1, 4, err, C_=Ct, ldc=N, split_k=split)
+    torch.cuda.synchronize()
+    assert int(err.item()) == 0
+    ref = Ae[:, :M].T @ Be
+    assert _rel(Ct.cpu().numpy(), ref) < 5e-6      # fp32 accumulation over K = 4168 plus the atomic partial sums
