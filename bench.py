@@ -128,6 +128,21 @@ def oracle_sample(w: wl.Workload, n: int, steps: int, warmup: int, params=None, 
     return ws.ntok / sec, sec, info
 
 
+def max_over_ranks(ms: float, dist, device) -> float:
+    """Step time of the whole job = the slowest replica's (the replicas never exchange data)."""
+    if dist is None:
+        return ms
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_tokens_per_s(tokens_per_rank_step: int, steps: int, world: int, ms: float) -> float:
+    """Whole-job throughput of `world` independent replicas over `steps` steps lasting `ms` (max over ranks)."""
+    return tokens_per_rank_step * steps * max(world, 1) / (ms * 1e-3)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -211,12 +226,7 @@ def main():
         end.record(s0)
         barrier()
         m.sync()
-        ms = start.elapsed_time(end)
-        if dist is not None:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(start.elapsed_time(end), dist, dev)
 
     run_steps(args.warmup, False)
     m.sync()
@@ -234,9 +244,8 @@ def main():
     run_steps(1, True)
     ms_e2e = timed(args.steps, True)
 
-    tokens = w.ntok * args.steps * max(world, 1)
-    value = tokens / (ms * 1e-3)
-    e2e = tokens / (ms_e2e * 1e-3)
+    value = job_tokens_per_s(w.ntok, args.steps, world, ms)
+    e2e = job_tokens_per_s(w.ntok, args.steps, world, ms_e2e)
     flops_tok = model_flops_per_token(w, n)
     peaks = {}
     try:
