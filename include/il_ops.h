@@ -25,7 +25,8 @@ extern "C" {
  * Leading dimensions in elements, multiples of 8; pointers 16-byte aligned.
  * Epilogues (the `epilogue` field):
  *   0 C(bf16) = acc + bias                         1 C(bf16) = gelu_tanh'(pre), C2(bf16) = gelu_tanh(pre), pre = acc + bias
- *   2 C(f32) = resid(f32) + acc + bias             3 C(bf16) = acc * aux[row % aux_rows, col]  (aux_rows >= 32)
+ *   2 C(f32) = resid(f32) + acc + bias             3 C(bf16) = acc * aux[row % aux_rows, col]  (aux_rows >= 32;
+ *                                                     optionally colsum[col] += sum over rows < aux_rows)
  *   4 C(f32) = acc (+ C when accumulate != 0)
  *   5 per-(row, 128-column block) softmax partials: part_max, part_sum [M, part_ld] at block index
  *     col0/128 + block (col0 % 128 == 0), and tgt_logit[row] = acc[row, targets[row] - col0] when that
@@ -42,6 +43,7 @@ typedef struct {
   const float* bias;
   const float* resid;
   const void* aux; int ld_aux; int aux_rows;
+  float* colsum; /* epilogue 3: optional [N] fp32, receives += the column sums of the output over rows < aux_rows */
   int accumulate;
   int split_k;   /* epilogue 4 without accumulate: > 1 splits the contraction over that many work units per
                     tile and adds the partial sums into C atomically (C must be zero on entry); 0/1 = off */

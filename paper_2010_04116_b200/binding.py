@@ -42,7 +42,7 @@ class il_gemm_desc(C.Structure):
                 ("C", C.c_void_p), ("ldc", C.c_int),
                 ("C2", C.c_void_p),
                 ("bias", C.c_void_p), ("resid", C.c_void_p),
-                ("aux", C.c_void_p), ("ld_aux", C.c_int), ("aux_rows", C.c_int),
+                ("aux", C.c_void_p), ("ld_aux", C.c_int), ("aux_rows", C.c_int), ("colsum", C.c_void_p),
                 ("accumulate", C.c_int), ("split_k", C.c_int),
                 ("targets", C.c_void_p),
                 ("part_max", C.c_void_p), ("part_sum", C.c_void_p), ("part_ld", C.c_int),
@@ -313,7 +313,7 @@ class Model:
 
 # ---------------------------------------------------------------------- operator-level calls
 def op_gemm(M, N, K, A, lda, a_mn, B, ldb, b_mn, epilogue, err_word, C_=None, ldc=0, C2=None, bias=None,
-            resid=None, aux=None, ld_aux=0, aux_rows=0, accumulate=0, split_k=0, targets=None, part_max=None,
+            resid=None, aux=None, ld_aux=0, aux_rows=0, colsum=None, accumulate=0, split_k=0, targets=None, part_max=None,
             part_sum=None, part_ld=0, tgt_logit=None, lse=None, scale=0.0, col0=0, stream=None):
     d = il_gemm_desc()
     d.M, d.N, d.K = M, N, K
@@ -323,6 +323,7 @@ def op_gemm(M, N, K, A, lda, a_mn, B, ldb, b_mn, epilogue, err_word, C_=None, ld
     d.C, d.ldc, d.C2 = _ptr(C_), ldc, _ptr(C2)
     d.bias, d.resid = _ptr(bias), _ptr(resid)
     d.aux, d.ld_aux, d.aux_rows = _ptr(aux), ld_aux, aux_rows
+    d.colsum = _ptr(colsum)
     d.accumulate = accumulate
     d.split_k = split_k
     d.targets = _ptr(targets)

@@ -112,24 +112,35 @@ __global__ void __launch_bounds__(128) attn_fwd_tc_kernel(const __grid_constant_
   float m = -INFINITY, l = 0.f;
   const float slack = 8.0f / c2;
 
+  // S_j = Q K_j^T; issued by thread 0 one step ahead (right after the previous block's P V) so that each sweep
+  // step waits for the tensor pipe only once
+  auto issue_s = [&](int j) {
+    const int st = j & 1;
+    if (!mbar_wait(bar_kv0 + 8 * st, (uint32_t)(j >> 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
+    tc_fence_after();
+#pragma unroll
+    for (int ks = 0; ks < DH / 16; ++ks) {
+      const uint64_t ad = make_smem_desc(sQ + (ks >> 2) * (TQ * 128) + (ks & 3) * 32, 16, 1024);
+      const uint64_t bd = make_smem_desc(sK0 + st * C::KV_BYTES + (ks >> 2) * (TK * 128) + (ks & 3) * 32, 16, 1024);
+      umma_bf16(tmem_base, ad, bd, idesc_s, ks ? 1u : 0u);
+    }
+    umma_commit(bar_s);
+  };
+  if (tid == 0) {
+    if (!mbar_wait(bar_q, 0, abortp)) { fail = 1; abort_flag = 1; }
+    issue_s(0);
+  }
+
   for (int j = 0; j < nkv; ++j) {
     const int st = j & 1;
     const uint32_t ph = (uint32_t)j & 1u;
-    if (tid == 0) {
-      bool ok = true;
-      if (j == 0) ok = mbar_wait(bar_q, 0, abortp);
-      ok = ok && mbar_wait(bar_kv0 + 8 * st, (uint32_t)(j >> 1) & 1u, abortp);
-      if (!ok) { fail = 1; abort_flag = 1; }
-      tc_fence_after();
-#pragma unroll
-      for (int ks = 0; ks < DH / 16; ++ks) {
-        const uint64_t ad = make_smem_desc(sQ + (ks >> 2) * (TQ * 128) + (ks & 3) * 32, 16, 1024);
-        const uint64_t bd = make_smem_desc(sK0 + st * C::KV_BYTES + (ks >> 2) * (TK * 128) + (ks & 3) * 32, 16, 1024);
-        umma_bf16(tmem_base, ad, bd, idesc_s, ks ? 1u : 0u);
-      }
-      umma_commit(bar_s);
-    }
     if (!mbar_wait(bar_s, ph, abortp)) { fail = 1; abort_flag = 1; }
+    // the previous block's P V was issued before these scores, so it has landed too: P's buffer, the O
+    // accumulator and the other K/V stage are free
+    if (j > 0) {
+      if (!mbar_wait(bar_o, (uint32_t)(j - 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
+      if (tid == 0 && j + 1 < nkv) load_kv(j + 1);
+    }
     tc_fence_after();
     // ---- softmax of this thread's row over the 64 keys of the block
     uint32_t r0[32], r1[32];
@@ -151,12 +162,6 @@ __global__ void __launch_bounds__(128) attn_fwd_tc_kernel(const __grid_constant_
       mx4[2] = fmaxf(mx4[2], s[i + 2]); mx4[3] = fmaxf(mx4[3], s[i + 3]);
     }
     const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-    // the previous block's P V must have landed before P's buffer is overwritten or O is rescaled
-    if (j > 0) {
-      if (!mbar_wait(bar_o, (uint32_t)(j - 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
-      tc_fence_after();
-      if (tid == 0 && j + 1 < nkv) load_kv(j + 1);            // both MMAs that read that stage have completed
-    }
     if (__any_sync(0xffffffffu, mx > m + slack)) {            // warp-uniform: raise the reference maximum
       const float mn = fmaxf(m, mx);
       const float alpha = ex2_fast((m - mn) * c2);            // 0 on the first block (m = -inf)
@@ -215,6 +220,7 @@ __global__ void __launch_bounds__(128) attn_fwd_tc_kernel(const __grid_constant_
         umma_bf16(tmem_base + 64, ad, bd, idesc_o, (j | ks) ? 1u : 0u);                            // O accumulates in TMEM
       }
       umma_commit(bar_o);
+      if (j + 1 < nkv) issue_s(j + 1);           // every thread has read S_j (barrier above): the buffer is free
     }
   }
   if (!fail && nkv > 0) {
@@ -389,12 +395,20 @@ __global__ void __launch_bounds__(256) attn_bwd_dkv_tc_kernel(const __grid_const
     tmem_alloc(smem_u32(&tmem_base_smem), C::TCOLS_KV);
     tmem_relinquish();
   }
-  auto load_vec = [&](int j) {       // lse (in log2 units) and delta of query block j into buffer j&1
+  // lse (in log2 units) and delta of a query block: fetched from global memory into a register one sweep
+  // step before they are put into shared memory (buffer j&1), two steps before they are used, so that no
+  // step waits on that load
+  auto fetch_vec = [&](int j) -> float {
     const int q = j * TK + (tid & 63);
-    if (tid < 64) s_lse[(j & 1) * 64 + tid] = q < T ? lse_b[q] * IL_LOG2E : 0.f;
-    else if (tid < 128) s_del[(j & 1) * 64 + (tid & 63)] = q < T ? del_b[q] : 0.f;
+    if (j >= nq || q >= T || tid >= 128) return 0.f;
+    return tid < 64 ? lse_b[q] * IL_LOG2E : del_b[q];
   };
-  if (q0 < nq) load_vec(q0);
+  auto put_vec = [&](int j, float v) {
+    if (tid < 64) s_lse[(j & 1) * 64 + tid] = v;
+    else if (tid < 128) s_del[(j & 1) * 64 + (tid & 63)] = v;
+  };
+  if (q0 < nq) put_vec(q0, fetch_vec(q0));
+  float vec_next = fetch_vec(q0 + 1);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -426,27 +440,39 @@ __global__ void __launch_bounds__(256) attn_bwd_dkv_tc_kernel(const __grid_const
   }
   const float c2 = scale * IL_LOG2E;
 
+  // S^T and dP^T of query block j; issued by thread 0 one step ahead (right after the previous block's dV/dK
+  // products) so that each sweep step waits for the tensor pipe only once
+  auto issue_s = [&](int j) {
+    const int it = j - q0, st = it & 1;
+    if (!mbar_wait(bar_q0 + 8 * st, (uint32_t)(it >> 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
+    tc_fence_after();
+#pragma unroll
+    for (int ks = 0; ks < DH / 16; ++ks) {
+      const uint32_t off_a = (ks >> 2) * (TQ * 128) + (ks & 3) * 32;
+      const uint32_t off_b = st * C::BLK_BYTES + (ks >> 2) * (TK * 128) + (ks & 3) * 32;
+      umma_bf16(tmem_base, make_smem_desc(sK + off_a, 16, 1024), make_smem_desc(sQ0 + off_b, 16, 1024), idesc_s, ks ? 1u : 0u);
+      umma_bf16(tmem_base + 64, make_smem_desc(sV + off_a, 16, 1024), make_smem_desc(sdO0 + off_b, 16, 1024), idesc_s,
+                ks ? 1u : 0u);
+    }
+    umma_commit(bar_s);
+  };
+  if (tid == 0 && q0 < nq) {
+    if (!mbar_wait(bar_kv, 0, abortp)) { fail = 1; abort_flag = 1; }
+    issue_s(q0);
+  }
+
   for (int j = q0; j < nq; ++j) {
     const int it = j - q0;
     const int st = it & 1;
-    if (tid == 0) {
-      bool ok = true;
-      if (it == 0) ok = mbar_wait(bar_kv, 0, abortp);
-      ok = ok && mbar_wait(bar_q0 + 8 * st, (uint32_t)(it >> 1) & 1u, abortp);
-      if (!ok) { fail = 1; abort_flag = 1; }
-      tc_fence_after();
-#pragma unroll
-      for (int ks = 0; ks < DH / 16; ++ks) {
-        const uint32_t off_a = (ks >> 2) * (TQ * 128) + (ks & 3) * 32;
-        const uint32_t off_b = st * C::BLK_BYTES + (ks >> 2) * (TK * 128) + (ks & 3) * 32;
-        umma_bf16(tmem_base, make_smem_desc(sK + off_a, 16, 1024), make_smem_desc(sQ0 + off_b, 16, 1024), idesc_s, ks ? 1u : 0u);
-        umma_bf16(tmem_base + 64, make_smem_desc(sV + off_a, 16, 1024), make_smem_desc(sdO0 + off_b, 16, 1024), idesc_s,
-                  ks ? 1u : 0u);
-      }
-      umma_commit(bar_s);
-    }
-    if (j + 1 < nq) load_vec(j + 1);               // visible after this step's barrier
+    if (j + 1 < nq) put_vec(j + 1, vec_next);      // visible after this step's barrier
+    vec_next = fetch_vec(j + 2);
     if (!mbar_wait(bar_s, (uint32_t)it & 1u, abortp)) { fail = 1; abort_flag = 1; }
+    // the previous step's dV/dK products were issued before these scores, so they have landed too: the
+    // P^T / dS^T tiles and the other Q/dO stage are free
+    if (it > 0) {
+      if (!mbar_wait(bar_acc, (uint32_t)(it - 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
+      if (tid == 0 && j + 1 < nq) load_q(j + 1);
+    }
     tc_fence_after();
     float p[32], ds[32];
     {
@@ -478,12 +504,6 @@ __global__ void __launch_bounds__(256) attn_bwd_dkv_tc_kernel(const __grid_const
 #pragma unroll
       for (int i = 0; i < 32; ++i) ds[i] *= p[i];
     }
-    // the previous step's dV/dK products must have finished reading P^T / dS^T before they are overwritten
-    if (it > 0) {
-      if (!mbar_wait(bar_acc, (uint32_t)(it - 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
-      tc_fence_after();
-      if (tid == 0 && j + 1 < nq) load_q(j + 1);   // ... and reading that Q/dO stage
-    }
     store_half_row_swizzled(sPT_gen, r, hf, p);
     store_half_row_swizzled(sdST_gen, r, hf, ds);
     fence_proxy_async();
@@ -500,6 +520,7 @@ __global__ void __launch_bounds__(256) attn_bwd_dkv_tc_kernel(const __grid_const
                   idesc_g, (it | ks) ? 1u : 0u);
       }
       umma_commit(bar_acc);
+      if (j + 1 < nq) issue_s(j + 1);              // every thread has read S^T / dP^T of this step (barrier above)
     }
   }
   const int nit = nq - q0;
@@ -639,25 +660,33 @@ __global__ void __launch_bounds__(256) attn_bwd_dq_tc_kernel(const __grid_consta
   const float lse2 = row < T ? lse[((size_t)bs * H + h) * T + row] * IL_LOG2E : 0.f;
   const float del = row < T ? delta[((size_t)nb * H + h) * T + row] : 0.f;
 
+  // S and dP of key block j; issued by thread 0 one step ahead (right after the previous block's dQ product)
+  auto issue_s = [&](int j) {
+    const int st = j & 1;
+    if (!mbar_wait(bar_kv0 + 8 * st, (uint32_t)(j >> 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
+    tc_fence_after();
+#pragma unroll
+    for (int ks = 0; ks < DH / 16; ++ks) {
+      const uint32_t off_a = (ks >> 2) * (TQ * 128) + (ks & 3) * 32;
+      const uint32_t off_b = st * C::BLK_BYTES + (ks >> 2) * (TK * 128) + (ks & 3) * 32;
+      umma_bf16(tmem_base, make_smem_desc(sQ + off_a, 16, 1024), make_smem_desc(sK0 + off_b, 16, 1024), idesc_s, ks ? 1u : 0u);
+      umma_bf16(tmem_base + 64, make_smem_desc(sdO + off_a, 16, 1024), make_smem_desc(sV0 + off_b, 16, 1024), idesc_s,
+                ks ? 1u : 0u);
+    }
+    umma_commit(bar_s);
+  };
+  if (tid == 0 && nkv > 0) {
+    if (!mbar_wait(bar_q, 0, abortp)) { fail = 1; abort_flag = 1; }
+    issue_s(0);
+  }
+
   for (int j = 0; j < nkv; ++j) {
     const int st = j & 1;
-    if (tid == 0) {
-      bool ok = true;
-      if (j == 0) ok = mbar_wait(bar_q, 0, abortp);
-      ok = ok && mbar_wait(bar_kv0 + 8 * st, (uint32_t)(j >> 1) & 1u, abortp);
-      if (!ok) { fail = 1; abort_flag = 1; }
-      tc_fence_after();
-#pragma unroll
-      for (int ks = 0; ks < DH / 16; ++ks) {
-        const uint32_t off_a = (ks >> 2) * (TQ * 128) + (ks & 3) * 32;
-        const uint32_t off_b = st * C::BLK_BYTES + (ks >> 2) * (TK * 128) + (ks & 3) * 32;
-        umma_bf16(tmem_base, make_smem_desc(sQ + off_a, 16, 1024), make_smem_desc(sK0 + off_b, 16, 1024), idesc_s, ks ? 1u : 0u);
-        umma_bf16(tmem_base + 64, make_smem_desc(sdO + off_a, 16, 1024), make_smem_desc(sV0 + off_b, 16, 1024), idesc_s,
-                  ks ? 1u : 0u);
-      }
-      umma_commit(bar_s);
-    }
     if (!mbar_wait(bar_s, (uint32_t)j & 1u, abortp)) { fail = 1; abort_flag = 1; }
+    if (j > 0) {                                     // issued before these scores: landed, dS and the other K/V stage are free
+      if (!mbar_wait(bar_acc, (uint32_t)(j - 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
+      if (tid == 0 && j + 1 < nkv) load_kv(j + 1);
+    }
     tc_fence_after();
     float ds[32];
     {
@@ -677,11 +706,6 @@ __global__ void __launch_bounds__(256) attn_bwd_dq_tc_kernel(const __grid_consta
 #pragma unroll
       for (int i = 0; i < 32; ++i) ds[i] *= (__uint_as_float(r1[i]) - del);
     }
-    if (j > 0) {
-      if (!mbar_wait(bar_acc, (uint32_t)(j - 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
-      tc_fence_after();
-      if (tid == 0 && j + 1 < nkv) load_kv(j + 1);
-    }
     store_half_row_swizzled(sdS_gen, r, hf, ds);
     fence_proxy_async();
     tc_fence_before();
@@ -693,6 +717,7 @@ __global__ void __launch_bounds__(256) attn_bwd_dq_tc_kernel(const __grid_consta
         umma_bf16(tmem_base + 128, make_smem_desc(sdS + ks * 32, 16, 1024),
                   make_smem_desc(sK0 + st * C::BLK_BYTES + ks * 2048, TK * 128, 1024), idesc_g, (j | ks) ? 1u : 0u);
       umma_commit(bar_acc);
+      if (j + 1 < nkv) issue_s(j + 1);
     }
   }
   if (!fail && nkv > 0) {

@@ -55,6 +55,7 @@ struct GemmDev {
   const float* resid;
   const bf16* aux;
   int ld_aux, aux_rows;
+  float* colsum;                 // EPI_BF16_DGELU: += column sums of the output over rows < aux_rows (or NULL)
   int accumulate;
   const int* targets;
   float* part_max;
@@ -175,6 +176,11 @@ __device__ __forceinline__ void epilogue_store4(const GemmDev& p, int grow, int 
     bf16* c = reinterpret_cast<bf16*>(p.C) + (size_t)grow * p.ldc + gcol;
     if constexpr (EPI == EPI_BF16_DGELU) {
       v[0] *= e.x; v[1] *= e.y; v[2] *= e.z; v[3] *= e.w;
+      if (p.colsum && grow < p.aux_rows) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          if (gcol + j < p.N) atomicAdd(p.colsum + gcol + j, v[j]);
+      }
     }
     float y[4] = {0.f, 0.f, 0.f, 0.f};
     if constexpr (EPI == EPI_BF16_GELU) {
@@ -491,11 +497,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
               }
             } else {
               uint2 o[8], g[8];
+              float4 cs = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
               for (int i = 0; i < 8; ++i) {
                 float x0 = a[i].x + b4.x, x1 = a[i].y + b4.y, x2 = a[i].z + b4.z, x3 = a[i].w + b4.w;
                 if constexpr (EPI == EPI_BF16_DGELU) {
                   x0 *= extra[i].x; x1 *= extra[i].y; x2 *= extra[i].z; x3 *= extra[i].w;
+                  if (row0 + 4 * i + lrow < p.aux_rows) { cs.x += x0; cs.y += x1; cs.z += x2; cs.w += x3; }
                 }
                 if constexpr (EPI == EPI_BF16_GELU) {
                   float y0, y1, y2, y3, d0, d1, d2, d3;
@@ -513,6 +521,15 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
               bf16* cbase = reinterpret_cast<bf16*>(p.C) + (size_t)(row0 + lrow) * p.ldc + gcol;
 #pragma unroll
               for (int i = 0; i < 8; ++i) *reinterpret_cast<uint2*>(cbase + (size_t)(4 * i) * p.ldc) = o[i];
+              if constexpr (EPI == EPI_BF16_DGELU) {
+                if (p.colsum && row0 < p.aux_rows) {     // bias gradient: column sums over the first gradient stream
+                  cs.x += __shfl_xor_sync(0xffffffffu, cs.x, 8);  cs.y += __shfl_xor_sync(0xffffffffu, cs.y, 8);
+                  cs.z += __shfl_xor_sync(0xffffffffu, cs.z, 8);  cs.w += __shfl_xor_sync(0xffffffffu, cs.w, 8);
+                  cs.x += __shfl_xor_sync(0xffffffffu, cs.x, 16); cs.y += __shfl_xor_sync(0xffffffffu, cs.y, 16);
+                  cs.z += __shfl_xor_sync(0xffffffffu, cs.z, 16); cs.w += __shfl_xor_sync(0xffffffffu, cs.w, 16);
+                  if (lane < 8) red_add_f32x4(p.colsum + gcol, cs);
+                }
+              }
               if constexpr (EPI == EPI_BF16_GELU) {
                 bf16* c2base = reinterpret_cast<bf16*>(p.C2) + (size_t)(row0 + lrow) * p.ldc + gcol;
 #pragma unroll
@@ -671,6 +688,7 @@ cudaError_t gemm_launch(const GemmArgs& a, unsigned* err_word, int num_sms, cuda
   if (a.epilogue == EPI_BF16_DGELU && (!a.aux || a.aux_rows < 32 || (a.ld_aux % 8) || ((uintptr_t)a.aux % 16)))
     return cudaErrorInvalidValue;
   if (a.bias && ((uintptr_t)a.bias % 16)) return cudaErrorInvalidValue;
+  if (a.colsum && (a.epilogue != EPI_BF16_DGELU || ((uintptr_t)a.colsum % 16))) return cudaErrorInvalidValue;
   if (a.epilogue == EPI_LSE && (!a.targets || !a.part_max || !a.part_sum || !a.tgt_logit || (a.col0 % (BN / 2))))
     return cudaErrorInvalidValue;
   if (a.epilogue == EPI_DZ && (!a.targets || !a.lse)) return cudaErrorInvalidValue;
@@ -695,6 +713,7 @@ cudaError_t gemm_launch(const GemmArgs& a, unsigned* err_word, int num_sms, cuda
   }
   p.C = a.C; p.ldc = a.ldc; p.C2 = a.C2; p.bias = a.bias; p.resid = a.resid;
   p.aux = reinterpret_cast<const bf16*>(a.aux); p.ld_aux = a.ld_aux; p.aux_rows = a.aux_rows > 0 ? a.aux_rows : 1;
+  p.colsum = a.colsum;
   p.accumulate = a.accumulate;
   p.targets = a.targets; p.part_max = a.part_max; p.part_sum = a.part_sum; p.part_ld = a.part_ld;
   p.tgt_logit = a.tgt_logit; p.lse = a.lse; p.scale = a.scale; p.col0 = a.col0;

@@ -36,6 +36,8 @@ struct GemmArgs {
   const float* resid; // EPI_F32_RESID: [M, ldc] fp32
   const void* aux;    // EPI_BF16_DGELU: bf16 [aux_rows, ld_aux]
   int ld_aux, aux_rows;
+  float* colsum;      // EPI_BF16_DGELU: [N] fp32, += column sums of the (unrounded) output over rows < aux_rows;
+                      // NULL = off.  Used for the bias gradient of the layer that produced aux.
   int accumulate;     // EPI_F32
   int split_k;        // EPI_F32 without accumulate: > 1 splits K over that many work units per tile; C must be
                       // zero on entry (partial sums are added atomically).  0/1 = off

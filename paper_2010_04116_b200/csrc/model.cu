@@ -764,9 +764,9 @@ il_status component_backward(il_model* m, int k, int s) {
     {
       GemmArgs g = gemm_args(R, F, d, c.dxb, d, 0, m->Pb + o.w2, F, 1, EPI_BF16_DGELU, c.dbig, F);
       g.aux = A.hgrad; g.ld_aux = F; g.aux_rows = N;
+      g.colsum = m->G + o.b1;                 // FC1 bias gradient: column sums of the first gradient stream
       IL_TRY(gemm(m, k, g));
     }
-    IL_K(m, colsum_bf16(c.dbig, F, m->G + o.b1, N, F, st));
     IL_TRY(wgrad(m, k, F, d, N, c.dbig, F, A.ln2, d, m->G + o.w1));
     IL_TRY(gemm(m, k, gemm_args(R, d, F, c.dbig, F, 0, m->Pb + o.w1, d, 1, EPI_BF16, c.dln, d)));
     IL_K(m, layernorm_bwd_params(c.dln, 0, A.x_mid, A.mean2, A.rstd2, m->G + o.ln2g, m->G + o.ln2b, N, d, st));
@@ -956,7 +956,7 @@ static il_status op_status(cudaError_t e) {
 extern "C" il_status il_op_gemm(const il_gemm_desc* q, unsigned* err_word, void* stream) {
   if (!q || !err_word) return IL_ERR_INVALID_ARG;
   GemmArgs g = gemm_args(q->M, q->N, q->K, q->A, q->lda, q->a_mn_major, q->B, q->ldb, q->b_mn_major, q->epilogue, q->C, q->ldc);
-  g.C2 = q->C2; g.bias = q->bias; g.resid = q->resid; g.aux = q->aux; g.ld_aux = q->ld_aux; g.aux_rows = q->aux_rows;
+  g.C2 = q->C2; g.bias = q->bias; g.resid = q->resid; g.aux = q->aux; g.ld_aux = q->ld_aux; g.aux_rows = q->aux_rows; g.colsum = q->colsum;
   g.accumulate = q->accumulate; g.split_k = q->split_k; g.targets = q->targets; g.part_max = q->part_max; g.part_sum = q->part_sum;
   g.part_ld = q->part_ld; g.tgt_logit = q->tgt_logit; g.lse = q->lse; g.scale = q->scale; g.col0 = q->col0;
   int dev = 0, sms = 0;

@@ -104,11 +104,13 @@ def test_gemm_multiply_epilogue_with_stacked_rows():
     Ht, He = _bf16(rng.standard_normal((rows, N)))
     Ct = torch.zeros((M, N), dtype=torch.bfloat16, device=DEV)
     err = _err_word()
-    il.op_gemm(M, N, K, At, K, 0, Wt, N, 1, 3, err, C_=Ct, ldc=N, aux=Ht, ld_aux=N, aux_rows=rows)
+    cs = torch.zeros(N, dtype=torch.float32, device=DEV)
+    il.op_gemm(M, N, K, At, K, 0, Wt, N, 1, 3, err, C_=Ct, ldc=N, aux=Ht, ld_aux=N, aux_rows=rows, colsum=cs)
     torch.cuda.synchronize()
     assert int(err.item()) == 0
     ref = (Ae @ We) * np.tile(He, (s, 1))
     assert _rel(Ct.float().cpu().numpy(), ref) < 3e-3
+    assert _rel(cs.cpu().numpy(), ref[:rows].sum(axis=0)) < 1e-5      # bias gradient from the first stream only
 
 
 @pytest.mark.parametrize("V", [512, 1000, 50257])
