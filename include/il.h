@@ -118,7 +118,10 @@ il_status il_get_boundary(il_model* m, int k, float* host, size_t count);
 /* Bytes of device memory obtained so far, and kernels launched since creation. */
 il_status il_stats(const il_model* m, long long* device_bytes, long long* kernel_launches);
 /* Device time of the GEMM kernels launched since the last reset, measured with CUDA events on
- * their own streams when profiling is switched on (adds event records; off by default). */
+ * their own streams when profiling is switched on (adds event records; off by default).
+ * enable = 1: events only (with several component streams busy a kernel's interval includes its wait for
+ * SMs); enable = 2: additionally every GEMM runs alone on the GPU (the other streams wait for it and it
+ * for them), so the intervals are kernel durations — slower steps, for measurement only. */
 il_status il_profile(il_model* m, int enable);
 il_status il_profile_read(il_model* m, double* gemm_ms, long long* gemm_launches, double* gemm_flops);
 /* Host-only helper (no device needed): the gradient streams component k carries under the n-wise rule

@@ -292,8 +292,9 @@ class Model:
         self._ck(self.L.il_stats(self._h, C.byref(b), C.byref(l)))
         return b.value, l.value
 
-    def profile(self, enable: bool):
-        self._ck(self.L.il_profile(self._h, 1 if enable else 0))
+    def profile(self, enable):
+        """0/False off, 1/True events around each GEMM, 2 the same with each GEMM alone on the GPU."""
+        self._ck(self.L.il_profile(self._h, int(enable)))
 
     def profile_read(self):
         ms, n, fl = C.c_double(0), C.c_longlong(0), C.c_double(0)

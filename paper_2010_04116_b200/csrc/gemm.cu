@@ -18,7 +18,7 @@
 // Operands may be K-major or MN-major in global memory (forward: K/K, dgrad: K/MN, wgrad: MN/MN); the
 // major-ness goes into the TMA box shape, the shared-memory descriptor and the instruction descriptor.
 // Ragged M/N/K edges rely on TMA zero fill for loads and on bounds checks in the epilogue.
-// No TMA load uses cluster multicast.  Every wait is bounded; on expiry the CTA sets the error word, and
+// Every CTA issues its own TMA loads (none is shared across a cluster).  Every wait is bounded; on expiry the CTA sets the error word, and
 // both CTAs meet at a cluster barrier before they return.
 #include <cstdio>
 #include <mutex>

@@ -98,7 +98,7 @@ struct il_model {
   std::vector<void*> allocs;
   long long bytes, launches;
   // profiling
-  bool prof;
+  int prof;                           // 0 off, 1 events around each GEMM, 2 the same with the GEMM alone on the GPU
   std::vector<ProfRec> prof_recs;
   std::vector<cudaEvent_t> prof_pool;
   std::string err;
@@ -183,6 +183,15 @@ il_status gemm(il_model* m, int k, const GemmArgs& g) {
       (i == 0 ? rec.a : rec.b) = e;
     }
     rec.flops = 2.0 * g.M * g.N * (double)g.K;
+    if (m->prof == 2) {
+      // exclusive timing: nothing else of this model runs while the GEMM does, so the event pair measures the
+      // kernel and not its wait for SMs held by other components' streams
+      for (int j = 0; j < m->K; ++j)
+        if (j != k) {
+          IL_CUDA(m, cudaEventRecord(m->ev_join[j], m->streams[j]));
+          IL_CUDA(m, cudaStreamWaitEvent(st, m->ev_join[j], 0));
+        }
+    }
     IL_CUDA(m, cudaEventRecord(rec.a, st));
   }
   cudaError_t e = gemm_launch(g, m->err_word, m->num_sms, st);
@@ -191,6 +200,9 @@ il_status gemm(il_model* m, int k, const GemmArgs& g) {
                 g.M, g.N, g.K, g.epilogue, cudaGetErrorString(e));
   if (m->prof) {
     IL_CUDA(m, cudaEventRecord(rec.b, st));
+    if (m->prof == 2)
+      for (int j = 0; j < m->K; ++j)
+        if (j != k) IL_CUDA(m, cudaStreamWaitEvent(m->streams[j], rec.b, 0));
     m->prof_recs.push_back(rec);
   }
   m->launches++;
@@ -299,7 +311,7 @@ extern "C" il_status il_create(int K, int Lc, int d, int H, int F, int V, int n,
   m->ntok_max = opt->max_batch * opt->max_seq;
   m->ln_eps = opt->ln_eps > 0 ? opt->ln_eps : 1e-5f;
   m->step = 0; m->bytes = 0; m->launches = 0; m->s_cap = 0;
-  m->prof = false; m->batch_set = false; m->bwd_done = false;
+  m->prof = 0; m->batch_set = false; m->bwd_done = false;
   m->B = m->T = m->ntok = 0;
   m->P = m->G = m->M1 = m->M2 = nullptr; m->Pb = nullptr;
   *out = m;   // returned even on failure below so that il_last_error/il_destroy work
@@ -898,7 +910,7 @@ extern "C" il_status il_profile(il_model* m, int enable) {
   IL_CUDA(m, cudaDeviceSynchronize());
   for (auto& r : m->prof_recs) { m->prof_pool.push_back(r.a); m->prof_pool.push_back(r.b); }
   m->prof_recs.clear();
-  m->prof = enable != 0;
+  m->prof = enable == 2 ? 2 : (enable != 0 ? 1 : 0);
   return IL_OK;
 }
 
