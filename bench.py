@@ -31,6 +31,14 @@ sys.path.insert(0, ROOT)
 import workloads as wl  # noqa: E402
 
 
+# DRAM bytes per algorithmic flop of the GEMM kernel, from one ncu capture (dram__bytes_read.sum +
+# dram__bytes_write.sum over 400 consecutive GEMM launches of the cfg4-2x1 step, whose launch shapes are cfg4's;
+# profiles/gemm_dram_traffic_cfg4_shapes.md).  Traffic grows with the flops of a launch at fixed shapes, so the
+# per-launch figure of another step mix is this ratio times that mix's flops per launch.  Set to None whenever
+# gemm.cu changes after the capture.
+GEMM_DRAM_BYTES_PER_FLOP = 1.0901e-3
+
+
 def model_flops_per_token(w: wl.Workload, n: int) -> float:
     """Algorithmic flops per token of one n-wise step: every contraction the method defines, counted once
     (forward, one wgrad per matrix, one dgrad per distinct gradient stream); recomputation is not counted."""
@@ -281,7 +289,11 @@ def main():
                                       "gemm_share_of_step": gemm_ms / ms if ms > 0 else None,
                                       "note": "events on the launch streams during the timed steps; intervals overlap "
                                               "across the component streams and include waiting for SMs"},
-                     "traffic": None},
+                     "traffic": (GEMM_DRAM_BYTES_PER_FLOP * x_flops / max(x_launches, 1)
+                                 if GEMM_DRAM_BYTES_PER_FLOP and w.name.startswith("cfg4") else None),
+                     "traffic_note": "DRAM bytes per launch = measured bytes/flop of the same launch shapes (ncu, "
+                                     "cfg4-2x1) x this run's flops per launch; algorithmic operand+output bytes are "
+                                     "of the same size (no re-reads)"},
         "model_flops": {"per_token_mflop": flops_tok / 1e6, "step_tflop": flops_tok * w.ntok / 1e12,
                         "tflops_per_gpu": per_gpu_tf, "frac_of_burst_peak": per_gpu_tf / peak_burst,
                         "frac_of_sustained_peak": per_gpu_tf / peak_sus, "burst_peak": peak_burst},
