@@ -75,6 +75,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
     if (globaltimer_ns() - t0 > limit_ns) return false;
+    __nanosleep(128);      // long waits (an idle role, a peer still busy) should not burn issue slots and power
   }
 }
 
