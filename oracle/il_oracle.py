@@ -289,14 +289,36 @@ def head_losses(P, tokens, targets, K: int, Lc: int, H: int) -> List[float]:
     return [head_loss(a[k + 1], targets, P, k, False)[0] for k in range(K)]
 
 
+def head_weight(k: int, h: int, n: int, K: int, rule: str) -> float:
+    """Weight of head h's gradient in the update of component k's parameters (0-based, k <= h <= k+n-1).
+
+    "sum"  : every head whose window covers the component counts once (the reading this build targets).
+    "far"  : the paper's main-text rule (Sec. 3): module k is updated from L_{c_{k+N-1}} alone; the window is
+             clamped at the last head, which makes N = number of modules end-to-end training of the final loss.
+    "mean" : the variant of the paper's Transformer experiments (Sec. 3, App. B.3): the mean of the
+             gradients from the module's own head and from head k+N-1.
+    """
+    far = min(k + n - 1, K - 1)
+    if rule == "sum":
+        return 1.0
+    if rule == "far":
+        return 1.0 if h == far else 0.0
+    if rule == "mean":
+        return 0.5 * (h == k) + 0.5 * (h == far)
+    raise ValueError("rule must be 'sum', 'far' or 'mean'")
+
+
 def nwise_gradients(P, tokens: np.ndarray, targets: np.ndarray, K: int, Lc: int, H: int, n: int,
-                    head_weights: Optional[Sequence[float]] = None):
+                    head_weights: Optional[Sequence[float]] = None, rule: str = "sum"):
     """One n-wise step's losses and parameter "gradients" (Sec. 3, Fig. 2).
 
     For every head h (0-based here) its loss is back-propagated through the head
     and then through components h, h-1, ..., max(h-n+1, 0); the gradient is dropped
     at the input of the last of these (the stop at the component boundary).  Each
-    head is a separate backward pass and all contributions are summed.
+    head is a separate backward pass; the parameter gradients it leaves in component k
+    enter the result with weight head_weight(k, h, n, K, rule) (all 1 for rule "sum").
+    Head parameters always receive their own loss's gradient with weight 1; the
+    embeddings belong to component 0.
     head_weights (default all 1) scales each head's loss before back-propagation.
     """
     if not (1 <= n <= K):
@@ -314,10 +336,22 @@ def nwise_gradients(P, tokens: np.ndarray, targets: np.ndarray, K: int, Lc: int,
         dx = da * wgt
         lowest = max(h - n + 1, 0)
         for k in range(h, lowest - 1, -1):
-            dx = component_bwd(dx, caches[k], P, k, B, T, H, G)
-        if lowest == 0:
-            embed_bwd(dx, tokens, P, G)
-        # else: dx is the gradient at a stopped boundary and is discarded.
+            wk = head_weight(k, h, n, K, rule)
+            if wk == 1.0:
+                dx = component_bwd(dx, caches[k], P, k, B, T, H, G)
+            else:
+                Gk: Dict[str, np.ndarray] = {}
+                dx_in = component_bwd(dx, caches[k], P, k, B, T, H, Gk)
+                if k == 0:
+                    embed_bwd(dx_in, tokens, P, Gk)
+                if wk != 0.0:
+                    for name, val in Gk.items():
+                        G[name] = G[name] + wk * val if name in G else wk * val
+                dx = dx_in
+                continue
+            if k == 0:
+                embed_bwd(dx, tokens, P, G)
+        # below `lowest` dx is the gradient at a stopped boundary and is discarded.
     for name in P:
         if name not in G:
             G[name] = np.zeros(P[name].shape, dtype=F64)

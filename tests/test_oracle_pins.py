@@ -407,3 +407,70 @@ def test_generators_are_seeded_and_shaped():
     w4 = wl.CONFIGS["cfg4"]
     per_block = sum(int(np.prod(s)) for nme, _, _, s in wl.tensor_specs(w4) if nme.startswith("c0.l0."))
     assert per_block == 12 * w4.d ** 2 + 13 * w4.d
+
+
+# ------------------------------------------------------------------ the paper's own head weightings
+
+def _rule_window_loss(P, tok, tgt, w, k, n, rule):
+    """Independent formula: the scalar whose plain derivative w.r.t. component k's parameters the rule asks for."""
+    L = orc.head_losses(P, tok, tgt, w.K, w.Lc, w.H)
+    far = min(k + n - 1, w.K - 1)
+    if rule == "far":
+        return L[far]
+    return 0.5 * L[k] + 0.5 * L[far]
+
+
+@pytest.mark.parametrize("rule", ["far", "mean"])
+@pytest.mark.parametrize("n", [2, 3])
+def test_paper_rules_finite_differences(rule, n):
+    """Sec. 3: module k updated from L_{k+N-1} ("far"), or from the mean of L_k and L_{k+N-1} ("mean")."""
+    w = TINY
+    P, tok, tgt = _setup(w)
+    _, G = orc.nwise_gradients(P, tok, tgt, w.K, w.Lc, w.H, n, rule=rule)
+    rng = np.random.default_rng(100 + n)
+    for name, comp, is_head, shape in wl.tensor_specs(w):
+        size = int(np.prod(shape))
+        for _ in range(2):
+            flat = int(rng.integers(0, size))
+            idx = np.unravel_index(flat, shape)
+            if name == "wte":
+                idx = (int(tok.reshape(-1)[flat % tok.size]), idx[1])
+            if is_head:
+                fn = lambda: orc.head_losses(P, tok, tgt, w.K, w.Lc, w.H)[comp]
+            else:
+                fn = lambda: _rule_window_loss(P, tok, tgt, w, comp, n, rule)
+            fd = _fd(P, name, idx, fn)
+            g = G[name][idx]
+            assert abs(fd - g) / max(abs(fd), abs(g), 1e-7) < 1e-6, (name, idx, fd, g)
+
+
+def test_paper_rules_relations():
+    w = TINY2
+    P, tok, tgt = _setup(w)
+    specs = wl.tensor_specs(w)
+    G = {(r, n): orc.nwise_gradients(P, tok, tgt, w.K, w.Lc, w.H, n, rule=r)[1]
+         for r in ("sum", "far", "mean") for n in (1, 2, w.K)}
+    for name, comp, is_head, _ in specs:
+        # n = 1: the three rules coincide (local learning)
+        assert np.array_equal(G[("far", 1)][name], G[("sum", 1)][name])
+        assert np.array_equal(G[("mean", 1)][name], G[("sum", 1)][name])
+        # head parameters never depend on the rule
+        if is_head:
+            assert np.array_equal(G[("far", 2)][name], G[("sum", 2)][name])
+            continue
+        # n = 2: the mean of the two heads is half their sum, except in the top component (one head only)
+        if comp < w.K - 1:
+            assert np.allclose(G[("mean", 2)][name], 0.5 * G[("sum", 2)][name], rtol=1e-12, atol=1e-15), name
+        else:
+            assert np.allclose(G[("mean", 2)][name], G[("sum", 2)][name], rtol=1e-12, atol=1e-15), name
+    # "far" with n = K is end-to-end training of the final loss alone (Sec. 3: N = number of modules)
+    Pt = {k: torch.tensor(v, dtype=torch.float64, requires_grad=True) for k, v in P.items()}
+    tt = torch.tensor(tok.reshape(-1), dtype=torch.long)
+    yy = torch.tensor(tgt.reshape(-1), dtype=torch.long)
+    x = Pt["wte"][tt] + Pt["wpe"][torch.arange(w.T).repeat(w.B)]
+    x = _torch_forward_from(Pt, x, 0, w.K, w)
+    u = Fnn.layer_norm(x, (w.d,), Pt[f"head{w.K - 1}.ln.g"], Pt[f"head{w.K - 1}.ln.b"], eps=1e-5)
+    Fnn.cross_entropy(Fnn.linear(u, Pt[f"head{w.K - 1}.w"]), yy).backward()
+    for name, comp, is_head, _ in specs:
+        if not is_head:
+            assert np.allclose(G[("far", w.K)][name], Pt[name].grad.numpy(), rtol=1e-9, atol=1e-13), name
