@@ -73,6 +73,15 @@ il_status il_destroy(il_model* m);
 /* Change n (1..K) between steps. */
 il_status il_set_n(il_model* m, int n);
 
+/* Which heads update the parameters of component k (Sec. 3).  Every rule uses the same windows (head h reaches
+ * components h .. h-n+1); they differ in the weight of head h in component k's parameter gradient:
+ *   IL_RULE_SUM  (default) every head whose window covers k, weight 1 (n = K: backprop of the summed losses);
+ *   IL_RULE_FAR  the paper's main-text rule: head min(k+n-1, K-1) alone (n = K: end-to-end on the last loss);
+ *   IL_RULE_MEAN the variant of the paper's Transformer experiments: mean of heads k and min(k+n-1, K-1).
+ * Head parameters always get their own loss's gradient.  Weighted rules need n <= 8. */
+enum { IL_RULE_SUM = 0, IL_RULE_FAR = 1, IL_RULE_MEAN = 2 };
+il_status il_set_rule(il_model* m, int rule);
+
 /* Parameter registry.  Order and names: "wte" [V,d], "wpe" [max_seq,d] (component 0: the first
  * module holds the input projection, App. B.3), then per component k and layer l
  * "c{k}.l{l}.{ln1.g,ln1.b,attn.wqkv,attn.bqkv,attn.wo,attn.bo,ln2.g,ln2.b,mlp.w1,mlp.b1,mlp.w2,mlp.b2}",

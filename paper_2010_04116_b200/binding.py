@@ -65,7 +65,7 @@ def lib() -> C.CDLL:
     vp, i, f, sz = C.c_void_p, C.c_int, C.c_float, C.c_size_t
     sig = {
         "il_create": [i, i, i, i, i, i, i, C.POINTER(il_options), C.POINTER(vp)],
-        "il_destroy": [vp], "il_set_n": [vp, i],
+        "il_destroy": [vp], "il_set_n": [vp, i], "il_set_rule": [vp, i],
         "il_tensor_info": [vp, i, C.POINTER(C.c_char_p), C.POINTER(i), C.POINTER(i), C.POINTER(i),
                            C.POINTER(C.c_longlong)],
         "il_set_param": [vp, i, vp, sz], "il_get_param": [vp, i, vp, sz], "il_get_grad": [vp, i, vp, sz],
@@ -228,6 +228,12 @@ class Model:
         m = np.ascontiguousarray(m, dtype=np.float32)
         v = np.ascontiguousarray(v, dtype=np.float32)
         self._ck(self.L.il_set_opt_state(self._h, self.index[name], m.ctypes.data, v.ctypes.data, step))
+
+    RULES = {"sum": 0, "far": 1, "mean": 2}
+
+    def set_rule(self, rule: str):
+        """'sum' (default), 'far' (the paper's main-text rule) or 'mean' (its Transformer variant)."""
+        self._ck(self.L.il_set_rule(self._h, self.RULES[rule]))
 
     def set_n(self, n: int):
         self._ck(self.L.il_set_n(self._h, n))

@@ -331,6 +331,45 @@ cudaError_t add_convert(const float* a, const float* b, float* out_f32, bf16* ou
   return cudaGetLastError();
 }
 
+struct LinComb { const float4* x[4]; float w[4]; int count; int accumulate; };
+
+__global__ void lincomb_convert_kernel(LinComb c, float4* out_f32, uint2* __restrict__ out_bf16, size_t n4) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+    float4 v = c.accumulate ? out_f32[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      if (j < c.count) {
+        const float4 a = c.x[j][i];
+        v.x += c.w[j] * a.x; v.y += c.w[j] * a.y; v.z += c.w[j] * a.z; v.w += c.w[j] * a.w;
+      }
+    out_f32[i] = v;
+    if (out_bf16) {
+      uint2 o;
+      o.x = pack_bf16x2(v.x, v.y);
+      o.y = pack_bf16x2(v.z, v.w);
+      out_bf16[i] = o;
+    }
+  }
+}
+
+cudaError_t lincomb_convert(const float* const* x, const float* w, int count, int accumulate, float* out_f32, bf16* out_bf16,
+                            size_t n, cudaStream_t s) {
+  if (count < 1 || count > 4 || !out_f32) return cudaErrorInvalidValue;
+  LinComb c;
+  for (int j = 0; j < 4; ++j) {
+    c.x[j] = reinterpret_cast<const float4*>(j < count ? x[j] : x[0]);
+    c.w[j] = j < count ? w[j] : 0.f;
+  }
+  c.count = count;
+  c.accumulate = accumulate;
+  const size_t n4 = n / 4;
+  int blocks = ceil_div(n4, 256);
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks < 1) blocks = 1;
+  lincomb_convert_kernel<<<blocks, 256, 0, s>>>(c, reinterpret_cast<float4*>(out_f32), reinterpret_cast<uint2*>(out_bf16), n4);
+  return cudaGetLastError();
+}
+
 cudaError_t f32_to_bf16(const float* in, bf16* out, size_t n, cudaStream_t s) {
   return add_convert(in, nullptr, nullptr, out, n, s);
 }

@@ -35,6 +35,10 @@ cudaError_t colsum_f32(const float* y, int ld, float* out, int rows, int cols, c
 // out_f32 = a + (b ? b : 0); out_bf16 (optional) = bf16 copy.   n elements (multiple of 4).
 cudaError_t add_convert(const float* a, const float* b, float* out_f32, __nv_bfloat16* out_bf16, size_t n,
                         cudaStream_t s);
+// out = (accumulate ? out : 0) + sum_{i<count} w[i] * x[i]   (count <= 4, host arrays of device pointers / weights);
+// out_bf16 (optional) = bf16 copy of the result.
+cudaError_t lincomb_convert(const float* const* x, const float* w, int count, int accumulate, float* out_f32,
+                            __nv_bfloat16* out_bf16, size_t n, cudaStream_t s);
 cudaError_t f32_to_bf16(const float* in, __nv_bfloat16* out, size_t n, cudaStream_t s);
 
 // Merge per-tile online-softmax partials: lse[r] = log sum_t exp(pm[r,t]) * ps[r,t];

@@ -62,6 +62,7 @@ struct ProfRec { cudaEvent_t a, b; double flops; };
 
 struct il_model {
   int K, Lc, d, H, F, V, n, dh;
+  int rule;                           // IL_RULE_*: which heads update a component's parameters
   int device, num_sms;
   int max_batch, max_seq, ntok_max;
   float ln_eps;
@@ -170,6 +171,14 @@ int s_cap_for(int K, int n) {
   size_t s = 1;
   for (int k = 0; k < K; ++k) s = std::max(s, terms_of(k, K, n).size());
   return (int)s;
+}
+
+// weight of head h's gradient in the parameter update of component k (k <= h <= min(k+n-1, K-1))
+float rule_weight(int rule, int k, int h, int n, int K) {
+  const int far = k + n - 1 < K - 1 ? k + n - 1 : K - 1;
+  if (rule == IL_RULE_FAR) return h == far ? 1.0f : 0.0f;
+  if (rule == IL_RULE_MEAN) return 0.5f * (h == k) + 0.5f * (h == far);
+  return 1.0f;
 }
 
 il_status gemm(il_model* m, int k, const GemmArgs& g) {
@@ -310,7 +319,7 @@ extern "C" il_status il_create(int K, int Lc, int d, int H, int F, int V, int n,
   m->max_batch = opt->max_batch; m->max_seq = opt->max_seq;
   m->ntok_max = opt->max_batch * opt->max_seq;
   m->ln_eps = opt->ln_eps > 0 ? opt->ln_eps : 1e-5f;
-  m->step = 0; m->bytes = 0; m->launches = 0; m->s_cap = 0;
+  m->rule = IL_RULE_SUM; m->step = 0; m->bytes = 0; m->launches = 0; m->s_cap = 0;
   m->prof = 0; m->batch_set = false; m->bwd_done = false;
   m->B = m->T = m->ntok = 0;
   m->P = m->G = m->M1 = m->M2 = nullptr; m->Pb = nullptr;
@@ -517,8 +526,19 @@ extern "C" il_status il_set_n(il_model* m, int n) {
   if (n < 1 || n > m->K) return fail(m, IL_ERR_INVALID_ARG, "n=%d outside [1, %d]", n, m->K);
   IL_CUDA(m, cudaSetDevice(m->device));
   IL_CUDA(m, cudaDeviceSynchronize());
-  IL_TRY(alloc_scratch(m, s_cap_for(m->K, n)));
+  IL_TRY(alloc_scratch(m, m->rule == IL_RULE_SUM ? s_cap_for(m->K, n) : n));
   m->n = n;
+  return IL_OK;
+}
+
+extern "C" il_status il_set_rule(il_model* m, int rule) {
+  IL_TRY(check_model(m));
+  if (rule != IL_RULE_SUM && rule != IL_RULE_FAR && rule != IL_RULE_MEAN) return fail(m, IL_ERR_INVALID_ARG, "unknown rule %d", rule);
+  if (m->n > 8 && rule != IL_RULE_SUM) return fail(m, IL_ERR_INVALID_ARG, "weighted rules support n <= 8");
+  IL_CUDA(m, cudaSetDevice(m->device));
+  IL_CUDA(m, cudaDeviceSynchronize());
+  IL_TRY(alloc_scratch(m, rule == IL_RULE_SUM ? s_cap_for(m->K, m->n) : m->n));
+  m->rule = rule;
   return IL_OK;
 }
 
@@ -822,31 +842,83 @@ extern "C" il_status il_backward_nwise(il_model* m) {
     }
     IL_TRY(head_backward(m, k));
   }
-  // components from the top down; component k needs the pass-down of component k+1 when any stream crosses
-  std::vector<int> above;   // termination levels of the streams of component k+1
-  for (int k = K - 1; k >= 0; --k) {
-    cudaStream_t st = m->streams[k];
-    const std::vector<int> terms = terms_of(k, K, n);
-    const int s = (int)terms.size();
-    bool needs_above = false;
-    for (int j = 0; j < s; ++j) {
-      int src = -1;
-      for (size_t q = 0; q < above.size(); ++q)
-        if (above[q] == terms[j]) src = (int)q;
-      if (src >= 0 && !needs_above) {
-        IL_CUDA(m, cudaStreamWaitEvent(st, m->ev_bwd[k + 1], 0));
-        needs_above = true;
+  if (m->rule == IL_RULE_SUM) {
+    // components from the top down; component k needs the pass-down of component k+1 when any stream crosses
+    std::vector<int> above;   // termination levels of the streams of component k+1
+    for (int k = K - 1; k >= 0; --k) {
+      cudaStream_t st = m->streams[k];
+      const std::vector<int> terms = terms_of(k, K, n);
+      const int s = (int)terms.size();
+      bool needs_above = false;
+      for (int j = 0; j < s; ++j) {
+        int src = -1;
+        for (size_t q = 0; q < above.size(); ++q)
+          if (above[q] == terms[j]) src = (int)q;
+        if (src >= 0 && !needs_above) {
+          IL_CUDA(m, cudaStreamWaitEvent(st, m->ev_bwd[k + 1], 0));
+          needs_above = true;
+        }
+        const float* passed = src >= 0 ? m->cs[k + 1].dx + (size_t)src * slice : nullptr;
+        IL_K(m, add_convert(m->hs[k].ghead, passed, m->cs[k].dx + (size_t)j * slice, m->cs[k].dxb + (size_t)j * slice, slice, st));
       }
-      const float* passed = src >= 0 ? m->cs[k + 1].dx + (size_t)src * slice : nullptr;
-      IL_K(m, add_convert(m->hs[k].ghead, passed, m->cs[k].dx + (size_t)j * slice, m->cs[k].dxb + (size_t)j * slice, slice, st));
+      IL_TRY(component_backward(m, k, s));
+      if (k == 0) {
+        IL_K(m, embed_bwd(m->tokens, m->cs[0].dx, m->G + m->off_wte, m->G + m->off_wpe, N, m->T, d, m->V, st));
+        m->launches++;
+      }
+      IL_CUDA(m, cudaEventRecord(m->ev_bwd[k], st));
+      above = terms;
     }
-    IL_TRY(component_backward(m, k, s));
-    if (k == 0) {
-      IL_K(m, embed_bwd(m->tokens, m->cs[0].dx, m->G + m->off_wte, m->G + m->off_wpe, N, m->T, d, m->V, st));
-      m->launches++;
+  } else {
+    // Weighted rules: component k carries slot 0 = sum_h W(k,h) g^(h) (drives every parameter gradient) and one
+    // slot per head that continues below k (all crossing heads but the one with h = k+n-1); the pass-down of a
+    // head is taken from its own slot of component k+1.
+    std::vector<int> above_heads;     // heads in slots 1.. of component k+1, ascending
+    for (int k = K - 1; k >= 0; --k) {
+      cudaStream_t st = m->streams[k];
+      const int hi = k + n - 1 < K - 1 ? k + n - 1 : K - 1;
+      auto grad_of = [&](int h) -> const float* {      // gradient of head h at the output of component k
+        if (h == k) return m->hs[k].ghead;
+        for (size_t q = 0; q < above_heads.size(); ++q)
+          if (above_heads[q] == h) return m->cs[k + 1].dx + (size_t)(q + 1) * slice;
+        return nullptr;
+      };
+      if (hi > k) IL_CUDA(m, cudaStreamWaitEvent(st, m->ev_bwd[k + 1], 0));
+      // slot 0: the weighted combination
+      {
+        const float* xs[8];
+        float ws[8];
+        int cnt = 0;
+        for (int h = k; h <= hi; ++h) {
+          const float wgt = rule_weight(m->rule, k, h, n, K);
+          if (wgt == 0.0f) continue;
+          xs[cnt] = grad_of(h);
+          if (!xs[cnt]) return fail(m, IL_ERR_STATE, "internal: gradient stream of head %d missing at component %d", h, k);
+          ws[cnt++] = wgt;
+        }
+        for (int c0 = 0; c0 < cnt; c0 += 4) {
+          const int c = cnt - c0 < 4 ? cnt - c0 : 4;
+          IL_K(m, lincomb_convert(xs + c0, ws + c0, c, c0 > 0, m->cs[k].dx, c0 + 4 >= cnt ? m->cs[k].dxb : nullptr, slice, st));
+        }
+      }
+      // slots 1..: heads that continue below this component
+      std::vector<int> mine;
+      if (k > 0)
+        for (int h = k; h <= hi; ++h)
+          if (h < k + n - 1) mine.push_back(h);
+      for (size_t q = 0; q < mine.size(); ++q) {
+        const float* src = grad_of(mine[q]);
+        if (!src) return fail(m, IL_ERR_STATE, "internal: gradient stream of head %d missing at component %d", mine[q], k);
+        IL_K(m, add_convert(src, nullptr, m->cs[k].dx + (q + 1) * slice, m->cs[k].dxb + (q + 1) * slice, slice, st));
+      }
+      IL_TRY(component_backward(m, k, 1 + (int)mine.size()));
+      if (k == 0) {
+        IL_K(m, embed_bwd(m->tokens, m->cs[0].dx, m->G + m->off_wte, m->G + m->off_wpe, N, m->T, d, m->V, st));
+        m->launches++;
+      }
+      IL_CUDA(m, cudaEventRecord(m->ev_bwd[k], st));
+      above_heads = mine;
     }
-    IL_CUDA(m, cudaEventRecord(m->ev_bwd[k], st));
-    above = terms;
   }
   m->bwd_done = true;
   return IL_OK;

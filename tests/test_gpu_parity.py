@@ -16,16 +16,18 @@ LOSS_RTOL = 1e-3
 GRAD_RTOL = 2e-2
 
 
-def _check_step(w, n, check_boundaries=True, adamw=False):
+def _check_step(w, n, check_boundaries=True, adamw=False, rule="sum"):
     P = wl.draw_params(w)
     tok, tgt = wl.draw_tokens(w)
     m = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, n, w.B, w.T)
     try:
         m.set_params(P)
+        if rule != "sum":
+            m.set_rule(rule)
         m.train_step(tok, tgt)
         losses = m.get_losses()
         m.sync()
-        ol, OG = orc.nwise_gradients(P, tok, tgt, w.K, w.Lc, w.H, n)
+        ol, OG = orc.nwise_gradients(P, tok, tgt, w.K, w.Lc, w.H, n, rule=rule)
         assert np.all(np.abs(losses - np.array(ol)) <= LOSS_RTOL * np.abs(np.array(ol))), (losses, ol)
         if check_boundaries:
             a, _ = orc.forward_all(P, tok, w.K, w.Lc, w.H)
@@ -75,6 +77,14 @@ def test_four_components_all_n(n):
     """K = 4 exercises every stream pattern: dropped, passed-down and stacked gradient streams."""
     w = wl.Workload("k4", K=4, Lc=1, d=128, H=2, F=256, V=1000, T=96, B=3, n=n, zipf=True)
     _check_step(w, n)
+
+
+@pytest.mark.parametrize("rule", ["far", "mean"])
+@pytest.mark.parametrize("n", [1, 2, 3, 4])
+def test_paper_head_weightings(rule, n):
+    """The paper's own rules (Sec. 3): update from head k+N-1 alone, or from the mean of heads k and k+N-1."""
+    w = wl.Workload("k4r", K=4, Lc=1, d=128, H=2, F=256, V=1000, T=96, B=3, n=n, zipf=True)
+    _check_step(w, n, check_boundaries=False, rule=rule)
 
 
 def test_gpt2_small_width_single_sequence():
