@@ -138,6 +138,16 @@ il_status il_profile_read(il_model* m, double* gemm_ms, long long* gemm_launches
  * k are grouped by that level.  Writes the distinct levels, descending, to terms[0..*count) (terms may be
  * NULL; it needs room for min(n, K) ints).  *count is the number of stacked backward passes of k. */
 il_status il_nwise_streams(int K, int n, int k, int* terms, int* count);
+/* Host-only: the paper's time-per-batch model of synchronous depthwise model parallelism (Sec. 3.1):
+ * A sequential accelerators (one module each), M micro-batches per mini-batch, N the n-wise parameter
+ * (N = 1 local learning, N >= A end-to-end / GPipe), micro-batch cost c(M) = c0 + c1 / M.
+ *   M = 1: 2N c;  M = 2 or A >= 2N-1: (N+1) M c;  otherwise (2+A-N) M c + 2 (2N-A-1) c.
+ * *out is in the unit of c0 and c1 (the paper fits c0 = 0.025 s, c1 = 1.279 s to its Transformer runs).  It
+ * models accelerators that idle while gradients travel; the single-GPU step of this library has no such idle
+ * time, so this is a planning aid for the multi-device placement, not a prediction of il_* step times. */
+il_status il_time_per_batch(int A, int M, int N, double c0, double c1, double* out);
+/* The power of two M in [1, 2^max_log2] that minimises il_time_per_batch (App. C of the paper). */
+il_status il_optimal_microbatches(int A, int N, double c0, double c1, int max_log2, int* M_out);
 const char* il_last_error(const il_model* m); /* library-owned, valid until the next call on m */
 const char* il_status_string(il_status s);
 

@@ -81,6 +81,8 @@ def lib() -> C.CDLL:
         "il_profile": [vp, i],
         "il_profile_read": [vp, C.POINTER(C.c_double), C.POINTER(C.c_longlong), C.POINTER(C.c_double)],
         "il_nwise_streams": [i, i, i, C.POINTER(i), C.POINTER(i)],
+        "il_time_per_batch": [i, i, i, C.c_double, C.c_double, C.POINTER(C.c_double)],
+        "il_optimal_microbatches": [i, i, C.c_double, C.c_double, i, C.POINTER(i)],
         "il_op_gemm": [C.POINTER(il_gemm_desc), vp, vp],
         "il_op_attention_fwd": [vp, vp, vp, i, i, i, i, vp],
         "il_op_attention_bwd": [vp, vp, vp, vp, vp, vp, i, i, i, i, i, vp],
@@ -111,6 +113,22 @@ def nwise_streams(K: int, n: int, k: int) -> List[int]:
     if st != IL_OK:
         raise ILError(st, "il_nwise_streams")
     return [terms[i] for i in range(cnt.value)]
+
+
+def time_per_batch(A: int, M: int, N: int, c0: float, c1: float) -> float:
+    out = C.c_double(0)
+    st = lib().il_time_per_batch(A, M, N, c0, c1, C.byref(out))
+    if st != IL_OK:
+        raise ILError(st, "il_time_per_batch")
+    return out.value
+
+
+def optimal_microbatches(A: int, N: int, c0: float, c1: float, max_log2: int = 10) -> int:
+    out = C.c_int(0)
+    st = lib().il_optimal_microbatches(A, N, c0, c1, max_log2, C.byref(out))
+    if st != IL_OK:
+        raise ILError(st, "il_optimal_microbatches")
+    return out.value
 
 
 def _ptr(t) -> Optional[int]:

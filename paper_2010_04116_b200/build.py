@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libil.so")
-SOURCES = ["gemm.cu", "elementwise.cu", "attention.cu", "model.cu", "noalloc.cu"]
+SOURCES = ["gemm.cu", "elementwise.cu", "attention.cu", "model.cu", "noalloc.cu", "timing.cu"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC"]
 

@@ -92,6 +92,15 @@ def test_gpt2_medium_shape_full_size(n):
     _check_against_golden("cfg4", n)
 
 
+def test_2p7b_shape_full_size():
+    """2.7B-shaped model (32 layers in 8 components, d 2560, seq 2048, batch 4), n = 2: about 110 GB on the device."""
+    _check_against_golden("cfg5", 2)
+    for m_ in _models.values():
+        m_.close()
+    _models.clear()
+    torch.cuda.empty_cache()
+
+
 def test_sweep_invariants_on_device_full_size():
     """Head gradients do not depend on n; the top component's gradient does not depend on n; with n = 1
     component k's gradient is that of its own head only, so n = 2 differs from it for every k < K-1."""
