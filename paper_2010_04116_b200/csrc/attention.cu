@@ -301,20 +301,7 @@ cudaError_t fwd_tc_launch(const bf16* qkv, bf16* o, float* lse, int B, int T, in
 // Probabilities are recomputed from the saved log-sum-exp; delta_i = sum_c dO_ic O_ic.
 // ------------------------------------------------------------------------------------------------
 
-// 64 fp32 values -> bf16 row `tid` of a [128 x 64] K-major tile with 128-byte swizzle
-__device__ __forceinline__ void store_row_swizzled(uint8_t* tile, int tid, const float (&v)[64]) {
-#pragma unroll
-  for (int c8 = 0; c8 < 8; ++c8) {
-    uint4 pk;
-    pk.x = pack_bf16x2(v[8 * c8], v[8 * c8 + 1]);
-    pk.y = pack_bf16x2(v[8 * c8 + 2], v[8 * c8 + 3]);
-    pk.z = pack_bf16x2(v[8 * c8 + 4], v[8 * c8 + 5]);
-    pk.w = pack_bf16x2(v[8 * c8 + 6], v[8 * c8 + 7]);
-    *reinterpret_cast<uint4*>(tile + tid * 128 + ((c8 ^ (tid & 7)) << 4)) = pk;
-  }
-}
-
-// 32 fp32 values -> bf16 columns [32 hf, 32 hf + 32) of row r of the same kind of tile
+// 32 fp32 values -> bf16 columns [32 hf, 32 hf + 32) of row r of a [128 x 64] K-major tile with 128-byte swizzle
 __device__ __forceinline__ void store_half_row_swizzled(uint8_t* tile, int r, int hf, const float (&v)[32]) {
 #pragma unroll
   for (int c = 0; c < 4; ++c) {

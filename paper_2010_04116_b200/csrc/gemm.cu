@@ -20,7 +20,6 @@
 // Ragged M/N/K edges rely on TMA zero fill for loads and on bounds checks in the epilogue.
 // Every CTA issues its own TMA loads (none is shared across a cluster).  Every wait is bounded; on expiry the CTA sets the error word, and
 // both CTAs meet at a cluster barrier before they return.
-#include <cstdio>
 #include <mutex>
 
 #include "common.cuh"
