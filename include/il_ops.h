@@ -30,7 +30,7 @@ extern "C" {
  *   4 C(f32) = acc (+ C when accumulate != 0)
  *   5 per-(row, 128-column block) softmax partials: part_max, part_sum [M, part_ld] at block index
  *     col0/128 + block (col0 % 128 == 0), and tgt_logit[row] = acc[row, targets[row] - col0] when that
- *     column is in range
+ *     column is in range; when C is not NULL, also C(bf16) = acc (the logits, ldc a multiple of 8)
  *   6 C(bf16) = (exp(acc - lse[row]) - [col + col0 == targets[row]]) * scale
  * (0,1) supports epilogues 0, 3, 4; (1,1) supports 4; (0,0) supports all. */
 typedef struct {

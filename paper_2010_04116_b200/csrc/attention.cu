@@ -6,13 +6,14 @@
 // that are not a multiple of 64 are all handled by the tensor map's bounds (zero fill).  Per key block:
 //   S = Q K^T        tcgen05.mma (M128 N64, both operands K-major in shared memory) -> TMEM columns [0, 64)
 //   softmax          thread r owns query row r: tcgen05.ld its 64 scores, running max / sum in registers
-//                    (no cross-lane reduction), P = exp2(...) rounded to bf16 and written to shared memory in
-//                    the K-major 128-byte-swizzled layout the next MMA expects
-//   O += P V         tcgen05.mma (M128 N=dh, A = P K-major, B = V MN-major), accumulated in TMEM columns
+//                    (no cross-lane reduction), P = exp2(...) rounded to bf16, packed in pairs and stored back
+//                    over the first 32 of the score columns (tcgen05.st)
+//   O += P V         tcgen05.mma (M128 N=dh, A = P read from TMEM, B = V MN-major), accumulated in TMEM columns
 //                    [64, 64+dh).  The reference maximum of a row is raised only when a block exceeds it by a
 //                    factor 2^8, so the accumulator is rescaled (tcgen05.ld / st) rarely.
-// A CTA runs these phases one after the other; several CTAs are resident per SM (128 threads, 64-112 KB of
+// A CTA runs these phases one after the other; several CTAs are resident per SM (128 threads, 64-144 KB of
 // shared memory, 128-256 TMEM columns each), which is what overlaps one CTA's softmax with another's MMAs.
+// K and V come through a ring of TMA stages filled two or more sweep steps ahead.
 // The T x T score matrix is never stored.  Every wait is bounded.
 #include "common.cuh"
 #include "kernels.h"
@@ -31,9 +32,9 @@ struct FwdCfg {
   static constexpr int NCH = (DH + 63) / 64;            // 64-column chunks of the head dimension
   static constexpr int Q_BYTES = NCH * TQ * 128;
   static constexpr int KV_BYTES = NCH * TK * 128;
-  static constexpr int P_BYTES = TQ * 128;
+  static constexpr int NST = (DH <= 64) ? 3 : 2;               // K/V ring depth: as deep as keeps three (dh <= 64) or two CTAs per SM
   static constexpr int TCOLS = (64 + DH <= 128) ? 128 : 256;   // 64 score columns + the O accumulator
-  static constexpr int SMEM = Q_BYTES + 4 * KV_BYTES + P_BYTES + 1024 + 64;
+  static constexpr int SMEM = Q_BYTES + NST * 2 * KV_BYTES + 1024 + 128;
 };
 
 template <int DH>
@@ -41,17 +42,16 @@ __global__ void __launch_bounds__(128) attn_fwd_tc_kernel(const __grid_constant_
                                                           const __grid_constant__ CUtensorMap tmKV, bf16* __restrict__ o,
                                                           float* __restrict__ lse, int T, int H, float scale, unsigned* err) {
   using C = FwdCfg<DH>;
+  constexpr int NST = C::NST;
   extern __shared__ uint8_t smem_raw[];
   __shared__ int abort_flag;
   __shared__ uint32_t tmem_base_smem;
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t sQ = base;
-  const uint32_t sK0 = sQ + C::Q_BYTES;                       // two K stages, then two V stages
-  const uint32_t sV0 = sK0 + 2 * C::KV_BYTES;
-  const uint32_t sP = sV0 + 2 * C::KV_BYTES;
-  const uint32_t bars = sP + C::P_BYTES;
-  const uint32_t bar_q = bars, bar_kv0 = bars + 8, bar_s = bars + 24, bar_o = bars + 32, bar_drain = bars + 40;
-  uint8_t* sP_gen = smem_raw + (sP - smem_u32(smem_raw));
+  const uint32_t sK0 = sQ + C::Q_BYTES;                       // the K stages, then the V stages
+  const uint32_t sV0 = sK0 + NST * C::KV_BYTES;
+  const uint32_t bars = sV0 + NST * C::KV_BYTES;
+  const uint32_t bar_q = bars, bar_s = bars + 8, bar_o = bars + 16, bar_drain = bars + 24, bar_kv0 = bars + 32;
 
   const int tid = threadIdx.x, warp = tid >> 5;
   const int qb = gridDim.x - 1 - blockIdx.x;                  // longest sweeps first
@@ -65,8 +65,7 @@ __global__ void __launch_bounds__(128) attn_fwd_tc_kernel(const __grid_constant_
   if (tid == 0) {
     abort_flag = 0;
     mbar_init(bar_q, 1);
-    mbar_init(bar_kv0, 1);
-    mbar_init(bar_kv0 + 8, 1);
+    for (int s = 0; s < NST; ++s) mbar_init(bar_kv0 + 8 * s, 1);
     mbar_init(bar_s, 1);
     mbar_init(bar_o, 1);
     mbar_init(bar_drain, 1);
@@ -81,7 +80,7 @@ __global__ void __launch_bounds__(128) attn_fwd_tc_kernel(const __grid_constant_
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem_base = tmem_base_smem;                  // scores at columns [0, 64), O at [64, 64 + dh)
+  const uint32_t tmem_base = tmem_base_smem;                  // scores at columns [0, 64) (then P packed in [0, 32)), O at [64, 64 + dh)
   const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
   volatile int* abortp = &abort_flag;
   constexpr uint32_t idesc_s = make_idesc_bf16(TQ, TK, 0, 0);
@@ -89,7 +88,7 @@ __global__ void __launch_bounds__(128) attn_fwd_tc_kernel(const __grid_constant_
   int fail = 0;
 
   auto load_kv = [&](int j) {
-    const int st = j & 1;
+    const int st = j % NST;
     mbar_expect_tx(bar_kv0 + 8 * st, 2 * C::KV_BYTES);
 #pragma unroll
     for (int c = 0; c < C::NCH; ++c) {
@@ -101,8 +100,8 @@ __global__ void __launch_bounds__(128) attn_fwd_tc_kernel(const __grid_constant_
     mbar_expect_tx(bar_q, C::Q_BYTES);
 #pragma unroll
     for (int c = 0; c < C::NCH; ++c) tma_load_4d(sQ + c * (TQ * 128), &tmQ, c * 64, h, qb * TQ, b, bar_q);
-    load_kv(0);
-    if (nkv > 1) load_kv(1);
+    for (int i = 0; i < NST; ++i)
+      if (i < nkv) load_kv(i);
   }
 
   const float c2 = scale * IL_LOG2E;
@@ -115,8 +114,8 @@ __global__ void __launch_bounds__(128) attn_fwd_tc_kernel(const __grid_constant_
   // S_j = Q K_j^T; issued by thread 0 one step ahead (right after the previous block's P V) so that each sweep
   // step waits for the tensor pipe only once
   auto issue_s = [&](int j) {
-    const int st = j & 1;
-    if (!mbar_wait(bar_kv0 + 8 * st, (uint32_t)(j >> 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
+    const int st = j % NST;
+    if (!mbar_wait(bar_kv0 + 8 * st, (uint32_t)(j / NST) & 1u, abortp)) { fail = 1; abort_flag = 1; }
     tc_fence_after();
 #pragma unroll
     for (int ks = 0; ks < DH / 16; ++ks) {
@@ -132,14 +131,14 @@ __global__ void __launch_bounds__(128) attn_fwd_tc_kernel(const __grid_constant_
   }
 
   for (int j = 0; j < nkv; ++j) {
-    const int st = j & 1;
+    const int st = j % NST;
     const uint32_t ph = (uint32_t)j & 1u;
     if (!mbar_wait(bar_s, ph, abortp)) { fail = 1; abort_flag = 1; }
-    // the previous block's P V was issued before these scores, so it has landed too: P's buffer, the O
-    // accumulator and the other K/V stage are free
+    // the previous block's P V was issued before these scores, so it has landed too: the packed P columns,
+    // the O accumulator and that block's K/V stage are free
     if (j > 0) {
       if (!mbar_wait(bar_o, (uint32_t)(j - 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
-      if (tid == 0 && j + 1 < nkv) load_kv(j + 1);
+      if (tid == 0 && j - 1 + NST < nkv) load_kv(j - 1 + NST);
     }
     tc_fence_after();
     // ---- softmax of this thread's row over the 64 keys of the block
@@ -198,29 +197,27 @@ __global__ void __launch_bounds__(128) attn_fwd_tc_kernel(const __grid_constant_
       ps4[0] += s[i]; ps4[1] += s[i + 1]; ps4[2] += s[i + 2]; ps4[3] += s[i + 3];
     }
     l += (ps4[0] + ps4[1]) + (ps4[2] + ps4[3]);
-    // P (bf16) into shared memory: row = tid, 16-byte chunk c8 lands at chunk (c8 ^ (row & 7)) of the 128-byte row
+    // P (bf16 pairs, even key in the low half) over the first 32 score columns of this thread's lane
+    {
+      uint32_t pw[32];
 #pragma unroll
-    for (int c8 = 0; c8 < 8; ++c8) {
-      uint4 pk;
-      pk.x = pack_bf16x2(s[8 * c8], s[8 * c8 + 1]);
-      pk.y = pack_bf16x2(s[8 * c8 + 2], s[8 * c8 + 3]);
-      pk.z = pack_bf16x2(s[8 * c8 + 4], s[8 * c8 + 5]);
-      pk.w = pack_bf16x2(s[8 * c8 + 6], s[8 * c8 + 7]);
-      *reinterpret_cast<uint4*>(sP_gen + tid * 128 + ((c8 ^ (tid & 7)) << 4)) = pk;
+      for (int i = 0; i < 32; ++i) pw[i] = pack_bf16x2(s[2 * i], s[2 * i + 1]);
+      tmem_st_32x32(t_lane, pw);
+      tmem_st_wait();
     }
-    fence_proxy_async();
     tc_fence_before();
     if (__syncthreads_or(fail)) { fail = 1; break; }     // uniform exit if any thread's wait expired
     if (tid == 0) {
       tc_fence_after();
 #pragma unroll
       for (int ks = 0; ks < TK / 16; ++ks) {
-        const uint64_t ad = make_smem_desc(sP + ks * 32, 16, 1024);
         const uint64_t bd = make_smem_desc(sV0 + st * C::KV_BYTES + ks * 2048, TK * 128, 1024);   // MN-major
-        umma_bf16(tmem_base + 64, ad, bd, idesc_o, (j | ks) ? 1u : 0u);                            // O accumulates in TMEM
+        umma_bf16_ts(tmem_base + 64, tmem_base + 8 * ks, bd, idesc_o, (j | ks) ? 1u : 0u);         // O accumulates in TMEM
       }
       umma_commit(bar_o);
-      if (j + 1 < nkv) issue_s(j + 1);           // every thread has read S_j (barrier above): the buffer is free
+      // every thread has read S_j (barrier above); the tensor pipe runs the P V just issued, which reads the
+      // packed columns, before it overwrites them with the next scores
+      if (j + 1 < nkv) issue_s(j + 1);
     }
   }
   if (!fail && nkv > 0) {
@@ -299,35 +296,33 @@ cudaError_t fwd_tc_launch(const bf16* qkv, bf16* o, float* lse, int B, int T, in
 // no row-wise reduction, so they never need to talk), all products run on tcgen05 and
 // — because the backward has no running maximum — every gradient accumulates in TMEM across the sweep.
 // Probabilities are recomputed from the saved log-sum-exp; delta_i = sum_c dO_ic O_ic.
+// P^T and dS^T (dS for dQ) never touch shared memory: a thread rounds its 32 values to bf16, packs them in
+// pairs and stores the 16 words back into the first half of the TMEM columns it has just read, from where
+// the next MMA takes them as its A operand.  The tiles of the swept index come through a 4-deep TMA ring.
 // ------------------------------------------------------------------------------------------------
-
-// 32 fp32 values -> bf16 columns [32 hf, 32 hf + 32) of row r of a [128 x 64] K-major tile with 128-byte swizzle
-__device__ __forceinline__ void store_half_row_swizzled(uint8_t* tile, int r, int hf, const float (&v)[32]) {
-#pragma unroll
-  for (int c = 0; c < 4; ++c) {
-    const int c8 = 4 * hf + c;
-    uint4 pk;
-    pk.x = pack_bf16x2(v[8 * c], v[8 * c + 1]);
-    pk.y = pack_bf16x2(v[8 * c + 2], v[8 * c + 3]);
-    pk.z = pack_bf16x2(v[8 * c + 4], v[8 * c + 5]);
-    pk.w = pack_bf16x2(v[8 * c + 6], v[8 * c + 7]);
-    *reinterpret_cast<uint4*>(tile + r * 128 + ((c8 ^ (r & 7)) << 4)) = pk;
-  }
-}
 
 template <int DH>
 struct BwdCfg {
   static constexpr int NCH = (DH + 63) / 64;
+  static constexpr int NST = 4;                         // ring depth of the swept tiles
   static constexpr int ROW_BYTES = NCH * TQ * 128;      // a 128-row operand (all chunks)
   static constexpr int BLK_BYTES = NCH * TK * 128;      // a 64-row operand
-  static constexpr int T_BYTES = TQ * 128;              // a [128 x 64] bf16 tile written by the threads
-  // dK/dV: K, V resident; Q, dO double-buffered; P^T, dS^T; lse/delta vectors.  TMEM: S^T, dP^T, dV, dK.
-  static constexpr int SMEM_KV = 2 * ROW_BYTES + 4 * BLK_BYTES + 2 * T_BYTES + 1024 + 2 * 2 * 64 * 4 + 64;
+  // dK/dV: K, V resident; ring of (Q, dO); lse/delta vectors.  TMEM: S^T, dP^T, dV, dK.
+  static constexpr int SMEM_KV = 2 * ROW_BYTES + NST * 2 * BLK_BYTES + 1024 + 2 * 2 * 64 * 4 + 128;
   static constexpr int TCOLS_KV = (128 + 2 * DH <= 256) ? 256 : 512;
-  // dQ: Q, dO resident; K, V double-buffered; dS.  TMEM: S, dP, dQ.
-  static constexpr int SMEM_Q = 2 * ROW_BYTES + 4 * BLK_BYTES + T_BYTES + 1024 + 64;
+  // dQ: Q, dO resident; ring of (K, V).  TMEM: S, dP, dQ.
+  static constexpr int SMEM_Q = 2 * ROW_BYTES + NST * 2 * BLK_BYTES + 1024 + 128;
   static constexpr int TCOLS_Q = 256;
 };
+
+// 32 fp32 values -> 16 words of bf16 pairs (even index in the low half)
+__device__ __forceinline__ void pack_row32(const float (&v)[32], uint32_t (&w)[16]) {
+#pragma unroll
+  for (int i = 0; i < 16; ++i) w[i] = pack_bf16x2(v[2 * i], v[2 * i + 1]);
+}
+// TMEM column offset (within a 64-column block whose two 32-column halves each hold their packed values in
+// their first 16 columns) of the A operand of K-step ks (16 elements = 8 columns)
+__device__ __forceinline__ constexpr uint32_t packed_col(int ks) { return (uint32_t)((ks >> 1) * 32 + (ks & 1) * 8); }
 
 template <int DH>
 __global__ void __launch_bounds__(256) attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmRow,   // qkv, 128-row box
@@ -337,19 +332,17 @@ __global__ void __launch_bounds__(256) attn_bwd_dkv_tc_kernel(const __grid_const
                                                               bf16* __restrict__ dqkv, int B, int T, int H, float scale,
                                                               unsigned* err) {
   using C = BwdCfg<DH>;
+  constexpr int NST = C::NST;
   extern __shared__ uint8_t smem_raw[];
   __shared__ int abort_flag;
   __shared__ uint32_t tmem_base_smem;
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t sK = base, sV = sK + C::ROW_BYTES;
-  const uint32_t sQ0 = sV + C::ROW_BYTES, sdO0 = sQ0 + 2 * C::BLK_BYTES;
-  const uint32_t sPT = sdO0 + 2 * C::BLK_BYTES, sdST = sPT + C::T_BYTES;
-  const uint32_t vecs = sdST + C::T_BYTES;                       // lse2[2][64], delta[2][64]
+  const uint32_t sQ0 = sV + C::ROW_BYTES, sdO0 = sQ0 + NST * C::BLK_BYTES;
+  const uint32_t vecs = sdO0 + NST * C::BLK_BYTES;               // lse2[2][64], delta[2][64]
   const uint32_t bars = vecs + 2 * 2 * 64 * 4;
-  const uint32_t bar_kv = bars, bar_q0 = bars + 8, bar_s = bars + 24, bar_acc = bars + 32, bar_drain = bars + 40;
+  const uint32_t bar_kv = bars, bar_s = bars + 8, bar_acc = bars + 16, bar_drain = bars + 24, bar_q0 = bars + 32;
   uint8_t* gen = smem_raw + (base - smem_u32(smem_raw));
-  uint8_t* sPT_gen = gen + (sPT - base);
-  uint8_t* sdST_gen = gen + (sdST - base);
   float* s_lse = reinterpret_cast<float*>(gen + (vecs - base));  // [2][64]
   float* s_del = s_lse + 128;                                    // [2][64]
 
@@ -368,11 +361,10 @@ __global__ void __launch_bounds__(256) attn_bwd_dkv_tc_kernel(const __grid_const
   if (tid == 0) {
     abort_flag = 0;
     mbar_init(bar_kv, 1);
-    mbar_init(bar_q0, 1);
-    mbar_init(bar_q0 + 8, 1);
     mbar_init(bar_s, 1);
     mbar_init(bar_acc, 1);
     mbar_init(bar_drain, 1);
+    for (int s = 0; s < NST; ++s) mbar_init(bar_q0 + 8 * s, 1);
     fence_mbar_init();
     tma_prefetch_desc(&tmRow);
     tma_prefetch_desc(&tmBlk);
@@ -399,7 +391,9 @@ __global__ void __launch_bounds__(256) attn_bwd_dkv_tc_kernel(const __grid_const
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem_base = tmem_base_smem;     // S^T [0,64), dP^T [64,128), dV [128,128+dh), dK [128+dh, 128+2dh)
+  // TMEM: S^T [0,64) and dP^T [64,128) (each later overwritten in part by its packed bf16 successor P^T,
+  // dS^T), dV [128,128+dh), dK [128+dh, 128+2dh)
+  const uint32_t tmem_base = tmem_base_smem;
   const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
   volatile int* abortp = &abort_flag;
   constexpr uint32_t idesc_s = make_idesc_bf16(TQ, TK, 0, 0);
@@ -407,7 +401,7 @@ __global__ void __launch_bounds__(256) attn_bwd_dkv_tc_kernel(const __grid_const
   int fail = 0;
 
   auto load_q = [&](int j) {
-    const int st = (j - q0) & 1;
+    const int st = (j - q0) % NST;
     mbar_expect_tx(bar_q0 + 8 * st, 2 * C::BLK_BYTES);
 #pragma unroll
     for (int c = 0; c < C::NCH; ++c) {
@@ -422,16 +416,16 @@ __global__ void __launch_bounds__(256) attn_bwd_dkv_tc_kernel(const __grid_const
       tma_load_4d(sK + c * (TQ * 128), &tmRow, c * 64, H + h, kb * TQ, bs, bar_kv);
       tma_load_4d(sV + c * (TQ * 128), &tmRow, c * 64, 2 * H + h, kb * TQ, bs, bar_kv);
     }
-    if (q0 < nq) load_q(q0);
-    if (q0 + 1 < nq) load_q(q0 + 1);
+    for (int i = 0; i < NST; ++i)
+      if (q0 + i < nq) load_q(q0 + i);
   }
   const float c2 = scale * IL_LOG2E;
 
   // S^T and dP^T of query block j; issued by thread 0 one step ahead (right after the previous block's dV/dK
   // products) so that each sweep step waits for the tensor pipe only once
   auto issue_s = [&](int j) {
-    const int it = j - q0, st = it & 1;
-    if (!mbar_wait(bar_q0 + 8 * st, (uint32_t)(it >> 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
+    const int it = j - q0, st = it % NST;
+    if (!mbar_wait(bar_q0 + 8 * st, (uint32_t)(it / NST) & 1u, abortp)) { fail = 1; abort_flag = 1; }
     tc_fence_after();
 #pragma unroll
     for (int ks = 0; ks < DH / 16; ++ks) {
@@ -450,25 +444,25 @@ __global__ void __launch_bounds__(256) attn_bwd_dkv_tc_kernel(const __grid_const
 
   for (int j = q0; j < nq; ++j) {
     const int it = j - q0;
-    const int st = it & 1;
+    const int st = it % NST;
     if (j + 1 < nq) put_vec(j + 1, vec_next);      // visible after this step's barrier
     vec_next = fetch_vec(j + 2);
     if (!mbar_wait(bar_s, (uint32_t)it & 1u, abortp)) { fail = 1; abort_flag = 1; }
-    // the previous step's dV/dK products were issued before these scores, so they have landed too: the
-    // P^T / dS^T tiles and the other Q/dO stage are free
+    // the previous step's dV/dK products were issued before these scores, so they have landed too: the packed
+    // P^T / dS^T columns and that step's Q/dO stage are free
     if (it > 0) {
       if (!mbar_wait(bar_acc, (uint32_t)(it - 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
-      if (tid == 0 && j + 1 < nq) load_q(j + 1);
+      if (tid == 0 && j - 1 + NST < nq) load_q(j - 1 + NST);
     }
     tc_fence_after();
-    float p[32], ds[32];
     {
+      float p[32], ds[32];
       uint32_t r0[32], r1[32];
       tmem_ld_32x32(t_lane + 32 * hf, r0);
       tmem_ld_32x32(t_lane + 64 + 32 * hf, r1);
       tmem_ld_wait();
-      const float4* lv = reinterpret_cast<const float4*>(s_lse + st * 64 + 32 * hf);
-      const float4* dv_ = reinterpret_cast<const float4*>(s_del + st * 64 + 32 * hf);
+      const float4* lv = reinterpret_cast<const float4*>(s_lse + (j & 1) * 64 + 32 * hf);
+      const float4* dv_ = reinterpret_cast<const float4*>(s_del + (j & 1) * 64 + 32 * hf);
       const bool diag = (j * TK < kb * TQ + TQ);   // some queries of this block precede some keys of this CTA
       const bool tail = (j * TK + TK > T);
       const int qbase = j * TK + 32 * hf;
@@ -490,10 +484,13 @@ __global__ void __launch_bounds__(256) attn_bwd_dkv_tc_kernel(const __grid_const
       }
 #pragma unroll
       for (int i = 0; i < 32; ++i) ds[i] *= p[i];
+      uint32_t pw[16], dw[16];
+      pack_row32(p, pw);
+      pack_row32(ds, dw);
+      tmem_st_32x16(t_lane + 32 * hf, pw);         // P^T over the first half of the S^T columns this thread read
+      tmem_st_32x16(t_lane + 64 + 32 * hf, dw);    // dS^T likewise over dP^T
+      tmem_st_wait();
     }
-    store_half_row_swizzled(sPT_gen, r, hf, p);
-    store_half_row_swizzled(sdST_gen, r, hf, ds);
-    fence_proxy_async();
     tc_fence_before();
     if (__syncthreads_or(fail)) { fail = 1; break; }
     if (tid == 0) {
@@ -501,13 +498,15 @@ __global__ void __launch_bounds__(256) attn_bwd_dkv_tc_kernel(const __grid_const
 #pragma unroll
       for (int ks = 0; ks < TK / 16; ++ks) {
         const uint32_t off_b = st * C::BLK_BYTES + ks * 2048;                               // MN-major: 16 queries
-        umma_bf16(tmem_base + 128, make_smem_desc(sPT + ks * 32, 16, 1024), make_smem_desc(sdO0 + off_b, TK * 128, 1024),
-                  idesc_g, (it | ks) ? 1u : 0u);
-        umma_bf16(tmem_base + 128 + DH, make_smem_desc(sdST + ks * 32, 16, 1024), make_smem_desc(sQ0 + off_b, TK * 128, 1024),
-                  idesc_g, (it | ks) ? 1u : 0u);
+        umma_bf16_ts(tmem_base + 128, tmem_base + packed_col(ks), make_smem_desc(sdO0 + off_b, TK * 128, 1024), idesc_g,
+                     (it | ks) ? 1u : 0u);
+        umma_bf16_ts(tmem_base + 128 + DH, tmem_base + 64 + packed_col(ks), make_smem_desc(sQ0 + off_b, TK * 128, 1024),
+                     idesc_g, (it | ks) ? 1u : 0u);
       }
       umma_commit(bar_acc);
-      if (j + 1 < nq) issue_s(j + 1);              // every thread has read S^T / dP^T of this step (barrier above)
+      // every thread has read S^T / dP^T of this step (barrier above); the tensor pipe runs the products just
+      // issued, which read the packed columns, before it overwrites them with the next scores
+      if (j + 1 < nq) issue_s(j + 1);
     }
   }
   const int nit = nq - q0;
@@ -575,16 +574,15 @@ __global__ void __launch_bounds__(256) attn_bwd_dq_tc_kernel(const __grid_consta
                                                              bf16* __restrict__ dqkv, int B, int T, int H, float scale,
                                                              unsigned* err) {
   using C = BwdCfg<DH>;
+  constexpr int NST = C::NST;
   extern __shared__ uint8_t smem_raw[];
   __shared__ int abort_flag;
   __shared__ uint32_t tmem_base_smem;
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t sQ = base, sdO = sQ + C::ROW_BYTES;
-  const uint32_t sK0 = sdO + C::ROW_BYTES, sV0 = sK0 + 2 * C::BLK_BYTES;
-  const uint32_t sdS = sV0 + 2 * C::BLK_BYTES;
-  const uint32_t bars = sdS + C::T_BYTES;
-  const uint32_t bar_q = bars, bar_kv0 = bars + 8, bar_s = bars + 24, bar_acc = bars + 32, bar_drain = bars + 40;
-  uint8_t* sdS_gen = smem_raw + (sdS - smem_u32(smem_raw));
+  const uint32_t sK0 = sdO + C::ROW_BYTES, sV0 = sK0 + NST * C::BLK_BYTES;
+  const uint32_t bars = sV0 + NST * C::BLK_BYTES;
+  const uint32_t bar_q = bars, bar_s = bars + 8, bar_acc = bars + 16, bar_drain = bars + 24, bar_kv0 = bars + 32;
 
   // 256 threads: thread (r, hf) owns row r = tid % 128 and columns [32 hf, 32 hf + 32) of each 64-wide block
   const int tid = threadIdx.x, warp = tid >> 5, r = tid & 127, hf = tid >> 7;
@@ -600,8 +598,7 @@ __global__ void __launch_bounds__(256) attn_bwd_dq_tc_kernel(const __grid_consta
   if (tid == 0) {
     abort_flag = 0;
     mbar_init(bar_q, 1);
-    mbar_init(bar_kv0, 1);
-    mbar_init(bar_kv0 + 8, 1);
+    for (int s = 0; s < NST; ++s) mbar_init(bar_kv0 + 8 * s, 1);
     mbar_init(bar_s, 1);
     mbar_init(bar_acc, 1);
     mbar_init(bar_drain, 1);
@@ -617,7 +614,7 @@ __global__ void __launch_bounds__(256) attn_bwd_dq_tc_kernel(const __grid_consta
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem_base = tmem_base_smem;     // S [0,64), dP [64,128), dQ [128,128+dh)
+  const uint32_t tmem_base = tmem_base_smem;     // S [0,64), dP [64,128) (later in part the packed dS), dQ [128,128+dh)
   const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
   volatile int* abortp = &abort_flag;
   constexpr uint32_t idesc_s = make_idesc_bf16(TQ, TK, 0, 0);
@@ -625,7 +622,7 @@ __global__ void __launch_bounds__(256) attn_bwd_dq_tc_kernel(const __grid_consta
   int fail = 0;
 
   auto load_kv = [&](int j) {
-    const int st = j & 1;
+    const int st = j % NST;
     mbar_expect_tx(bar_kv0 + 8 * st, 2 * C::BLK_BYTES);
 #pragma unroll
     for (int c = 0; c < C::NCH; ++c) {
@@ -640,8 +637,8 @@ __global__ void __launch_bounds__(256) attn_bwd_dq_tc_kernel(const __grid_consta
       tma_load_4d(sQ + c * (TQ * 128), &tmRow, c * 64, h, qb * TQ, bs, bar_q);
       tma_load_4d(sdO + c * (TQ * 128), &tmdO, c * 64, h, qb * TQ, nb, bar_q);
     }
-    load_kv(0);
-    if (nkv > 1) load_kv(1);
+    for (int i = 0; i < NST; ++i)
+      if (i < nkv) load_kv(i);
   }
   const float c2 = scale * IL_LOG2E;
   const float lse2 = row < T ? lse[((size_t)bs * H + h) * T + row] * IL_LOG2E : 0.f;
@@ -649,8 +646,8 @@ __global__ void __launch_bounds__(256) attn_bwd_dq_tc_kernel(const __grid_consta
 
   // S and dP of key block j; issued by thread 0 one step ahead (right after the previous block's dQ product)
   auto issue_s = [&](int j) {
-    const int st = j & 1;
-    if (!mbar_wait(bar_kv0 + 8 * st, (uint32_t)(j >> 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
+    const int st = j % NST;
+    if (!mbar_wait(bar_kv0 + 8 * st, (uint32_t)(j / NST) & 1u, abortp)) { fail = 1; abort_flag = 1; }
     tc_fence_after();
 #pragma unroll
     for (int ks = 0; ks < DH / 16; ++ks) {
@@ -668,15 +665,15 @@ __global__ void __launch_bounds__(256) attn_bwd_dq_tc_kernel(const __grid_consta
   }
 
   for (int j = 0; j < nkv; ++j) {
-    const int st = j & 1;
+    const int st = j % NST;
     if (!mbar_wait(bar_s, (uint32_t)j & 1u, abortp)) { fail = 1; abort_flag = 1; }
-    if (j > 0) {                                     // issued before these scores: landed, dS and the other K/V stage are free
+    if (j > 0) {                                     // issued before these scores: landed, the packed dS and that step's K/V stage are free
       if (!mbar_wait(bar_acc, (uint32_t)(j - 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
-      if (tid == 0 && j + 1 < nkv) load_kv(j + 1);
+      if (tid == 0 && j - 1 + NST < nkv) load_kv(j - 1 + NST);
     }
     tc_fence_after();
-    float ds[32];
     {
+      float ds[32];
       uint32_t r0[32], r1[32];
       tmem_ld_32x32(t_lane + 32 * hf, r0);
       tmem_ld_32x32(t_lane + 64 + 32 * hf, r1);
@@ -692,17 +689,19 @@ __global__ void __launch_bounds__(256) attn_bwd_dq_tc_kernel(const __grid_consta
       }
 #pragma unroll
       for (int i = 0; i < 32; ++i) ds[i] *= (__uint_as_float(r1[i]) - del);
+      uint32_t dw[16];
+      pack_row32(ds, dw);
+      tmem_st_32x16(t_lane + 64 + 32 * hf, dw);      // dS over the first half of the dP columns this thread read
+      tmem_st_wait();
     }
-    store_half_row_swizzled(sdS_gen, r, hf, ds);
-    fence_proxy_async();
     tc_fence_before();
     if (__syncthreads_or(fail)) { fail = 1; break; }
     if (tid == 0) {
       tc_fence_after();
 #pragma unroll
       for (int ks = 0; ks < TK / 16; ++ks)
-        umma_bf16(tmem_base + 128, make_smem_desc(sdS + ks * 32, 16, 1024),
-                  make_smem_desc(sK0 + st * C::BLK_BYTES + ks * 2048, TK * 128, 1024), idesc_g, (j | ks) ? 1u : 0u);
+        umma_bf16_ts(tmem_base + 128, tmem_base + 64 + packed_col(ks),
+                     make_smem_desc(sK0 + st * C::BLK_BYTES + ks * 2048, TK * 128, 1024), idesc_g, (j | ks) ? 1u : 0u);
       umma_commit(bar_acc);
       if (j + 1 < nkv) issue_s(j + 1);
     }

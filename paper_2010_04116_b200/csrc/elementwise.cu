@@ -418,6 +418,42 @@ cudaError_t lse_finalize(const float* part_max, const float* part_sum, int part_
 }
 
 // ---------------------------------------------------------------------------------------------
+// Gradient of the mean cross-entropy with respect to the logits, in place on the saved bf16 logits:
+// z[r, c] <- (exp(z[r, c] - lse[r]) - [c == target[r]]) * scale.  One CTA per row, 8 columns per thread and
+// trip; the padding columns [V, ld) are zeroed.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) dz_from_logits_kernel(bf16* __restrict__ z, int ld, const float* __restrict__ lse,
+                                                             const int* __restrict__ targets, int V, float scale) {
+  const int row = blockIdx.x;
+  const float l = lse[row];
+  const int tgt = targets[row];
+  uint4* zr = reinterpret_cast<uint4*>(z + (size_t)row * ld);
+  for (int c8 = threadIdx.x; c8 < ld / 8; c8 += 256) {
+    const int c0 = c8 * 8;
+    uint4 raw = zr[c8];
+    uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[i]));
+      const int c = c0 + 2 * i;
+      float a = (__expf(f.x - l) - (c == tgt ? 1.0f : 0.0f)) * scale;
+      float b = (__expf(f.y - l) - (c + 1 == tgt ? 1.0f : 0.0f)) * scale;
+      if (c >= V) a = 0.0f;
+      if (c + 1 >= V) b = 0.0f;
+      w[i] = pack_bf16x2(a, b);
+    }
+    zr[c8] = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+
+cudaError_t dz_from_logits(bf16* z, int ld, const float* lse, const int* targets, int rows, int V, float scale,
+                           cudaStream_t s) {
+  if ((ld % 8) || ((uintptr_t)z % 16)) return cudaErrorInvalidValue;
+  dz_from_logits_kernel<<<rows, 256, 0, s>>>(z, ld, lse, targets, V, scale);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
 // AdamW: 16 bytes/param read (p, m, v, g), 12 written (p, m, v) + 2 (bf16 shadow) = 30 B/param
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) adamw_kernel(float4* __restrict__ p, float4* __restrict__ m, float4* __restrict__ v,

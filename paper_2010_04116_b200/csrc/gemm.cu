@@ -85,7 +85,8 @@ struct RowState {   // per-thread state carried across the 32-column chunks of o
 };
 
 // Row-wise part of the epilogue, in the accumulator's own layout (thread = one row, v = 32 consecutive
-// columns starting at `col`): the softmax statistics (EPI_LSE, nothing stored) and dZ (EPI_DZ, in place).
+// columns starting at `col`): the softmax statistics (EPI_LSE; the logits themselves are stored only when
+// C is given) and dZ (EPI_DZ, in place).
 template <int EPI>
 __device__ __forceinline__ void epilogue_rowwise(const GemmDev& p, int col, float (&v)[32], RowState& st) {
   const bool full = (col + 32 <= p.N);
@@ -171,7 +172,7 @@ __device__ __forceinline__ void epilogue_store4(const GemmDev& p, int grow, int 
       }
     }
   }
-  if constexpr (EPI == EPI_BF16 || EPI == EPI_BF16_GELU || EPI == EPI_DZ || EPI == EPI_BF16_DGELU) {
+  if constexpr (EPI == EPI_BF16 || EPI == EPI_BF16_GELU || EPI == EPI_DZ || EPI == EPI_BF16_DGELU || EPI == EPI_LSE) {
     bf16* c = reinterpret_cast<bf16*>(p.C) + (size_t)grow * p.ldc + gcol;
     if constexpr (EPI == EPI_BF16_DGELU) {
       v[0] *= e.x; v[1] *= e.y; v[2] *= e.z; v[3] *= e.w;
@@ -468,7 +469,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
         for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
         if constexpr (EPI == EPI_LSE || EPI == EPI_DZ) epilogue_rowwise<EPI>(p, col, v, st);
-        if constexpr (EPI != EPI_LSE) {
+        if (EPI != EPI_LSE || p.C != nullptr) {      // EPI_LSE keeps the logits (bf16) only when asked to
           // transpose through shared memory: lane (= row) writes its 32 columns, then lane l reads 4
           // columns of row 4i + l/8
 #pragma unroll
@@ -679,7 +680,7 @@ cudaError_t gemm_launch(const GemmArgs& a, unsigned* err_word, int num_sms, cuda
   KernelFn kern = pick_kernel(a.A.mn_major, a.B.mn_major, a.epilogue);
   if (!kern) return cudaErrorInvalidValue;
   const bool out_f32 = (a.epilogue == EPI_F32 || a.epilogue == EPI_F32_RESID);
-  if (a.epilogue != EPI_LSE) {
+  if (a.epilogue != EPI_LSE || a.C) {
     if (!a.C || (a.ldc % (out_f32 ? 4 : 8)) || ((uintptr_t)a.C % 16)) return cudaErrorInvalidValue;
   }
   if (a.epilogue == EPI_BF16_GELU && (!a.C2 || ((uintptr_t)a.C2 % 16))) return cudaErrorInvalidValue;

@@ -12,7 +12,7 @@ enum GemmEpilogue : int {
   EPI_F32_RESID = 2,   // C(f32)  = resid(f32) + acc + bias        (C may alias resid)
   EPI_BF16_DGELU = 3,  // C(bf16) = acc * aux[row % aux_rows, col]   (aux = saved gelu'(pre))
   EPI_F32 = 4,         // C(f32)  = acc (+ C if accumulate)
-  EPI_LSE = 5,         // online-softmax partials per (row, column tile) + logit of the target column
+  EPI_LSE = 5,         // online-softmax partials per (row, column tile) + logit of the target column; C (bf16, optional) = acc
   EPI_DZ = 6,          // C(bf16) = (exp(acc - lse[row]) - [col + col0 == target[row]]) * scale
   EPI_COUNT = 7
 };

@@ -30,9 +30,6 @@ using namespace il;
 
 namespace {
 
-// Columns of dZ held at once in the head backward (bf16 [Ntok, chunk], L2-sized).  18 tiles of 256 columns:
-// with d_model 1024 the chunk's weight-gradient GEMM then has 72 output tiles for 74 CTA pairs.
-constexpr int VOCAB_CHUNK = 4608;
 
 struct TensorRec {
   std::string name;
@@ -53,7 +50,8 @@ struct CompScratch {     // backward scratch of one component, rows = s_cap * nt
   float* dx; bf16* dxb; bf16* dbig; bf16* dln; bf16* dattn; bf16* dqkv; float* delta;
 };
 struct HeadScratch {
-  bf16* u; float *mean, *rstd, *pmax, *psum, *tgt_logit, *lse, *du, *ghead; bf16* dz;
+  bf16* u; float *mean, *rstd, *pmax, *psum, *tgt_logit, *lse, *du, *ghead;
+  bf16* z;   // [Ntok, ldz]: the logits kept by the loss pass, turned into dZ in place by the backward
 };
 
 struct ProfRec { cudaEvent_t a, b; double flops; };
@@ -91,6 +89,7 @@ struct il_model {
   float* losses;                     // device [K]
   unsigned* err_word;
   int part_ld;
+  int ldz;                            // row stride of the saved logits (vocabulary rounded up to 64)
   // step state
   int B, T, ntok;
   bool batch_set, bwd_done;
@@ -474,6 +473,7 @@ extern "C" il_status il_create(int K, int Lc, int d, int H, int F, int V, int n,
       if (l == Lc - 1) m->a[k + 1] = A.x_out;
     }
   m->part_ld = (V + 127) / 128;
+  m->ldz = (V + 63) / 64 * 64;
   m->hs.assign(K, HeadScratch{});
   for (int k = 0; k < K; ++k) {
     HeadScratch& h = m->hs[k];
@@ -486,7 +486,7 @@ extern "C" il_status il_create(int K, int Lc, int d, int H, int F, int V, int n,
     IL_TRY(dev_alloc_t(m, &h.lse, N));
     IL_TRY(dev_alloc_t(m, &h.du, N * d));
     IL_TRY(dev_alloc_t(m, &h.ghead, N * d));
-    IL_TRY(dev_alloc_t(m, &h.dz, N * (size_t)VOCAB_CHUNK));
+    IL_TRY(dev_alloc_t(m, &h.z, N * (size_t)m->ldz));
   }
   IL_TRY(alloc_scratch(m, s_cap_for(K, n)));
   IL_TRY(dev_alloc_t(m, &m->tokens, N));
@@ -704,7 +704,7 @@ extern "C" il_status il_aux_head_loss(il_model* m, int k, float* loss_host) {
     const HeadOff& o = m->head_off[k];
     HeadScratch& h = m->hs[k];
     IL_K(m, layernorm_fwd(m->a[k + 1], m->P + o.lng, m->P + o.lnb, h.u, h.mean, h.rstd, N, d, m->ln_eps, st));
-    GemmArgs g = gemm_args(N, V, d, h.u, d, 0, m->Pb + o.w, d, 0, EPI_LSE, nullptr, 0);
+    GemmArgs g = gemm_args(N, V, d, h.u, d, 0, m->Pb + o.w, d, 0, EPI_LSE, h.z, m->ldz);
     g.targets = m->targets;
     g.part_max = h.pmax; g.part_sum = h.psum; g.part_ld = m->part_ld;
     g.tgt_logit = h.tgt_logit;
@@ -748,32 +748,22 @@ extern "C" il_status il_get_losses(il_model* m, float* losses_host) {
 
 namespace {
 
-// Head k backward on stream k: dZ chunk by chunk over the vocabulary -> dW_h, dU; LayerNorm backward -> ghead.
+// Head k backward on stream k: the saved logits become dZ = (softmax - onehot) / Ntok in place, then
+// dU = dZ W and dW_h = dZ^T U over the whole vocabulary; LayerNorm backward -> ghead.
 il_status head_backward(il_model* m, int k) {
   cudaStream_t st = m->streams[k];
   const int N = m->ntok, d = m->d, V = m->V;
   const HeadOff& o = m->head_off[k];
   HeadScratch& h = m->hs[k];
-  for (int v0 = 0; v0 < V; v0 += VOCAB_CHUNK) {
-    const int nv = V - v0 < VOCAB_CHUNK ? V - v0 : VOCAB_CHUNK;
-    const bf16* Wc = m->Pb + o.w + (size_t)v0 * d;
-    {  // logits of the chunk recomputed, turned into dZ = (softmax - onehot) / Ntok in the epilogue
-      GemmArgs g = gemm_args(N, nv, d, h.u, d, 0, Wc, d, 0, EPI_DZ, h.dz, VOCAB_CHUNK);
-      g.targets = m->targets;
-      g.lse = h.lse;
-      g.scale = 1.0f / (float)N;
-      g.col0 = v0;
-      IL_TRY(gemm(m, k, g));
-    }
-    {  // dU += dZ_chunk * W_chunk
-      GemmArgs g = gemm_args(N, d, nv, h.dz, VOCAB_CHUNK, 0, Wc, d, 1, EPI_F32, h.du, d);
-      g.accumulate = v0 > 0;
-      IL_TRY(gemm(m, k, g));
-    }
-    {  // dW_chunk = dZ_chunk^T * U
-      GemmArgs g = gemm_args(nv, d, N, h.dz, VOCAB_CHUNK, 1, h.u, d, 1, EPI_F32, m->G + o.w + (size_t)v0 * d, d);
-      IL_TRY(gemm(m, k, g));
-    }
+  IL_K(m, dz_from_logits(h.z, m->ldz, h.lse, m->targets, N, V, 1.0f / (float)N, st));
+  {  // dU = dZ * W.  Not split over the contraction: atomically added partial sums would make dU, and with it
+     // every gradient below this head, depend on the order the work units finish in.
+    GemmArgs g = gemm_args(N, d, V, h.z, m->ldz, 0, m->Pb + o.w, d, 1, EPI_F32, h.du, d);
+    IL_TRY(gemm(m, k, g));
+  }
+  {  // dW = dZ^T * U
+    GemmArgs g = gemm_args(V, d, N, h.z, m->ldz, 1, h.u, d, 1, EPI_F32, m->G + o.w, d);
+    IL_TRY(gemm(m, k, g));
   }
   IL_K(m, layernorm_bwd_params(h.du, 1, m->a[k + 1], h.mean, h.rstd, m->G + o.lng, m->G + o.lnb, N, d, st));
   IL_K(m, layernorm_bwd_rows(h.du, 1, m->a[k + 1], h.mean, h.rstd, m->P + o.lng, nullptr, h.ghead, nullptr, N, N, d, st));

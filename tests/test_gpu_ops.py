@@ -139,6 +139,18 @@ def test_gemm_softmax_epilogues(V):
     lse = gmax + np.log((psn * np.exp(pmn - gmax[:, None])).sum(axis=1))
     assert np.max(np.abs(lse - lse_ref)) < 2e-5 * max(1.0, np.abs(lse_ref).max())
     assert np.max(np.abs(tl.cpu().numpy() - z[np.arange(M), tgt])) < 1e-4
+    # the same call with C given also keeps the logits (bf16, padded row stride); statistics unchanged
+    ldz = (V + 63) // 64 * 64
+    zt = torch.full((M, ldz), 7.0, dtype=torch.bfloat16, device=DEV)
+    pm2, ps2, tl2 = torch.zeros_like(pm), torch.zeros_like(ps), torch.zeros_like(tl)
+    il.op_gemm(M, V, K, Ut, K, 0, Wt, K, 0, 5, err, C_=zt, ldc=ldz, targets=tt, part_max=pm2, part_sum=ps2,
+               part_ld=ntiles, tgt_logit=tl2)
+    torch.cuda.synchronize()
+    assert int(err.item()) == 0
+    assert torch.equal(pm2, pm) and torch.equal(ps2, ps) and torch.equal(tl2, tl)
+    zg = zt.float().cpu().numpy()
+    assert np.max(np.abs(zg[:, :V] - z)) <= 2.0 ** -8 * np.abs(z).max() + 1e-6     # one bf16 rounding
+    assert np.all(zg[:, V:] == 7.0)
     # dZ on a chunk that starts mid-vocabulary and runs past its end
     col0 = (V // 2) // 8 * 8
     nv = V - col0
