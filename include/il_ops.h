@@ -53,6 +53,8 @@ typedef struct {
   const float* lse;
   float scale;
   int col0;
+  int tile_blocks; /* output tile: 1 = 256 x 256, 2 = 256 x 512 (fewer operand bytes per product, epilogue less
+                      hidden), 0 = chosen from the shape; results do not depend on it */
 } il_gemm_desc;
 
 /* err_word: device word (unsigned) the kernel sets non-zero if one of its bounded waits expired. */

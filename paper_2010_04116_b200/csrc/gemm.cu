@@ -31,17 +31,27 @@ constexpr int BM = 128;                          // rows of A (and of the accumu
 constexpr int TILE_M = 2 * BM;                   // rows of the output tile of a CTA pair
 constexpr int BN = 256;                          // columns of the output tile; each CTA stages half of B
 constexpr int BK = 64;
-constexpr int STAGES = 5;
 constexpr int A_BYTES = BM * BK * 2;             // 16 KB
 constexpr int B_BYTES = (BN / 2) * BK * 2;       // 16 KB
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;   // 32 KB per CTA and stage
 constexpr int TMEM_COLS = 2 * BN;                // 512 columns: two accumulators
+// NT = accumulators (256-column blocks) per tile.  NT 1: a tile is 256 x 256 and the two accumulators alternate
+// between consecutive tiles, so a tile's epilogue hides behind the next tile's main loop.  NT 2: a tile is
+// 256 x 512, both accumulators belong to it and every A slab feeds two MMAs: a CTA takes 48 KB instead of
+// 64 KB from L2 per 2 x (128 x 256 x 64) products.  One SM's L2 port delivers a 32 KB slab in about the time the
+// tensor pipe needs for it, so with NT 1 the two run neck and neck and stall each other; NT 2 leaves the loads
+// 25 % slack at the price of an epilogue that overlaps only the start of the next tile.
+template <int NT> struct TileCfg {
+  static constexpr int STAGES = (NT == 1) ? 6 : 4;
+  static constexpr int STAGE_BYTES = A_BYTES + NT * B_BYTES;   // 32 / 48 KB per CTA and stage
+};
 constexpr int EPI_WARPS = 8;
 constexpr int GEMM_THREADS = 64 + 32 * EPI_WARPS;   // producer warp, MMA warp, epilogue warps
 constexpr int BAR_BYTES = 256;
-constexpr int STG_LD = 36;                       // floats per row of an epilogue warp's 32 x 32 staging tile
+constexpr int STG_LD = 32;                       // floats per row of an epilogue warp's 32 x 32 staging tile (16-byte slots XOR-swizzled by row)
 constexpr int STG_BYTES = EPI_WARPS * 32 * STG_LD * 4;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + BAR_BYTES + STG_BYTES;
+template <int NT> constexpr int smem_bytes() {
+  return TileCfg<NT>::STAGES * TileCfg<NT>::STAGE_BYTES + 1024 /*alignment slack*/ + BAR_BYTES + STG_BYTES;
+}
 
 struct GemmDev {
   int M, N, K;
@@ -228,10 +238,12 @@ __device__ __forceinline__ void epilogue_store4(const GemmDev& p, int grow, int 
   }
 }
 
-template <bool A_MN, bool B_MN, int EPI>
+template <bool A_MN, bool B_MN, int EPI, int NT>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const GemmDev p) {
+  constexpr int STAGES = TileCfg<NT>::STAGES;
+  constexpr int STAGE_BYTES = TileCfg<NT>::STAGE_BYTES;
   extern __shared__ uint8_t smem_raw[];
   __shared__ int abort_flag;
   __shared__ uint32_t tmem_base_smem;
@@ -289,7 +301,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         int m_blk, n_blk;
         tile_coords(t / p.split_k, p.tiles_m, p.tiles_n, m_blk, n_blk);
         const int m0 = m_blk * TILE_M + (int)rank * BM;       // this CTA's 128 rows of A
-        const int n0 = n_blk * BN + (int)rank * (BN / 2);     // this CTA's 128 rows of B
+        const int n0 = n_blk * (NT * BN) + (int)rank * (BN / 2);   // this CTA's 128 rows of the (first) 256-row block of B
         const int kb0 = (t % p.split_k) * p.kb_per_split;
         const int kb1 = min(num_kb_all, kb0 + p.kb_per_split);
         for (int kb = kb0; kb < kb1; ++kb) {
@@ -306,11 +318,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
             for (int i = 0; i < BM / 64; ++i) tma_load_2d_pair(sa + i * 8192, &tmA, m0 + 64 * i, k0, fb);
           }
-          if constexpr (!B_MN) {
-            tma_load_2d_pair(sb, &tmB, k0, n0, fb);
-          } else {
 #pragma unroll
-            for (int i = 0; i < BN / 128; ++i) tma_load_2d_pair(sb + i * 8192, &tmB, n0 + 64 * i, k0, fb);
+          for (int h = 0; h < NT; ++h) {          // block h of the tile's columns (past N: zero fill)
+            if constexpr (!B_MN) {
+              tma_load_2d_pair(sb + h * B_BYTES, &tmB, k0, n0 + h * BN, fb);
+            } else {
+#pragma unroll
+              for (int i = 0; i < BN / 128; ++i) tma_load_2d_pair(sb + h * B_BYTES + i * 8192, &tmB, n0 + h * BN + 64 * i, k0, fb);
+            }
           }
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -329,8 +344,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       int it = 0;
       bool ok = true;
       for (int t = pair; t < num_tiles && ok; t += num_pairs, ++it) {
-        const int as = it & 1;
-        const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
+        // NT 1: the tile uses accumulator it % 2.  NT 2: it uses both; block 0 is waited for first and handed to
+        // the epilogue as soon as its last MMAs are issued, block 1 is only waited for before its first MMA, so
+        // the first products of a tile overlap the draining of the previous tile's second block.
+        const int as = (NT == 1) ? (it & 1) : 0;
+        const uint32_t aphase = (NT == 1) ? ((uint32_t)(it >> 1) & 1u) : ((uint32_t)it & 1u);
         if (!mbar_wait(acc_empty_bar(as), aphase ^ 1u, abortp)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(as * BN);
@@ -342,17 +360,27 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           const uint32_t sa = smem_base + stage * STAGE_BYTES;
           const uint32_t sb = sa + A_BYTES;
 #pragma unroll
-          for (int k = 0; k < BK / 16; ++k) {
-            // K-major: 16 k-elements = 32 bytes along the swizzled row; 8-row groups 1024 B apart.
-            // MN-major: 16 k = two groups of 8 k-rows (1024 B each); 64-element MN chunks 8192 B apart.
-            const uint64_t ad = A_MN ? make_smem_desc(sa + k * 2048, 8192, 1024) : make_smem_desc(sa + k * 32, 16, 1024);
-            const uint64_t bd = B_MN ? make_smem_desc(sb + k * 2048, 8192, 1024) : make_smem_desc(sb + k * 32, 16, 1024);
-            umma_bf16_pair(d_tmem, ad, bd, idesc, (kb > kb0 || k != 0) ? 1u : 0u);
+          for (int h = 0; h < NT; ++h) {
+            if (NT == 2 && h == 1 && kb == kb0) {
+              if (!mbar_wait(acc_empty_bar(1), aphase ^ 1u, abortp)) { ok = false; break; }
+              tc_fence_after();
+            }
+#pragma unroll
+            for (int k = 0; k < BK / 16; ++k) {
+              // K-major: 16 k-elements = 32 bytes along the swizzled row; 8-row groups 1024 B apart.
+              // MN-major: 16 k = two groups of 8 k-rows (1024 B each); 64-element MN chunks 8192 B apart.
+              const uint32_t sbh = sb + h * B_BYTES;
+              const uint64_t ad = A_MN ? make_smem_desc(sa + k * 2048, 8192, 1024) : make_smem_desc(sa + k * 32, 16, 1024);
+              const uint64_t bd = B_MN ? make_smem_desc(sbh + k * 2048, 8192, 1024) : make_smem_desc(sbh + k * 32, 16, 1024);
+              umma_bf16_pair(d_tmem + (uint32_t)(h * BN), ad, bd, idesc, (kb > kb0 || k != 0) ? 1u : 0u);
+            }
+            if (NT == 2 && h == 0 && kb == kb1 - 1) umma_commit_pair(acc_full_bar(0), 3);
           }
+          if (!ok) break;
           umma_commit_pair(empty_bar(stage), 3);   // slab reusable in both CTAs once these MMAs have read it
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
-        if (ok) umma_commit_pair(acc_full_bar(as), 3);
+        if (ok) umma_commit_pair(acc_full_bar(NT == 1 ? as : 1), 3);
       }
       if (!ok) {
         atomicExch(p.err, DEV_TIMEOUT_MMA);
@@ -374,10 +402,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     int it = 0;
     bool ok = true;
     for (int t = pair; t < num_tiles && ok; t += num_pairs, ++it) {
-      int m_blk, n_blk;
-      tile_coords(t / p.split_k, p.tiles_m, p.tiles_n, m_blk, n_blk);
-      const int as = it & 1;
-      const uint32_t aphase = (uint32_t)(it >> 1) & 1u;
+      int m_blk, n_tile;
+      tile_coords(t / p.split_k, p.tiles_m, p.tiles_n, m_blk, n_tile);
+      for (int h = 0; h < NT && ok; ++h) {           // the tile's 256-column blocks, one accumulator each
+      const int n_blk = n_tile * NT + h;
+      const int as = (NT == 1) ? (it & 1) : h;
+      const uint32_t aphase = (NT == 1) ? ((uint32_t)(it >> 1) & 1u) : ((uint32_t)it & 1u);
       const int row0 = m_blk * TILE_M + (int)rank * BM + q * 32;     // first row of this warp's 32
       const int col_base = n_blk * BN + half * (BN / 2);
       const int lrow = lane >> 3;                  // row within a group of 4 after the transpose
@@ -474,11 +504,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           // columns of row 4i + l/8
 #pragma unroll
           for (int j = 0; j < 8; ++j)
-            *reinterpret_cast<float4*>(stg + lane * STG_LD + 4 * j) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+            *reinterpret_cast<float4*>(stg + lane * STG_LD + 4 * (j ^ (lane & 7))) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
           __syncwarp();
           float4 a[8];
 #pragma unroll
-          for (int i = 0; i < 8; ++i) a[i] = *reinterpret_cast<const float4*>(stg + (4 * i + lrow) * STG_LD + gcol_off);
+          for (int i = 0; i < 8; ++i)          // row 4i + lrow, slot (lane & 7) ^ (row & 7); row & 7 = (4i + lrow) & 7
+            a[i] = *reinterpret_cast<const float4*>(stg + (4 * i + lrow) * STG_LD + 4 * ((lane & 7) ^ ((4 * i + lrow) & 7)));
           if (interior) {
             float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f);
             if constexpr (EPI == EPI_BF16 || EPI == EPI_BF16_GELU || EPI == EPI_F32_RESID)
@@ -558,6 +589,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(mapa_cluster(acc_empty_bar(as), 0));
+      }
     }
     if (!ok && lane == 0) {
       atomicExch(p.err, DEV_TIMEOUT_EPILOGUE);
@@ -588,16 +620,16 @@ static cudaError_t g_init_err = cudaSuccess;
 
 typedef void (*KernelFn)(const CUtensorMap, const CUtensorMap, const GemmDev);
 
-template <bool A_MN, bool B_MN>
+template <bool A_MN, bool B_MN, int NT>
 static KernelFn pick_epi(int epi) {
   switch (epi) {
-    case EPI_BF16: return gemm_tcgen05_kernel<A_MN, B_MN, EPI_BF16>;
-    case EPI_BF16_GELU: return gemm_tcgen05_kernel<A_MN, B_MN, EPI_BF16_GELU>;
-    case EPI_F32_RESID: return gemm_tcgen05_kernel<A_MN, B_MN, EPI_F32_RESID>;
-    case EPI_BF16_DGELU: return gemm_tcgen05_kernel<A_MN, B_MN, EPI_BF16_DGELU>;
-    case EPI_F32: return gemm_tcgen05_kernel<A_MN, B_MN, EPI_F32>;
-    case EPI_LSE: return gemm_tcgen05_kernel<A_MN, B_MN, EPI_LSE>;
-    case EPI_DZ: return gemm_tcgen05_kernel<A_MN, B_MN, EPI_DZ>;
+    case EPI_BF16: return gemm_tcgen05_kernel<A_MN, B_MN, EPI_BF16, NT>;
+    case EPI_BF16_GELU: return gemm_tcgen05_kernel<A_MN, B_MN, EPI_BF16_GELU, NT>;
+    case EPI_F32_RESID: return gemm_tcgen05_kernel<A_MN, B_MN, EPI_F32_RESID, NT>;
+    case EPI_BF16_DGELU: return gemm_tcgen05_kernel<A_MN, B_MN, EPI_BF16_DGELU, NT>;
+    case EPI_F32: return gemm_tcgen05_kernel<A_MN, B_MN, EPI_F32, NT>;
+    case EPI_LSE: return gemm_tcgen05_kernel<A_MN, B_MN, EPI_LSE, NT>;
+    case EPI_DZ: return gemm_tcgen05_kernel<A_MN, B_MN, EPI_DZ, NT>;
   }
   return nullptr;
 }
@@ -605,18 +637,22 @@ static KernelFn pick_epi(int epi) {
 // Only the operand layouts the training step uses are instantiated:
 //   forward (K/K): every epilogue but the wgrad-only ones; dgrad (K/MN): bf16, dgelu, f32;
 //   wgrad (MN/MN): f32.
-static KernelFn pick_kernel(int a_mn, int b_mn, int epi) {
-  if (!a_mn && !b_mn) return pick_epi<false, false>(epi);
+template <int NT>
+static KernelFn pick_kernel_nt(int a_mn, int b_mn, int epi) {
+  if (!a_mn && !b_mn) return pick_epi<false, false, NT>(epi);
   if (!a_mn && b_mn) {
     switch (epi) {
-      case EPI_BF16: return gemm_tcgen05_kernel<false, true, EPI_BF16>;
-      case EPI_BF16_DGELU: return gemm_tcgen05_kernel<false, true, EPI_BF16_DGELU>;
-      case EPI_F32: return gemm_tcgen05_kernel<false, true, EPI_F32>;
+      case EPI_BF16: return gemm_tcgen05_kernel<false, true, EPI_BF16, NT>;
+      case EPI_BF16_DGELU: return gemm_tcgen05_kernel<false, true, EPI_BF16_DGELU, NT>;
+      case EPI_F32: return gemm_tcgen05_kernel<false, true, EPI_F32, NT>;
     }
     return nullptr;
   }
-  if (a_mn && b_mn && epi == EPI_F32) return gemm_tcgen05_kernel<true, true, EPI_F32>;
+  if (a_mn && b_mn && epi == EPI_F32) return gemm_tcgen05_kernel<true, true, EPI_F32, NT>;
   return nullptr;
+}
+static KernelFn pick_kernel(int a_mn, int b_mn, int epi, int nt) {
+  return nt == 2 ? pick_kernel_nt<2>(a_mn, b_mn, epi) : pick_kernel_nt<1>(a_mn, b_mn, epi);
 }
 
 cudaError_t gemm_init() {
@@ -632,11 +668,13 @@ cudaError_t gemm_init() {
     for (int a = 0; a < 2; ++a)
       for (int b = 0; b < 2; ++b)
         for (int epi = 0; epi < EPI_COUNT; ++epi) {
-          KernelFn k = pick_kernel(a, b, epi);
-          if (!k) continue;
-          e = cudaFuncSetAttribute(reinterpret_cast<const void*>(k), cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   SMEM_BYTES);
-          if (e != cudaSuccess) { g_init_err = e; return; }
+          for (int nt = 1; nt <= 2; ++nt) {
+            KernelFn k = pick_kernel(a, b, epi, nt);
+            if (!k) continue;
+            e = cudaFuncSetAttribute(reinterpret_cast<const void*>(k), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     nt == 2 ? smem_bytes<2>() : smem_bytes<1>());
+            if (e != cudaSuccess) { g_init_err = e; return; }
+          }
         }
   });
   return g_init_err;
@@ -677,7 +715,12 @@ cudaError_t gemm_launch(const GemmArgs& a, unsigned* err_word, int num_sms, cuda
   if (e != cudaSuccess) return e;
   if (a.M <= 0 || a.N <= 0 || a.K <= 0 || !a.A.ptr || !a.B.ptr || !err_word) return cudaErrorInvalidValue;
   if ((a.A.ld % 8) || (a.B.ld % 8) || ((uintptr_t)a.A.ptr % 16) || ((uintptr_t)a.B.ptr % 16)) return cudaErrorInvalidValue;
-  KernelFn kern = pick_kernel(a.A.mn_major, a.B.mn_major, a.epilogue);
+  // Tile width.  256 x 512 tiles cut the operand bytes per product by a quarter but expose most of the epilogue,
+  // so they pay when the main loop of a tile is long (K) and the output is at least one such tile wide.
+  int nt = a.tile_blocks;
+  if (nt < 1 || nt > 2) nt = (a.N > BN && a.K >= 2048) ? 2 : 1;
+  if (a.N <= BN) nt = 1;
+  KernelFn kern = pick_kernel(a.A.mn_major, a.B.mn_major, a.epilogue, nt);
   if (!kern) return cudaErrorInvalidValue;
   const bool out_f32 = (a.epilogue == EPI_F32 || a.epilogue == EPI_F32_RESID);
   if (a.epilogue != EPI_LSE || a.C) {
@@ -700,7 +743,7 @@ cudaError_t gemm_launch(const GemmArgs& a, unsigned* err_word, int num_sms, cuda
   GemmDev p;
   p.M = a.M; p.N = a.N; p.K = a.K;
   p.tiles_m = (a.M + TILE_M - 1) / TILE_M;
-  p.tiles_n = (a.N + BN - 1) / BN;
+  p.tiles_n = (a.N + nt * BN - 1) / (nt * BN);
   {
     // Split the contraction when the tile count leaves most CTA pairs idle (fp32 outputs only; the caller
     // zeroes C and the partial sums are added with red.global.add).
@@ -721,7 +764,7 @@ cudaError_t gemm_launch(const GemmArgs& a, unsigned* err_word, int num_sms, cuda
   const long long tiles = (long long)p.tiles_m * p.tiles_n * p.split_k;
   const int pairs = (int)(tiles < num_sms / 2 ? tiles : num_sms / 2);
   const int grid = 2 * pairs;
-  kern<<<grid, GEMM_THREADS, SMEM_BYTES, stream>>>(tmA, tmB, p);
+  kern<<<grid, GEMM_THREADS, nt == 2 ? smem_bytes<2>() : smem_bytes<1>(), stream>>>(tmA, tmB, p);
   return cudaGetLastError();
 }
 

@@ -50,6 +50,7 @@ struct GemmArgs {
   const float* lse;   // [M]
   float scale;        // EPI_DZ: 1 / Ntok
   int col0;
+  int tile_blocks;    // 256-column blocks per output tile: 1 (256 x 256), 2 (256 x 512), 0 = chosen from the shape
 };
 
 // Enqueue one GEMM on `stream`.  `err_word` is a device word set non-zero when a bounded wait in

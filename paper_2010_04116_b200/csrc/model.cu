@@ -236,23 +236,33 @@ GemmArgs gemm_args(int M, int N, int K, const void* A, int lda, int a_mn, const 
     (m)->launches++;                                                                                    \
   } while (0)
 
-// Weight-gradient GEMM dW[M,N] = dY^T X over K tokens.  When the output has far fewer 256 x 256 tiles than the
-// GPU has CTA pairs, the token axis is split over several work units per tile (partial sums are added
-// atomically into the zeroed gradient).
+// Weight-gradient GEMM dW[M,N] = dY^T X over K tokens.  The output has few tiles compared with the number of CTA
+// pairs, so the tile width (256 or 512 columns) and the number of work units per tile the token axis is split
+// into (partial sums are added atomically into the zeroed gradient) are chosen together, by a small model of
+// the kernel: waves of units over the pairs, times the k-slabs of a unit (a 512-wide slab costs 1.72 of a
+// 256-wide one) plus the unit's exposed prologue / epilogue.
 il_status wgrad(il_model* m, int k, int M, int N, int K, const bf16* dY, int ld_dy, const bf16* X, int ld_x, float* dW) {
-  const int tiles = ((M + 255) / 256) * ((N + 255) / 256);
   const int pairs = m->num_sms / 2;
-  int best = 1;
-  double best_cost = (double)((tiles + pairs - 1) / pairs);
-  for (int s = 2; s <= 4; ++s) {
-    if (K / 64 / s < 16) break;
-    const double cost = (double)((tiles * s + pairs - 1) / pairs) / s;
-    if (cost < best_cost * 0.9) { best_cost = cost; best = s; }
+  const int slabs = (K + 63) / 64;
+  int best_nt = 1, best_s = 1;
+  double best_cost = 1e300;
+  for (int nt = 1; nt <= 2; ++nt) {
+    if (nt == 2 && N <= 256) break;
+    const int tiles = ((M + 255) / 256) * ((N + 256 * nt - 1) / (256 * nt));
+    const double slab_cost = nt == 1 ? 1.0 : 1.72, unit_cost = nt == 1 ? 2.0 : 10.0;
+    for (int s = 1; s <= 8; ++s) {
+      if (s > 1 && slabs / s < 16) break;
+      const int per = (slabs + s - 1) / s;
+      const int waves = (tiles * s + pairs - 1) / pairs;
+      const double cost = waves * (per * slab_cost + unit_cost) + (s > 1 ? 4.0 : 0.0);   // + zeroing the output
+      if (cost < best_cost * 0.97) { best_cost = cost; best_nt = nt; best_s = s; }
+    }
   }
   GemmArgs g = gemm_args(M, N, K, dY, ld_dy, 1, X, ld_x, 1, EPI_F32, dW, N);
-  if (best > 1) {
+  g.tile_blocks = best_nt;
+  if (best_s > 1) {
     IL_CUDA(m, cudaMemsetAsync(dW, 0, (size_t)M * N * sizeof(float), m->streams[k]));
-    g.split_k = best;
+    g.split_k = best_s;
   }
   return gemm(m, k, g);
 }
@@ -1033,6 +1043,7 @@ extern "C" il_status il_op_gemm(const il_gemm_desc* q, unsigned* err_word, void*
   g.C2 = q->C2; g.bias = q->bias; g.resid = q->resid; g.aux = q->aux; g.ld_aux = q->ld_aux; g.aux_rows = q->aux_rows; g.colsum = q->colsum;
   g.accumulate = q->accumulate; g.split_k = q->split_k; g.targets = q->targets; g.part_max = q->part_max; g.part_sum = q->part_sum;
   g.part_ld = q->part_ld; g.tgt_logit = q->tgt_logit; g.lse = q->lse; g.scale = q->scale; g.col0 = q->col0;
+  g.tile_blocks = q->tile_blocks;
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return IL_ERR_CUDA;
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return IL_ERR_CUDA;

@@ -260,3 +260,51 @@ def test_gemm_split_k_adds_partial_sums(split):
     assert int(err.item()) == 0
     ref = Ae[:, :M].T @ Be
     assert _rel(Ct.cpu().numpy(), ref) < 5e-6      # fp32 accumulation over K = 4168 plus the atomic partial sums
+
+
+@pytest.mark.parametrize("M,N,K,layout,epi", [
+    (512, 512, 128, (0, 0), 4),        # exactly one wide tile
+    (1000, 700, 200, (0, 0), 0),       # ragged: the second wide tile has one and a bit column blocks
+    (777, 1304, 136, (0, 1), 4),       # dgrad layout, three wide tiles, ragged rows
+    (1304, 560, 264, (1, 1), 4),       # wgrad layout
+    (640, 900, 320, (0, 0), 2),        # fp32 residual epilogue
+    (300, 1000, 128, (0, 0), 5),       # softmax partials: block index must follow the column, not the tile
+])
+def test_gemm_wide_tiles_match_square_tiles(M, N, K, layout, epi):
+    """256 x 512 output tiles (two accumulators per tile, shared A slab) compute each element exactly as
+    256 x 256 tiles do: same products, same order."""
+    rng = np.random.default_rng(M + N + K)
+    a_mn, b_mn = layout
+    At, _ = _bf16(rng.standard_normal((K, M) if a_mn else (M, K)))
+    Bt, _ = _bf16(rng.standard_normal((K, N) if b_mn else (N, K)) * 0.2)
+    lda, ldb = (M if a_mn else K), (N if b_mn else K)
+    ldc = (N + 7) // 8 * 8
+    outs = []
+    for tb in (1, 2):
+        err = _err_word()
+        kw = {}
+        extra = []
+        if epi == 0:
+            Ct = torch.zeros((M, ldc), dtype=torch.bfloat16, device=DEV)
+            kw["bias"] = torch.linspace(-1, 1, N, device=DEV)
+        elif epi == 5:
+            nt = (N + 127) // 128
+            Ct = torch.zeros((M, ldc), dtype=torch.bfloat16, device=DEV)
+            pm = torch.zeros((M, nt), device=DEV); ps = torch.zeros((M, nt), device=DEV); tl = torch.zeros(M, device=DEV)
+            kw.update(targets=torch.tensor(rng.integers(0, N, size=M).astype(np.int32), device=DEV) if not outs else outs[0][1][3],
+                      part_max=pm, part_sum=ps, part_ld=nt, tgt_logit=tl)
+            extra = [pm, ps, tl, kw["targets"]]
+        else:
+            Ct = torch.zeros((M, ldc), dtype=torch.float32, device=DEV)
+            if epi == 2:
+                kw["resid"] = torch.full((M, ldc), 0.5, device=DEV)
+        il.op_gemm(M, N, K, At, lda, a_mn, Bt, ldb, b_mn, epi, err, C_=Ct, ldc=ldc, tile_blocks=tb, **kw)
+        torch.cuda.synchronize()
+        assert int(err.item()) == 0
+        outs.append((Ct.clone(), extra))
+    assert torch.equal(outs[0][0], outs[1][0])
+    for x, y in zip(outs[0][1], outs[1][1]):
+        assert torch.equal(x, y)
+    ref = (At.float().T if a_mn else At.float()) @ (Bt.float() if b_mn else Bt.float().T)
+    got = outs[1][0][:, :N].float() - (0.5 if epi == 2 else 0.0) - (kw["bias"] if epi == 0 else 0.0)
+    assert torch.linalg.norm(got - ref) / torch.linalg.norm(ref) < (4e-3 if epi in (0, 5) else 1e-5)
