@@ -46,7 +46,7 @@ typedef enum {
   IL_ERR_OOM = 3,         /* the allocator returned NULL                                            */
   IL_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed; see il_last_error                   */
   IL_ERR_TIMEOUT = 5,     /* a bounded device-side wait expired (kernel returned early)             */
-  IL_ERR_NONFINITE = 6    /* reserved                                                               */
+  IL_ERR_NONFINITE = 6    /* a head's log-sum-exp left [-80, 80] (the backward keeps exp(logit) in bf16)  */
 } il_status;
 
 typedef struct {
@@ -120,7 +120,8 @@ il_status il_backward_nwise(il_model* m);
 /* AdamW (decoupled weight decay on rank-2 tensors; weight_decay = 0 is the paper's Adam,
  * App. B.3: beta1 0.9, beta2 0.98, eps 1e-9).  Needs il_backward_nwise.  Increments the step. */
 il_status il_adamw_step(il_model* m, float lr, float beta1, float beta2, float eps, float weight_decay);
-/* Wait for all enqueued work; reports device-side timeouts as IL_ERR_TIMEOUT. */
+/* Wait for all enqueued work; reports device-side timeouts as IL_ERR_TIMEOUT and a head whose
+ * log-sum-exp left [-80, 80] in il_backward_nwise as IL_ERR_NONFINITE (that step's gradients are invalid). */
 il_status il_sync(il_model* m);
 /* Boundary activation a_k, k = 0..K (a_0 = embeddings), fp32 [B*T, d] to host; synchronises. */
 il_status il_get_boundary(il_model* m, int k, float* host, size_t count);

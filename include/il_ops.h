@@ -27,10 +27,11 @@ extern "C" {
  *   0 C(bf16) = acc + bias                         1 C(bf16) = gelu_tanh'(pre), C2(bf16) = gelu_tanh(pre), pre = acc + bias
  *   2 C(f32) = resid(f32) + acc + bias             3 C(bf16) = acc * aux[row % aux_rows, col]  (aux_rows >= 32;
  *                                                     optionally colsum[col] += sum over rows < aux_rows)
- *   4 C(f32) = acc (+ C when accumulate != 0)
+ *   4 C(f32) = acc * rowscale[row] (+ C when accumulate != 0); rowscale [M] fp32, optional
  *   5 per-(row, 128-column block) softmax partials: part_max, part_sum [M, part_ld] at block index
  *     col0/128 + block (col0 % 128 == 0), and tgt_logit[row] = acc[row, targets[row] - col0] when that
- *     column is in range; when C is not NULL, also C(bf16) = acc (the logits, ldc a multiple of 8)
+ *     column is in range; when C is not NULL, also C(bf16) = acc (the logits, ldc a multiple of 8), or
+ *     exp(acc) when store_exp != 0
  *   6 C(bf16) = (exp(acc - lse[row]) - [col + col0 == targets[row]]) * scale
  * (0,1) supports epilogues 0, 3, 4; (1,1) supports 4; (0,0) supports all. */
 typedef struct {
@@ -55,6 +56,8 @@ typedef struct {
   int col0;
   int tile_blocks; /* output tile: 1 = 256 x 256, 2 = 256 x 512 (fewer operand bytes per product, epilogue less
                       hidden), 0 = chosen from the shape; results do not depend on it */
+  const float* rowscale; /* epilogue 4 */
+  int store_exp;         /* epilogue 5 */
 } il_gemm_desc;
 
 /* err_word: device word (unsigned) the kernel sets non-zero if one of its bounded waits expired. */

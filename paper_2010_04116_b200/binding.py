@@ -47,7 +47,8 @@ class il_gemm_desc(C.Structure):
                 ("targets", C.c_void_p),
                 ("part_max", C.c_void_p), ("part_sum", C.c_void_p), ("part_ld", C.c_int),
                 ("tgt_logit", C.c_void_p), ("lse", C.c_void_p),
-                ("scale", C.c_float), ("col0", C.c_int), ("tile_blocks", C.c_int)]
+                ("scale", C.c_float), ("col0", C.c_int), ("tile_blocks", C.c_int),
+                ("rowscale", C.c_void_p), ("store_exp", C.c_int)]
 
 
 _lib = None
@@ -339,7 +340,7 @@ class Model:
 # ---------------------------------------------------------------------- operator-level calls
 def op_gemm(M, N, K, A, lda, a_mn, B, ldb, b_mn, epilogue, err_word, C_=None, ldc=0, C2=None, bias=None,
             resid=None, aux=None, ld_aux=0, aux_rows=0, colsum=None, accumulate=0, split_k=0, targets=None, part_max=None,
-            part_sum=None, part_ld=0, tgt_logit=None, lse=None, scale=0.0, col0=0, tile_blocks=0, stream=None):
+            part_sum=None, part_ld=0, tgt_logit=None, lse=None, scale=0.0, col0=0, tile_blocks=0, rowscale=None, store_exp=0, stream=None):
     d = il_gemm_desc()
     d.M, d.N, d.K = M, N, K
     d.A, d.lda, d.a_mn_major = _ptr(A), lda, a_mn
@@ -356,6 +357,7 @@ def op_gemm(M, N, K, A, lda, a_mn, B, ldb, b_mn, epilogue, err_word, C_=None, ld
     d.tgt_logit, d.lse = _ptr(tgt_logit), _ptr(lse)
     d.scale, d.col0 = scale, col0
     d.tile_blocks = tile_blocks
+    d.rowscale, d.store_exp = _ptr(rowscale), store_exp
     st = lib().il_op_gemm(C.byref(d), _ptr(err_word), stream)
     if st != IL_OK:
         raise ILError(st, "il_op_gemm")

@@ -10,7 +10,7 @@ namespace il {
 typedef __nv_bfloat16 bf16;
 
 // Values of the device-side error word (0 = no error).
-enum : unsigned { DEV_OK = 0u, DEV_TIMEOUT_PRODUCER = 1u, DEV_TIMEOUT_MMA = 2u, DEV_TIMEOUT_EPILOGUE = 3u };
+enum : unsigned { DEV_OK = 0u, DEV_TIMEOUT_PRODUCER = 1u, DEV_TIMEOUT_MMA = 2u, DEV_TIMEOUT_EPILOGUE = 3u, DEV_LOGIT_RANGE = 4u };
 
 // Every device-side wait gives up after this long, sets the error word and lets the CTA return.
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;

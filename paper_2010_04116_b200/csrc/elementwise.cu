@@ -418,38 +418,51 @@ cudaError_t lse_finalize(const float* part_max, const float* part_sum, int part_
 }
 
 // ---------------------------------------------------------------------------------------------
-// Gradient of the mean cross-entropy with respect to the logits, in place on the saved bf16 logits:
-// z[r, c] <- (exp(z[r, c] - lse[r]) - [c == target[r]]) * scale.  One CTA per row, 8 columns per thread and
-// trip; the padding columns [V, ld) are zeroed.
+// Head backward set-up.  The loss pass kept E = exp(logits) (bf16).  With s_r = exp(-lse_r) / rows the gradient
+// of the mean cross-entropy is dZ[r, c] = s_r * (E[r, c] - [c == target_r] * exp(lse_r)), so one warp per row
+//   * subtracts exp(lse_r) from the target's entry of E (the bf16 rounding of that difference is, relative to
+//     the entry, what rounding dZ itself would be),
+//   * writes s_r for the epilogue of dU = diag(s) (E W),
+//   * writes U'[r, :] = s_r * U[r, :] (bf16) for dW = E^T U'.
+// exp(logit) must stay inside the bf16 / fp32 range: rows whose lse leaves [-80, 80] raise the error word.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) dz_from_logits_kernel(bf16* __restrict__ z, int ld, const float* __restrict__ lse,
-                                                             const int* __restrict__ targets, int V, float scale) {
-  const int row = blockIdx.x;
+__global__ void __launch_bounds__(256) head_backward_prepare_kernel(bf16* __restrict__ e, int ld, const float* __restrict__ lse,
+                                                                    const int* __restrict__ targets, const bf16* __restrict__ u,
+                                                                    bf16* __restrict__ u_scaled, float* __restrict__ rowscale,
+                                                                    int rows, int d, float inv_rows, unsigned* err) {
+  const int lane = threadIdx.x & 31;
+  const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (row >= rows) return;
   const float l = lse[row];
-  const int tgt = targets[row];
-  uint4* zr = reinterpret_cast<uint4*>(z + (size_t)row * ld);
-  for (int c8 = threadIdx.x; c8 < ld / 8; c8 += 256) {
-    const int c0 = c8 * 8;
-    uint4 raw = zr[c8];
+  if (!(l >= -80.0f && l <= 80.0f)) {
+    if (lane == 0) atomicExch(err, DEV_LOGIT_RANGE);
+    return;
+  }
+  const float s = __expf(-l) * inv_rows;
+  if (lane == 0) {
+    rowscale[row] = s;
+    bf16* et = e + (size_t)row * ld + targets[row];
+    *et = __float2bfloat16(__bfloat162float(*et) - __expf(l));
+  }
+  const uint4* ur = reinterpret_cast<const uint4*>(u + (size_t)row * d);
+  uint4* us = reinterpret_cast<uint4*>(u_scaled + (size_t)row * d);
+  for (int c8 = lane; c8 < d / 8; c8 += 32) {
+    const uint4 raw = ur[c8];
     uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[i]));
-      const int c = c0 + 2 * i;
-      float a = (__expf(f.x - l) - (c == tgt ? 1.0f : 0.0f)) * scale;
-      float b = (__expf(f.y - l) - (c + 1 == tgt ? 1.0f : 0.0f)) * scale;
-      if (c >= V) a = 0.0f;
-      if (c + 1 >= V) b = 0.0f;
-      w[i] = pack_bf16x2(a, b);
+      w[i] = pack_bf16x2(f.x * s, f.y * s);
     }
-    zr[c8] = make_uint4(w[0], w[1], w[2], w[3]);
+    us[c8] = make_uint4(w[0], w[1], w[2], w[3]);
   }
 }
 
-cudaError_t dz_from_logits(bf16* z, int ld, const float* lse, const int* targets, int rows, int V, float scale,
-                           cudaStream_t s) {
-  if ((ld % 8) || ((uintptr_t)z % 16)) return cudaErrorInvalidValue;
-  dz_from_logits_kernel<<<rows, 256, 0, s>>>(z, ld, lse, targets, V, scale);
+cudaError_t head_backward_prepare(bf16* e, int ld, const float* lse, const int* targets, const bf16* u, bf16* u_scaled,
+                                  float* rowscale, int rows, int d, unsigned* err, cudaStream_t s) {
+  if ((d % 8) || ((uintptr_t)u % 16) || ((uintptr_t)u_scaled % 16) || !err) return cudaErrorInvalidValue;
+  head_backward_prepare_kernel<<<ceil_div(rows, 8), 256, 0, s>>>(e, ld, lse, targets, u, u_scaled, rowscale, rows, d,
+                                                                 1.0f / (float)rows, err);
   return cudaGetLastError();
 }
 

@@ -74,6 +74,8 @@ struct GemmDev {
   const float* lse;
   float scale;
   int col0;
+  const float* rowscale;
+  int store_exp;
   unsigned* err;
 };
 
@@ -119,6 +121,10 @@ __device__ __forceinline__ void epilogue_rowwise(const GemmDev& p, int col, floa
 #pragma unroll
       for (int j = 0; j < 32; ++j)
         if (j == tj) st.tl = v[j];
+    }
+    if (p.store_exp) {       // what is kept for the backward is exp(logit): softmax up to a per-row factor
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] = __expf(v[j]);
     }
   } else if constexpr (EPI == EPI_DZ) {
     const float l = st.m;   // lse of this row
@@ -461,6 +467,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           if constexpr (EPI == EPI_DZ) st.m = __ldg(p.lse + row);
         }
       }
+      float rs = 1.0f;                           // EPI_F32: factor of this thread's row
+      if constexpr (EPI == EPI_F32) {
+        if (p.rowscale && row_ok) rs = __ldg(p.rowscale + row);
+      }
       const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * BN + half * (BN / 2));
 #pragma unroll
       for (int c = 0; c < BN / 64; ++c) {
@@ -499,6 +509,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
         for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
         if constexpr (EPI == EPI_LSE || EPI == EPI_DZ) epilogue_rowwise<EPI>(p, col, v, st);
+        if constexpr (EPI == EPI_F32) {
+          if (p.rowscale) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] *= rs;
+          }
+        }
         if (EPI != EPI_LSE || p.C != nullptr) {      // EPI_LSE keeps the logits (bf16) only when asked to
           // transpose through shared memory: lane (= row) writes its 32 columns, then lane l reads 4
           // columns of row 4i + l/8
@@ -735,6 +751,8 @@ cudaError_t gemm_launch(const GemmArgs& a, unsigned* err_word, int num_sms, cuda
   if (a.epilogue == EPI_LSE && (!a.targets || !a.part_max || !a.part_sum || !a.tgt_logit || (a.col0 % (BN / 2))))
     return cudaErrorInvalidValue;
   if (a.epilogue == EPI_DZ && (!a.targets || !a.lse)) return cudaErrorInvalidValue;
+  if (a.rowscale && a.epilogue != EPI_F32) return cudaErrorInvalidValue;
+  if (a.store_exp && (a.epilogue != EPI_LSE || !a.C)) return cudaErrorInvalidValue;
 
   CUtensorMap tmA, tmB;
   if (!encode_operand(&tmA, a.A, a.M, a.K, BM)) return cudaErrorInvalidValue;
@@ -760,6 +778,7 @@ cudaError_t gemm_launch(const GemmArgs& a, unsigned* err_word, int num_sms, cuda
   p.accumulate = a.accumulate;
   p.targets = a.targets; p.part_max = a.part_max; p.part_sum = a.part_sum; p.part_ld = a.part_ld;
   p.tgt_logit = a.tgt_logit; p.lse = a.lse; p.scale = a.scale; p.col0 = a.col0;
+  p.rowscale = a.rowscale; p.store_exp = a.store_exp;
   p.err = err_word;
   const long long tiles = (long long)p.tiles_m * p.tiles_n * p.split_k;
   const int pairs = (int)(tiles < num_sms / 2 ? tiles : num_sms / 2);

@@ -11,8 +11,9 @@ enum GemmEpilogue : int {
   EPI_BF16_GELU = 1,   // pre = acc + bias ; C(bf16) = gelu'(pre) ; C2(bf16) = gelu(pre)
   EPI_F32_RESID = 2,   // C(f32)  = resid(f32) + acc + bias        (C may alias resid)
   EPI_BF16_DGELU = 3,  // C(bf16) = acc * aux[row % aux_rows, col]   (aux = saved gelu'(pre))
-  EPI_F32 = 4,         // C(f32)  = acc (+ C if accumulate)
-  EPI_LSE = 5,         // online-softmax partials per (row, column tile) + logit of the target column; C (bf16, optional) = acc
+  EPI_F32 = 4,         // C(f32)  = acc * rowscale[row] (+ C if accumulate); rowscale optional
+  EPI_LSE = 5,         // online-softmax partials per (row, column tile) + logit of the target column; C (bf16, optional) =
+                       // acc, or exp(acc) with store_exp
   EPI_DZ = 6,          // C(bf16) = (exp(acc - lse[row]) - [col + col0 == target[row]]) * scale
   EPI_COUNT = 7
 };
@@ -50,6 +51,8 @@ struct GemmArgs {
   const float* lse;   // [M]
   float scale;        // EPI_DZ: 1 / Ntok
   int col0;
+  const float* rowscale;  // EPI_F32: [M] fp32 or NULL
+  int store_exp;      // EPI_LSE with C: store exp(acc) instead of acc
   int tile_blocks;    // 256-column blocks per output tile: 1 (256 x 256), 2 (256 x 512), 0 = chosen from the shape
 };
 

@@ -43,9 +43,10 @@ cudaError_t f32_to_bf16(const float* in, __nv_bfloat16* out, size_t n, cudaStrea
 
 // Merge per-tile online-softmax partials: lse[r] = log sum_t exp(pm[r,t]) * ps[r,t];
 // loss_out += (1/rows) * sum_r (lse[r] - tgt_logit[r])   (loss_out zeroed by the caller).
-// z (bf16 logits [rows, ld], in place) <- (exp(z - lse[row]) - [col == targets[row]]) * scale; columns >= V zeroed
-cudaError_t dz_from_logits(__nv_bfloat16* z, int ld, const float* lse, const int* targets, int rows, int V, float scale,
-                           cudaStream_t s);
+// Head backward set-up on E = exp(logits) (bf16 [rows, ld]): E[r, target_r] -= exp(lse_r); rowscale[r] =
+// exp(-lse_r) / rows; u_scaled[r, :] = rowscale[r] * u[r, :].  Sets *err when an lse lies outside [-80, 80].
+cudaError_t head_backward_prepare(__nv_bfloat16* e, int ld, const float* lse, const int* targets, const __nv_bfloat16* u,
+                                  __nv_bfloat16* u_scaled, float* rowscale, int rows, int d, unsigned* err, cudaStream_t s);
 cudaError_t lse_finalize(const float* part_max, const float* part_sum, int part_ld, int ntiles, const float* tgt_logit,
                          float* lse, float* loss_out, int rows, cudaStream_t s);
 

@@ -51,7 +51,9 @@ struct CompScratch {     // backward scratch of one component, rows = s_cap * nt
 };
 struct HeadScratch {
   bf16* u; float *mean, *rstd, *pmax, *psum, *tgt_logit, *lse, *du, *ghead;
-  bf16* z;   // [Ntok, ldz]: the logits kept by the loss pass, turned into dZ in place by the backward
+  bf16* z;   // [Ntok, ldz]: exp(logits) kept by the loss pass; the backward patches the target column in place
+  bf16* us;  // [Ntok, d]: rows of u scaled by exp(-lse) / Ntok
+  float* rs; // [Ntok]: exp(-lse) / Ntok
 };
 
 struct ProfRec { cudaEvent_t a, b; double flops; };
@@ -497,6 +499,8 @@ extern "C" il_status il_create(int K, int Lc, int d, int H, int F, int V, int n,
     IL_TRY(dev_alloc_t(m, &h.du, N * d));
     IL_TRY(dev_alloc_t(m, &h.ghead, N * d));
     IL_TRY(dev_alloc_t(m, &h.z, N * (size_t)m->ldz));
+    IL_TRY(dev_alloc_t(m, &h.us, N * d));
+    IL_TRY(dev_alloc_t(m, &h.rs, N));
   }
   IL_TRY(alloc_scratch(m, s_cap_for(K, n)));
   IL_TRY(dev_alloc_t(m, &m->tokens, N));
@@ -719,6 +723,7 @@ extern "C" il_status il_aux_head_loss(il_model* m, int k, float* loss_host) {
     g.part_max = h.pmax; g.part_sum = h.psum; g.part_ld = m->part_ld;
     g.tgt_logit = h.tgt_logit;
     g.col0 = 0;
+    g.store_exp = 1;
     IL_TRY(gemm(m, k, g));
     IL_K(m, lse_finalize(h.pmax, h.psum, m->part_ld, m->part_ld, h.tgt_logit, h.lse, m->losses + k, N, st));
     m->loss_done[k] = 1;
@@ -758,21 +763,24 @@ extern "C" il_status il_get_losses(il_model* m, float* losses_host) {
 
 namespace {
 
-// Head k backward on stream k: the saved logits become dZ = (softmax - onehot) / Ntok in place, then
-// dU = dZ W and dW_h = dZ^T U over the whole vocabulary; LayerNorm backward -> ghead.
+// Head k backward on stream k.  The loss pass kept E = exp(logits); dZ = (softmax - onehot) / Ntok equals
+// diag(s) E' with s = exp(-lse) / Ntok and E' = E with exp(lse) subtracted at the target, so after a per-row
+// set-up kernel dU = diag(s) (E' W) and dW_h = E'^T (diag(s) U) run straight on E' — no pass over the
+// [Ntok, V] matrix other than the two GEMMs.  LayerNorm backward -> ghead.
 il_status head_backward(il_model* m, int k) {
   cudaStream_t st = m->streams[k];
   const int N = m->ntok, d = m->d, V = m->V;
   const HeadOff& o = m->head_off[k];
   HeadScratch& h = m->hs[k];
-  IL_K(m, dz_from_logits(h.z, m->ldz, h.lse, m->targets, N, V, 1.0f / (float)N, st));
-  {  // dU = dZ * W.  Not split over the contraction: atomically added partial sums would make dU, and with it
-     // every gradient below this head, depend on the order the work units finish in.
+  IL_K(m, head_backward_prepare(h.z, m->ldz, h.lse, m->targets, h.u, h.us, h.rs, N, d, m->err_word, st));
+  {  // dU = diag(s) (E' W).  Not split over the contraction: atomically added partial sums would make dU, and
+     // with it every gradient below this head, depend on the order the work units finish in.
     GemmArgs g = gemm_args(N, d, V, h.z, m->ldz, 0, m->Pb + o.w, d, 1, EPI_F32, h.du, d);
+    g.rowscale = h.rs;
     IL_TRY(gemm(m, k, g));
   }
-  {  // dW = dZ^T * U
-    GemmArgs g = gemm_args(V, d, N, h.z, m->ldz, 1, h.u, d, 1, EPI_F32, m->G + o.w, d);
+  {  // dW = E'^T (diag(s) U)
+    GemmArgs g = gemm_args(V, d, N, h.z, m->ldz, 1, h.us, d, 1, EPI_F32, m->G + o.w, d);
     IL_TRY(gemm(m, k, g));
   }
   IL_K(m, layernorm_bwd_params(h.du, 1, m->a[k + 1], h.mean, h.rstd, m->G + o.lng, m->G + o.lnb, N, d, st));
@@ -953,6 +961,8 @@ extern "C" il_status il_sync(il_model* m) {
   if (w) {
     IL_CUDA(m, cudaMemsetAsync(m->err_word, 0, 4, m->streams[0]));
     IL_CUDA(m, cudaStreamSynchronize(m->streams[0]));
+    if (w == DEV_LOGIT_RANGE)
+      return fail(m, IL_ERR_NONFINITE, "a head's log-sum-exp left [-80, 80]: exp(logit) is not representable");
     return fail(m, IL_ERR_TIMEOUT, "a bounded device-side wait expired (code %u)", w);
   }
   return IL_OK;
@@ -1043,7 +1053,7 @@ extern "C" il_status il_op_gemm(const il_gemm_desc* q, unsigned* err_word, void*
   g.C2 = q->C2; g.bias = q->bias; g.resid = q->resid; g.aux = q->aux; g.ld_aux = q->ld_aux; g.aux_rows = q->aux_rows; g.colsum = q->colsum;
   g.accumulate = q->accumulate; g.split_k = q->split_k; g.targets = q->targets; g.part_max = q->part_max; g.part_sum = q->part_sum;
   g.part_ld = q->part_ld; g.tgt_logit = q->tgt_logit; g.lse = q->lse; g.scale = q->scale; g.col0 = q->col0;
-  g.tile_blocks = q->tile_blocks;
+  g.tile_blocks = q->tile_blocks; g.rowscale = q->rowscale; g.store_exp = q->store_exp;
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return IL_ERR_CUDA;
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return IL_ERR_CUDA;

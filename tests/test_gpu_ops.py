@@ -151,6 +151,16 @@ def test_gemm_softmax_epilogues(V):
     zg = zt.float().cpu().numpy()
     assert np.max(np.abs(zg[:, :V] - z)) <= 2.0 ** -8 * np.abs(z).max() + 1e-6     # one bf16 rounding
     assert np.all(zg[:, V:] == 7.0)
+    # store_exp: what is kept is exp(logit), rounded once to bf16
+    et = torch.full((M, ldz), 7.0, dtype=torch.bfloat16, device=DEV)
+    il.op_gemm(M, V, K, Ut, K, 0, Wt, K, 0, 5, err, C_=et, ldc=ldz, targets=tt, part_max=pm2, part_sum=ps2,
+               part_ld=ntiles, tgt_logit=tl2, store_exp=1)
+    torch.cuda.synchronize()
+    assert int(err.item()) == 0
+    assert torch.equal(pm2, pm) and torch.equal(ps2, ps) and torch.equal(tl2, tl)
+    eg = et.float().cpu().numpy()
+    assert np.max(np.abs(eg[:, :V] / np.exp(z) - 1.0)) < 2.0 ** -8 + 1e-5
+    assert np.all(eg[:, V:] == 7.0)
     # dZ on a chunk that starts mid-vocabulary and runs past its end
     col0 = (V // 2) // 8 * 8
     nv = V - col0
@@ -308,3 +318,23 @@ def test_gemm_wide_tiles_match_square_tiles(M, N, K, layout, epi):
     ref = (At.float().T if a_mn else At.float()) @ (Bt.float() if b_mn else Bt.float().T)
     got = outs[1][0][:, :N].float() - (0.5 if epi == 2 else 0.0) - (kw["bias"] if epi == 0 else 0.0)
     assert torch.linalg.norm(got - ref) / torch.linalg.norm(ref) < (4e-3 if epi in (0, 5) else 1e-5)
+
+
+def test_gemm_row_scale_on_fp32_output():
+    """Epilogue 4 with a per-row factor (the head's input gradient dU = diag(s) (E W)), with and without accumulation."""
+    rng = np.random.default_rng(11)
+    M, N, K = 300, 264, 520
+    At, Ae = _bf16(rng.standard_normal((M, K)))
+    Bt, Be = _bf16(rng.standard_normal((K, N)) * 0.3)          # MN-major B, as in dgrad
+    sc = rng.uniform(0.1, 3.0, size=M)
+    st = torch.tensor(sc, dtype=torch.float32, device=DEV)
+    Ct = torch.full((M, N), 2.0, dtype=torch.float32, device=DEV)
+    err = _err_word()
+    il.op_gemm(M, N, K, At, K, 0, Bt, N, 1, 4, err, C_=Ct, ldc=N, rowscale=st)
+    torch.cuda.synchronize()
+    ref = (Ae @ Be) * st.cpu().numpy().astype(np.float64)[:, None]
+    assert _rel(Ct.cpu().numpy(), ref) < 2e-6
+    il.op_gemm(M, N, K, At, K, 0, Bt, N, 1, 4, err, C_=Ct, ldc=N, rowscale=st, accumulate=1)
+    torch.cuda.synchronize()
+    assert int(err.item()) == 0
+    assert _rel(Ct.cpu().numpy(), 2 * ref) < 2e-6

@@ -187,3 +187,27 @@ def test_zero_weight_head_gives_ln_vocab():
         assert abs(losses[1] - np.log(w.V)) < 1e-5 * np.log(w.V)
     finally:
         m.close()
+
+
+def test_logit_range_is_checked():
+    """The backward keeps exp(logit) in bf16; a head whose log-sum-exp leaves [-80, 80] must be reported, not
+    silently turned into inf / nan gradients."""
+    from paper_2010_04116_b200.binding import ILError
+    w = wl.CONFIGS["cfg1"]
+    P = wl.draw_params(w)
+    tok, tgt = wl.draw_tokens(w)
+    m = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, 1, w.B, w.T)
+    try:
+        m.set_params(P)
+        m.set_param("head0.w", (P["head0.w"] * 4000.0).astype(np.float32))
+        with pytest.raises(ILError) as ei:
+            m.train_step(tok, tgt)
+            m.sync()
+        assert "IL_ERR_NONFINITE" in str(ei.value)
+        # the model stays usable: with sane parameters the next step is clean
+        m.set_param("head0.w", P["head0.w"])
+        m.train_step(tok, tgt)
+        m.sync()
+        assert np.all(np.isfinite(m.get_grad("head0.w")))
+    finally:
+        m.close()
