@@ -56,6 +56,7 @@ template <int NT> constexpr int smem_bytes() {
 struct GemmDev {
   int M, N, K;
   int tiles_m, tiles_n;
+  int group_m;                   // row blocks per group of the tile order
   int split_k, kb_per_split;     // work unit = (tile, k-range); split_k > 1 adds into C with red.add
   void* C;
   int ldc;
@@ -79,15 +80,17 @@ struct GemmDev {
   unsigned* err;
 };
 
-// Tile order: groups of TILE_GROUP_M row blocks are swept across all column blocks before the next group
-// starts, so that the pairs running at the same time share a small set of A rows and the whole of B in L2.
-constexpr int TILE_GROUP_M = 8;
-__device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int& m_blk, int& n_blk) {
-  const int per_group = TILE_GROUP_M * tiles_n;
+// Tile order: groups of group_m row blocks are swept across all column blocks before the next group starts, so
+// that the pairs running at the same time share a small set of A rows and the whole of B in L2.  B is read from
+// DRAM once per group, A once in total: the host makes the group as tall as the matrix when all of A fits in
+// L2 beside the streams passing through it (the heads' [Ntok, V, d] projection: W would otherwise be read four
+// times), and 8 row blocks otherwise.
+__device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int group_m, int& m_blk, int& n_blk) {
+  const int per_group = group_m * tiles_n;
   const int g = t / per_group;
   const int within = t - g * per_group;
-  const int gm = min(TILE_GROUP_M, tiles_m - g * TILE_GROUP_M);
-  m_blk = g * TILE_GROUP_M + within % gm;
+  const int gm = min(group_m, tiles_m - g * group_m);
+  m_blk = g * group_m + within % gm;
   n_blk = within / gm;
 }
 
@@ -305,7 +308,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       bool ok = true;
       for (int t = pair; t < num_tiles && ok; t += num_pairs) {
         int m_blk, n_blk;
-        tile_coords(t / p.split_k, p.tiles_m, p.tiles_n, m_blk, n_blk);
+        tile_coords(t / p.split_k, p.tiles_m, p.tiles_n, p.group_m, m_blk, n_blk);
         const int m0 = m_blk * TILE_M + (int)rank * BM;       // this CTA's 128 rows of A
         const int n0 = n_blk * (NT * BN) + (int)rank * (BN / 2);   // this CTA's 128 rows of the (first) 256-row block of B
         const int kb0 = (t % p.split_k) * p.kb_per_split;
@@ -409,7 +412,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     bool ok = true;
     for (int t = pair; t < num_tiles && ok; t += num_pairs, ++it) {
       int m_blk, n_tile;
-      tile_coords(t / p.split_k, p.tiles_m, p.tiles_n, m_blk, n_tile);
+      tile_coords(t / p.split_k, p.tiles_m, p.tiles_n, p.group_m, m_blk, n_tile);
       for (int h = 0; h < NT && ok; ++h) {           // the tile's 256-column blocks, one accumulator each
       const int n_blk = n_tile * NT + h;
       const int as = (NT == 1) ? (it & 1) : h;
@@ -762,6 +765,7 @@ cudaError_t gemm_launch(const GemmArgs& a, unsigned* err_word, int num_sms, cuda
   p.M = a.M; p.N = a.N; p.K = a.K;
   p.tiles_m = (a.M + TILE_M - 1) / TILE_M;
   p.tiles_n = (a.N + nt * BN - 1) / (nt * BN);
+  p.group_m = ((long long)a.M * a.K * 2 <= (48ll << 20)) ? p.tiles_m : 8;
   {
     // Split the contraction when the tile count leaves most CTA pairs idle (fp32 outputs only; the caller
     // zeroes C and the partial sums are added with red.global.add).
