@@ -113,16 +113,19 @@ __global__ void __launch_bounds__(128) attn_fwd_tc_kernel(const __grid_constant_
 
   // S_j = Q K_j^T; issued by thread 0 one step ahead (right after the previous block's P V) so that each sweep
   // step waits for the tensor pipe only once
+  // descriptors of the operands at their first stage; a sweep step adds its stage's offset (one add per MMA:
+  // the issuing thread's own instruction stream is on every step's critical path)
+  const SmemDescBase dq_k = make_smem_desc_base(sQ, 16, 1024), dk_k = make_smem_desc_base(sK0, 16, 1024);
+  const SmemDescBase dv_mn = make_smem_desc_base(sV0, TK * 128, 1024);
   auto issue_s = [&](int j) {
     const int st = j % NST;
     if (!mbar_wait(bar_kv0 + 8 * st, (uint32_t)(j / NST) & 1u, abortp)) { fail = 1; abort_flag = 1; }
     tc_fence_after();
+    const uint32_t so = (uint32_t)(st * C::KV_BYTES);
 #pragma unroll
-    for (int ks = 0; ks < DH / 16; ++ks) {
-      const uint64_t ad = make_smem_desc(sQ + (ks >> 2) * (TQ * 128) + (ks & 3) * 32, 16, 1024);
-      const uint64_t bd = make_smem_desc(sK0 + st * C::KV_BYTES + (ks >> 2) * (TK * 128) + (ks & 3) * 32, 16, 1024);
-      umma_bf16(tmem_base, ad, bd, idesc_s, ks ? 1u : 0u);
-    }
+    for (int ks = 0; ks < DH / 16; ++ks)
+      umma_bf16(tmem_base, desc_at(dq_k, (ks >> 2) * (TQ * 128) + (ks & 3) * 32),
+                desc_at(dk_k, so + (ks >> 2) * (TK * 128) + (ks & 3) * 32), idesc_s, ks ? 1u : 0u);
     umma_commit(bar_s);
   };
   if (tid == 0) {
@@ -209,11 +212,10 @@ __global__ void __launch_bounds__(128) attn_fwd_tc_kernel(const __grid_constant_
     if (__syncthreads_or(fail)) { fail = 1; break; }     // uniform exit if any thread's wait expired
     if (tid == 0) {
       tc_fence_after();
+      const uint32_t so = (uint32_t)(st * C::KV_BYTES);
 #pragma unroll
-      for (int ks = 0; ks < TK / 16; ++ks) {
-        const uint64_t bd = make_smem_desc(sV0 + st * C::KV_BYTES + ks * 2048, TK * 128, 1024);   // MN-major
-        umma_bf16_ts(tmem_base + 64, tmem_base + 8 * ks, bd, idesc_o, (j | ks) ? 1u : 0u);         // O accumulates in TMEM
-      }
+      for (int ks = 0; ks < TK / 16; ++ks)       // B = V read MN-major; O accumulates in TMEM
+        umma_bf16_ts(tmem_base + 64, tmem_base + 8 * ks, desc_at(dv_mn, so + ks * 2048), idesc_o, (j | ks) ? 1u : 0u);
       umma_commit(bar_o);
       // every thread has read S_j (barrier above); the tensor pipe runs the P V just issued, which reads the
       // packed columns, before it overwrites them with the next scores
@@ -423,17 +425,22 @@ __global__ void __launch_bounds__(256) attn_bwd_dkv_tc_kernel(const __grid_const
 
   // S^T and dP^T of query block j; issued by thread 0 one step ahead (right after the previous block's dV/dK
   // products) so that each sweep step waits for the tensor pipe only once
+  // descriptors of the operands at their first stage; a sweep step adds its stage's offset (one add per MMA:
+  // the issuing thread's own instruction stream is on every step's critical path)
+  const SmemDescBase dk_k = make_smem_desc_base(sK, 16, 1024), dv_k = make_smem_desc_base(sV, 16, 1024);
+  const SmemDescBase dq_k = make_smem_desc_base(sQ0, 16, 1024), ddo_k = make_smem_desc_base(sdO0, 16, 1024);
+  const SmemDescBase dq_mn = make_smem_desc_base(sQ0, TK * 128, 1024), ddo_mn = make_smem_desc_base(sdO0, TK * 128, 1024);
   auto issue_s = [&](int j) {
     const int it = j - q0, st = it % NST;
     if (!mbar_wait(bar_q0 + 8 * st, (uint32_t)(it / NST) & 1u, abortp)) { fail = 1; abort_flag = 1; }
     tc_fence_after();
+    const uint32_t so = (uint32_t)(st * C::BLK_BYTES);
 #pragma unroll
     for (int ks = 0; ks < DH / 16; ++ks) {
       const uint32_t off_a = (ks >> 2) * (TQ * 128) + (ks & 3) * 32;
-      const uint32_t off_b = st * C::BLK_BYTES + (ks >> 2) * (TK * 128) + (ks & 3) * 32;
-      umma_bf16(tmem_base, make_smem_desc(sK + off_a, 16, 1024), make_smem_desc(sQ0 + off_b, 16, 1024), idesc_s, ks ? 1u : 0u);
-      umma_bf16(tmem_base + 64, make_smem_desc(sV + off_a, 16, 1024), make_smem_desc(sdO0 + off_b, 16, 1024), idesc_s,
-                ks ? 1u : 0u);
+      const uint32_t off_b = so + (ks >> 2) * (TK * 128) + (ks & 3) * 32;
+      umma_bf16(tmem_base, desc_at(dk_k, off_a), desc_at(dq_k, off_b), idesc_s, ks ? 1u : 0u);
+      umma_bf16(tmem_base + 64, desc_at(dv_k, off_a), desc_at(ddo_k, off_b), idesc_s, ks ? 1u : 0u);
     }
     umma_commit(bar_s);
   };
@@ -495,13 +502,13 @@ __global__ void __launch_bounds__(256) attn_bwd_dkv_tc_kernel(const __grid_const
     if (__syncthreads_or(fail)) { fail = 1; break; }
     if (tid == 0) {
       tc_fence_after();
+      const uint32_t so = (uint32_t)(st * C::BLK_BYTES);
 #pragma unroll
       for (int ks = 0; ks < TK / 16; ++ks) {
-        const uint32_t off_b = st * C::BLK_BYTES + ks * 2048;                               // MN-major: 16 queries
-        umma_bf16_ts(tmem_base + 128, tmem_base + packed_col(ks), make_smem_desc(sdO0 + off_b, TK * 128, 1024), idesc_g,
+        const uint32_t off_b = so + ks * 2048;                                              // MN-major: 16 queries
+        umma_bf16_ts(tmem_base + 128, tmem_base + packed_col(ks), desc_at(ddo_mn, off_b), idesc_g, (it | ks) ? 1u : 0u);
+        umma_bf16_ts(tmem_base + 128 + DH, tmem_base + 64 + packed_col(ks), desc_at(dq_mn, off_b), idesc_g,
                      (it | ks) ? 1u : 0u);
-        umma_bf16_ts(tmem_base + 128 + DH, tmem_base + 64 + packed_col(ks), make_smem_desc(sQ0 + off_b, TK * 128, 1024),
-                     idesc_g, (it | ks) ? 1u : 0u);
       }
       umma_commit(bar_acc);
       // every thread has read S^T / dP^T of this step (barrier above); the tensor pipe runs the products just
@@ -645,17 +652,21 @@ __global__ void __launch_bounds__(256) attn_bwd_dq_tc_kernel(const __grid_consta
   const float del = row < T ? delta[((size_t)nb * H + h) * T + row] : 0.f;
 
   // S and dP of key block j; issued by thread 0 one step ahead (right after the previous block's dQ product)
+  // descriptors at the first stage; a sweep step adds its stage's offset (one add per MMA)
+  const SmemDescBase dq_k = make_smem_desc_base(sQ, 16, 1024), ddo_k = make_smem_desc_base(sdO, 16, 1024);
+  const SmemDescBase dk_k = make_smem_desc_base(sK0, 16, 1024), dv_k = make_smem_desc_base(sV0, 16, 1024);
+  const SmemDescBase dk_mn = make_smem_desc_base(sK0, TK * 128, 1024);
   auto issue_s = [&](int j) {
     const int st = j % NST;
     if (!mbar_wait(bar_kv0 + 8 * st, (uint32_t)(j / NST) & 1u, abortp)) { fail = 1; abort_flag = 1; }
     tc_fence_after();
+    const uint32_t so = (uint32_t)(st * C::BLK_BYTES);
 #pragma unroll
     for (int ks = 0; ks < DH / 16; ++ks) {
       const uint32_t off_a = (ks >> 2) * (TQ * 128) + (ks & 3) * 32;
-      const uint32_t off_b = st * C::BLK_BYTES + (ks >> 2) * (TK * 128) + (ks & 3) * 32;
-      umma_bf16(tmem_base, make_smem_desc(sQ + off_a, 16, 1024), make_smem_desc(sK0 + off_b, 16, 1024), idesc_s, ks ? 1u : 0u);
-      umma_bf16(tmem_base + 64, make_smem_desc(sdO + off_a, 16, 1024), make_smem_desc(sV0 + off_b, 16, 1024), idesc_s,
-                ks ? 1u : 0u);
+      const uint32_t off_b = so + (ks >> 2) * (TK * 128) + (ks & 3) * 32;
+      umma_bf16(tmem_base, desc_at(dq_k, off_a), desc_at(dk_k, off_b), idesc_s, ks ? 1u : 0u);
+      umma_bf16(tmem_base + 64, desc_at(ddo_k, off_a), desc_at(dv_k, off_b), idesc_s, ks ? 1u : 0u);
     }
     umma_commit(bar_s);
   };
@@ -698,10 +709,11 @@ __global__ void __launch_bounds__(256) attn_bwd_dq_tc_kernel(const __grid_consta
     if (__syncthreads_or(fail)) { fail = 1; break; }
     if (tid == 0) {
       tc_fence_after();
+      const uint32_t so = (uint32_t)(st * C::BLK_BYTES);
 #pragma unroll
       for (int ks = 0; ks < TK / 16; ++ks)
-        umma_bf16_ts(tmem_base + 128, tmem_base + 64 + packed_col(ks),
-                     make_smem_desc(sK0 + st * C::BLK_BYTES + ks * 2048, TK * 128, 1024), idesc_g, (j | ks) ? 1u : 0u);
+        umma_bf16_ts(tmem_base + 128, tmem_base + 64 + packed_col(ks), desc_at(dk_mn, so + ks * 2048), idesc_g,
+                     (j | ks) ? 1u : 0u);
       umma_commit(bar_acc);
       if (j + 1 < nkv) issue_s(j + 1);
     }

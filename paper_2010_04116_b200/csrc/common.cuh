@@ -256,6 +256,19 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr, uint32_t 
   d |= (uint64_t)2 << 61;   // SWIZZLE_128B
   return d;
 }
+// The same descriptor split so that a loop only adds to the address field: base once, then desc_at(base, bytes)
+// costs one integer add (the 14-bit address field cannot overflow for addresses inside shared memory).
+struct SmemDescBase { uint32_t lo, hi; };
+__device__ __forceinline__ SmemDescBase make_smem_desc_base(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  const uint64_t d = make_smem_desc(smem_addr, lbo_bytes, sbo_bytes);
+  SmemDescBase b;
+  b.lo = (uint32_t)d;
+  b.hi = (uint32_t)(d >> 32);
+  return b;
+}
+__device__ __forceinline__ uint64_t desc_at(SmemDescBase b, uint32_t byte_offset) {
+  return ((uint64_t)b.hi << 32) | (uint64_t)(b.lo + (byte_offset >> 4));
+}
 // Instruction descriptor: bf16 x bf16 -> fp32, M x N tile, operand major-ness (0 = K, 1 = MN).
 __host__ __device__ constexpr uint32_t make_idesc_bf16(int M, int N, int a_mn, int b_mn) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
