@@ -15,7 +15,11 @@ What it follows
 * Auxiliary network h_ck after every component and the local loss
   L_ck(x, y) = L(h_ck(f_ck o ... o f_c1 (x)), y), Sec. 3 (unnumbered equations);
   L is the mean next-token cross-entropy.  The auxiliary network here is
-  LayerNorm followed by an untied linear map to the vocabulary.
+  LayerNorm followed by an untied linear map to the vocabulary; with
+  head_layers > 0 that many Transformer blocks come first, which is the
+  auxiliary network of the paper's Transformer runs (App. B.3).
+* Micro-batching (Sec. 3.1): nwise_gradients_microbatched averages the
+  gradients of equal groups of sequences before the single update.
 * n-wise rule, Sec. 3 and Fig. 2: the gradient of head h flows through its own
   component and across n-1 component boundaries, then stops.  Reading used here:
   the gradients of all heads whose window covers a component are summed with
@@ -27,7 +31,7 @@ What it follows
 * Optimiser: Adam with the hyper-parameters of App. B.3, written as AdamW
   (decoupled weight decay; weight decay 0 gives the paper's Adam).
 
-Pins (tests/test_oracle_*.py): central finite differences of the windowed loss
+Pins (tests/test_oracle_pins.py, tests/test_oracle_aux_blocks.py): central finite differences of the windowed loss
 sums on tiny nets, brute-force softmax/attention/cross-entropy on tiny inputs,
 the locality / nesting / n=K invariants of the rule, ln(V) for a zero-weight
 head, causal-mask independence, closed-form first AdamW step.  No numeric
@@ -231,8 +235,15 @@ def component_bwd(dx: np.ndarray, caches, P, k: int, B: int, T: int, H: int, G):
     return dx
 
 
-def head_loss(a: np.ndarray, targets: np.ndarray, P, k: int, want_grad: bool, row_block: int = 1024):
-    """Auxiliary head k: z = LN(a) W^T, L = mean_i (logsumexp_v z_iv - z_i,y_i).
+def head_loss(a: np.ndarray, targets: np.ndarray, P, k: int, want_grad: bool, row_block: int = 1024,
+              head_layers: int = 0, B: int = 0, T: int = 0, H: int = 0):
+    """Auxiliary head k: z = LN(t(a)) W^T, L = mean_i (logsumexp_v z_iv - z_i,y_i).
+
+    t is the identity for head_layers = 0 (LayerNorm + linear head).  For head_layers > 0 it is that many
+    pre-LN Transformer blocks of the main network's shape with parameters head{k}.l{j}.* — the auxiliary
+    network of the paper's Transformer runs (App. B.3: main network output -> 2 Transformer blocks ->
+    embedding matrix -> logits; the LayerNorm before the matrix is this build's, as pre-LN blocks need one).
+    B, T, H are needed by the blocks' attention only.
 
     Returns (loss, da, grads dict) — the last two None unless want_grad.
     Rows are independent, so they are processed in blocks to bound memory.
@@ -242,6 +253,10 @@ def head_loss(a: np.ndarray, targets: np.ndarray, P, k: int, want_grad: bool, ro
     W = _f64(P[f"head{k}.w"])
     y = targets.reshape(-1)
     N = a.shape[0]
+    hcaches = []
+    for j in range(head_layers):
+        a, c = block_fwd(a, P, f"head{k}.l{j}.", B, T, H)
+        hcaches.append(c)
     u, cache = layernorm_fwd(a, g, b)
     loss = 0.0
     du = np.zeros_like(u) if want_grad else None
@@ -265,7 +280,10 @@ def head_loss(a: np.ndarray, targets: np.ndarray, P, k: int, want_grad: bool, ro
     if not want_grad:
         return loss, None, None
     da, dg, db = layernorm_bwd(du, cache, g)
-    return loss, da, {f"head{k}.ln.g": dg, f"head{k}.ln.b": db, f"head{k}.w": dW}
+    hg = {f"head{k}.ln.g": dg, f"head{k}.ln.b": db, f"head{k}.w": dW}
+    for j in reversed(range(head_layers)):
+        da = block_bwd(da, hcaches[j], P, f"head{k}.l{j}.", B, T, H, hg)
+    return loss, da, hg
 
 
 # ----------------------------------------------------------------------------
@@ -284,9 +302,10 @@ def forward_all(P, tokens: np.ndarray, K: int, Lc: int, H: int):
     return a, caches
 
 
-def head_losses(P, tokens, targets, K: int, Lc: int, H: int) -> List[float]:
+def head_losses(P, tokens, targets, K: int, Lc: int, H: int, head_layers: int = 0) -> List[float]:
+    B, T = tokens.shape
     a, _ = forward_all(P, tokens, K, Lc, H)
-    return [head_loss(a[k + 1], targets, P, k, False)[0] for k in range(K)]
+    return [head_loss(a[k + 1], targets, P, k, False, head_layers=head_layers, B=B, T=T, H=H)[0] for k in range(K)]
 
 
 def head_weight(k: int, h: int, n: int, K: int, rule: str) -> float:
@@ -309,7 +328,7 @@ def head_weight(k: int, h: int, n: int, K: int, rule: str) -> float:
 
 
 def nwise_gradients(P, tokens: np.ndarray, targets: np.ndarray, K: int, Lc: int, H: int, n: int,
-                    head_weights: Optional[Sequence[float]] = None, rule: str = "sum"):
+                    head_weights: Optional[Sequence[float]] = None, rule: str = "sum", head_layers: int = 0):
     """One n-wise step's losses and parameter "gradients" (Sec. 3, Fig. 2).
 
     For every head h (0-based here) its loss is back-propagated through the head
@@ -320,6 +339,8 @@ def nwise_gradients(P, tokens: np.ndarray, targets: np.ndarray, K: int, Lc: int,
     Head parameters always receive their own loss's gradient with weight 1; the
     embeddings belong to component 0.
     head_weights (default all 1) scales each head's loss before back-propagation.
+    head_layers > 0 puts that many Transformer blocks inside every auxiliary head (see head_loss); they are
+    head parameters and so receive only their own loss's gradient.
     """
     if not (1 <= n <= K):
         raise ValueError("n must be in [1, K]")
@@ -328,7 +349,7 @@ def nwise_gradients(P, tokens: np.ndarray, targets: np.ndarray, K: int, Lc: int,
     losses: List[float] = []
     G: Dict[str, np.ndarray] = {}
     for h in range(K):
-        loss, da, hg = head_loss(a[h + 1], targets, P, h, True)
+        loss, da, hg = head_loss(a[h + 1], targets, P, h, True, head_layers=head_layers, B=B, T=T, H=H)
         losses.append(loss)
         wgt = 1.0 if head_weights is None else float(head_weights[h])
         for name, val in hg.items():
@@ -356,6 +377,27 @@ def nwise_gradients(P, tokens: np.ndarray, targets: np.ndarray, K: int, Lc: int,
         if name not in G:
             G[name] = np.zeros(P[name].shape, dtype=F64)
     return losses, G
+
+
+def nwise_gradients_microbatched(P, tokens: np.ndarray, targets: np.ndarray, K: int, Lc: int, H: int, n: int,
+                                 micro_batches: int, rule: str = "sum", head_layers: int = 0):
+    """The same step with the mini-batch split into `micro_batches` equal groups of sequences (Sec. 3.1:
+    micro-batching as in pipeline parallelism): every group is a separate forward/backward, the parameter
+    gradients of the groups are averaged and one update follows.  Returns (mean losses, gradients).
+    With equal group sizes this is the gradient of the whole mini-batch; a test pins that identity."""
+    Bfull = tokens.shape[0]
+    if micro_batches < 1 or Bfull % micro_batches:
+        raise ValueError("the batch must split into equal micro-batches")
+    per = Bfull // micro_batches
+    losses = np.zeros(K, dtype=F64)
+    G: Dict[str, np.ndarray] = {}
+    for mb in range(micro_batches):
+        sl = slice(mb * per, (mb + 1) * per)
+        l, g = nwise_gradients(P, tokens[sl], targets[sl], K, Lc, H, n, rule=rule, head_layers=head_layers)
+        losses += np.asarray(l, dtype=F64) / micro_batches
+        for name, val in g.items():
+            G[name] = G[name] + val / micro_batches if name in G else val / micro_batches
+    return [float(x) for x in losses], G
 
 
 def adamw_step(P: Dict[str, np.ndarray], G: Dict[str, np.ndarray], state: Dict[str, Tuple[np.ndarray, np.ndarray]],

@@ -39,6 +39,9 @@ class Workload:
     n: int            # n-wise parameter (1 = local learning, K = full backprop)
     zipf: bool = True  # token law: Zipf(1.1) if True, uniform otherwise
     adamw: bool = False
+    Lh: int = 0       # Transformer blocks inside every auxiliary head (App. B.3: 2); 0 = LayerNorm + linear head
+    M: int = 1        # micro-batches a mini-batch of B sequences is processed in (Sec. 3.1)
+    rule: str = "sum"  # head weighting: "sum", "far" (Sec. 3 main text) or "mean" (App. B.3)
 
     @property
     def ntok(self) -> int:
@@ -62,6 +65,12 @@ CONFIGS: Dict[str, Workload] = {
     # cfg4's widths, sequence length, batch and vocabulary with only two one-layer components: every kernel
     # runs at cfg4's shapes while the model holds ~3 GB, small enough for profiler captures.
     "cfg4-2x1": Workload("cfg4-2x1", K=2, Lc=1, d=1024, H=16, F=4096, V=50257, T=1024, B=8, n=2, adamw=True),
+    # The shape of the paper's own Transformer runs (App. B.3): modules of 6 blocks, d 1024, 4 attention heads,
+    # sequence length 128, an auxiliary network of 2 blocks + embedding matrix per module, the mean-of-two-heads
+    # rule, Adam; A = 4 modules, a mini-batch of 1024 sequences in 4 micro-batches (Sec. 3.1).  The vocabulary
+    # size is not printed in the paper; the other configurations' 50257 is used.
+    "cfgP": Workload("cfgP", K=4, Lc=6, d=1024, H=4, F=4096, V=50257, T=128, B=1024, n=2, adamw=True, Lh=2, M=4,
+                     rule="mean"),
 }
 
 
@@ -96,6 +105,22 @@ def tensor_specs(w: Workload, max_seq: int | None = None) -> List[Tuple[str, int
                 (p + "mlp.b2", k, False, (w.d,)),
             ]
     for k in range(w.K):
+        for l in range(w.Lh):
+            p = f"head{k}.l{l}."
+            specs += [
+                (p + "ln1.g", k, True, (w.d,)),
+                (p + "ln1.b", k, True, (w.d,)),
+                (p + "attn.wqkv", k, True, (3 * w.d, w.d)),
+                (p + "attn.bqkv", k, True, (3 * w.d,)),
+                (p + "attn.wo", k, True, (w.d, w.d)),
+                (p + "attn.bo", k, True, (w.d,)),
+                (p + "ln2.g", k, True, (w.d,)),
+                (p + "ln2.b", k, True, (w.d,)),
+                (p + "mlp.w1", k, True, (w.F, w.d)),
+                (p + "mlp.b1", k, True, (w.F,)),
+                (p + "mlp.w2", k, True, (w.d, w.F)),
+                (p + "mlp.b2", k, True, (w.d,)),
+            ]
         specs += [
             (f"head{k}.ln.g", k, True, (w.d,)),
             (f"head{k}.ln.b", k, True, (w.d,)),
