@@ -60,6 +60,11 @@ typedef struct {
   int n_streams;
   int use_bias;                     /* reserved, must be 1 (GPT-2 style biases)                      */
   float ln_eps;                     /* <= 0 => 1e-5                                                  */
+  int head_layers;                  /* Transformer blocks inside every auxiliary head, 0..64.  0: the  */
+                                    /* head is LayerNorm + linear.  2 is the auxiliary network of the  */
+                                    /* paper's Transformer runs (App. B.3: main network output ->      */
+                                    /* 2 Transformer blocks -> embedding matrix -> logits); the blocks */
+                                    /* have the main network's shape, the head's LayerNorm follows them */
 } il_options;
 
 /* Build a model: K components x layers_per_component blocks, d_model, n_heads, d_ff, vocab, and the
@@ -85,7 +90,9 @@ il_status il_set_rule(il_model* m, int rule);
 /* Parameter registry.  Order and names: "wte" [V,d], "wpe" [max_seq,d] (component 0: the first
  * module holds the input projection, App. B.3), then per component k and layer l
  * "c{k}.l{l}.{ln1.g,ln1.b,attn.wqkv,attn.bqkv,attn.wo,attn.bo,ln2.g,ln2.b,mlp.w1,mlp.b1,mlp.w2,mlp.b2}",
- * then per head "head{k}.{ln.g,ln.b,w}".  Host fp32 buffers; `count` must equal the tensor size.
+ * then per head k its blocks "head{k}.l{j}.{the same twelve names}" (j < head_layers) followed by
+ * "head{k}.{ln.g,ln.b,w}".  Everything named head{k}.* is a parameter of the auxiliary network of
+ * component k and is updated from L_ck alone (Sec. 3).  Host fp32 buffers; `count` must equal the tensor size.
  * These calls synchronise the device. */
 int il_num_tensors(const il_model* m);
 il_status il_tensor_info(const il_model* m, int idx, const char** name, int* component, int* is_head,
@@ -117,6 +124,14 @@ il_status il_get_losses(il_model* m, float* losses_host);
  * the n components below it, a stop at each window's lowest component input, contributions of
  * overlapping heads summed.  Overwrites all gradients.  Needs all K forwards and head losses. */
 il_status il_backward_nwise(il_model* m);
+/* Micro-batching (Sec. 3.1: a mini-batch is split into M micro-batches and one update follows).  With
+ * M > 1 an update is M rounds of il_set_batch .. il_backward_nwise, one per micro-batch of equal size,
+ * then il_adamw_step: the first il_backward_nwise of an update overwrites the gradients, the later ones
+ * add to them, and each is scaled by 1/M, so that il_get_grad and il_adamw_step see the gradient of the
+ * mean loss over the whole mini-batch.  An (M+1)-th il_backward_nwise and an il_adamw_step after fewer
+ * than M return IL_ERR_STATE.  Calling this function (M >= 1; 1 is the default) starts a new update and
+ * abandons gradients accumulated so far.  Losses are reported per micro-batch. */
+il_status il_set_micro_batches(il_model* m, int micro_batches);
 /* AdamW (decoupled weight decay on rank-2 tensors; weight_decay = 0 is the paper's Adam,
  * App. B.3: beta1 0.9, beta2 0.98, eps 1e-9).  Needs il_backward_nwise.  Increments the step. */
 il_status il_adamw_step(il_model* m, float lr, float beta1, float beta2, float eps, float weight_decay);
@@ -139,6 +154,9 @@ il_status il_profile_read(il_model* m, double* gemm_ms, long long* gemm_launches
  * k are grouped by that level.  Writes the distinct levels, descending, to terms[0..*count) (terms may be
  * NULL; it needs room for min(n, K) ints).  *count is the number of stacked backward passes of k. */
 il_status il_nwise_streams(int K, int n, int k, int* terms, int* count);
+/* Host-only: the learning-rate schedule of the paper's Transformer runs (App. B.3),
+ *   lr = d_model^-0.5 * min(step^-0.5, step * warmup_steps^-1.5),   step >= 1 (the paper: d_model 1024, warm-up 4000). */
+il_status il_lr_schedule(long long step, int d_model, int warmup_steps, double* lr);
 /* Host-only: the paper's time-per-batch model of synchronous depthwise model parallelism (Sec. 3.1):
  * A sequential accelerators (one module each), M micro-batches per mini-batch, N the n-wise parameter
  * (N = 1 local learning, N >= A end-to-end / GPipe), micro-batch cost c(M) = c0 + c1 / M.

@@ -1,2 +1,2 @@
 """B200-native n-wise interlocking-backpropagation training step (CUDA library + thin ctypes binding)."""
-from .binding import ILError, Model, lib, nwise_streams  # noqa: F401
+from .binding import ILError, Model, lib, lr_schedule, nwise_streams  # noqa: F401

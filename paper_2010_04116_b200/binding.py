@@ -31,7 +31,7 @@ class il_options(C.Structure):
     _fields_ = [("device", C.c_int), ("max_batch", C.c_int), ("max_seq", C.c_int),
                 ("alloc", ALLOC_FN), ("free_", FREE_FN), ("alloc_ctx", C.c_void_p),
                 ("streams", C.POINTER(C.c_void_p)), ("n_streams", C.c_int),
-                ("use_bias", C.c_int), ("ln_eps", C.c_float)]
+                ("use_bias", C.c_int), ("ln_eps", C.c_float), ("head_layers", C.c_int)]
 
 
 class il_gemm_desc(C.Structure):
@@ -66,7 +66,8 @@ def lib() -> C.CDLL:
     vp, i, f, sz = C.c_void_p, C.c_int, C.c_float, C.c_size_t
     sig = {
         "il_create": [i, i, i, i, i, i, i, C.POINTER(il_options), C.POINTER(vp)],
-        "il_destroy": [vp], "il_set_n": [vp, i], "il_set_rule": [vp, i],
+        "il_destroy": [vp], "il_set_n": [vp, i], "il_set_rule": [vp, i], "il_set_micro_batches": [vp, i],
+        "il_lr_schedule": [C.c_longlong, i, i, C.POINTER(C.c_double)],
         "il_tensor_info": [vp, i, C.POINTER(C.c_char_p), C.POINTER(i), C.POINTER(i), C.POINTER(i),
                            C.POINTER(C.c_longlong)],
         "il_set_param": [vp, i, vp, sz], "il_get_param": [vp, i, vp, sz], "il_get_grad": [vp, i, vp, sz],
@@ -124,6 +125,14 @@ def time_per_batch(A: int, M: int, N: int, c0: float, c1: float) -> float:
     return out.value
 
 
+def lr_schedule(step: int, d_model: int, warmup_steps: int = 4000) -> float:
+    out = C.c_double(0)
+    st = lib().il_lr_schedule(step, d_model, warmup_steps, C.byref(out))
+    if st != IL_OK:
+        raise ILError(st, "il_lr_schedule")
+    return out.value
+
+
 def optimal_microbatches(A: int, N: int, c0: float, c1: float, max_log2: int = 10) -> int:
     out = C.c_int(0)
     st = lib().il_optimal_microbatches(A, N, c0, c1, max_log2, C.byref(out))
@@ -143,7 +152,7 @@ class Model:
     the K per-component streams are torch streams."""
 
     def __init__(self, K: int, Lc: int, d: int, H: int, F: int, V: int, n: int, max_batch: int, max_seq: int,
-                 device: int = 0, torch_alloc: bool = True, torch_streams: bool = True):
+                 device: int = 0, torch_alloc: bool = True, torch_streams: bool = True, head_layers: int = 0):
         import torch
         self._torch = torch
         self.L = lib()
@@ -156,6 +165,7 @@ class Model:
         opt.max_batch, opt.max_seq = max_batch, max_seq
         opt.use_bias = 1
         opt.ln_eps = 1e-5
+        opt.head_layers = head_layers
         dev = torch.device("cuda", device)
         if torch_alloc:
             def _alloc(nbytes, ctx):
@@ -254,6 +264,10 @@ class Model:
         """'sum' (default), 'far' (the paper's main-text rule) or 'mean' (its Transformer variant)."""
         self._ck(self.L.il_set_rule(self._h, self.RULES[rule]))
 
+    def set_micro_batches(self, micro_batches: int):
+        """Process every mini-batch as this many micro-batch steps before one update (Sec. 3.1)."""
+        self._ck(self.L.il_set_micro_batches(self._h, micro_batches))
+
     def set_n(self, n: int):
         self._ck(self.L.il_set_n(self._h, n))
         self.n = n
@@ -333,6 +347,15 @@ class Model:
             self.forward_component(k)
             self.aux_head_loss(k)
         self.backward_nwise()
+        if adamw is not None:
+            self.adamw_step(**adamw)
+
+    def train_minibatch(self, tokens, targets, micro_batches: int, adamw: Optional[dict] = None):
+        """One update from a mini-batch processed as `micro_batches` equal groups of sequences (Sec. 3.1);
+        il_set_micro_batches(micro_batches) must be in effect.  Asynchronous."""
+        per = tokens.shape[0] // micro_batches
+        for mb in range(micro_batches):
+            self.train_step(tokens[mb * per:(mb + 1) * per], targets[mb * per:(mb + 1) * per])
         if adamw is not None:
             self.adamw_step(**adamw)
 

@@ -46,11 +46,12 @@ __global__ void embed_bwd_wte_kernel(const int* __restrict__ tok, const float* _
     atomicAdd(dwte + (size_t)t * d + c, dx[i]);
   }
 }
-__global__ void embed_bwd_wpe_kernel(const float* __restrict__ dx, float* __restrict__ dwpe, int B, int T, int d) {
+__global__ void embed_bwd_wpe_kernel(const float* __restrict__ dx, float* __restrict__ dwpe, int B, int T, int d,
+                                     int accumulate) {
   const int d4 = d >> 2;
   const size_t total = (size_t)T * d4;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float4 acc = accumulate ? reinterpret_cast<const float4*>(dwpe)[i] : make_float4(0.f, 0.f, 0.f, 0.f);
     for (int b = 0; b < B; ++b) {
       const float4 v = reinterpret_cast<const float4*>(dx + (size_t)b * T * d)[i];
       acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
@@ -60,12 +61,12 @@ __global__ void embed_bwd_wpe_kernel(const float* __restrict__ dx, float* __rest
 }
 
 cudaError_t embed_bwd(const int* tok, const float* dx, float* dwte, float* dwpe, int ntok, int T, int d, int V,
-                      cudaStream_t s) {
+                      int accumulate, cudaStream_t s) {
   int blocks = ceil_div((size_t)ntok * d, 256);
   if (blocks > 148 * 16) blocks = 148 * 16;
   embed_bwd_wte_kernel<<<blocks, 256, 0, s>>>(tok, dx, dwte, ntok, d, V);
   int blocks2 = ceil_div((size_t)T * (d / 4), 256);
-  embed_bwd_wpe_kernel<<<blocks2, 256, 0, s>>>(dx, dwpe, ntok / T, T, d);
+  embed_bwd_wpe_kernel<<<blocks2, 256, 0, s>>>(dx, dwpe, ntok / T, T, d, accumulate);
   return cudaGetLastError();
 }
 
@@ -459,10 +460,10 @@ __global__ void __launch_bounds__(256) head_backward_prepare_kernel(bf16* __rest
 }
 
 cudaError_t head_backward_prepare(bf16* e, int ld, const float* lse, const int* targets, const bf16* u, bf16* u_scaled,
-                                  float* rowscale, int rows, int d, unsigned* err, cudaStream_t s) {
+                                  float* rowscale, int rows, int d, float scale, unsigned* err, cudaStream_t s) {
   if ((d % 8) || ((uintptr_t)u % 16) || ((uintptr_t)u_scaled % 16) || !err) return cudaErrorInvalidValue;
   head_backward_prepare_kernel<<<ceil_div(rows, 8), 256, 0, s>>>(e, ld, lse, targets, u, u_scaled, rowscale, rows, d,
-                                                                 1.0f / (float)rows, err);
+                                                                 scale / (float)rows, err);
   return cudaGetLastError();
 }
 

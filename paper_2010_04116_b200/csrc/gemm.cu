@@ -106,28 +106,50 @@ template <int EPI>
 __device__ __forceinline__ void epilogue_rowwise(const GemmDev& p, int col, float (&v)[32], RowState& st) {
   const bool full = (col + 32 <= p.N);
   if constexpr (EPI == EPI_LSE) {
+    constexpr float L2E = 1.4426950408889634f;
     float cm = -INFINITY;
 #pragma unroll
     for (int j = 0; j < 32; ++j)
       if (full || col + j < p.N) cm = fmaxf(cm, v[j]);
-    if (cm > -INFINITY) {
-      float nm = fmaxf(st.m, cm);
-      float acc = 0.0f;
-#pragma unroll
-      for (int j = 0; j < 32; ++j)
-        if (full || col + j < p.N) acc += __expf(v[j] - nm);
-      st.s = st.s * __expf(st.m - nm) + acc;
-      st.m = nm;
-    }
     int tj = st.tgt - (p.col0 + col);
     if (tj >= 0 && tj < 32) {
 #pragma unroll
       for (int j = 0; j < 32; ++j)
         if (j == tj) st.tl = v[j];
     }
-    if (p.store_exp) {       // what is kept for the backward is exp(logit): softmax up to a per-row factor
+    if (p.store_exp) {
+      // What is kept for the backward is E = exp(logit) (softmax up to a per-row factor), so each element needs
+      // one exponential only: while the running maximum stays where exp() of it is far from the fp32 range, the
+      // chunk's share of the softmax sum is the sum of the stored values times one factor per chunk.
+      const float nm = fmaxf(st.m, cm);
+      const bool direct = fabsf(nm) < 64.0f;      // nm = -inf (nothing valid yet) takes the general branch
+      float acc = 0.0f;
+      if (direct) {
 #pragma unroll
-      for (int j = 0; j < 32; ++j) v[j] = __expf(v[j]);
+        for (int j = 0; j < 32; ++j) {
+          v[j] = ex2_fast(v[j] * L2E);
+          if (full || col + j < p.N) acc += v[j];
+        }
+        acc *= ex2_fast(-nm * L2E);
+      } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          if (full || col + j < p.N) acc += ex2_fast((v[j] - nm) * L2E);
+          v[j] = ex2_fast(v[j] * L2E);
+        }
+      }
+      if (cm > -INFINITY) {
+        st.s = st.s * ex2_fast((st.m - nm) * L2E) + acc;
+        st.m = nm;
+      }
+    } else if (cm > -INFINITY) {
+      const float nm = fmaxf(st.m, cm);
+      float acc = 0.0f;
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (full || col + j < p.N) acc += ex2_fast((v[j] - nm) * L2E);
+      st.s = st.s * ex2_fast((st.m - nm) * L2E) + acc;
+      st.m = nm;
     }
   } else if constexpr (EPI == EPI_DZ) {
     const float l = st.m;   // lse of this row

@@ -10,9 +10,10 @@ namespace il {
 // a_0[i,:] = wte[clamp(tok[i]),:] + wpe[i % T,:]  (fp32 residual stream)
 cudaError_t embed_fwd(const int* tok, const float* wte, const float* wpe, float* x, int ntok, int T, int d, int V,
                       cudaStream_t s);
-// dwte[tok[i],:] += dx[i,:] (atomic), dwpe[t,:] = sum_b dx[b*T+t,:];  dwte must be zeroed by the caller.
+// dwte[tok[i],:] += dx[i,:] (atomic), dwpe[t,:] = (accumulate ? dwpe[t,:] : 0) + sum_b dx[b*T+t,:];  dwte must be
+// zeroed by the caller (or hold the sum it is to be added to).
 cudaError_t embed_bwd(const int* tok, const float* dx, float* dwte, float* dwpe, int ntok, int T, int d, int V,
-                      cudaStream_t s);
+                      int accumulate, cudaStream_t s);
 
 // y(bf16) = gamma * (x - mean) * rstd + beta per row; mean/rstd saved in fp32.
 cudaError_t layernorm_fwd(const float* x, const float* gamma, const float* beta, __nv_bfloat16* y, float* mean,
@@ -44,9 +45,10 @@ cudaError_t f32_to_bf16(const float* in, __nv_bfloat16* out, size_t n, cudaStrea
 // Merge per-tile online-softmax partials: lse[r] = log sum_t exp(pm[r,t]) * ps[r,t];
 // loss_out += (1/rows) * sum_r (lse[r] - tgt_logit[r])   (loss_out zeroed by the caller).
 // Head backward set-up on E = exp(logits) (bf16 [rows, ld]): E[r, target_r] -= exp(lse_r); rowscale[r] =
-// exp(-lse_r) / rows; u_scaled[r, :] = rowscale[r] * u[r, :].  Sets *err when an lse lies outside [-80, 80].
+// scale * exp(-lse_r) / rows; u_scaled[r, :] = rowscale[r] * u[r, :].  Sets *err when an lse lies outside [-80, 80].
 cudaError_t head_backward_prepare(__nv_bfloat16* e, int ld, const float* lse, const int* targets, const __nv_bfloat16* u,
-                                  __nv_bfloat16* u_scaled, float* rowscale, int rows, int d, unsigned* err, cudaStream_t s);
+                                  __nv_bfloat16* u_scaled, float* rowscale, int rows, int d, float scale, unsigned* err,
+                                  cudaStream_t s);
 cudaError_t lse_finalize(const float* part_max, const float* part_sum, int part_ld, int ntiles, const float* tgt_logit,
                          float* lse, float* loss_out, int rows, cudaStream_t s);
 

@@ -62,6 +62,8 @@ struct ProfRec { cudaEvent_t a, b; double flops; };
 
 struct il_model {
   int K, Lc, d, H, F, V, n, dh;
+  int Lh;                             // Transformer blocks inside every auxiliary head (0 = LayerNorm + linear)
+  int micro, micro_done;              // micro-batches per update, backward passes since the last update
   int rule;                           // IL_RULE_*: which heads update a component's parameters
   int device, num_sms;
   int max_batch, max_seq, ntok_max;
@@ -73,7 +75,7 @@ struct il_model {
   cudaEvent_t ev_batch;
   // parameters
   std::vector<TensorRec> tensors;
-  std::vector<LayerOff> layer_off;   // K*Lc
+  std::vector<LayerOff> layer_off;   // K*Lc main layers, then K*Lh head layers (head k's at K*Lc + k*Lh)
   std::vector<HeadOff> head_off;     // K
   size_t off_wte, off_wpe;
   std::vector<size_t> comp_begin, comp_mat_end, comp_end;   // flat ranges per component
@@ -83,7 +85,7 @@ struct il_model {
   long long step;
   // activations
   std::vector<float*> a;             // K+1 boundaries; a[k+1] aliases the last layer's x_out
-  std::vector<LayerActs> acts;       // K*Lc
+  std::vector<LayerActs> acts;       // same indexing as layer_off
   std::vector<CompScratch> cs;
   std::vector<HeadScratch> hs;
   int s_cap;
@@ -243,7 +245,8 @@ GemmArgs gemm_args(int M, int N, int K, const void* A, int lda, int a_mn, const 
 // into (partial sums are added atomically into the zeroed gradient) are chosen together, by a small model of
 // the kernel: waves of units over the pairs, times the k-slabs of a unit (a 512-wide slab costs 1.72 of a
 // 256-wide one) plus the unit's exposed prologue / epilogue.
-il_status wgrad(il_model* m, int k, int M, int N, int K, const bf16* dY, int ld_dy, const bf16* X, int ld_x, float* dW) {
+il_status wgrad(il_model* m, int k, int M, int N, int K, const bf16* dY, int ld_dy, const bf16* X, int ld_x, float* dW,
+                bool acc) {
   const int pairs = m->num_sms / 2;
   const int slabs = (K + 63) / 64;
   int best_nt = 1, best_s = 1;
@@ -263,8 +266,11 @@ il_status wgrad(il_model* m, int k, int M, int N, int K, const bf16* dY, int ld_
   GemmArgs g = gemm_args(M, N, K, dY, ld_dy, 1, X, ld_x, 1, EPI_F32, dW, N);
   g.tile_blocks = best_nt;
   if (best_s > 1) {
-    IL_CUDA(m, cudaMemsetAsync(dW, 0, (size_t)M * N * sizeof(float), m->streams[k]));
+    // split units add their partial sums into the output: zero it first, unless this pass adds to the last one's
+    if (!acc) IL_CUDA(m, cudaMemsetAsync(dW, 0, (size_t)M * N * sizeof(float), m->streams[k]));
     g.split_k = best_s;
+  } else {
+    g.accumulate = acc ? 1 : 0;
   }
   return gemm(m, k, g);
 }
@@ -298,6 +304,12 @@ il_status join_all(il_model* m) {
   return IL_OK;
 }
 
+// input of head k's LayerNorm: the component's output, or the output of the head's own blocks
+const float* head_input(const il_model* m, int k) {
+  if (m->Lh == 0) return m->a[k + 1];
+  return m->acts[(size_t)m->K * m->Lc + (size_t)k * m->Lh + m->Lh - 1].x_out;
+}
+
 il_status check_model(const il_model* m) { return m ? IL_OK : IL_ERR_INVALID_ARG; }
 
 // Stream-ordered copy on stream 0 followed by a wait: the data is in place when this returns.
@@ -316,6 +328,7 @@ extern "C" il_status il_create(int K, int Lc, int d, int H, int F, int V, int n,
   if (!out) return IL_ERR_INVALID_ARG;
   *out = nullptr;
   if (!opt || K < 1 || Lc < 1 || d < 8 || H < 1 || F < 8 || V < 2 || n < 1 || n > K) return IL_ERR_INVALID_ARG;
+  if (opt->head_layers < 0 || opt->head_layers > 64) return IL_ERR_INVALID_ARG;
   if (d % H || d % 8 || F % 8 || opt->max_batch < 1 || opt->max_seq < 1) return IL_ERR_INVALID_ARG;
   const int dh = d / H;
   if (!(dh == 32 || dh == 64 || dh == 80 || dh == 128)) return IL_ERR_INVALID_ARG;
@@ -325,6 +338,7 @@ extern "C" il_status il_create(int K, int Lc, int d, int H, int F, int V, int n,
   il_model* m = new (std::nothrow) il_model();
   if (!m) return IL_ERR_OOM;
   m->K = K; m->Lc = Lc; m->d = d; m->H = H; m->F = F; m->V = V; m->n = n; m->dh = dh;
+  m->Lh = opt->head_layers; m->micro = 1; m->micro_done = 0;
   m->opt = *opt;
   m->device = opt->device;
   m->max_batch = opt->max_batch; m->max_seq = opt->max_seq;
@@ -363,16 +377,21 @@ extern "C" il_status il_create(int K, int Lc, int d, int H, int F, int V, int n,
   add("wpe", 0, 0, 2, m->max_seq, d);
   const char* lnames[12] = {"ln1.g", "ln1.b", "attn.wqkv", "attn.bqkv", "attn.wo", "attn.bo",
                             "ln2.g", "ln2.b", "mlp.w1", "mlp.b1", "mlp.w2", "mlp.b2"};
+  const long long ls0[12] = {d, d, 3LL * d, 3LL * d, d, d, d, d, F, F, d, d};
+  const long long ls1[12] = {0, 0, d, 0, d, 0, 0, 0, d, 0, F, 0};
+  const int Lh = m->Lh;
   for (int k = 0; k < K; ++k)
     for (int l = 0; l < Lc; ++l) {
       char pre[64];
       snprintf(pre, sizeof pre, "c%d.l%d.", k, l);
-      const long long s0[12] = {d, d, 3LL * d, 3LL * d, d, d, d, d, F, F, d, d};
-      const long long s1[12] = {0, 0, d, 0, d, 0, 0, 0, d, 0, F, 0};
-      for (int i = 0; i < 12; ++i) add(std::string(pre) + lnames[i], k, 0, s1[i] ? 2 : 1, s0[i], s1[i]);
+      for (int i = 0; i < 12; ++i) add(std::string(pre) + lnames[i], k, 0, ls1[i] ? 2 : 1, ls0[i], ls1[i]);
     }
   for (int k = 0; k < K; ++k) {
     char pre[64];
+    for (int l = 0; l < Lh; ++l) {       // the auxiliary network's own blocks (App. B.3), same shape as the main ones
+      snprintf(pre, sizeof pre, "head%d.l%d.", k, l);
+      for (int i = 0; i < 12; ++i) add(std::string(pre) + lnames[i], k, 1, ls1[i] ? 2 : 1, ls0[i], ls1[i]);
+    }
     snprintf(pre, sizeof pre, "head%d.", k);
     add(std::string(pre) + "ln.g", k, 1, 1, d, 0);
     add(std::string(pre) + "ln.b", k, 1, 1, d, 0);
@@ -393,20 +412,21 @@ extern "C" il_status il_create(int K, int Lc, int d, int H, int F, int V, int n,
     m->comp_end[k] = cur;
   }
   m->total = cur;
-  m->layer_off.resize((size_t)K * Lc);
+  m->layer_off.resize((size_t)K * (Lc + Lh));
   m->head_off.resize(K);
   {
     size_t i = 0;
     m->off_wte = m->tensors[i++].off;
     m->off_wpe = m->tensors[i++].off;
-    for (int kl = 0; kl < K * Lc; ++kl) {
-      LayerOff& o = m->layer_off[kl];
+    auto take_layer = [&](LayerOff& o) {
       o.ln1g = m->tensors[i++].off; o.ln1b = m->tensors[i++].off; o.wqkv = m->tensors[i++].off;
       o.bqkv = m->tensors[i++].off; o.wo = m->tensors[i++].off; o.bo = m->tensors[i++].off;
       o.ln2g = m->tensors[i++].off; o.ln2b = m->tensors[i++].off; o.w1 = m->tensors[i++].off;
       o.b1 = m->tensors[i++].off; o.w2 = m->tensors[i++].off; o.b2 = m->tensors[i++].off;
-    }
+    };
+    for (int kl = 0; kl < K * Lc; ++kl) take_layer(m->layer_off[kl]);
     for (int k = 0; k < K; ++k) {
+      for (int l = 0; l < Lh; ++l) take_layer(m->layer_off[(size_t)K * Lc + (size_t)k * Lh + l]);
       HeadOff& o = m->head_off[k];
       o.lng = m->tensors[i++].off; o.lnb = m->tensors[i++].off; o.w = m->tensors[i++].off;
     }
@@ -465,10 +485,10 @@ extern "C" il_status il_create(int K, int Lc, int d, int H, int F, int V, int n,
   const size_t N = m->ntok_max;
   m->a.assign(K + 1, nullptr);
   IL_TRY(dev_alloc_t(m, &m->a[0], N * d));
-  m->acts.resize((size_t)K * Lc);
+  m->acts.resize((size_t)K * (Lc + Lh));
   for (int k = 0; k < K; ++k)
-    for (int l = 0; l < Lc; ++l) {
-      LayerActs& A = m->acts[(size_t)k * Lc + l];
+    for (int l = 0; l < Lc + Lh; ++l) {
+      LayerActs& A = l < Lc ? m->acts[(size_t)k * Lc + l] : m->acts[(size_t)K * Lc + (size_t)k * Lh + (l - Lc)];
       IL_TRY(dev_alloc_t(m, &A.ln1, N * d));
       IL_TRY(dev_alloc_t(m, &A.qkv, N * 3 * d));
       IL_TRY(dev_alloc_t(m, &A.attn_o, N * d));
@@ -482,7 +502,7 @@ extern "C" il_status il_create(int K, int Lc, int d, int H, int F, int V, int n,
       IL_TRY(dev_alloc_t(m, &A.lse, N * H));
       IL_TRY(dev_alloc_t(m, &A.x_mid, N * d));
       IL_TRY(dev_alloc_t(m, &A.x_out, N * d));
-      if (l == Lc - 1) m->a[k + 1] = A.x_out;
+      if (l == Lc - 1) m->a[k + 1] = A.x_out;   // the component's output; head blocks (l >= Lc) follow it
     }
   m->part_ld = (V + 127) / 128;
   m->ldz = (V + 63) / 64 * 64;
@@ -656,24 +676,15 @@ extern "C" il_status il_set_batch(il_model* m, const int* tokens, const int* tar
   return IL_OK;
 }
 
-extern "C" il_status il_forward_component(il_model* m, int k) {
-  IL_TRY(check_model(m));
-  if (k < 0 || k >= m->K) return fail(m, IL_ERR_INVALID_ARG, "component %d out of range", k);
-  if (!m->batch_set) return fail(m, IL_ERR_STATE, "il_forward_component before il_set_batch");
-  if (k > 0 && !m->fwd_done[k - 1]) return fail(m, IL_ERR_STATE, "component %d forward needs component %d first", k, k - 1);
-  if (m->fwd_done[k]) return fail(m, IL_ERR_STATE, "component %d already forwarded in this step", k);
-  IL_CUDA(m, cudaSetDevice(m->device));
+namespace {
+
+// `count` consecutive pre-LN blocks (layer records base .. base+count-1) applied to x_in on stream k.
+il_status layers_forward(il_model* m, int k, size_t base, int count, const float* x_in) {
   cudaStream_t st = m->streams[k];
   const int N = m->ntok, d = m->d, F = m->F;
-  if (k == 0) {
-    IL_K(m, embed_fwd(m->tokens, m->P + m->off_wte, m->P + m->off_wpe, m->a[0], N, m->T, d, m->V, st));
-  } else {
-    IL_CUDA(m, cudaStreamWaitEvent(st, m->ev_fwd[k - 1], 0));
-  }
-  const float* x_in = m->a[k];
-  for (int l = 0; l < m->Lc; ++l) {
-    const LayerOff& o = m->layer_off[(size_t)k * m->Lc + l];
-    LayerActs& A = m->acts[(size_t)k * m->Lc + l];
+  for (int l = 0; l < count; ++l) {
+    const LayerOff& o = m->layer_off[base + l];
+    LayerActs& A = m->acts[base + l];
     IL_K(m, layernorm_fwd(x_in, m->P + o.ln1g, m->P + o.ln1b, A.ln1, A.mean1, A.rstd1, N, d, m->ln_eps, st));
     {
       GemmArgs g = gemm_args(N, 3 * d, d, A.ln1, d, 0, m->Pb + o.wqkv, d, 0, EPI_BF16, A.qkv, 3 * d);
@@ -702,6 +713,26 @@ extern "C" il_status il_forward_component(il_model* m, int k) {
     }
     x_in = A.x_out;
   }
+  return IL_OK;
+}
+
+}  // namespace
+
+extern "C" il_status il_forward_component(il_model* m, int k) {
+  IL_TRY(check_model(m));
+  if (k < 0 || k >= m->K) return fail(m, IL_ERR_INVALID_ARG, "component %d out of range", k);
+  if (!m->batch_set) return fail(m, IL_ERR_STATE, "il_forward_component before il_set_batch");
+  if (k > 0 && !m->fwd_done[k - 1]) return fail(m, IL_ERR_STATE, "component %d forward needs component %d first", k, k - 1);
+  if (m->fwd_done[k]) return fail(m, IL_ERR_STATE, "component %d already forwarded in this step", k);
+  IL_CUDA(m, cudaSetDevice(m->device));
+  cudaStream_t st = m->streams[k];
+  const int N = m->ntok, d = m->d;
+  if (k == 0) {
+    IL_K(m, embed_fwd(m->tokens, m->P + m->off_wte, m->P + m->off_wpe, m->a[0], N, m->T, d, m->V, st));
+  } else {
+    IL_CUDA(m, cudaStreamWaitEvent(st, m->ev_fwd[k - 1], 0));
+  }
+  IL_TRY(layers_forward(m, k, (size_t)k * m->Lc, m->Lc, m->a[k]));
   IL_CUDA(m, cudaEventRecord(m->ev_fwd[k], st));
   m->fwd_done[k] = 1;
   return IL_OK;
@@ -717,7 +748,10 @@ extern "C" il_status il_aux_head_loss(il_model* m, int k, float* loss_host) {
     const int N = m->ntok, d = m->d, V = m->V;
     const HeadOff& o = m->head_off[k];
     HeadScratch& h = m->hs[k];
-    IL_K(m, layernorm_fwd(m->a[k + 1], m->P + o.lng, m->P + o.lnb, h.u, h.mean, h.rstd, N, d, m->ln_eps, st));
+    const size_t hbase = (size_t)m->K * m->Lc + (size_t)k * m->Lh;
+    if (m->Lh > 0) IL_TRY(layers_forward(m, k, hbase, m->Lh, m->a[k + 1]));
+    const float* hx = head_input(m, k);
+    IL_K(m, layernorm_fwd(hx, m->P + o.lng, m->P + o.lnb, h.u, h.mean, h.rstd, N, d, m->ln_eps, st));
     GemmArgs g = gemm_args(N, V, d, h.u, d, 0, m->Pb + o.w, d, 0, EPI_LSE, h.z, m->ldz);
     g.targets = m->targets;
     g.part_max = h.pmax; g.part_sum = h.psum; g.part_ld = m->part_ld;
@@ -763,16 +797,59 @@ extern "C" il_status il_get_losses(il_model* m, float* losses_host) {
 
 namespace {
 
+// Backward on stream k through `count` consecutive blocks (layer records base .. base+count-1, whose first block
+// read x_first) for s stacked gradient streams already placed in cs[k].dx / dxb; the result is left there.
+// acc: parameter gradients are added to what the buffers hold (a later micro-batch) instead of replacing it.
+il_status layers_backward(il_model* m, int k, int s, size_t base, int count, const float* x_first, bool acc) {
+  cudaStream_t st = m->streams[k];
+  const int N = m->ntok, d = m->d, F = m->F;
+  const int R = s * N;
+  CompScratch& c = m->cs[k];
+  for (int l = count - 1; l >= 0; --l) {
+    const LayerOff& o = m->layer_off[base + l];
+    LayerActs& A = m->acts[base + l];
+    const float* x_in = (l == 0) ? x_first : m->acts[base + l - 1].x_out;
+    // ---- MLP: x_out = x_mid + W2 gelu(W1 ln2 + b1) + b2
+    IL_K(m, colsum_f32(c.dx, d, m->G + o.b2, N, d, st));
+    IL_TRY(wgrad(m, k, d, F, N, c.dxb, d, A.hact, F, m->G + o.w2, acc));
+    {
+      GemmArgs g = gemm_args(R, F, d, c.dxb, d, 0, m->Pb + o.w2, F, 1, EPI_BF16_DGELU, c.dbig, F);
+      g.aux = A.hgrad; g.ld_aux = F; g.aux_rows = N;
+      g.colsum = m->G + o.b1;                 // FC1 bias gradient: column sums of the first gradient stream
+      IL_TRY(gemm(m, k, g));
+    }
+    IL_TRY(wgrad(m, k, F, d, N, c.dbig, F, A.ln2, d, m->G + o.w1, acc));
+    IL_TRY(gemm(m, k, gemm_args(R, d, F, c.dbig, F, 0, m->Pb + o.w1, d, 1, EPI_BF16, c.dln, d)));
+    IL_K(m, layernorm_bwd_params(c.dln, 0, A.x_mid, A.mean2, A.rstd2, m->G + o.ln2g, m->G + o.ln2b, N, d, st));
+    IL_K(m, layernorm_bwd_rows(c.dln, 0, A.x_mid, A.mean2, A.rstd2, m->P + o.ln2g, c.dx, c.dx, c.dxb, R, N, d, st));
+    // ---- attention: x_mid = x_in + Wo attn(Wqkv ln1 + bqkv) + bo
+    IL_K(m, colsum_f32(c.dx, d, m->G + o.bo, N, d, st));
+    IL_TRY(wgrad(m, k, d, d, N, c.dxb, d, A.attn_o, d, m->G + o.wo, acc));
+    IL_TRY(gemm(m, k, gemm_args(R, d, d, c.dxb, d, 0, m->Pb + o.wo, d, 1, EPI_BF16, c.dattn, d)));
+    IL_K(m, attention_bwd(A.qkv, A.attn_o, A.lse, c.dattn, c.dqkv, c.delta, s * m->B, m->B, m->T, m->H, m->dh, m->err_word, st));
+    m->launches += 2;
+    IL_K(m, colsum_bf16(c.dqkv, 3 * d, m->G + o.bqkv, N, 3 * d, st));
+    IL_TRY(wgrad(m, k, 3 * d, d, N, c.dqkv, 3 * d, A.ln1, d, m->G + o.wqkv, acc));
+    IL_TRY(gemm(m, k, gemm_args(R, d, 3 * d, c.dqkv, 3 * d, 0, m->Pb + o.wqkv, d, 1, EPI_BF16, c.dln, d)));
+    IL_K(m, layernorm_bwd_params(c.dln, 0, x_in, A.mean1, A.rstd1, m->G + o.ln1g, m->G + o.ln1b, N, d, st));
+    IL_K(m, layernorm_bwd_rows(c.dln, 0, x_in, A.mean1, A.rstd1, m->P + o.ln1g, c.dx, c.dx, c.dxb, R, N, d, st));
+  }
+  return IL_OK;
+}
+
 // Head k backward on stream k.  The loss pass kept E = exp(logits); dZ = (softmax - onehot) / Ntok equals
 // diag(s) E' with s = exp(-lse) / Ntok and E' = E with exp(lse) subtracted at the target, so after a per-row
 // set-up kernel dU = diag(s) (E' W) and dW_h = E'^T (diag(s) U) run straight on E' — no pass over the
 // [Ntok, V] matrix other than the two GEMMs.  LayerNorm backward -> ghead.
-il_status head_backward(il_model* m, int k) {
+// With blocks inside the head (App. B.3) the gradient then runs through them, in the component's backward
+// scratch (free at this point of stream k), and ghead is the gradient at the component's output either way.
+// acc / scale: this pass adds scale * gradient to the buffers (micro-batch 2.. of an update) or overwrites them.
+il_status head_backward(il_model* m, int k, bool acc, float scale) {
   cudaStream_t st = m->streams[k];
   const int N = m->ntok, d = m->d, V = m->V;
   const HeadOff& o = m->head_off[k];
   HeadScratch& h = m->hs[k];
-  IL_K(m, head_backward_prepare(h.z, m->ldz, h.lse, m->targets, h.u, h.us, h.rs, N, d, m->err_word, st));
+  IL_K(m, head_backward_prepare(h.z, m->ldz, h.lse, m->targets, h.u, h.us, h.rs, N, d, scale, m->err_word, st));
   {  // dU = diag(s) (E' W).  Not split over the contraction: atomically added partial sums would make dU, and
      // with it every gradient below this head, depend on the order the work units finish in.
     GemmArgs g = gemm_args(N, d, V, h.z, m->ldz, 0, m->Pb + o.w, d, 1, EPI_F32, h.du, d);
@@ -781,49 +858,24 @@ il_status head_backward(il_model* m, int k) {
   }
   {  // dW = E'^T (diag(s) U)
     GemmArgs g = gemm_args(V, d, N, h.z, m->ldz, 1, h.us, d, 1, EPI_F32, m->G + o.w, d);
+    g.accumulate = acc ? 1 : 0;
     IL_TRY(gemm(m, k, g));
   }
-  IL_K(m, layernorm_bwd_params(h.du, 1, m->a[k + 1], h.mean, h.rstd, m->G + o.lng, m->G + o.lnb, N, d, st));
-  IL_K(m, layernorm_bwd_rows(h.du, 1, m->a[k + 1], h.mean, h.rstd, m->P + o.lng, nullptr, h.ghead, nullptr, N, N, d, st));
+  const float* hx = head_input(m, k);
+  IL_K(m, layernorm_bwd_params(h.du, 1, hx, h.mean, h.rstd, m->G + o.lng, m->G + o.lnb, N, d, st));
+  if (m->Lh == 0) {
+    IL_K(m, layernorm_bwd_rows(h.du, 1, hx, h.mean, h.rstd, m->P + o.lng, nullptr, h.ghead, nullptr, N, N, d, st));
+    return IL_OK;
+  }
+  CompScratch& c = m->cs[k];
+  IL_K(m, layernorm_bwd_rows(h.du, 1, hx, h.mean, h.rstd, m->P + o.lng, nullptr, c.dx, c.dxb, N, N, d, st));
+  IL_TRY(layers_backward(m, k, 1, (size_t)m->K * m->Lc + (size_t)k * m->Lh, m->Lh, m->a[k + 1], acc));
+  IL_CUDA(m, cudaMemcpyAsync(h.ghead, c.dx, (size_t)N * d * sizeof(float), cudaMemcpyDeviceToDevice, st));
   return IL_OK;
 }
 
-// Component k backward on stream k for s stacked gradient streams already placed in cs[k].dx / dxb.
-il_status component_backward(il_model* m, int k, int s) {
-  cudaStream_t st = m->streams[k];
-  const int N = m->ntok, d = m->d, F = m->F;
-  const int R = s * N;
-  CompScratch& c = m->cs[k];
-  for (int l = m->Lc - 1; l >= 0; --l) {
-    const LayerOff& o = m->layer_off[(size_t)k * m->Lc + l];
-    LayerActs& A = m->acts[(size_t)k * m->Lc + l];
-    const float* x_in = (l == 0) ? m->a[k] : m->acts[(size_t)k * m->Lc + l - 1].x_out;
-    // ---- MLP: x_out = x_mid + W2 gelu(W1 ln2 + b1) + b2
-    IL_K(m, colsum_f32(c.dx, d, m->G + o.b2, N, d, st));
-    IL_TRY(wgrad(m, k, d, F, N, c.dxb, d, A.hact, F, m->G + o.w2));
-    {
-      GemmArgs g = gemm_args(R, F, d, c.dxb, d, 0, m->Pb + o.w2, F, 1, EPI_BF16_DGELU, c.dbig, F);
-      g.aux = A.hgrad; g.ld_aux = F; g.aux_rows = N;
-      g.colsum = m->G + o.b1;                 // FC1 bias gradient: column sums of the first gradient stream
-      IL_TRY(gemm(m, k, g));
-    }
-    IL_TRY(wgrad(m, k, F, d, N, c.dbig, F, A.ln2, d, m->G + o.w1));
-    IL_TRY(gemm(m, k, gemm_args(R, d, F, c.dbig, F, 0, m->Pb + o.w1, d, 1, EPI_BF16, c.dln, d)));
-    IL_K(m, layernorm_bwd_params(c.dln, 0, A.x_mid, A.mean2, A.rstd2, m->G + o.ln2g, m->G + o.ln2b, N, d, st));
-    IL_K(m, layernorm_bwd_rows(c.dln, 0, A.x_mid, A.mean2, A.rstd2, m->P + o.ln2g, c.dx, c.dx, c.dxb, R, N, d, st));
-    // ---- attention: x_mid = x_in + Wo attn(Wqkv ln1 + bqkv) + bo
-    IL_K(m, colsum_f32(c.dx, d, m->G + o.bo, N, d, st));
-    IL_TRY(wgrad(m, k, d, d, N, c.dxb, d, A.attn_o, d, m->G + o.wo));
-    IL_TRY(gemm(m, k, gemm_args(R, d, d, c.dxb, d, 0, m->Pb + o.wo, d, 1, EPI_BF16, c.dattn, d)));
-    IL_K(m, attention_bwd(A.qkv, A.attn_o, A.lse, c.dattn, c.dqkv, c.delta, s * m->B, m->B, m->T, m->H, m->dh, m->err_word, st));
-    m->launches += 2;
-    IL_K(m, colsum_bf16(c.dqkv, 3 * d, m->G + o.bqkv, N, 3 * d, st));
-    IL_TRY(wgrad(m, k, 3 * d, d, N, c.dqkv, 3 * d, A.ln1, d, m->G + o.wqkv));
-    IL_TRY(gemm(m, k, gemm_args(R, d, 3 * d, c.dqkv, 3 * d, 0, m->Pb + o.wqkv, d, 1, EPI_BF16, c.dln, d)));
-    IL_K(m, layernorm_bwd_params(c.dln, 0, x_in, A.mean1, A.rstd1, m->G + o.ln1g, m->G + o.ln1b, N, d, st));
-    IL_K(m, layernorm_bwd_rows(c.dln, 0, x_in, A.mean1, A.rstd1, m->P + o.ln1g, c.dx, c.dx, c.dxb, R, N, d, st));
-  }
-  return IL_OK;
+il_status component_backward(il_model* m, int k, int s, bool acc) {
+  return layers_backward(m, k, s, (size_t)k * m->Lc, m->Lc, m->a[k], acc);
 }
 
 }  // namespace
@@ -835,20 +887,28 @@ extern "C" il_status il_backward_nwise(il_model* m) {
     if (!m->fwd_done[k] || !m->loss_done[k])
       return fail(m, IL_ERR_STATE, "il_backward_nwise needs all %d forwards and head losses (component %d missing)", m->K, k);
   if (m->bwd_done) return fail(m, IL_ERR_STATE, "il_backward_nwise already called in this step");
+  if (m->micro > 1 && m->micro_done >= m->micro)
+    return fail(m, IL_ERR_STATE, "all %d micro-batches of this update have been back-propagated; call il_adamw_step", m->micro);
   IL_CUDA(m, cudaSetDevice(m->device));
   const int K = m->K, n = m->n, N = m->ntok, d = m->d;
   const size_t slice = (size_t)N * d;
+  // Micro-batching (Sec. 3.1): the first backward pass of an update overwrites the gradients, the later ones add
+  // to them; each pass is scaled by 1 / micro-batches so that the buffers end up holding the mini-batch mean.
+  const bool acc = m->micro > 1 && m->micro_done > 0;
+  const float gscale = 1.0f / (float)m->micro;
 
   // every head's own backward is independent of the others: enqueue all of them first
   for (int k = 0; k < K; ++k) {
     cudaStream_t st = m->streams[k];
-    IL_CUDA(m, cudaMemsetAsync(m->G + m->comp_mat_end[k], 0, (m->comp_end[k] - m->comp_mat_end[k]) * 4, st));
-    if (k == 0) {
-      const size_t emb = (size_t)m->V * d;
-      IL_CUDA(m, cudaMemsetAsync(m->G + m->off_wte, 0, emb * 4, st));
-      IL_CUDA(m, cudaMemsetAsync(m->G + m->off_wpe, 0, (size_t)m->max_seq * d * 4, st));
+    if (!acc) {   // vectors and embeddings are summed into atomically
+      IL_CUDA(m, cudaMemsetAsync(m->G + m->comp_mat_end[k], 0, (m->comp_end[k] - m->comp_mat_end[k]) * 4, st));
+      if (k == 0) {
+        const size_t emb = (size_t)m->V * d;
+        IL_CUDA(m, cudaMemsetAsync(m->G + m->off_wte, 0, emb * 4, st));
+        IL_CUDA(m, cudaMemsetAsync(m->G + m->off_wpe, 0, (size_t)m->max_seq * d * 4, st));
+      }
     }
-    IL_TRY(head_backward(m, k));
+    IL_TRY(head_backward(m, k, acc, gscale));
   }
   if (m->rule == IL_RULE_SUM) {
     // components from the top down; component k needs the pass-down of component k+1 when any stream crosses
@@ -869,9 +929,9 @@ extern "C" il_status il_backward_nwise(il_model* m) {
         const float* passed = src >= 0 ? m->cs[k + 1].dx + (size_t)src * slice : nullptr;
         IL_K(m, add_convert(m->hs[k].ghead, passed, m->cs[k].dx + (size_t)j * slice, m->cs[k].dxb + (size_t)j * slice, slice, st));
       }
-      IL_TRY(component_backward(m, k, s));
+      IL_TRY(component_backward(m, k, s, acc));
       if (k == 0) {
-        IL_K(m, embed_bwd(m->tokens, m->cs[0].dx, m->G + m->off_wte, m->G + m->off_wpe, N, m->T, d, m->V, st));
+        IL_K(m, embed_bwd(m->tokens, m->cs[0].dx, m->G + m->off_wte, m->G + m->off_wpe, N, m->T, d, m->V, acc ? 1 : 0, st));
         m->launches++;
       }
       IL_CUDA(m, cudaEventRecord(m->ev_bwd[k], st));
@@ -919,9 +979,9 @@ extern "C" il_status il_backward_nwise(il_model* m) {
         if (!src) return fail(m, IL_ERR_STATE, "internal: gradient stream of head %d missing at component %d", mine[q], k);
         IL_K(m, add_convert(src, nullptr, m->cs[k].dx + (q + 1) * slice, m->cs[k].dxb + (q + 1) * slice, slice, st));
       }
-      IL_TRY(component_backward(m, k, 1 + (int)mine.size()));
+      IL_TRY(component_backward(m, k, 1 + (int)mine.size(), acc));
       if (k == 0) {
-        IL_K(m, embed_bwd(m->tokens, m->cs[0].dx, m->G + m->off_wte, m->G + m->off_wpe, N, m->T, d, m->V, st));
+        IL_K(m, embed_bwd(m->tokens, m->cs[0].dx, m->G + m->off_wte, m->G + m->off_wpe, N, m->T, d, m->V, acc ? 1 : 0, st));
         m->launches++;
       }
       IL_CUDA(m, cudaEventRecord(m->ev_bwd[k], st));
@@ -929,12 +989,31 @@ extern "C" il_status il_backward_nwise(il_model* m) {
     }
   }
   m->bwd_done = true;
+  m->micro_done = m->micro > 1 ? m->micro_done + 1 : 1;
+  return IL_OK;
+}
+
+extern "C" il_status il_set_micro_batches(il_model* m, int micro_batches) {
+  IL_TRY(check_model(m));
+  if (micro_batches < 1) return fail(m, IL_ERR_INVALID_ARG, "micro_batches must be >= 1");
+  m->micro = micro_batches;
+  m->micro_done = 0;      // gradients accumulated so far are abandoned: the next backward pass overwrites them
+  return IL_OK;
+}
+
+extern "C" il_status il_lr_schedule(long long step, int d_model, int warmup_steps, double* lr) {
+  if (step < 1 || d_model < 1 || warmup_steps < 1 || !lr) return IL_ERR_INVALID_ARG;
+  const double s = (double)step, w = (double)warmup_steps;
+  const double a = 1.0 / sqrt(s), b = s / (w * sqrt(w));
+  *lr = (a < b ? a : b) / sqrt((double)d_model);
   return IL_OK;
 }
 
 extern "C" il_status il_adamw_step(il_model* m, float lr, float beta1, float beta2, float eps, float wd) {
   IL_TRY(check_model(m));
   if (!m->bwd_done || !m->batch_set) return fail(m, IL_ERR_STATE, "il_adamw_step needs il_backward_nwise of the current step");
+  if (m->micro_done != m->micro)
+    return fail(m, IL_ERR_STATE, "il_adamw_step after %d of %d micro-batches", m->micro_done, m->micro);
   if (!(beta1 >= 0 && beta1 < 1 && beta2 >= 0 && beta2 < 1 && eps >= 0)) return fail(m, IL_ERR_INVALID_ARG, "bad AdamW hyper-parameters");
   IL_CUDA(m, cudaSetDevice(m->device));
   m->step += 1;
@@ -949,6 +1028,7 @@ extern "C" il_status il_adamw_step(il_model* m, float lr, float beta1, float bet
                   (float)bc2, m->streams[k]));
   }
   m->batch_set = false;   // a new batch is required for the next step
+  m->micro_done = 0;
   return IL_OK;
 }
 

@@ -157,7 +157,10 @@ def test_gemm_softmax_epilogues(V):
                part_ld=ntiles, tgt_logit=tl2, store_exp=1)
     torch.cuda.synchronize()
     assert int(err.item()) == 0
-    assert torch.equal(pm2, pm) and torch.equal(ps2, ps) and torch.equal(tl2, tl)
+    # with store_exp the partial sums are formed from the stored exponentials times one factor per 32-column
+    # chunk: the same numbers up to rounding order
+    assert torch.equal(pm2, pm) and torch.equal(tl2, tl)
+    assert torch.allclose(ps2, ps, rtol=2e-6, atol=0)
     eg = et.float().cpu().numpy()
     assert np.max(np.abs(eg[:, :V] / np.exp(z) - 1.0)) < 2.0 ** -8 + 1e-5
     assert np.all(eg[:, V:] == 7.0)

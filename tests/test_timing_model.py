@@ -61,3 +61,20 @@ def test_library_matches_oracle_everywhere():
         il.time_per_batch(0, 1, 1, C0, C1)
     with pytest.raises(il.ILError):
         il.optimal_microbatches(4, 2, -1.0, C1)
+
+
+def test_lr_schedule_matches_the_paper_formula():
+    """App. B.3: lr = 1024^-0.5 min(step^-0.5, step warmup^-1.5) with 4000 warm-up steps: linear warm-up to
+    the peak (d warmup)^-0.5 at step = warmup, inverse square root decay afterwards."""
+    import math
+
+    from oracle import il_oracle as orc
+    assert il.lr_schedule(4000, 1024, 4000) == pytest.approx((1024 * 4000) ** -0.5, rel=1e-14)
+    assert il.lr_schedule(1, 1024, 4000) == pytest.approx(1024 ** -0.5 * 4000 ** -1.5, rel=1e-14)
+    assert il.lr_schedule(16000, 1024, 4000) == pytest.approx(0.5 * il.lr_schedule(4000, 1024, 4000), rel=1e-14)
+    for step in (1, 7, 3999, 4000, 4001, 123456):
+        assert il.lr_schedule(step, 1024, 4000) == pytest.approx(orc.inverse_sqrt_lr(step, 1024, 4000), rel=1e-14)
+        assert il.lr_schedule(step, 768, 100) == pytest.approx(
+            768 ** -0.5 * min(1 / math.sqrt(step), step / 100 ** 1.5), rel=1e-14)
+    with pytest.raises(il.ILError):
+        il.lr_schedule(0, 1024, 4000)
