@@ -69,7 +69,7 @@ typedef struct {
 
 /* Build a model: K components x layers_per_component blocks, d_model, n_heads, d_ff, vocab, and the
  * n of the n-wise rule (Sec. 3: N in [1, number of modules]).  Requires d_model % n_heads == 0,
- * head dim in {32, 64, 80, 128}, d_model % 8 == 0, d_ff % 8 == 0.  opt must be non-NULL with
+ * head dim in {32, 64, 80, 128, 256}, d_model % 8 == 0, d_ff % 8 == 0.  opt must be non-NULL with
  * max_batch, max_seq > 0.  Parameters start at zero (LayerNorm gains at one); set them with
  * il_set_param. */
 il_status il_create(int K, int layers_per_component, int d_model, int n_heads, int d_ff, int vocab,

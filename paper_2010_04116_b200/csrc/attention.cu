@@ -33,7 +33,7 @@ struct FwdCfg {
   static constexpr int Q_BYTES = NCH * TQ * 128;
   static constexpr int KV_BYTES = NCH * TK * 128;
   static constexpr int NST = (DH <= 64) ? 3 : 2;               // K/V ring depth: as deep as keeps three (dh <= 64) or two CTAs per SM
-  static constexpr int TCOLS = (64 + DH <= 128) ? 128 : 256;   // 64 score columns + the O accumulator
+  static constexpr int TCOLS = (64 + DH <= 128) ? 128 : (64 + DH <= 256) ? 256 : 512;   // 64 score columns + the O accumulator
   static constexpr int SMEM = Q_BYTES + NST * 2 * KV_BYTES + 1024 + 128;
 };
 
@@ -306,15 +306,16 @@ cudaError_t fwd_tc_launch(const bf16* qkv, bf16* o, float* lse, int B, int T, in
 template <int DH>
 struct BwdCfg {
   static constexpr int NCH = (DH + 63) / 64;
-  static constexpr int NST = 4;                         // ring depth of the swept tiles
+  static constexpr int NST = (DH > 128) ? 1 : 4;        // ring depth of the swept tiles (one 64 KB stage is all that fits at dh 256)
+  static constexpr bool AHEAD = NST > 1;                // the next step's scores are issued one step ahead (needs a second stage)
   static constexpr int ROW_BYTES = NCH * TQ * 128;      // a 128-row operand (all chunks)
   static constexpr int BLK_BYTES = NCH * TK * 128;      // a 64-row operand
   // dK/dV: K, V resident; ring of (Q, dO); lse/delta vectors.  TMEM: S^T, dP^T, dV, dK.
   static constexpr int SMEM_KV = 2 * ROW_BYTES + NST * 2 * BLK_BYTES + 1024 + 2 * 2 * 64 * 4 + 128;
-  static constexpr int TCOLS_KV = (128 + 2 * DH <= 256) ? 256 : 512;
+  static constexpr int TCOLS_KV = (128 + 2 * DH <= 256) ? 256 : 512;   // dh 256: one accumulator per launch (PART)
   // dQ: Q, dO resident; ring of (K, V).  TMEM: S, dP, dQ.
   static constexpr int SMEM_Q = 2 * ROW_BYTES + NST * 2 * BLK_BYTES + 1024 + 128;
-  static constexpr int TCOLS_Q = 256;
+  static constexpr int TCOLS_Q = (128 + DH <= 256) ? 256 : 512;
 };
 
 // 32 fp32 values -> 16 words of bf16 pairs (even index in the low half)
@@ -326,7 +327,9 @@ __device__ __forceinline__ void pack_row32(const float (&v)[32], uint32_t (&w)[1
 // their first 16 columns) of the A operand of K-step ks (16 elements = 8 columns)
 __device__ __forceinline__ constexpr uint32_t packed_col(int ks) { return (uint32_t)((ks >> 1) * 32 + (ks & 1) * 8); }
 
-template <int DH>
+// PART: 0 = dV and dK in one launch; 1 = dV only; 2 = dK only (head dimensions whose two accumulators do not fit
+// the 512 TMEM columns together run as two launches, each recomputing the scores).
+template <int DH, int PART>
 __global__ void __launch_bounds__(256) attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmRow,   // qkv, 128-row box
                                                               const __grid_constant__ CUtensorMap tmBlk,   // qkv, 64-row box
                                                               const __grid_constant__ CUtensorMap tmdO,    // dout, 64-row box
@@ -440,13 +443,13 @@ __global__ void __launch_bounds__(256) attn_bwd_dkv_tc_kernel(const __grid_const
       const uint32_t off_a = (ks >> 2) * (TQ * 128) + (ks & 3) * 32;
       const uint32_t off_b = so + (ks >> 2) * (TK * 128) + (ks & 3) * 32;
       umma_bf16(tmem_base, desc_at(dk_k, off_a), desc_at(dq_k, off_b), idesc_s, ks ? 1u : 0u);
-      umma_bf16(tmem_base + 64, desc_at(dv_k, off_a), desc_at(ddo_k, off_b), idesc_s, ks ? 1u : 0u);
+      if (PART != 1) umma_bf16(tmem_base + 64, desc_at(dv_k, off_a), desc_at(ddo_k, off_b), idesc_s, ks ? 1u : 0u);
     }
     umma_commit(bar_s);
   };
   if (tid == 0 && q0 < nq) {
     if (!mbar_wait(bar_kv, 0, abortp)) { fail = 1; abort_flag = 1; }
-    issue_s(q0);
+    if (C::AHEAD) issue_s(q0);
   }
 
   for (int j = q0; j < nq; ++j) {
@@ -454,10 +457,19 @@ __global__ void __launch_bounds__(256) attn_bwd_dkv_tc_kernel(const __grid_const
     const int st = it % NST;
     if (j + 1 < nq) put_vec(j + 1, vec_next);      // visible after this step's barrier
     vec_next = fetch_vec(j + 2);
+    if (!C::AHEAD) {
+      // single stage: the previous step's products must have retired before its tiles are replaced and the
+      // new scores overwrite the packed columns; only then are this step's scores issued
+      if (it > 0) {
+        if (!mbar_wait(bar_acc, (uint32_t)(it - 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
+        if (tid == 0) load_q(j);
+      }
+      if (tid == 0) issue_s(j);
+    }
     if (!mbar_wait(bar_s, (uint32_t)it & 1u, abortp)) { fail = 1; abort_flag = 1; }
     // the previous step's dV/dK products were issued before these scores, so they have landed too: the packed
     // P^T / dS^T columns and that step's Q/dO stage are free
-    if (it > 0) {
+    if (C::AHEAD && it > 0) {
       if (!mbar_wait(bar_acc, (uint32_t)(it - 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
       if (tid == 0 && j - 1 + NST < nq) load_q(j - 1 + NST);
     }
@@ -466,7 +478,7 @@ __global__ void __launch_bounds__(256) attn_bwd_dkv_tc_kernel(const __grid_const
       float p[32], ds[32];
       uint32_t r0[32], r1[32];
       tmem_ld_32x32(t_lane + 32 * hf, r0);
-      tmem_ld_32x32(t_lane + 64 + 32 * hf, r1);
+      if (PART != 1) tmem_ld_32x32(t_lane + 64 + 32 * hf, r1);
       tmem_ld_wait();
       const float4* lv = reinterpret_cast<const float4*>(s_lse + (j & 1) * 64 + 32 * hf);
       const float4* dv_ = reinterpret_cast<const float4*>(s_del + (j & 1) * 64 + 32 * hf);
@@ -481,7 +493,7 @@ __global__ void __launch_bounds__(256) attn_bwd_dkv_tc_kernel(const __grid_const
         for (int e = 0; e < 4; ++e) {
           const int i = 4 * i4 + e;
           p[i] = ex2_fast(fmaf(__uint_as_float(r0[i]), c2, -ll[e]));
-          ds[i] = __uint_as_float(r1[i]) - dd[e];
+          ds[i] = PART != 1 ? __uint_as_float(r1[i]) - dd[e] : 0.f;
         }
       }
       if (diag || tail) {                          // uniform: only blocks on the diagonal or past the sequence end
@@ -492,10 +504,14 @@ __global__ void __launch_bounds__(256) attn_bwd_dkv_tc_kernel(const __grid_const
 #pragma unroll
       for (int i = 0; i < 32; ++i) ds[i] *= p[i];
       uint32_t pw[16], dw[16];
-      pack_row32(p, pw);
-      pack_row32(ds, dw);
-      tmem_st_32x16(t_lane + 32 * hf, pw);         // P^T over the first half of the S^T columns this thread read
-      tmem_st_32x16(t_lane + 64 + 32 * hf, dw);    // dS^T likewise over dP^T
+      if (PART != 2) {
+        pack_row32(p, pw);
+        tmem_st_32x16(t_lane + 32 * hf, pw);       // P^T over the first half of the S^T columns this thread read
+      }
+      if (PART != 1) {
+        pack_row32(ds, dw);
+        tmem_st_32x16(t_lane + 64 + 32 * hf, dw);  // dS^T likewise over dP^T
+      }
       tmem_st_wait();
     }
     tc_fence_before();
@@ -506,14 +522,16 @@ __global__ void __launch_bounds__(256) attn_bwd_dkv_tc_kernel(const __grid_const
 #pragma unroll
       for (int ks = 0; ks < TK / 16; ++ks) {
         const uint32_t off_b = so + ks * 2048;                                              // MN-major: 16 queries
-        umma_bf16_ts(tmem_base + 128, tmem_base + packed_col(ks), desc_at(ddo_mn, off_b), idesc_g, (it | ks) ? 1u : 0u);
-        umma_bf16_ts(tmem_base + 128 + DH, tmem_base + 64 + packed_col(ks), desc_at(dq_mn, off_b), idesc_g,
-                     (it | ks) ? 1u : 0u);
+        if (PART != 2)
+          umma_bf16_ts(tmem_base + 128, tmem_base + packed_col(ks), desc_at(ddo_mn, off_b), idesc_g, (it | ks) ? 1u : 0u);
+        if (PART != 1)
+          umma_bf16_ts(tmem_base + 128 + (PART == 0 ? DH : 0), tmem_base + 64 + packed_col(ks), desc_at(dq_mn, off_b), idesc_g,
+                       (it | ks) ? 1u : 0u);
       }
       umma_commit(bar_acc);
       // every thread has read S^T / dP^T of this step (barrier above); the tensor pipe runs the products just
       // issued, which read the packed columns, before it overwrites them with the next scores
-      if (j + 1 < nq) issue_s(j + 1);
+      if (C::AHEAD && j + 1 < nq) issue_s(j + 1);
     }
   }
   const int nit = nq - q0;
@@ -525,12 +543,15 @@ __global__ void __launch_bounds__(256) attn_bwd_dkv_tc_kernel(const __grid_const
   if (!fail) {
     bf16* rowp = dqkv + ((size_t)nb * T + key) * (3 * d) + h * DH;
     {
-      const int which = hf;                          // first half of the threads writes dV, second half dK
-      const uint32_t tcol = t_lane + 128 + which * DH;
+      // one launch for both: the first half of the threads writes dV, the second half dK; a launch that holds
+      // one of them splits its columns between the two halves
+      const int which = PART == 0 ? hf : PART - 1;
+      const uint32_t tcol = t_lane + 128 + (PART == 0 ? which * DH : 0);
       bf16* dst = rowp + (which == 0 ? 2 * d : d);
       const float f = which == 0 ? 1.0f : scale;
+      const int cbeg = PART == 0 ? 0 : hf * (DH / 2), cend = PART == 0 ? DH : cbeg + DH / 2;
 #pragma unroll
-      for (int c0 = 0; c0 < DH; c0 += 32) {
+      for (int c0 = cbeg; c0 < cend; c0 += 32) {
         float v[32];
         if (c0 + 32 <= DH) {
           uint32_t rr[32];
@@ -672,13 +693,20 @@ __global__ void __launch_bounds__(256) attn_bwd_dq_tc_kernel(const __grid_consta
   };
   if (tid == 0 && nkv > 0) {
     if (!mbar_wait(bar_q, 0, abortp)) { fail = 1; abort_flag = 1; }
-    issue_s(0);
+    if (C::AHEAD) issue_s(0);
   }
 
   for (int j = 0; j < nkv; ++j) {
     const int st = j % NST;
+    if (!C::AHEAD) {      // single stage: retire the previous step's product, replace its tiles, then issue these scores
+      if (j > 0) {
+        if (!mbar_wait(bar_acc, (uint32_t)(j - 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
+        if (tid == 0) load_kv(j);
+      }
+      if (tid == 0) issue_s(j);
+    }
     if (!mbar_wait(bar_s, (uint32_t)j & 1u, abortp)) { fail = 1; abort_flag = 1; }
-    if (j > 0) {                                     // issued before these scores: landed, the packed dS and that step's K/V stage are free
+    if (C::AHEAD && j > 0) {                         // issued before these scores: landed, the packed dS and that step's K/V stage are free
       if (!mbar_wait(bar_acc, (uint32_t)(j - 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
       if (tid == 0 && j - 1 + NST < nkv) load_kv(j - 1 + NST);
     }
@@ -715,7 +743,7 @@ __global__ void __launch_bounds__(256) attn_bwd_dq_tc_kernel(const __grid_consta
         umma_bf16_ts(tmem_base + 128, tmem_base + 64 + packed_col(ks), desc_at(dk_mn, so + ks * 2048), idesc_g,
                      (j | ks) ? 1u : 0u);
       umma_commit(bar_acc);
-      if (j + 1 < nkv) issue_s(j + 1);
+      if (C::AHEAD && j + 1 < nkv) issue_s(j + 1);
     }
   }
   if (!fail && nkv > 0) {
@@ -816,7 +844,15 @@ cudaError_t bwd_tc_launch(const bf16* qkv, const bf16* o, const float* lse, cons
   if (!tma_encode_bf16(&tmRow, qkv, 4, dims, strides, box128) || !tma_encode_bf16(&tmBlk, qkv, 4, dims, strides, box64) ||
       !tma_encode_bf16(&tmdO64, dout, 4, ddims, dstrides, box64) || !tma_encode_bf16(&tmdO128, dout, 4, ddims, dstrides, box128))
     return cudaErrorInvalidValue;
-  cudaError_t e = cudaFuncSetAttribute(attn_bwd_dkv_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_KV);
+  constexpr bool SPLIT = 128 + 2 * DH > 512;      // dV and dK accumulators do not fit TMEM together: one launch each
+  cudaError_t e = cudaSuccess;
+  if constexpr (SPLIT) {
+    e = cudaFuncSetAttribute(attn_bwd_dkv_tc_kernel<DH, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_KV);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(attn_bwd_dkv_tc_kernel<DH, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_KV);
+  } else {
+    e = cudaFuncSetAttribute(attn_bwd_dkv_tc_kernel<DH, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_KV);
+  }
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(attn_bwd_dq_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_Q);
   if (e != cudaSuccess) return e;
@@ -825,7 +861,12 @@ cudaError_t bwd_tc_launch(const bf16* qkv, const bf16* o, const float* lse, cons
   attn_delta_tc_kernel<DH><<<(unsigned)((nthreads + 255) / 256), 256, 0, s>>>(dout, o, delta, NB, B, T, H);
   dim3 grid((T + TQ - 1) / TQ, NB * H);
   const float scale = rsqrtf((float)DH);
-  attn_bwd_dkv_tc_kernel<DH><<<grid, 256, C::SMEM_KV, s>>>(tmRow, tmBlk, tmdO64, lse, delta, dqkv, B, T, H, scale, err);
+  if constexpr (SPLIT) {
+    attn_bwd_dkv_tc_kernel<DH, 1><<<grid, 256, C::SMEM_KV, s>>>(tmRow, tmBlk, tmdO64, lse, delta, dqkv, B, T, H, scale, err);
+    attn_bwd_dkv_tc_kernel<DH, 2><<<grid, 256, C::SMEM_KV, s>>>(tmRow, tmBlk, tmdO64, lse, delta, dqkv, B, T, H, scale, err);
+  } else {
+    attn_bwd_dkv_tc_kernel<DH, 0><<<grid, 256, C::SMEM_KV, s>>>(tmRow, tmBlk, tmdO64, lse, delta, dqkv, B, T, H, scale, err);
+  }
   attn_bwd_dq_tc_kernel<DH><<<grid, 256, C::SMEM_Q, s>>>(tmRow, tmBlk, tmdO128, lse, delta, dqkv, B, T, H, scale, err);
   return cudaGetLastError();
 }
@@ -840,6 +881,7 @@ cudaError_t attention_fwd(const bf16* qkv, bf16* o, float* lse, int B, int T, in
     case 64: return fwd_tc_launch<64>(qkv, o, lse, B, T, H, err, s);
     case 80: return fwd_tc_launch<80>(qkv, o, lse, B, T, H, err, s);
     case 128: return fwd_tc_launch<128>(qkv, o, lse, B, T, H, err, s);
+    case 256: return fwd_tc_launch<256>(qkv, o, lse, B, T, H, err, s);
   }
   return cudaErrorInvalidValue;
 }
@@ -852,6 +894,7 @@ cudaError_t attention_bwd(const bf16* qkv, const bf16* o, const float* lse, cons
     case 64: return bwd_tc_launch<64>(qkv, o, lse, dout, dqkv, delta, NB, B, T, H, err, s);
     case 80: return bwd_tc_launch<80>(qkv, o, lse, dout, dqkv, delta, NB, B, T, H, err, s);
     case 128: return bwd_tc_launch<128>(qkv, o, lse, dout, dqkv, delta, NB, B, T, H, err, s);
+    case 256: return bwd_tc_launch<256>(qkv, o, lse, dout, dqkv, delta, NB, B, T, H, err, s);
   }
   return cudaErrorInvalidValue;
 }

@@ -57,7 +57,7 @@ cudaError_t adamw(float* p, float* m, float* v, const float* g, __nv_bfloat16* p
                   float lr, float beta1, float beta2, float eps, float wd, float bc1, float bc2, cudaStream_t s);
 
 // Causal attention on packed qkv [B*T, 3d] (Q | K | V, head h at columns h*dh) on the tcgen05 tensor cores.
-// dh in {32, 64, 80, 128}; pointers 16-byte aligned.
+// dh in {32, 64, 80, 128, 256}; pointers 16-byte aligned.
 //   o [B*T, d] bf16, lse [B, H, T] fp32 (natural log of the softmax denominator, scores scaled by 1/sqrt(dh)).
 // err (may be NULL): device word set non-zero if a bounded wait in the kernel expired.
 cudaError_t attention_fwd(const __nv_bfloat16* qkv, __nv_bfloat16* o, float* lse, int B, int T, int H, int dh,

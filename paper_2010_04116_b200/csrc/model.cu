@@ -331,7 +331,7 @@ extern "C" il_status il_create(int K, int Lc, int d, int H, int F, int V, int n,
   if (opt->head_layers < 0 || opt->head_layers > 64) return IL_ERR_INVALID_ARG;
   if (d % H || d % 8 || F % 8 || opt->max_batch < 1 || opt->max_seq < 1) return IL_ERR_INVALID_ARG;
   const int dh = d / H;
-  if (!(dh == 32 || dh == 64 || dh == 80 || dh == 128)) return IL_ERR_INVALID_ARG;
+  if (!(dh == 32 || dh == 64 || dh == 80 || dh == 128 || dh == 256)) return IL_ERR_INVALID_ARG;
   if (opt->streams && opt->n_streams < K) return IL_ERR_INVALID_ARG;
   if ((opt->alloc == nullptr) != (opt->free_ == nullptr)) return IL_ERR_INVALID_ARG;
 

@@ -89,3 +89,23 @@ def test_micro_batched_update_matches_the_whole_mini_batch(M, Lh, rule):
             m.train_step(tok[:per], tgt[:per])
     finally:
         m.close()
+
+
+def test_paper_head_shape_dh256_short_sequences():
+    """The paper's Transformer shape has 4 attention heads at d 1024, i.e. head dimension 256, on sequences of
+    128 tokens (App. B.3): one module pair with 2-block auxiliary networks at those widths and a small vocabulary."""
+    w = wl.Workload("dh256", K=2, Lc=1, d=1024, H=4, F=4096, V=1200, T=128, B=2, n=2, zipf=True, Lh=2)
+    P = wl.draw_params(w)
+    tok, tgt = wl.draw_tokens(w)
+    m = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, 2, w.B, w.T, head_layers=w.Lh)
+    try:
+        m.set_params(P)
+        m.set_rule("mean")
+        m.train_step(tok, tgt)
+        losses = m.get_losses()
+        m.sync()
+        ol, OG = orc.nwise_gradients(P, tok, tgt, w.K, w.Lc, w.H, 2, rule="mean", head_layers=w.Lh)
+        assert np.all(np.abs(losses - np.array(ol)) <= LOSS_RTOL * np.abs(np.array(ol))), (losses, ol)
+        _compare(m, OG)
+    finally:
+        m.close()

@@ -182,7 +182,8 @@ def test_gemm_softmax_epilogues(V):
     assert np.all(got[:, nv:] == 3.0)
 
 
-@pytest.mark.parametrize("B,T,H,dh", [(2, 64, 2, 32), (1, 200, 2, 64), (2, 256, 3, 64), (1, 192, 2, 80), (1, 130, 1, 128)])
+@pytest.mark.parametrize("B,T,H,dh", [(2, 64, 2, 32), (1, 200, 2, 64), (2, 256, 3, 64), (1, 192, 2, 80), (1, 130, 1, 128),
+                                      (3, 128, 2, 256), (1, 300, 1, 256)])
 def test_attention_forward_backward(B, T, H, dh):
     rng = np.random.default_rng(B * 1000 + T + dh)
     d = H * dh
