@@ -48,9 +48,17 @@ def model_flops_per_token(w: wl.Workload, n: int) -> float:
     total = 0.0
     for k in range(w.K):
         heads = [h for h in range(w.K) if max(h - n + 1, 0) <= k <= h]
-        s_k = len({max(h - n + 1, 0) for h in heads})
+        if w.rule == "sum":
+            s_k = len({max(h - n + 1, 0) for h in heads})
+        else:
+            # weighted rules: one stream for the weighted combination that drives the parameter gradients plus
+            # one per head that continues below the component (the two coincide when a single head is involved)
+            below = [h for h in heads if k > 0 and h < k + n - 1]
+            s_k = 1 + len(below) - (1 if len(heads) == 1 and below else 0)
         total += w.Lc * (gemm + att_f) + w.Lc * gemm + s_k * w.Lc * (gemm + att_b)
     total += w.K * 6.0 * w.d * w.V
+    # blocks inside the auxiliary heads: forward, wgrad and one dgrad each
+    total += w.K * w.Lh * ((gemm + att_f) + gemm + (gemm + att_b))
     return total
 
 
@@ -125,7 +133,7 @@ def oracle_sample(w: wl.Workload, n: int, steps: int, warmup: int, params=None, 
     times = []
     for i in range(warmup + steps):
         t0 = time.perf_counter()
-        orc.nwise_gradients(P, tok, tgt, ws.K, ws.Lc, ws.H, n)
+        orc.nwise_gradients(P, tok, tgt, ws.K, ws.Lc, ws.H, n, rule=ws.rule, head_layers=ws.Lh)
         if i >= warmup:
             times.append(time.perf_counter() - t0)
     sec = float(np.mean(times))
@@ -169,8 +177,10 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     metric = "training tokens/s per n-wise step"
+    extra = (f", {w.Lh} blocks per auxiliary head, rule={w.rule}, {w.M} micro-batches per update"
+             if (w.Lh or w.M > 1 or w.rule != "sum") else "")
     cfg_desc = {"workload": f"{w.name}: {w.K}x{w.Lc} layers, d={w.d}, H={w.H}, F={w.F}, T={w.T}, B={w.B}, V={w.V}, "
-                            f"n={n}, adamw={bool(w.adamw and not args.no_adamw)}",
+                            f"n={n}, adamw={bool(w.adamw and not args.no_adamw)}{extra}",
                 "global_batch": w.B * max(world, 1), "seq_len": w.T, "parallelism": f"replicas x{max(world, 1)}",
                 "l2": "inputs larger than L2 (each step streams several GB of weights and activations)"}
 
@@ -199,8 +209,12 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
     use_adamw = bool(w.adamw and not args.no_adamw)
-    hp = dict(lr=1e-4, beta1=0.9, beta2=0.98, eps=1e-9, weight_decay=0.01) if use_adamw else None
-    m = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, n, w.B, w.T, device=local_rank)
+    hp = dict(lr=1e-4, beta1=0.9, beta2=0.98, eps=1e-9, weight_decay=w.weight_decay) if use_adamw else None
+    m = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, n, w.B // w.M, w.T, device=local_rank, head_layers=w.Lh)
+    if w.rule != "sum":
+        m.set_rule(w.rule)
+    if w.M > 1:
+        m.set_micro_batches(w.M)
     # parameters drawn on the host by the seeded generator, copied once
     params = wl.draw_params(w)
     m.set_params(params)
@@ -220,7 +234,12 @@ def main():
     def run_steps(count, e2e):
         for i in range(count):
             tok, tgt = (pin_batches if e2e else dev_batches)[i % nb]
-            m.train_step(tok, tgt, adamw=hp)
+            if w.M > 1:
+                if hp is None:
+                    m.set_micro_batches(w.M)     # no update follows: start the next accumulation explicitly
+                m.train_minibatch(tok, tgt, w.M, adamw=hp)
+            else:
+                m.train_step(tok, tgt, adamw=hp)
             if e2e:
                 m.get_losses()          # device -> host read of the step's result (waits for the heads)
 

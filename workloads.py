@@ -42,6 +42,7 @@ class Workload:
     Lh: int = 0       # Transformer blocks inside every auxiliary head (App. B.3: 2); 0 = LayerNorm + linear head
     M: int = 1        # micro-batches a mini-batch of B sequences is processed in (Sec. 3.1)
     rule: str = "sum"  # head weighting: "sum", "far" (Sec. 3 main text) or "mean" (App. B.3)
+    weight_decay: float = 0.01   # decoupled decay of the AdamW step; 0 gives the paper's Adam (App. B.3)
 
     @property
     def ntok(self) -> int:
@@ -70,7 +71,7 @@ CONFIGS: Dict[str, Workload] = {
     # rule, Adam; A = 4 modules, a mini-batch of 1024 sequences in 4 micro-batches (Sec. 3.1).  The vocabulary
     # size is not printed in the paper; the other configurations' 50257 is used.
     "cfgP": Workload("cfgP", K=4, Lc=6, d=1024, H=4, F=4096, V=50257, T=128, B=1024, n=2, adamw=True, Lh=2, M=4,
-                     rule="mean"),
+                     rule="mean", weight_decay=0.0),
 }
 
 
