@@ -193,6 +193,126 @@ cudaError_t layernorm_bwd_rows(const void* dy, int dy_is_f32, const float* x, co
 }
 
 // ---------------------------------------------------------------------------------------------
+// LayerNorm backward in one pass over the rows (bf16 dy, d = 128 NV with NV <= 8): the row part as above and, for
+// the rows of the first gradient stream (row < x_rows), the column reductions that otherwise take three more
+// kernels over the same data: dgamma += dy * xhat, dbeta += dy, and colsum += the kernel's own output (the bias
+// gradient of the linear layer whose output this residual-stream gradient belongs to).  A warp walks rows with a
+// grid-wide stride, keeps a row's values in registers between the two passes and its column partials in
+// registers across rows; the block combines its eight warps through shared memory and adds one value per
+// column and output to global memory.  dgamma / dbeta / colsum must be zeroed (or hold a sum to add to).
+// ---------------------------------------------------------------------------------------------
+template <int NV>
+__global__ void __launch_bounds__(256, 1) layernorm_bwd_fused_kernel(const bf16* __restrict__ dy, const float* __restrict__ x,
+                                                                     const float* __restrict__ mean,
+                                                                     const float* __restrict__ rstd,
+                                                                     const float* __restrict__ gamma, const float* resid,
+                                                                     float* dx_out, bf16* __restrict__ dx_bf16,
+                                                                     float* __restrict__ dgamma, float* __restrict__ dbeta,
+                                                                     float* __restrict__ colsum, int rows, int x_rows) {
+  constexpr int d = NV * 128;
+  __shared__ float4 red[8][NV * 32];
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int warps = gridDim.x * 8;
+  float4 g4[NV];
+#pragma unroll
+  for (int i = 0; i < NV; ++i) g4[i] = __ldg(reinterpret_cast<const float4*>(gamma) + lane + 32 * i);
+  float4 ag[NV], ab[NV], ac[NV];
+#pragma unroll
+  for (int i = 0; i < NV; ++i) ag[i] = ab[i] = ac[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int row = blockIdx.x * 8 + w; row < rows; row += warps) {
+    const int xrow = row % x_rows;
+    const bool first = row < x_rows;              // rows of the first stream feed the parameter gradients
+    const float mu = mean[xrow], rs = rstd[xrow];
+    const float4* xr = reinterpret_cast<const float4*>(x + (size_t)xrow * d);
+    float4 dv[NV], xh[NV];
+    float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+      dv[i] = load_dy4<false>(dy, (size_t)row, d, lane + 32 * i);
+      const float4 xv = xr[lane + 32 * i];
+      xh[i] = make_float4((xv.x - mu) * rs, (xv.y - mu) * rs, (xv.z - mu) * rs, (xv.w - mu) * rs);
+    }
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+      const float a0 = dv[i].x * g4[i].x, a1 = dv[i].y * g4[i].y, a2 = dv[i].z * g4[i].z, a3 = dv[i].w * g4[i].w;
+      s1 += (a0 + a1) + (a2 + a3);
+      s2 += (a0 * xh[i].x + a1 * xh[i].y) + (a2 * xh[i].z + a3 * xh[i].w);
+      if (first) {
+        ag[i].x += dv[i].x * xh[i].x; ag[i].y += dv[i].y * xh[i].y; ag[i].z += dv[i].z * xh[i].z; ag[i].w += dv[i].w * xh[i].w;
+        ab[i].x += dv[i].x; ab[i].y += dv[i].y; ab[i].z += dv[i].z; ab[i].w += dv[i].w;
+      }
+    }
+    const float m1 = warp_sum(s1) / d;
+    const float m2 = warp_sum(s2) / d;          // mean of dxhat * xhat
+    const float4* rr = resid ? reinterpret_cast<const float4*>(resid + (size_t)row * d) : nullptr;
+    float4* outr = reinterpret_cast<float4*>(dx_out + (size_t)row * d);
+    uint2* outb = dx_bf16 ? reinterpret_cast<uint2*>(dx_bf16 + (size_t)row * d) : nullptr;
+    float4 r4[NV];
+    if (rr) {
+#pragma unroll
+      for (int i = 0; i < NV; ++i) r4[i] = rr[lane + 32 * i];
+    }
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+      float4 o;
+      o.x = (dv[i].x * g4[i].x - m1 - xh[i].x * m2) * rs;
+      o.y = (dv[i].y * g4[i].y - m1 - xh[i].y * m2) * rs;
+      o.z = (dv[i].z * g4[i].z - m1 - xh[i].z * m2) * rs;
+      o.w = (dv[i].w * g4[i].w - m1 - xh[i].w * m2) * rs;
+      if (rr) { o.x += r4[i].x; o.y += r4[i].y; o.z += r4[i].z; o.w += r4[i].w; }
+      outr[lane + 32 * i] = o;
+      if (outb) {
+        uint2 b;
+        b.x = pack_bf16x2(o.x, o.y);
+        b.y = pack_bf16x2(o.z, o.w);
+        outb[lane + 32 * i] = b;
+      }
+      if (first) { ac[i].x += o.x; ac[i].y += o.y; ac[i].z += o.z; ac[i].w += o.w; }
+    }
+  }
+  // block-level combination, one quantity after the other through the same buffer
+#pragma unroll
+  for (int q = 0; q < 3; ++q) {
+    float* out = q == 0 ? dgamma : q == 1 ? dbeta : colsum;
+    if (!out) continue;                           // uniform across the block
+#pragma unroll
+    for (int i = 0; i < NV; ++i) red[w][lane + 32 * i] = q == 0 ? ag[i] : q == 1 ? ab[i] : ac[i];
+    __syncthreads();
+    for (int c = threadIdx.x; c < NV * 32; c += 256) {
+      float4 t = red[0][c];
+#pragma unroll
+      for (int k = 1; k < 8; ++k) {
+        const float4 v = red[k][c];
+        t.x += v.x; t.y += v.y; t.z += v.z; t.w += v.w;
+      }
+      red_add_f32x4(out + 4 * c, t);
+    }
+    __syncthreads();
+  }
+}
+
+// Fused LayerNorm backward for bf16 dy when d is a multiple of 128 up to 1024; returns cudaErrorNotSupported for
+// other widths (the caller then uses the separate row and column kernels).  dgamma, dbeta, colsum: fp32 [d],
+// summed into (colsum may be NULL).
+cudaError_t layernorm_bwd_fused(const bf16* dy, const float* x, const float* mean, const float* rstd, const float* gamma,
+                                const float* resid, float* dx_out, bf16* dx_bf16, float* dgamma, float* dbeta,
+                                float* colsum, int rows, int x_rows, int d, cudaStream_t s) {
+  if (d % 128 || d > 1024 || d < 128) return cudaErrorNotSupported;
+  int blocks = ceil_div(rows, 8);
+  if (blocks > 148) blocks = 148;
+#define IL_LNF(NV)                                                                                                        \
+  case NV:                                                                                                                \
+    layernorm_bwd_fused_kernel<NV><<<blocks, 256, 0, s>>>(dy, x, mean, rstd, gamma, resid, dx_out, dx_bf16, dgamma, dbeta, \
+                                                          colsum, rows, x_rows);                                          \
+    break;
+  switch (d / 128) {
+    IL_LNF(1) IL_LNF(2) IL_LNF(3) IL_LNF(4) IL_LNF(5) IL_LNF(6) IL_LNF(7) IL_LNF(8)
+  }
+#undef IL_LNF
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
 // Column reductions.  Block = 32 lanes x 8 warps; a lane owns 4 consecutive columns, a block 128 columns;
 // the rows are split over gridDim.y; partial sums are combined through shared memory and one atomicAdd
 // per column per block.

@@ -28,6 +28,11 @@ cudaError_t layernorm_bwd_rows(const void* dy, int dy_is_f32, const float* x, co
 // Outputs are accumulated atomically and must be zeroed by the caller.
 cudaError_t layernorm_bwd_params(const void* dy, int dy_is_f32, const float* x, const float* mean, const float* rstd,
                                  float* dgamma, float* dbeta, int rows, int d, cudaStream_t s);
+// Both of the above in one pass for bf16 dy and d a multiple of 128 up to 1024 (cudaErrorNotSupported otherwise),
+// plus, when colsum != NULL, colsum[c] += sum over the first x_rows rows of dx_out[r,c].
+cudaError_t layernorm_bwd_fused(const __nv_bfloat16* dy, const float* x, const float* mean, const float* rstd,
+                                const float* gamma, const float* resid, float* dx_out, __nv_bfloat16* dx_bf16, float* dgamma,
+                                float* dbeta, float* colsum, int rows, int x_rows, int d, cudaStream_t s);
 // out[c] += sum_r y[r,c] for bf16 y [rows, ld] (bias gradients).  out zeroed by the caller.
 cudaError_t colsum_bf16(const __nv_bfloat16* y, int ld, float* out, int rows, int cols, cudaStream_t s);
 // out[c] += sum_r y[r,c] for fp32 y.

@@ -805,12 +805,15 @@ il_status layers_backward(il_model* m, int k, int s, size_t base, int count, con
   const int N = m->ntok, d = m->d, F = m->F;
   const int R = s * N;
   CompScratch& c = m->cs[k];
+  const bool fused_ln = d % 128 == 0 && d <= 1024;     // widths the one-pass LayerNorm backward covers
   for (int l = count - 1; l >= 0; --l) {
     const LayerOff& o = m->layer_off[base + l];
     LayerActs& A = m->acts[base + l];
     const float* x_in = (l == 0) ? x_first : m->acts[base + l - 1].x_out;
     // ---- MLP: x_out = x_mid + W2 gelu(W1 ln2 + b1) + b2
-    IL_K(m, colsum_f32(c.dx, d, m->G + o.b2, N, d, st));
+    // bias gradient of FC2: column sums of the incoming gradient (first stream).  Below the top block they come
+    // out of the LayerNorm backward that produced this gradient.
+    if (l == count - 1 || !fused_ln) IL_K(m, colsum_f32(c.dx, d, m->G + o.b2, N, d, st));
     IL_TRY(wgrad(m, k, d, F, N, c.dxb, d, A.hact, F, m->G + o.w2, acc));
     {
       GemmArgs g = gemm_args(R, F, d, c.dxb, d, 0, m->Pb + o.w2, F, 1, EPI_BF16_DGELU, c.dbig, F);
@@ -820,10 +823,15 @@ il_status layers_backward(il_model* m, int k, int s, size_t base, int count, con
     }
     IL_TRY(wgrad(m, k, F, d, N, c.dbig, F, A.ln2, d, m->G + o.w1, acc));
     IL_TRY(gemm(m, k, gemm_args(R, d, F, c.dbig, F, 0, m->Pb + o.w1, d, 1, EPI_BF16, c.dln, d)));
-    IL_K(m, layernorm_bwd_params(c.dln, 0, A.x_mid, A.mean2, A.rstd2, m->G + o.ln2g, m->G + o.ln2b, N, d, st));
-    IL_K(m, layernorm_bwd_rows(c.dln, 0, A.x_mid, A.mean2, A.rstd2, m->P + o.ln2g, c.dx, c.dx, c.dxb, R, N, d, st));
-    // ---- attention: x_mid = x_in + Wo attn(Wqkv ln1 + bqkv) + bo
-    IL_K(m, colsum_f32(c.dx, d, m->G + o.bo, N, d, st));
+    if (fused_ln) {   // LayerNorm backward with its parameter gradients and the bias gradient of Wo in one pass
+      IL_K(m, layernorm_bwd_fused(c.dln, A.x_mid, A.mean2, A.rstd2, m->P + o.ln2g, c.dx, c.dx, c.dxb, m->G + o.ln2g,
+                                  m->G + o.ln2b, m->G + o.bo, R, N, d, st));
+    } else {
+      IL_K(m, layernorm_bwd_params(c.dln, 0, A.x_mid, A.mean2, A.rstd2, m->G + o.ln2g, m->G + o.ln2b, N, d, st));
+      IL_K(m, layernorm_bwd_rows(c.dln, 0, A.x_mid, A.mean2, A.rstd2, m->P + o.ln2g, c.dx, c.dx, c.dxb, R, N, d, st));
+      // ---- attention: x_mid = x_in + Wo attn(Wqkv ln1 + bqkv) + bo
+      IL_K(m, colsum_f32(c.dx, d, m->G + o.bo, N, d, st));
+    }
     IL_TRY(wgrad(m, k, d, d, N, c.dxb, d, A.attn_o, d, m->G + o.wo, acc));
     IL_TRY(gemm(m, k, gemm_args(R, d, d, c.dxb, d, 0, m->Pb + o.wo, d, 1, EPI_BF16, c.dattn, d)));
     IL_K(m, attention_bwd(A.qkv, A.attn_o, A.lse, c.dattn, c.dqkv, c.delta, s * m->B, m->B, m->T, m->H, m->dh, m->err_word, st));
@@ -831,8 +839,14 @@ il_status layers_backward(il_model* m, int k, int s, size_t base, int count, con
     IL_K(m, colsum_bf16(c.dqkv, 3 * d, m->G + o.bqkv, N, 3 * d, st));
     IL_TRY(wgrad(m, k, 3 * d, d, N, c.dqkv, 3 * d, A.ln1, d, m->G + o.wqkv, acc));
     IL_TRY(gemm(m, k, gemm_args(R, d, 3 * d, c.dqkv, 3 * d, 0, m->Pb + o.wqkv, d, 1, EPI_BF16, c.dln, d)));
-    IL_K(m, layernorm_bwd_params(c.dln, 0, x_in, A.mean1, A.rstd1, m->G + o.ln1g, m->G + o.ln1b, N, d, st));
-    IL_K(m, layernorm_bwd_rows(c.dln, 0, x_in, A.mean1, A.rstd1, m->P + o.ln1g, c.dx, c.dx, c.dxb, R, N, d, st));
+    if (fused_ln) {   // ... and the FC2 bias gradient of the block below
+      float* b2_below = l > 0 ? m->G + m->layer_off[base + l - 1].b2 : nullptr;
+      IL_K(m, layernorm_bwd_fused(c.dln, x_in, A.mean1, A.rstd1, m->P + o.ln1g, c.dx, c.dx, c.dxb, m->G + o.ln1g,
+                                  m->G + o.ln1b, b2_below, R, N, d, st));
+    } else {
+      IL_K(m, layernorm_bwd_params(c.dln, 0, x_in, A.mean1, A.rstd1, m->G + o.ln1g, m->G + o.ln1b, N, d, st));
+      IL_K(m, layernorm_bwd_rows(c.dln, 0, x_in, A.mean1, A.rstd1, m->P + o.ln1g, c.dx, c.dx, c.dxb, R, N, d, st));
+    }
   }
   return IL_OK;
 }
