@@ -108,9 +108,55 @@ __global__ void __launch_bounds__(256) layernorm_fwd_kernel(const float* __restr
   }
 }
 
+// The same for d = 128 NV (NV <= 8): a row is read once and held in registers between the passes.
+template <int NV>
+__global__ void __launch_bounds__(256) layernorm_fwd_reg_kernel(const float* __restrict__ x, const float* __restrict__ gamma,
+                                                                const float* __restrict__ beta, bf16* __restrict__ y,
+                                                                float* __restrict__ mean, float* __restrict__ rstd,
+                                                                int rows, float eps) {
+  constexpr int d = NV * 128;
+  const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (row >= rows) return;
+  const float4* xr = reinterpret_cast<const float4*>(x + (size_t)row * d);
+  float4 v[NV];
+#pragma unroll
+  for (int i = 0; i < NV; ++i) v[i] = xr[lane + 32 * i];
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < NV; ++i) s += (v[i].x + v[i].y) + (v[i].z + v[i].w);
+  const float mu = warp_sum(s) / d;
+  float q = 0.f;
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+    v[i].x -= mu; v[i].y -= mu; v[i].z -= mu; v[i].w -= mu;
+    q += (v[i].x * v[i].x + v[i].y * v[i].y) + (v[i].z * v[i].z + v[i].w * v[i].w);
+  }
+  const float rs = rsqrtf(warp_sum(q) / d + eps);
+  if (lane == 0) { mean[row] = mu; rstd[row] = rs; }
+  uint2* yr = reinterpret_cast<uint2*>(y + (size_t)row * d);
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+    const float4 g = __ldg(reinterpret_cast<const float4*>(gamma) + lane + 32 * i);
+    const float4 b = __ldg(reinterpret_cast<const float4*>(beta) + lane + 32 * i);
+    uint2 o;
+    o.x = pack_bf16x2(v[i].x * rs * g.x + b.x, v[i].y * rs * g.y + b.y);
+    o.y = pack_bf16x2(v[i].z * rs * g.z + b.z, v[i].w * rs * g.w + b.w);
+    yr[lane + 32 * i] = o;
+  }
+}
+
 cudaError_t layernorm_fwd(const float* x, const float* gamma, const float* beta, bf16* y, float* mean, float* rstd,
                           int rows, int d, float eps, cudaStream_t s) {
-  layernorm_fwd_kernel<<<ceil_div(rows, 8), 256, 0, s>>>(x, gamma, beta, y, mean, rstd, rows, d, eps);
+  const int blocks = ceil_div(rows, 8);
+#define IL_LNR(NV) \
+  case NV: layernorm_fwd_reg_kernel<NV><<<blocks, 256, 0, s>>>(x, gamma, beta, y, mean, rstd, rows, eps); break;
+  if (d % 128 == 0 && d <= 1024) {
+    switch (d / 128) { IL_LNR(1) IL_LNR(2) IL_LNR(3) IL_LNR(4) IL_LNR(5) IL_LNR(6) IL_LNR(7) IL_LNR(8) }
+  } else {
+    layernorm_fwd_kernel<<<blocks, 256, 0, s>>>(x, gamma, beta, y, mean, rstd, rows, d, eps);
+  }
+#undef IL_LNR
   return cudaGetLastError();
 }
 
@@ -389,7 +435,14 @@ __global__ void __launch_bounds__(256) colsum_kernel(const void* __restrict__ y,
   const int r1 = min(rows, r0 + rows_per_block);
   float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
   if (col_ok) {
-    for (int r = r0 + w; r < r1; r += 8) {
+    int r = r0 + w;
+    for (; r + 24 < r1; r += 32) {               // four independent loads in flight per lane
+      const float4 v0 = load_dy4<IN_F32>(y, (size_t)r, ld, c4), v1 = load_dy4<IN_F32>(y, (size_t)r + 8, ld, c4);
+      const float4 v2 = load_dy4<IN_F32>(y, (size_t)r + 16, ld, c4), v3 = load_dy4<IN_F32>(y, (size_t)r + 24, ld, c4);
+      a.x += (v0.x + v1.x) + (v2.x + v3.x); a.y += (v0.y + v1.y) + (v2.y + v3.y);
+      a.z += (v0.z + v1.z) + (v2.z + v3.z); a.w += (v0.w + v1.w) + (v2.w + v3.w);
+    }
+    for (; r < r1; r += 8) {
       const float4 v = load_dy4<IN_F32>(y, (size_t)r, ld, c4);
       a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
     }

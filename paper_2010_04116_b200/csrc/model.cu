@@ -954,19 +954,22 @@ extern "C" il_status il_backward_nwise(il_model* m) {
   } else {
     // Weighted rules: component k carries slot 0 = sum_h W(k,h) g^(h) (drives every parameter gradient) and one
     // slot per head that continues below k (all crossing heads but the one with h = k+n-1); the pass-down of a
-    // head is taken from its own slot of component k+1.
-    std::vector<int> above_heads;     // heads in slots 1.. of component k+1, ascending
+    // head is taken from its own slot of component k+1.  When the combination is a single head with weight one that
+    // also continues below (the top component under the mean rule), slot 0 serves as that head's slot too.
+    std::vector<int> above_heads;     // heads carried by component k+1 ...
+    std::vector<int> above_slots;     // ... and the slot each of them occupies there
     for (int k = K - 1; k >= 0; --k) {
       cudaStream_t st = m->streams[k];
       const int hi = k + n - 1 < K - 1 ? k + n - 1 : K - 1;
       auto grad_of = [&](int h) -> const float* {      // gradient of head h at the output of component k
         if (h == k) return m->hs[k].ghead;
         for (size_t q = 0; q < above_heads.size(); ++q)
-          if (above_heads[q] == h) return m->cs[k + 1].dx + (size_t)(q + 1) * slice;
+          if (above_heads[q] == h) return m->cs[k + 1].dx + (size_t)above_slots[q] * slice;
         return nullptr;
       };
       if (hi > k) IL_CUDA(m, cudaStreamWaitEvent(st, m->ev_bwd[k + 1], 0));
       // slot 0: the weighted combination
+      int single = -1;                  // the head slot 0 equals exactly, if any
       {
         const float* xs[8];
         float ws[8];
@@ -976,6 +979,7 @@ extern "C" il_status il_backward_nwise(il_model* m) {
           if (wgt == 0.0f) continue;
           xs[cnt] = grad_of(h);
           if (!xs[cnt]) return fail(m, IL_ERR_STATE, "internal: gradient stream of head %d missing at component %d", h, k);
+          single = (cnt == 0 && wgt == 1.0f) ? h : -1;
           ws[cnt++] = wgt;
         }
         for (int c0 = 0; c0 < cnt; c0 += 4) {
@@ -984,22 +988,26 @@ extern "C" il_status il_backward_nwise(il_model* m) {
         }
       }
       // slots 1..: heads that continue below this component
-      std::vector<int> mine;
+      std::vector<int> mine, mine_slots;
+      int used = 1;
       if (k > 0)
         for (int h = k; h <= hi; ++h)
-          if (h < k + n - 1) mine.push_back(h);
-      for (size_t q = 0; q < mine.size(); ++q) {
-        const float* src = grad_of(mine[q]);
-        if (!src) return fail(m, IL_ERR_STATE, "internal: gradient stream of head %d missing at component %d", mine[q], k);
-        IL_K(m, add_convert(src, nullptr, m->cs[k].dx + (q + 1) * slice, m->cs[k].dxb + (q + 1) * slice, slice, st));
-      }
-      IL_TRY(component_backward(m, k, 1 + (int)mine.size(), acc));
+          if (h < k + n - 1) {
+            mine.push_back(h);
+            if (h == single) { mine_slots.push_back(0); continue; }
+            const float* src = grad_of(h);
+            if (!src) return fail(m, IL_ERR_STATE, "internal: gradient stream of head %d missing at component %d", h, k);
+            IL_K(m, add_convert(src, nullptr, m->cs[k].dx + (size_t)used * slice, m->cs[k].dxb + (size_t)used * slice, slice, st));
+            mine_slots.push_back(used++);
+          }
+      IL_TRY(component_backward(m, k, used, acc));
       if (k == 0) {
         IL_K(m, embed_bwd(m->tokens, m->cs[0].dx, m->G + m->off_wte, m->G + m->off_wpe, N, m->T, d, m->V, acc ? 1 : 0, st));
         m->launches++;
       }
       IL_CUDA(m, cudaEventRecord(m->ev_bwd[k], st));
       above_heads = mine;
+      above_slots = mine_slots;
     }
   }
   m->bwd_done = true;
