@@ -137,10 +137,10 @@ __global__ void __launch_bounds__(128) attn_fwd_tc_kernel(const __grid_constant_
     const int st = j % NST;
     const uint32_t ph = (uint32_t)j & 1u;
     if (!mbar_wait(bar_s, ph, abortp)) { fail = 1; abort_flag = 1; }
-    // the previous block's P V was issued before these scores, so it has landed too: the packed P columns,
-    // the O accumulator and that block's K/V stage are free
+    // the previous block's P V was issued before these scores and the tensor pipe retires in order, so it has
+    // landed too (bar_s covers it; only the last P V is committed on its own): the packed P columns, the O
+    // accumulator and that block's K/V stage are free
     if (j > 0) {
-      if (!mbar_wait(bar_o, (uint32_t)(j - 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
       if (tid == 0 && j - 1 + NST < nkv) load_kv(j - 1 + NST);
     }
     tc_fence_after();
@@ -216,14 +216,14 @@ __global__ void __launch_bounds__(128) attn_fwd_tc_kernel(const __grid_constant_
 #pragma unroll
       for (int ks = 0; ks < TK / 16; ++ks)       // B = V read MN-major; O accumulates in TMEM
         umma_bf16_ts(tmem_base + 64, tmem_base + 8 * ks, desc_at(dv_mn, so + ks * 2048), idesc_o, (j | ks) ? 1u : 0u);
-      umma_commit(bar_o);
       // every thread has read S_j (barrier above); the tensor pipe runs the P V just issued, which reads the
       // packed columns, before it overwrites them with the next scores
       if (j + 1 < nkv) issue_s(j + 1);
+      else umma_commit(bar_o);
     }
   }
   if (!fail && nkv > 0) {
-    if (!mbar_wait(bar_o, (uint32_t)(nkv - 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
+    if (!mbar_wait(bar_o, 0, abortp)) { fail = 1; abort_flag = 1; }
     tc_fence_after();
   }
   fail = __syncthreads_or(fail);
@@ -469,8 +469,8 @@ __global__ void __launch_bounds__(256) attn_bwd_dkv_tc_kernel(const __grid_const
     if (!mbar_wait(bar_s, (uint32_t)it & 1u, abortp)) { fail = 1; abort_flag = 1; }
     // the previous step's dV/dK products were issued before these scores, so they have landed too: the packed
     // P^T / dS^T columns and that step's Q/dO stage are free
+    // (the tensor pipe retires in order: bar_s covers them, only the last step's products are committed on their own)
     if (C::AHEAD && it > 0) {
-      if (!mbar_wait(bar_acc, (uint32_t)(it - 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
       if (tid == 0 && j - 1 + NST < nq) load_q(j - 1 + NST);
     }
     tc_fence_after();
@@ -528,15 +528,15 @@ __global__ void __launch_bounds__(256) attn_bwd_dkv_tc_kernel(const __grid_const
           umma_bf16_ts(tmem_base + 128 + (PART == 0 ? DH : 0), tmem_base + 64 + packed_col(ks), desc_at(dq_mn, off_b), idesc_g,
                        (it | ks) ? 1u : 0u);
       }
-      umma_commit(bar_acc);
       // every thread has read S^T / dP^T of this step (barrier above); the tensor pipe runs the products just
       // issued, which read the packed columns, before it overwrites them with the next scores
       if (C::AHEAD && j + 1 < nq) issue_s(j + 1);
+      else umma_commit(bar_acc);
     }
   }
   const int nit = nq - q0;
   if (!fail && nit > 0) {
-    if (!mbar_wait(bar_acc, (uint32_t)(nit - 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
+    if (!mbar_wait(bar_acc, C::AHEAD ? 0u : ((uint32_t)(nit - 1) & 1u), abortp)) { fail = 1; abort_flag = 1; }
     tc_fence_after();
   }
   fail = __syncthreads_or(fail);
@@ -706,8 +706,7 @@ __global__ void __launch_bounds__(256) attn_bwd_dq_tc_kernel(const __grid_consta
       if (tid == 0) issue_s(j);
     }
     if (!mbar_wait(bar_s, (uint32_t)j & 1u, abortp)) { fail = 1; abort_flag = 1; }
-    if (C::AHEAD && j > 0) {                         // issued before these scores: landed, the packed dS and that step's K/V stage are free
-      if (!mbar_wait(bar_acc, (uint32_t)(j - 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
+    if (C::AHEAD && j > 0) {                         // issued before these scores: landed (bar_s covers it), the packed dS and that step's K/V stage are free
       if (tid == 0 && j - 1 + NST < nkv) load_kv(j - 1 + NST);
     }
     tc_fence_after();
@@ -742,12 +741,12 @@ __global__ void __launch_bounds__(256) attn_bwd_dq_tc_kernel(const __grid_consta
       for (int ks = 0; ks < TK / 16; ++ks)
         umma_bf16_ts(tmem_base + 128, tmem_base + 64 + packed_col(ks), desc_at(dk_mn, so + ks * 2048), idesc_g,
                      (j | ks) ? 1u : 0u);
-      umma_commit(bar_acc);
       if (C::AHEAD && j + 1 < nkv) issue_s(j + 1);
+      else umma_commit(bar_acc);
     }
   }
   if (!fail && nkv > 0) {
-    if (!mbar_wait(bar_acc, (uint32_t)(nkv - 1) & 1u, abortp)) { fail = 1; abort_flag = 1; }
+    if (!mbar_wait(bar_acc, C::AHEAD ? 0u : ((uint32_t)(nkv - 1) & 1u), abortp)) { fail = 1; abort_flag = 1; }
     tc_fence_after();
   }
   fail = __syncthreads_or(fail);
