@@ -1,0 +1,76 @@
+"""Time one operator of the library at the GPT-2-medium-shaped sizes (8192 tokens, d 1024, 16 heads of 64, vocab 50257)
+through the C ABI: useful for comparing kernel changes and as a small case for profiler captures.
+
+    python -m paper_2010_04116_b200.opbench <op> [iterations] [gradient batches]
+
+ops: logits (auxiliary head: vocabulary projection with the softmax / exp(logit) epilogue), plain (the same
+contraction with a plain bf16 output), attn_fwd, attn_bwd (gradient batches = stacked gradient streams x 8).
+"""
+from __future__ import annotations
+
+import sys
+
+import torch
+
+from . import binding as il
+
+DEV = "cuda:0"
+
+
+def _timeit(name, fn, flops, iters, err):
+    for _ in range(2):
+        fn()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(iters):
+        fn()
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / iters
+    print(f"{name}: {ms * 1e3:.1f} us, {flops / ms / 1e9:.1f} TFLOP/s, device error word {int(err.item())}")
+
+
+def main(argv):
+    which = argv[1] if len(argv) > 1 else "logits"
+    iters = int(argv[2]) if len(argv) > 2 else 10
+    err = torch.zeros(1, dtype=torch.int32, device=DEV)
+    if which in ("logits", "plain"):
+        M, V, K = 8192, 50257, 1024
+        ldz = (V + 63) // 64 * 64
+        U = torch.randn(M, K, device=DEV).to(torch.bfloat16)
+        W = (torch.randn(V, K, device=DEV) * 0.02).to(torch.bfloat16)
+        E = torch.empty(M, ldz, dtype=torch.bfloat16, device=DEV)
+        if which == "logits":
+            tt = torch.randint(0, V, (M,), dtype=torch.int32, device=DEV)
+            nt = (V + 127) // 128
+            pm, ps = torch.zeros(M, nt, device=DEV), torch.zeros(M, nt, device=DEV)
+            tl = torch.zeros(M, device=DEV)
+            fn = lambda: il.op_gemm(M, V, K, U, K, 0, W, K, 0, 5, err, C_=E, ldc=ldz, targets=tt, part_max=pm,
+                                    part_sum=ps, part_ld=nt, tgt_logit=tl, store_exp=1)
+        else:
+            fn = lambda: il.op_gemm(M, V, K, U, K, 0, W, K, 0, 0, err, C_=E, ldc=ldz)
+        _timeit(which, fn, 2.0 * M * V * K, iters, err)
+    elif which in ("attn_fwd", "attn_bwd"):
+        B, T, H, dh = 8, 1024, 16, 64
+        NB = int(argv[3]) if len(argv) > 3 else B
+        d = H * dh
+        qkv = torch.randn(B * T, 3 * d, device=DEV).to(torch.bfloat16)
+        o = torch.empty(B * T, d, dtype=torch.bfloat16, device=DEV)
+        lse = torch.empty(B * H * T, device=DEV)
+        il.op_attention_fwd(qkv, o, lse, B, T, H, dh)
+        causal = 2.0 * B * H * T * T * dh          # QK^T and PV over the lower triangle
+        if which == "attn_fwd":
+            _timeit(which, lambda: il.op_attention_fwd(qkv, o, lse, B, T, H, dh), causal, iters, err)
+        else:
+            do = torch.randn(NB * T, d, device=DEV).to(torch.bfloat16)
+            dqkv = torch.empty(NB * T, 3 * d, dtype=torch.bfloat16, device=DEV)
+            delta = torch.empty(NB * H * T, device=DEV)
+            _timeit(which, lambda: il.op_attention_bwd(qkv, o, lse, do, dqkv, delta, NB, B, T, H, dh),
+                    2.5 * causal * NB / B, iters, err)
+    else:
+        raise SystemExit(__doc__)
+
+
+if __name__ == "__main__":
+    main(sys.argv)

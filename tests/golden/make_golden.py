@@ -44,8 +44,8 @@ def main():
     t0 = time.time()
     P = wl.draw_params(w)
     tok, tgt = wl.draw_tokens(w)
-    losses, G = orc.nwise_gradients(P, tok, tgt, w.K, w.Lc, w.H, n)
-    out = {"config": cfg, "n": n, "weight_seed": wl.WEIGHT_SEED, "token_seed": wl.TOKEN_SEED,
+    losses, G = orc.nwise_gradients(P, tok, tgt, w.K, w.Lc, w.H, n, rule=w.rule, head_layers=w.Lh)
+    out = {"config": cfg, "n": n, "rule": w.rule, "head_layers": w.Lh, "weight_seed": wl.WEIGHT_SEED, "token_seed": wl.TOKEN_SEED,
            "oracle_seconds": None, "losses": [float(x) for x in losses], "tensors": {}}
     for i, (name, _, _, _) in enumerate(wl.tensor_specs(w)):
         out["tensors"][name] = summarize(name, i, G[name])

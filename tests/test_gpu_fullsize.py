@@ -37,9 +37,13 @@ def _model(cfg):
         _models.clear()
         torch.cuda.empty_cache()
         w = wl.CONFIGS[cfg]
-        m = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, 1, w.B, w.T)
+        m = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, 1, w.B // w.M, w.T, head_layers=w.Lh)
         for i, (name, _, _, shape) in enumerate(wl.tensor_specs(w)):
             m.set_param(name, wl.draw_tensor(name, i, shape))
+        if w.rule != "sum":
+            m.set_rule(w.rule)
+        if w.M > 1:
+            m.set_micro_batches(w.M)
         _models[cfg] = m
     return _models[cfg]
 
@@ -50,15 +54,28 @@ def _check_against_golden(cfg, n):
     m = _model(cfg)
     m.set_n(n)
     tok, tgt = wl.draw_tokens(w)
-    m.train_step(torch.tensor(tok, device="cuda:0"), torch.tensor(tgt, device="cuda:0"))
-    losses = m.get_losses()
-    m.sync()
+    dt, dg = torch.tensor(tok, device="cuda:0"), torch.tensor(tgt, device="cuda:0")
     ref = np.array(gold["losses"])
-    assert np.all(np.abs(losses - ref) <= 1e-3 * np.abs(ref)), (losses, ref)
-    # the per-token losses average to the head loss (holds at any size)
-    tl = m.get_token_losses(w.K - 1, w.ntok)
-    assert abs(float(tl.astype(np.float64).mean()) - losses[-1]) < 1e-4 * losses[-1]
-    assert np.all(tl > 0)
+    if w.M > 1:
+        # the mini-batch as bench.py runs it: M micro-batch passes accumulating into one gradient; the stored
+        # losses are the whole mini-batch's, i.e. the mean of the micro-batches'
+        m.set_micro_batches(w.M)
+        per = w.B // w.M
+        losses = np.zeros(w.K)
+        for mb in range(w.M):
+            m.train_step(dt[mb * per:(mb + 1) * per], dg[mb * per:(mb + 1) * per])
+            losses += m.get_losses() / w.M
+        m.sync()
+        assert np.all(np.abs(losses - ref) <= 1e-3 * np.abs(ref)), (losses, ref)
+    else:
+        m.train_step(dt, dg)
+        losses = m.get_losses()
+        m.sync()
+        assert np.all(np.abs(losses - ref) <= 1e-3 * np.abs(ref)), (losses, ref)
+        # the per-token losses average to the head loss (holds at any size)
+        tl = m.get_token_losses(w.K - 1, w.ntok)
+        assert abs(float(tl.astype(np.float64).mean()) - losses[-1]) < 1e-4 * losses[-1]
+        assert np.all(tl > 0)
     bad = []
     for i, (name, _, _, _) in enumerate(wl.tensor_specs(w)):
         g = m.get_grad(name).astype(np.float64).reshape(-1)
@@ -90,6 +107,12 @@ def test_gpt2_small_shape_full_size(n):
 @pytest.mark.parametrize("n", [2, 3])
 def test_gpt2_medium_shape_full_size(n):
     _check_against_golden("cfg4", n)
+
+
+def test_paper_shape_full_model_reduced_batch():
+    """The paper-shaped model at full size (4 modules x 6 blocks, d 1024, 4 heads of 256, 2-block auxiliary networks,
+    vocabulary 50257, mean rule) on a mini-batch of 8 sequences of 128 tokens in 4 micro-batches."""
+    _check_against_golden("cfgP-b8", 2)
 
 
 def test_2p7b_shape_full_size():

@@ -72,6 +72,10 @@ CONFIGS: Dict[str, Workload] = {
     # size is not printed in the paper; the other configurations' 50257 is used.
     "cfgP": Workload("cfgP", K=4, Lc=6, d=1024, H=4, F=4096, V=50257, T=128, B=1024, n=2, adamw=True, Lh=2, M=4,
                      rule="mean", weight_decay=0.0),
+    # cfgP's model at full size on a mini-batch of 8 sequences (4 micro-batches of 2): what the fp64 oracle can
+    # run at full widths, depth and vocabulary in minutes, for the stored expected values.
+    "cfgP-b8": Workload("cfgP-b8", K=4, Lc=6, d=1024, H=4, F=4096, V=50257, T=128, B=8, n=2, adamw=True, Lh=2, M=4,
+                        rule="mean", weight_decay=0.0),
 }
 
 
