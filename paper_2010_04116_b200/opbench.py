@@ -4,7 +4,9 @@ through the C ABI: useful for comparing kernel changes and as a small case for p
     python -m paper_2010_04116_b200.opbench <op> [iterations] [gradient batches]
 
 ops: logits (auxiliary head: vocabulary projection with the softmax / exp(logit) epilogue), plain (the same
-contraction with a plain bf16 output), attn_fwd, attn_bwd (gradient batches = stacked gradient streams x 8).
+contraction with a plain bf16 output), fc1 (first MLP projection with the GELU epilogue and its two outputs),
+fc1_plain (the same contraction, bias and bf16 output only), attn_fwd, attn_bwd (gradient batches = stacked
+gradient streams x 8).
 """
 from __future__ import annotations
 
@@ -51,6 +53,17 @@ def main(argv):
         else:
             fn = lambda: il.op_gemm(M, V, K, U, K, 0, W, K, 0, 0, err, C_=E, ldc=ldz)
         _timeit(which, fn, 2.0 * M * V * K, iters, err)
+    elif which in ("fc1", "fc1_plain"):
+        M, N, K = 8192, 4096, 1024
+        X = torch.randn(M, K, device=DEV).to(torch.bfloat16)
+        W = (torch.randn(N, K, device=DEV) * 0.02).to(torch.bfloat16)
+        bias = torch.randn(N, device=DEV) * 0.02
+        Y, Y2 = (torch.empty(M, N, dtype=torch.bfloat16, device=DEV) for _ in range(2))
+        if which == "fc1":
+            fn = lambda: il.op_gemm(M, N, K, X, K, 0, W, K, 0, 1, err, C_=Y, ldc=N, C2=Y2, bias=bias)
+        else:
+            fn = lambda: il.op_gemm(M, N, K, X, K, 0, W, K, 0, 0, err, C_=Y, ldc=N, bias=bias)
+        _timeit(which, fn, 2.0 * M * N * K, iters, err)
     elif which in ("attn_fwd", "attn_bwd"):
         B, T, H, dh = 8, 1024, 16, 64
         NB = int(argv[3]) if len(argv) > 3 else B
