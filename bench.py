@@ -36,7 +36,7 @@ import workloads as wl  # noqa: E402
 # profiles/gemm_dram_traffic_cfg4_shapes.md).  Traffic grows with the flops of a launch at fixed shapes, so the
 # per-launch figure of another step mix is this ratio times that mix's flops per launch.  Set to None whenever
 # gemm.cu changes after the capture.
-GEMM_DRAM_BYTES_PER_FLOP = 1.2564e-3
+GEMM_DRAM_BYTES_PER_FLOP = 1.2568e-3
 
 
 def model_flops_per_token(w: wl.Workload, n: int) -> float:
