@@ -497,10 +497,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         if (p.rowscale && row_ok) rs = __ldg(p.rowscale + row);
       }
       const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * BN + half * (BN / 2));
-#pragma unroll
-      for (int c = 0; c < BN / 64; ++c) {
+      // One 32-column chunk of this warp's 32 rows; returns false once the chunk lies past the last column.
+      auto do_chunk = [&](const int c) -> bool {
         const int col = col_base + c * 32;
-        if (col >= p.N) break;               // uniform across the warp
+        if (col >= p.N) return false;        // uniform across the warp
         uint32_t r[32];
         tmem_ld_32x32(t_addr + (uint32_t)(c * 32), r);
         const int gcol = col + gcol_off;
@@ -617,6 +617,19 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           }
           __syncwarp();
         }
+        return true;
+      };
+      // Epilogues that prefetch a second operand index their register buffers by the chunk number, so their four
+      // chunks are unrolled; the others run the chunk body as a loop, a quarter of the code to keep in the
+      // instruction cache beside the main loop's.
+      if constexpr (EPI == EPI_BF16_DGELU || EPI == EPI_F32_RESID || EPI == EPI_F32) {
+#pragma unroll
+        for (int c = 0; c < BN / 64; ++c)
+          if (!do_chunk(c)) break;
+      } else {
+#pragma unroll 1
+        for (int c = 0; c < BN / 64; ++c)
+          if (!do_chunk(c)) break;
       }
       if constexpr (EPI == EPI_LSE) {
         if (row_ok && n_blk * BN + half * (BN / 2) < p.N) {
