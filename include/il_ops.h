@@ -97,6 +97,15 @@ il_status il_op_layernorm_bwd(const void* dy, int dy_is_f32, const float* x, con
                               const float* gamma, const float* resid, float* dx, void* dx_bf16, float* dgamma,
                               float* dbeta, int rows, int x_rows, int d, void* stream);
 
+/* The same in one pass over the rows for bf16 dy and d a multiple of 128 up to 1024 (IL_ERR_INVALID_ARG
+ * otherwise), as the training step runs it inside the blocks: dx and dx_bf16 as above, dgamma / dbeta summed into
+ * over the first x_rows rows, and, when colsum != NULL, colsum[c] += sum over the first x_rows rows of dx[r, c]
+ * (the bias gradient of the linear layer whose output this position of the residual stream is).  dgamma, dbeta
+ * and colsum are fp32 [d], zeroed by the caller or holding a sum to add to. */
+il_status il_op_layernorm_bwd_fused(const void* dy, const float* x, const float* mean, const float* rstd,
+                                    const float* gamma, const float* resid, float* dx, void* dx_bf16, float* dgamma,
+                                    float* dbeta, float* colsum, int rows, int x_rows, int d, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -91,6 +91,7 @@ def lib() -> C.CDLL:
         "il_op_attention_bwd_noalloc": [vp, vp, vp, vp, vp, i, i, i, i, i, vp],
         "il_op_layernorm_fwd": [vp, vp, vp, vp, vp, vp, i, i, f, vp],
         "il_op_layernorm_bwd": [vp, i, vp, vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, vp],
+        "il_op_layernorm_bwd_fused": [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, vp],
     }
     for name, args in sig.items():
         fn = getattr(L, name)
@@ -420,3 +421,11 @@ def op_layernorm_bwd(dy, dy_is_f32, x, mean, rstd, gamma, resid, dx, dx_bf16, dg
                                    _ptr(dx), _ptr(dx_bf16), _ptr(dgamma), _ptr(dbeta), rows, x_rows, d, stream)
     if st != IL_OK:
         raise ILError(st, "il_op_layernorm_bwd")
+
+
+def op_layernorm_bwd_fused(dy, x, mean, rstd, gamma, resid, dx, dx_bf16, dgamma, dbeta, colsum, rows, x_rows, d,
+                           stream=None):
+    st = lib().il_op_layernorm_bwd_fused(_ptr(dy), _ptr(x), _ptr(mean), _ptr(rstd), _ptr(gamma), _ptr(resid), _ptr(dx),
+                                         _ptr(dx_bf16), _ptr(dgamma), _ptr(dbeta), _ptr(colsum), rows, x_rows, d, stream)
+    if st != IL_OK:
+        raise ILError(st, "il_op_layernorm_bwd_fused")

@@ -466,7 +466,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           for (int i = 0; i < 8; ++i) {
             const int grow = row0 + 4 * i + lrow;
             int arow = arow0 + 4 * i + lrow;          // grow % aux_rows without a division
-            if (arow >= p.aux_rows) arow -= p.aux_rows;
+            while (arow >= p.aux_rows) arow -= p.aux_rows;   // more than once only for fewer than 32 saved rows
             pre_h[c][i] = make_uint2(0u, 0u);
             if (grow < p.M && gcol + 4 <= p.N)
               pre_h[c][i] = *reinterpret_cast<const uint2*>(p.aux + (size_t)arow * p.ld_aux + gcol);
@@ -520,7 +520,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             for (int i = 0; i < 8; ++i) {
               const int grow = row0 + 4 * i + lrow;
               int arow = arow0 + 4 * i + lrow;
-              if (arow >= p.aux_rows) arow -= p.aux_rows;
+              while (arow >= p.aux_rows) arow -= p.aux_rows;   // more than once only for fewer than 32 saved rows
               if (grow < p.M) extra[i] = epilogue_load4<EPI>(p, grow, arow, gcol);
             }
           }
@@ -782,7 +782,7 @@ cudaError_t gemm_launch(const GemmArgs& a, unsigned* err_word, int num_sms, cuda
   }
   if (a.epilogue == EPI_BF16_GELU && (!a.C2 || ((uintptr_t)a.C2 % 16))) return cudaErrorInvalidValue;
   if (a.epilogue == EPI_F32_RESID && (!a.resid || ((uintptr_t)a.resid % 16))) return cudaErrorInvalidValue;
-  if (a.epilogue == EPI_BF16_DGELU && (!a.aux || a.aux_rows < 32 || (a.ld_aux % 8) || ((uintptr_t)a.aux % 16)))
+  if (a.epilogue == EPI_BF16_DGELU && (!a.aux || a.aux_rows < 1 || (a.ld_aux % 8) || ((uintptr_t)a.aux % 16)))
     return cudaErrorInvalidValue;
   if (a.bias && ((uintptr_t)a.bias % 16)) return cudaErrorInvalidValue;
   if (a.colsum && (a.epilogue != EPI_BF16_DGELU || ((uintptr_t)a.colsum % 16))) return cudaErrorInvalidValue;

@@ -1191,3 +1191,13 @@ extern "C" il_status il_op_layernorm_bwd(const void* dy, int dy_is_f32, const fl
   }
   return op_status(layernorm_bwd_rows(dy, dy_is_f32, x, mean, rstd, gamma, resid, dx, (bf16*)dx_bf16, rows, x_rows, d, st));
 }
+
+extern "C" il_status il_op_layernorm_bwd_fused(const void* dy, const float* x, const float* mean, const float* rstd,
+                                               const float* gamma, const float* resid, float* dx, void* dx_bf16,
+                                               float* dgamma, float* dbeta, float* colsum, int rows, int x_rows, int d,
+                                               void* stream) {
+  if (!dy || !x || !mean || !rstd || !gamma || !dx || !dgamma || !dbeta || rows < 1 || x_rows < 1) return IL_ERR_INVALID_ARG;
+  if (d < 128 || d > 1024 || d % 128) return IL_ERR_INVALID_ARG;
+  return op_status(layernorm_bwd_fused((const bf16*)dy, x, mean, rstd, gamma, resid, dx, (bf16*)dx_bf16, dgamma, dbeta, colsum,
+                                       rows, x_rows, d, reinterpret_cast<cudaStream_t>(stream)));
+}

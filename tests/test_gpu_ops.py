@@ -260,6 +260,41 @@ def test_layernorm_forward_backward(rows, d):
         assert _rel(dxb.float().cpu().numpy(), got.astype(np.float64)) < 3e-3
 
 
+@pytest.mark.parametrize("rows,d,s", [(40, 128, 1), (1000, 768, 2), (8192 + 13, 1024, 2), (300, 384, 3)])
+def test_layernorm_backward_one_pass(rows, d, s):
+    """The one-pass LayerNorm backward of the blocks: row part for s stacked streams, gamma / beta gradients and the
+    column sums of its own output over the first stream, added to what the outputs already hold."""
+    rng = np.random.default_rng(rows * 3 + d + s)
+    x = (rng.standard_normal((rows, d)) * 2 + 0.5).astype(np.float32)
+    g = (1 + 0.1 * rng.standard_normal(d)).astype(np.float32)
+    xt, gt = torch.tensor(x, device=DEV), torch.tensor(g, device=DEV)
+    y = torch.zeros((rows, d), dtype=torch.bfloat16, device=DEV)
+    mean = torch.zeros(rows, dtype=torch.float32, device=DEV)
+    rstd = torch.zeros(rows, dtype=torch.float32, device=DEV)
+    il.op_layernorm_fwd(xt, gt, torch.zeros(d, device=DEV), y, mean, rstd, rows, d)
+    _, cache = orc.layernorm_fwd(x.astype(np.float64), g.astype(np.float64), np.zeros(d))
+    dyt, dye = _bf16(rng.standard_normal((s * rows, d)))
+    res = torch.tensor(rng.standard_normal((s * rows, d)), dtype=torch.float32, device=DEV)
+    res0 = res.cpu().numpy().astype(np.float64)
+    dxb = torch.zeros((s * rows, d), dtype=torch.bfloat16, device=DEV)
+    start = [rng.standard_normal(d).astype(np.float32) for _ in range(3)]     # sums the outputs are added to
+    dg, db, cs = [torch.tensor(v, device=DEV) for v in start]
+    il.op_layernorm_bwd_fused(dyt, xt, mean, rstd, gt, res, res, dxb, dg, db, cs, s * rows, rows, d)   # dx aliases resid
+    torch.cuda.synchronize()
+    got = res.cpu().numpy().astype(np.float64)
+    for j in range(s):
+        dxr, dgr, dbr = orc.layernorm_bwd(dye[j * rows:(j + 1) * rows], cache, g.astype(np.float64))
+        ref = res0[j * rows:(j + 1) * rows] + dxr
+        assert _rel(got[j * rows:(j + 1) * rows], ref) < 1e-5
+        if j == 0:
+            assert _rel(dg.cpu().numpy() - start[0], dgr) < 1e-4
+            assert _rel(db.cpu().numpy() - start[1], dbr) < 1e-4
+            assert _rel(cs.cpu().numpy() - start[2], ref.sum(axis=0)) < 1e-4
+    assert _rel(dxb.float().cpu().numpy(), got) < 3e-3
+    with pytest.raises(il.ILError):          # widths outside its range are refused, not mishandled
+        il.op_layernorm_bwd_fused(dyt, xt, mean, rstd, gt, res, res, dxb, dg, db, cs, s * rows, rows, 2560)
+
+
 @pytest.mark.parametrize("split", [2, 4])
 def test_gemm_split_k_adds_partial_sums(split):
     """wgrad layout with the contraction split over several work units per tile (atomic fp32 accumulation)."""
