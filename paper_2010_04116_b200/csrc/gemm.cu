@@ -445,9 +445,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const int gcol_off = 4 * (lane & 7);
       const int arow0 = (EPI == EPI_BF16_DGELU) ? row0 % p.aux_rows : 0;
       // While the main loop of this tile is still running, fetch the epilogue's second operand in the
-      // coalesced (transposed) layout: the saved pre-activation for all four chunks (bf16, 64 registers), or
-      // the first chunk of the fp32 residual / accumulated C (the later chunks are fetched one chunk ahead).
-      uint2 pre_h[EPI == EPI_BF16_DGELU ? 4 : 1][8];
+      // coalesced (transposed) layout: the first chunk of the saved gelu' (bf16) or of the fp32 residual /
+      // accumulated C; the later chunks are fetched one chunk ahead.
+      uint2 cur_h[8], nxt_h[8];      // saved gelu' of the chunk being processed and of the next one
       float4 pre_f[2][8];
       auto load_f32_chunk = [&](int c, float4 (&dst)[8]) {
         const int gcol = col_base + c * 32 + gcol_off;
@@ -458,20 +458,20 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           if (grow < p.M && gcol < p.N) dst[i] = epilogue_load4<EPI>(p, grow, 0, gcol);
         }
       };
-      if constexpr (EPI == EPI_BF16_DGELU) {
+      auto load_h_chunk = [&](int c, uint2 (&dst)[8]) {
+        const int gcol = col_base + c * 32 + gcol_off;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const int gcol = col_base + c * 32 + gcol_off;
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const int grow = row0 + 4 * i + lrow;
-            int arow = arow0 + 4 * i + lrow;          // grow % aux_rows without a division
-            while (arow >= p.aux_rows) arow -= p.aux_rows;   // more than once only for fewer than 32 saved rows
-            pre_h[c][i] = make_uint2(0u, 0u);
-            if (grow < p.M && gcol + 4 <= p.N)
-              pre_h[c][i] = *reinterpret_cast<const uint2*>(p.aux + (size_t)arow * p.ld_aux + gcol);
-          }
+        for (int i = 0; i < 8; ++i) {
+          const int grow = row0 + 4 * i + lrow;
+          int arow = arow0 + 4 * i + lrow;          // grow % aux_rows without a division
+          while (arow >= p.aux_rows) arow -= p.aux_rows;   // more than once only for fewer than 32 saved rows
+          dst[i] = make_uint2(0u, 0u);
+          if (grow < p.M && gcol + 4 <= p.N)
+            dst[i] = *reinterpret_cast<const uint2*>(p.aux + (size_t)arow * p.ld_aux + gcol);
         }
+      };
+      if constexpr (EPI == EPI_BF16_DGELU) {
+        load_h_chunk(0, cur_h);
       } else if constexpr (EPI == EPI_F32_RESID || EPI == EPI_F32) {
         load_f32_chunk(0, pre_f[0]);
       }
@@ -511,10 +511,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         if constexpr (EPI == EPI_BF16_DGELU) {
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
-            const float2 h0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pre_h[c][i].x));
-            const float2 h1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pre_h[c][i].y));
+            const float2 h0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&cur_h[i].x));
+            const float2 h1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&cur_h[i].y));
             extra[i] = make_float4(h0.x, h0.y, h1.x, h1.y);
           }
+          // the next chunk's values travel while this one is processed
+          if (c + 1 < BN / 64 && col + 32 < p.N) load_h_chunk(c + 1, nxt_h);
           if (!interior && gcol < p.N && gcol + 4 > p.N) {    // ragged last columns: element-wise reload
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
@@ -617,12 +619,16 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           }
           __syncwarp();
         }
+        if constexpr (EPI == EPI_BF16_DGELU) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) cur_h[i] = nxt_h[i];
+        }
         return true;
       };
       // Epilogues that prefetch a second operand index their register buffers by the chunk number, so their four
       // chunks are unrolled; the others run the chunk body as a loop, a quarter of the code to keep in the
       // instruction cache beside the main loop's.
-      if constexpr (EPI == EPI_BF16_DGELU || EPI == EPI_F32_RESID || EPI == EPI_F32) {
+      if constexpr (EPI == EPI_F32_RESID || EPI == EPI_F32) {
 #pragma unroll
         for (int c = 0; c < BN / 64; ++c)
           if (!do_chunk(c)) break;

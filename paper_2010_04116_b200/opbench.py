@@ -5,7 +5,9 @@ through the C ABI: useful for comparing kernel changes and as a small case for p
 
 ops: logits (auxiliary head: vocabulary projection with the softmax / exp(logit) epilogue), plain (the same
 contraction with a plain bf16 output), fc1 (first MLP projection with the GELU epilogue and its two outputs),
-fc1_plain (the same contraction, bias and bf16 output only), attn_fwd, attn_bwd (gradient batches = stacked
+fc1_plain (the same contraction, bias and bf16 output only), dgelu (gradient through the second MLP projection,
+multiplied by the saved GELU derivative, with the bias-gradient column sums; dgelu_nosum without them; dgelu_plain
+the bare contraction), attn_fwd, attn_bwd (gradient batches = stacked
 gradient streams x 8).
 """
 from __future__ import annotations
@@ -64,6 +66,19 @@ def main(argv):
         else:
             fn = lambda: il.op_gemm(M, N, K, X, K, 0, W, K, 0, 0, err, C_=Y, ldc=N, bias=bias)
         _timeit(which, fn, 2.0 * M * N * K, iters, err)
+    elif which in ("dgelu", "dgelu_nosum", "dgelu_plain"):
+        R, N, K = 16384, 4096, 1024            # two stacked gradient streams of 8192 tokens
+        dY = torch.randn(R, K, device=DEV).to(torch.bfloat16)
+        W2 = (torch.randn(K, N, device=DEV) * 0.02).to(torch.bfloat16)      # [d, F]: read MN-major
+        aux = torch.randn(R // 2, N, device=DEV).to(torch.bfloat16)
+        out = torch.empty(R, N, dtype=torch.bfloat16, device=DEV)
+        cs = torch.zeros(N, device=DEV)
+        if which == "dgelu_plain":
+            fn = lambda: il.op_gemm(R, N, K, dY, K, 0, W2, N, 1, 0, err, C_=out, ldc=N, tile_blocks=1)
+        else:
+            fn = lambda: il.op_gemm(R, N, K, dY, K, 0, W2, N, 1, 3, err, C_=out, ldc=N, aux=aux, ld_aux=N,
+                                    aux_rows=R // 2, colsum=cs if which == "dgelu" else None)
+        _timeit(which, fn, 2.0 * R * N * K, iters, err)
     elif which in ("attn_fwd", "attn_bwd"):
         B, T, H, dh = 8, 1024, 16, 64
         NB = int(argv[3]) if len(argv) > 3 else B
