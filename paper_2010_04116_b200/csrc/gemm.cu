@@ -448,7 +448,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       // coalesced (transposed) layout: the first chunk of the saved gelu' (bf16) or of the fp32 residual /
       // accumulated C; the later chunks are fetched one chunk ahead.
       uint2 cur_h[8], nxt_h[8];      // saved gelu' of the chunk being processed and of the next one
-      float4 pre_f[2][8];
+      float4 cur_f[8], nxt_f[8];     // fp32 second operand of the chunk being processed and of the next one
       auto load_f32_chunk = [&](int c, float4 (&dst)[8]) {
         const int gcol = col_base + c * 32 + gcol_off;
 #pragma unroll
@@ -473,7 +473,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       if constexpr (EPI == EPI_BF16_DGELU) {
         load_h_chunk(0, cur_h);
       } else if constexpr (EPI == EPI_F32_RESID || EPI == EPI_F32) {
-        load_f32_chunk(0, pre_f[0]);
+        load_f32_chunk(0, cur_f);
       }
       {   // one lane polls the barrier (keeps 255 pollers off the shared-memory pipe the main loop lives on)
         int got = 1;
@@ -528,8 +528,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           }
         } else if constexpr (EPI == EPI_F32_RESID || EPI == EPI_F32) {
 #pragma unroll
-          for (int i = 0; i < 8; ++i) extra[i] = pre_f[c & 1][i];
-          if (c + 1 < BN / 64 && col + 32 < p.N) load_f32_chunk(c + 1, pre_f[(c + 1) & 1]);
+          for (int i = 0; i < 8; ++i) extra[i] = cur_f[i];
+          if (c + 1 < BN / 64 && col + 32 < p.N) load_f32_chunk(c + 1, nxt_f);
         }
         tmem_ld_wait();
         float v[32];
@@ -623,20 +623,17 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
           for (int i = 0; i < 8; ++i) cur_h[i] = nxt_h[i];
         }
+        if constexpr (EPI == EPI_F32_RESID || EPI == EPI_F32) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) cur_f[i] = nxt_f[i];
+        }
         return true;
       };
-      // Epilogues that prefetch a second operand index their register buffers by the chunk number, so their four
-      // chunks are unrolled; the others run the chunk body as a loop, a quarter of the code to keep in the
-      // instruction cache beside the main loop's.
-      if constexpr (EPI == EPI_F32_RESID || EPI == EPI_F32) {
-#pragma unroll
-        for (int c = 0; c < BN / 64; ++c)
-          if (!do_chunk(c)) break;
-      } else {
+      // The chunk body is a loop, not four copies: it is the largest code in the kernel and has to stay in the
+      // instruction cache beside the main loop's (second operands are handed from chunk to chunk in registers).
 #pragma unroll 1
-        for (int c = 0; c < BN / 64; ++c)
-          if (!do_chunk(c)) break;
-      }
+      for (int c = 0; c < BN / 64; ++c)
+        if (!do_chunk(c)) break;
       if constexpr (EPI == EPI_LSE) {
         if (row_ok && n_blk * BN + half * (BN / 2) < p.N) {
           const size_t pi = (size_t)row * p.part_ld + (p.col0 / (BN / 2) + n_blk * 2 + half);
