@@ -507,6 +507,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         // fast path: the whole 32 x 32 chunk is inside the matrix (uniform across the warp), so nothing below
         // is predicated and the 32 element chains of a lane are independent straight-line code
         const bool interior = (row0 + 32 <= p.M) && (col + 32 <= p.N);
+        // the chunk's bias values are requested before the accumulator columns are waited for
+        float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        if constexpr (EPI == EPI_BF16 || EPI == EPI_BF16_GELU || EPI == EPI_F32_RESID)
+          if (interior && p.bias) b4 = __ldg(reinterpret_cast<const float4*>(p.bias + gcol));
         float4 extra[8];
         if constexpr (EPI == EPI_BF16_DGELU) {
 #pragma unroll
@@ -554,9 +558,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           for (int i = 0; i < 8; ++i)          // row 4i + lrow, slot (lane & 7) ^ (row & 7); row & 7 = (4i + lrow) & 7
             a[i] = *reinterpret_cast<const float4*>(stg + (4 * i + lrow) * STG_LD + 4 * ((lane & 7) ^ ((4 * i + lrow) & 7)));
           if (interior) {
-            float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f);
-            if constexpr (EPI == EPI_BF16 || EPI == EPI_BF16_GELU || EPI == EPI_F32_RESID)
-              if (p.bias) b4 = __ldg(reinterpret_cast<const float4*>(p.bias + gcol));
             if constexpr (EPI == EPI_F32_RESID || EPI == EPI_F32) {
               float* cbase = reinterpret_cast<float*>(p.C) + (size_t)(row0 + lrow) * p.ldc + gcol;
               if (EPI == EPI_F32 && p.split_k > 1) {       // partial sums of a k-range: add into the zeroed output
