@@ -335,12 +335,15 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const int n0 = n_blk * (NT * BN) + (int)rank * (BN / 2);   // this CTA's 128 rows of the (first) 256-row block of B
         const int kb0 = (t % p.split_k) * p.kb_per_split;
         const int kb1 = min(num_kb_all, kb0 + p.kb_per_split);
+        // a wide tile whose second 256-column block lies wholly past N carries that block neither through shared
+        // memory nor through the tensor pipe
+        const int nh = (NT == 2 && n_blk * (NT * BN) + BN >= p.N) ? 1 : NT;
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abortp)) { ok = false; break; }
           const uint32_t sa = smem_base + stage * STAGE_BYTES;
           const uint32_t sb = sa + A_BYTES;
           // both CTAs' bytes are credited to the leader's barrier, which expects the pair's total
-          if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * STAGE_BYTES);
+          if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * (A_BYTES + nh * B_BYTES));
           const uint32_t fb = mapa_cluster(full_bar(stage), 0);
           const int k0 = kb * BK;
           if constexpr (!A_MN) {
@@ -351,6 +354,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           }
 #pragma unroll
           for (int h = 0; h < NT; ++h) {          // block h of the tile's columns (past N: zero fill)
+            if (h >= nh) break;
             if constexpr (!B_MN) {
               tma_load_2d_pair(sb + h * B_BYTES, &tmB, k0, n0 + h * BN, fb);
             } else {
@@ -385,6 +389,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const uint32_t d_tmem = tmem_base + (uint32_t)(as * BN);
         const int kb0 = (t % p.split_k) * p.kb_per_split;
         const int kb1 = min(num_kb_all, kb0 + p.kb_per_split);
+        int m_blk_, n_tile_;
+        tile_coords(t / p.split_k, p.tiles_m, p.tiles_n, p.group_m, m_blk_, n_tile_);
+        const bool skip_h1 = (NT == 2 && n_tile_ * (NT * BN) + BN >= p.N);   // second block wholly past N: not loaded
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abortp)) { ok = false; break; }
           tc_fence_after();
@@ -396,6 +403,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
               if (!mbar_wait(acc_empty_bar(1), aphase ^ 1u, abortp)) { ok = false; break; }
               tc_fence_after();
             }
+            if (h == 1 && skip_h1) continue;      // the accumulator is still handed over below; nothing reads it
 #pragma unroll
             for (int k = 0; k < BK / 16; ++k) {
               // K-major: 16 k-elements = 32 bytes along the swizzled row; 8-row groups 1024 B apart.

@@ -317,6 +317,7 @@ def test_gemm_split_k_adds_partial_sums(split):
     (777, 1304, 136, (0, 1), 4),       # dgrad layout, three wide tiles, ragged rows
     (1304, 560, 264, (1, 1), 4),       # wgrad layout
     (640, 900, 320, (0, 0), 2),        # fp32 residual epilogue
+    (600, 768, 192, (0, 1), 0),        # one and a half wide tiles: the last tile's second block is skipped whole
     (300, 1000, 128, (0, 0), 5),       # softmax partials: block index must follow the column, not the tile
 ])
 def test_gemm_wide_tiles_match_square_tiles(M, N, K, layout, epi):
