@@ -3,6 +3,9 @@ through the C ABI: useful for comparing kernel changes and as a small case for p
 
     python -m paper_2010_04116_b200.opbench <op> [iterations] [gradient batches]
 
+The environment variable IL_OPBENCH_TILE (1 or 2) forces the GEMM tile width (256 or 512 columns) where the op
+takes one; unset, the library chooses.
+
 ops: logits (auxiliary head: vocabulary projection with the softmax / exp(logit) epilogue), plain (the same
 contraction with a plain bf16 output), fc1 (first MLP projection with the GELU epilogue and its two outputs),
 fc1_plain (the same contraction, bias and bf16 output only), dgelu (gradient through the second MLP projection,
@@ -12,6 +15,7 @@ gradient streams x 8).
 """
 from __future__ import annotations
 
+import os
 import sys
 
 import torch
@@ -19,6 +23,7 @@ import torch
 from . import binding as il
 
 DEV = "cuda:0"
+TILE = int(os.environ.get("IL_OPBENCH_TILE", "0"))
 
 
 def _timeit(name, fn, flops, iters, err):
@@ -51,9 +56,9 @@ def main(argv):
             pm, ps = torch.zeros(M, nt, device=DEV), torch.zeros(M, nt, device=DEV)
             tl = torch.zeros(M, device=DEV)
             fn = lambda: il.op_gemm(M, V, K, U, K, 0, W, K, 0, 5, err, C_=E, ldc=ldz, targets=tt, part_max=pm,
-                                    part_sum=ps, part_ld=nt, tgt_logit=tl, store_exp=1)
+                                    part_sum=ps, part_ld=nt, tgt_logit=tl, store_exp=1, tile_blocks=TILE)
         else:
-            fn = lambda: il.op_gemm(M, V, K, U, K, 0, W, K, 0, 0, err, C_=E, ldc=ldz)
+            fn = lambda: il.op_gemm(M, V, K, U, K, 0, W, K, 0, 0, err, C_=E, ldc=ldz, tile_blocks=TILE)
         _timeit(which, fn, 2.0 * M * V * K, iters, err)
     elif which in ("fc1", "fc1_plain"):
         M, N, K = 8192, 4096, 1024
@@ -62,9 +67,9 @@ def main(argv):
         bias = torch.randn(N, device=DEV) * 0.02
         Y, Y2 = (torch.empty(M, N, dtype=torch.bfloat16, device=DEV) for _ in range(2))
         if which == "fc1":
-            fn = lambda: il.op_gemm(M, N, K, X, K, 0, W, K, 0, 1, err, C_=Y, ldc=N, C2=Y2, bias=bias)
+            fn = lambda: il.op_gemm(M, N, K, X, K, 0, W, K, 0, 1, err, C_=Y, ldc=N, C2=Y2, bias=bias, tile_blocks=TILE)
         else:
-            fn = lambda: il.op_gemm(M, N, K, X, K, 0, W, K, 0, 0, err, C_=Y, ldc=N, bias=bias)
+            fn = lambda: il.op_gemm(M, N, K, X, K, 0, W, K, 0, 0, err, C_=Y, ldc=N, bias=bias, tile_blocks=TILE)
         _timeit(which, fn, 2.0 * M * N * K, iters, err)
     elif which in ("dgelu", "dgelu_nosum", "dgelu_plain"):
         R, N, K = 16384, 4096, 1024            # two stacked gradient streams of 8192 tokens
@@ -74,10 +79,10 @@ def main(argv):
         out = torch.empty(R, N, dtype=torch.bfloat16, device=DEV)
         cs = torch.zeros(N, device=DEV)
         if which == "dgelu_plain":
-            fn = lambda: il.op_gemm(R, N, K, dY, K, 0, W2, N, 1, 0, err, C_=out, ldc=N, tile_blocks=1)
+            fn = lambda: il.op_gemm(R, N, K, dY, K, 0, W2, N, 1, 0, err, C_=out, ldc=N, tile_blocks=TILE or 1)
         else:
             fn = lambda: il.op_gemm(R, N, K, dY, K, 0, W2, N, 1, 3, err, C_=out, ldc=N, aux=aux, ld_aux=N,
-                                    aux_rows=R // 2, colsum=cs if which == "dgelu" else None)
+                                    aux_rows=R // 2, colsum=cs if which == "dgelu" else None, tile_blocks=TILE)
         _timeit(which, fn, 2.0 * R * N * K, iters, err)
     elif which in ("attn_fwd", "attn_bwd"):
         B, T, H, dh = 8, 1024, 16, 64
