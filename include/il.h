@@ -58,14 +58,27 @@ typedef struct {
   void* alloc_ctx;
   void** streams;                   /* K cudaStream_t owned by the caller; NULL => library-created   */
   int n_streams;
-  int use_bias;                     /* reserved, must be 1 (GPT-2 style biases)                      */
+  int use_bias;                     /* must be 1 (GPT-2 style biases on every projection); anything else is refused  */
   float ln_eps;                     /* <= 0 => 1e-5                                                  */
   int head_layers;                  /* Transformer blocks inside every auxiliary head, 0..64.  0: the  */
                                     /* head is LayerNorm + linear.  2 is the auxiliary network of the  */
                                     /* paper's Transformer runs (App. B.3: main network output ->      */
                                     /* 2 Transformer blocks -> embedding matrix -> logits); the blocks */
                                     /* have the main network's shape, the head's LayerNorm follows them */
+  int head_mode;                    /* IL_HEAD_STORED (0, default) or IL_HEAD_RECOMPUTE (1): see il_aux_head_loss     */
+  int placement;                    /* IL_PLACE_SINGLE (0, default): all components on `device`, component k+1 reads   */
+                                    /* component k's output in place.  IL_PLACE_PIPELINE (1): the paper's placement,   */
+                                    /* one module per accelerator (Sec. 3): component k lives on devices[k] with its   */
+                                    /* parameters, optimiser state and activations; a_k travels forward and at most    */
+                                    /* n-1 gradient tensors travel backward per boundary, each copied into a buffer    */
+                                    /* the receiving device owns (see il_pipeline_transfers)                           */
+  const int* devices;               /* IL_PLACE_PIPELINE: K device ordinals (n_devices == K), or NULL: every component */
+  int n_devices;                    /* on `device`, still exchanged through the copy path.  Caller-owned streams[k]    */
+                                    /* must belong to devices[k]; the alloc hook is called with that device current    */
 } il_options;
+
+enum { IL_HEAD_STORED = 0, IL_HEAD_RECOMPUTE = 1 };
+enum { IL_PLACE_SINGLE = 0, IL_PLACE_PIPELINE = 1 };
 
 /* Build a model: K components x layers_per_component blocks, d_model, n_heads, d_ff, vocab, and the
  * n of the n-wise rule (Sec. 3: N in [1, number of modules]).  Requires d_model % n_heads == 0,
@@ -111,9 +124,20 @@ il_status il_set_batch(il_model* m, const int* tokens, const int* targets, int B
 /* Forward of component k (Sec. 3: a_k = f_ck(a_{k-1}); k = 0 also performs the embedding lookup).
  * Must be called for k = 0..K-1 in order. */
 il_status il_forward_component(il_model* m, int k);
-/* Auxiliary head k: LayerNorm, vocabulary projection and mean cross-entropy, with the logits
- * consumed tile by tile (never stored).  Needs il_forward_component(k).  loss_host != NULL makes the
- * call wait for this head and return its loss; NULL leaves it asynchronous. */
+/* Auxiliary head k (Sec. 3: h_ck and the local loss L_ck): LayerNorm, vocabulary projection and mean
+ * cross-entropy.  The projection's epilogue turns each output tile into per-row softmax partials and the
+ * target logit; the logits themselves are never stored.  What is kept for il_backward_nwise depends on
+ * il_options.head_mode:
+ *   IL_HEAD_STORED    the same epilogue also writes exp(logit) as a bf16 [B*T, vocab] matrix per head
+ *                     (vocab * 2 bytes per token and head: 824 MB per head at 8192 tokens and a 50257-word
+ *                     vocabulary); the backward runs its two contractions on that matrix without recomputing
+ *                     anything.  Price besides the memory: every row's log-sum-exp must lie in [-80, 80]
+ *                     (checked; a violation makes il_sync return IL_ERR_NONFINITE and skips the update).
+ *   IL_HEAD_RECOMPUTE nothing of size [B*T, vocab] is ever held: the backward walks the vocabulary in chunks of
+ *                     8192 columns, forms the chunk's logits again, turns them into dZ in the epilogue and
+ *                     feeds dZ to the two gradient contractions (one third more head flops, no range limit).
+ * Needs il_forward_component(k).  loss_host != NULL makes the call wait for this head and return its loss;
+ * NULL leaves it asynchronous. */
 il_status il_aux_head_loss(il_model* m, int k, float* loss_host);
 /* Per-token negative log-likelihood of head k for the current step, fp32 [B*T] to host (their mean is
  * the head's loss).  Needs il_aux_head_loss(k); waits for it. */
@@ -133,10 +157,16 @@ il_status il_backward_nwise(il_model* m);
  * abandons gradients accumulated so far.  Losses are reported per micro-batch. */
 il_status il_set_micro_batches(il_model* m, int micro_batches);
 /* AdamW (decoupled weight decay on rank-2 tensors; weight_decay = 0 is the paper's Adam,
- * App. B.3: beta1 0.9, beta2 0.98, eps 1e-9).  Needs il_backward_nwise.  Increments the step. */
+ * App. B.3: beta1 0.9, beta2 0.98, eps 1e-9).  Needs il_backward_nwise.  Increments the step.
+ * The update kernels read the device-side error word: while it is set (a bounded wait expired, or a head left
+ * the exp(logit) range) a component's parameters, Adam moments and bf16 copies are left untouched, and the next
+ * il_sync reports the error and takes the skipped updates back off the step counter.  The check is per component
+ * and per launch: a component whose update ran before another component raised the error keeps that update
+ * (il_last_error then says so). */
 il_status il_adamw_step(il_model* m, float lr, float beta1, float beta2, float eps, float weight_decay);
 /* Wait for all enqueued work; reports device-side timeouts as IL_ERR_TIMEOUT and a head whose
- * log-sum-exp left [-80, 80] in il_backward_nwise as IL_ERR_NONFINITE (that step's gradients are invalid). */
+ * log-sum-exp left [-80, 80] in il_backward_nwise as IL_ERR_NONFINITE (that step's gradients are invalid).
+ * Reporting clears the error: the next step starts clean. */
 il_status il_sync(il_model* m);
 /* Boundary activation a_k, k = 0..K (a_0 = embeddings), fp32 [B*T, d] to host; synchronises. */
 il_status il_get_boundary(il_model* m, int k, float* host, size_t count);
@@ -154,6 +184,22 @@ il_status il_profile_read(il_model* m, double* gemm_ms, long long* gemm_launches
  * k are grouped by that level.  Writes the distinct levels, descending, to terms[0..*count) (terms may be
  * NULL; it needs room for min(n, K) ints).  *count is the number of stacked backward passes of k. */
 il_status il_nwise_streams(int K, int n, int k, int* terms, int* count);
+/* Host-only: the tensors that cross component boundaries in one step of the pipeline placement (Sec. 3 and the
+ * schedule of Fig. 3: activations are sent to the next accelerator, gradients back to the previous one), in the
+ * order the step issues them.  Record i is records[3i .. 3i+2] = (direction, boundary, id): direction 0 = the
+ * activation a_{boundary+1} from component `boundary` to component boundary+1 (id -1); direction 1 = one [B*T, d]
+ * fp32 gradient tensor from component boundary+1 down to component `boundary`; id is, under IL_RULE_SUM, the
+ * termination level of the gradient stream (the sum of the gradients of all heads crossing component boundary+1
+ * that stop at or below the input of component id), and under the weighted rules the head whose gradient it is.
+ * At most n-1 gradient tensors cross a boundary.  *count receives the number of records; at most `capacity` are
+ * written (records may be NULL). */
+il_status il_pipeline_transfers(int K, int n, int rule, int* records, int capacity, int* count);
+/* The copies between components the pipeline placement actually issued since the last il_set_batch, in the same
+ * record format (empty for IL_PLACE_SINGLE). */
+il_status il_pipeline_last_transfers(il_model* m, int* records, int capacity, int* count);
+/* Device address of the error word the kernels of component k report to (unsigned; 0 = no error; see il_sync).
+ * For diagnostics and for tests of the error path: a caller may hand it to il_op_* calls as their err_word. */
+il_status il_error_word(il_model* m, int k, void** device_ptr);
 /* Host-only: the learning-rate schedule of the paper's Transformer runs (App. B.3),
  *   lr = d_model^-0.5 * min(step^-0.5, step * warmup_steps^-1.5),   step >= 1 (the paper: d_model 1024, warm-up 4000). */
 il_status il_lr_schedule(long long step, int d_model, int warmup_steps, double* lr);

@@ -64,10 +64,12 @@ typedef struct {
 il_status il_op_gemm(const il_gemm_desc* desc, unsigned* err_word, void* stream);
 
 /* Causal multi-head self-attention of the Transformer blocks on packed qkv [B*T, 3*H*dh] bf16
- * (Q | K | V; head h at columns h*dh): o [B*T, H*dh] bf16, lse [B, H, T] fp32.  dh in {32,64,80,128}. */
+ * (Q | K | V; head h at columns h*dh): o [B*T, H*dh] bf16, lse [B, H, T] fp32.  dh in {32, 64, 80, 128, 256};
+ * qkv and o 16-byte aligned, lse 4-byte aligned. */
 il_status il_op_attention_fwd(const void* qkv, void* o, float* lse, int B, int T, int H, int dh, void* stream);
 /* Its backward.  NB gradient batches may share the saved forward of B sequences (gradient batch b uses
- * sequence b % B): dout [NB*T, H*dh] bf16 -> dqkv [NB*T, 3*H*dh] bf16.  delta: scratch [NB*H*T] fp32. */
+ * sequence b % B): dout [NB*T, H*dh] bf16 -> dqkv [NB*T, 3*H*dh] bf16.  delta: scratch [NB*H*T] fp32.
+ * qkv, o, dout and dqkv must be 16-byte aligned (IL_ERR_INVALID_ARG otherwise, before anything is launched). */
 il_status il_op_attention_bwd(const void* qkv, const void* o, const float* lse, const void* dout, void* dqkv,
                               float* delta, int NB, int B, int T, int H, int dh, void* stream);
 
@@ -85,6 +87,17 @@ il_status il_op_attention_bwd(const void* qkv, const void* o, const float* lse, 
 il_status il_op_attention_bwd_noalloc(const void* qkv, const void* o, const float* lse, const void* dout, void* dqkv,
                                       int NB, int B, int T, int H, int dh, void* stream);
 size_t il_op_attention_bwd_noalloc_max_rows(void);
+/* Whether a bounded wait expired in any il_op_attention_bwd_noalloc call on the current device since the last
+ * call of this function (the allocation-free variant reports to an error word that also lives inside the library
+ * image).  Waits for `stream`, copies the word to the host and clears it: IL_OK, or IL_ERR_TIMEOUT when the
+ * results of those calls are not valid.  Allocates nothing. */
+il_status il_op_attention_bwd_noalloc_status(void* stream);
+
+/* Error-path probe: launches one thread that waits limit_us microseconds (1 .. 1,000,000) on a barrier nobody
+ * arrives at — the bounded wait every pipelined kernel of this library uses — and then writes a time-out code to
+ * *err_word, exactly as a kernel whose producer never delivered would.  The kernel returns normally; the GPU
+ * context stays usable.  With err_word = il_error_word(model, k) the model's next il_sync returns IL_ERR_TIMEOUT. */
+il_status il_op_wait_probe(unsigned* err_word, unsigned limit_us, void* stream);
 
 /* LayerNorm over the last axis (biased variance, eps inside the square root): y bf16 [rows, d],
  * mean/rstd fp32 [rows].  d % 8 == 0. */

@@ -31,7 +31,9 @@ class il_options(C.Structure):
     _fields_ = [("device", C.c_int), ("max_batch", C.c_int), ("max_seq", C.c_int),
                 ("alloc", ALLOC_FN), ("free_", FREE_FN), ("alloc_ctx", C.c_void_p),
                 ("streams", C.POINTER(C.c_void_p)), ("n_streams", C.c_int),
-                ("use_bias", C.c_int), ("ln_eps", C.c_float), ("head_layers", C.c_int)]
+                ("use_bias", C.c_int), ("ln_eps", C.c_float), ("head_layers", C.c_int),
+                ("head_mode", C.c_int), ("placement", C.c_int),
+                ("devices", C.POINTER(C.c_int)), ("n_devices", C.c_int)]
 
 
 class il_gemm_desc(C.Structure):
@@ -83,6 +85,11 @@ def lib() -> C.CDLL:
         "il_profile": [vp, i],
         "il_profile_read": [vp, C.POINTER(C.c_double), C.POINTER(C.c_longlong), C.POINTER(C.c_double)],
         "il_nwise_streams": [i, i, i, C.POINTER(i), C.POINTER(i)],
+        "il_pipeline_transfers": [i, i, i, C.POINTER(i), i, C.POINTER(i)],
+        "il_pipeline_last_transfers": [vp, C.POINTER(i), i, C.POINTER(i)],
+        "il_error_word": [vp, i, C.POINTER(vp)],
+        "il_op_wait_probe": [vp, C.c_uint, vp],
+        "il_op_attention_bwd_noalloc_status": [vp],
         "il_time_per_batch": [i, i, i, C.c_double, C.c_double, C.POINTER(C.c_double)],
         "il_optimal_microbatches": [i, i, C.c_double, C.c_double, i, C.POINTER(i)],
         "il_op_gemm": [C.POINTER(il_gemm_desc), vp, vp],
@@ -116,6 +123,23 @@ def nwise_streams(K: int, n: int, k: int) -> List[int]:
     if st != IL_OK:
         raise ILError(st, "il_nwise_streams")
     return [terms[i] for i in range(cnt.value)]
+
+
+RULES = {"sum": 0, "far": 1, "mean": 2}
+
+
+def pipeline_transfers(K: int, n: int, rule: str = "sum") -> List[tuple]:
+    """(direction, boundary, id) of every tensor that crosses a component boundary in one step of the pipeline
+    placement, in issue order (host-only)."""
+    cnt = C.c_int(0)
+    st = lib().il_pipeline_transfers(K, n, RULES[rule], None, 0, C.byref(cnt))
+    if st != IL_OK:
+        raise ILError(st, "il_pipeline_transfers")
+    rec = (C.c_int * (3 * max(cnt.value, 1)))()
+    st = lib().il_pipeline_transfers(K, n, RULES[rule], rec, cnt.value, C.byref(cnt))
+    if st != IL_OK:
+        raise ILError(st, "il_pipeline_transfers")
+    return [(rec[3 * i], rec[3 * i + 1], rec[3 * i + 2]) for i in range(cnt.value)]
 
 
 def time_per_batch(A: int, M: int, N: int, c0: float, c1: float) -> float:
@@ -153,7 +177,13 @@ class Model:
     the K per-component streams are torch streams."""
 
     def __init__(self, K: int, Lc: int, d: int, H: int, F: int, V: int, n: int, max_batch: int, max_seq: int,
-                 device: int = 0, torch_alloc: bool = True, torch_streams: bool = True, head_layers: int = 0):
+                 device: int = 0, torch_alloc: bool = True, torch_streams: bool = True, head_layers: int = 0,
+                 head_mode: str = "stored", placement: str = "single", devices: Optional[Sequence[int]] = None,
+                 alloc_fail_at: Optional[int] = None):
+        """head_mode: 'stored' (exp(logits) kept for the backward) or 'recompute' (vocabulary-chunked backward that
+        forms the logits again).  placement: 'single', or 'pipeline' = one component per entry of `devices`
+        (default: all on `device`, still exchanged through the copy path).  alloc_fail_at: make the allocator
+        hook return NULL at its i-th call (0-based), for tests of the out-of-memory path."""
         import torch
         self._torch = torch
         self.L = lib()
@@ -167,11 +197,26 @@ class Model:
         opt.use_bias = 1
         opt.ln_eps = 1e-5
         opt.head_layers = head_layers
+        opt.head_mode = {"stored": 0, "recompute": 1}[head_mode]
+        opt.placement = {"single": 0, "pipeline": 1}[placement]
+        self.head_mode, self.placement = head_mode, placement
+        self.devices = list(devices) if devices is not None else [device] * K
+        if devices is not None:
+            self._dev_arr = (C.c_int * K)(*self.devices)
+            opt.devices = C.cast(self._dev_arr, C.POINTER(C.c_int))
+            opt.n_devices = K
         dev = torch.device("cuda", device)
+        self._alloc_calls = 0
         if torch_alloc:
             def _alloc(nbytes, ctx):
+                i = self._alloc_calls
+                self._alloc_calls += 1
+                if alloc_fail_at is not None and i == alloc_fail_at:
+                    return None
                 try:
-                    t = torch.empty(int(nbytes), dtype=torch.uint8, device=dev)
+                    # the library calls the hook with the target device current
+                    cur = torch.device("cuda", torch.cuda.current_device()) if devices is not None else dev
+                    t = torch.empty(int(nbytes), dtype=torch.uint8, device=cur)
                 except Exception:
                     return None
                 self._blocks[t.data_ptr()] = t
@@ -184,7 +229,7 @@ class Model:
             opt.alloc, opt.free_ = self._alloc_cb, self._free_cb
         self.streams = []
         if torch_streams:
-            self.streams = [torch.cuda.Stream(device=dev) for _ in range(K)]
+            self.streams = [torch.cuda.Stream(device=torch.device("cuda", self.devices[k])) for k in range(K)]
             self._stream_arr = (C.c_void_p * K)(*[s.cuda_stream for s in self.streams])
             opt.streams = C.cast(self._stream_arr, C.POINTER(C.c_void_p))
             opt.n_streams = K
@@ -259,7 +304,21 @@ class Model:
         v = np.ascontiguousarray(v, dtype=np.float32)
         self._ck(self.L.il_set_opt_state(self._h, self.index[name], m.ctypes.data, v.ctypes.data, step))
 
-    RULES = {"sum": 0, "far": 1, "mean": 2}
+    RULES = RULES
+
+    def error_word(self, k: int = 0) -> int:
+        """Device address of the error word component k's kernels report to."""
+        out = C.c_void_p(None)
+        self._ck(self.L.il_error_word(self._h, k, C.byref(out)))
+        return out.value
+
+    def last_transfers(self) -> List[tuple]:
+        """(direction, boundary, id) of the copies between components issued since the last set_batch."""
+        cnt = C.c_int(0)
+        self._ck(self.L.il_pipeline_last_transfers(self._h, None, 0, C.byref(cnt)))
+        rec = (C.c_int * (3 * max(cnt.value, 1)))()
+        self._ck(self.L.il_pipeline_last_transfers(self._h, rec, cnt.value, C.byref(cnt)))
+        return [(rec[3 * i], rec[3 * i + 1], rec[3 * i + 2]) for i in range(cnt.value)]
 
     def set_rule(self, rule: str):
         """'sum' (default), 'far' (the paper's main-text rule) or 'mean' (its Transformer variant)."""
@@ -398,6 +457,19 @@ def op_attention_bwd(qkv, o, lse, dout, dqkv, delta, NB, B, T, H, dh, stream=Non
                                    dh, stream)
     if st != IL_OK:
         raise ILError(st, "il_op_attention_bwd")
+
+
+def op_wait_probe(err_word_ptr: int, limit_us: int, stream=None):
+    """Launch the error-path probe: a bounded wait that runs out after limit_us and writes a time-out code to the
+    device word at err_word_ptr."""
+    st = lib().il_op_wait_probe(err_word_ptr, limit_us, stream)
+    if st != IL_OK:
+        raise ILError(st, "il_op_wait_probe")
+
+
+def op_attention_bwd_noalloc_status(stream=None) -> int:
+    """il_status of the allocation-free attention backward calls since the last query (0 = fine)."""
+    return lib().il_op_attention_bwd_noalloc_status(stream)
 
 
 def op_attention_bwd_noalloc(qkv, o, lse, dout, dqkv, NB, B, T, H, dh, stream=None):

@@ -874,7 +874,7 @@ cudaError_t bwd_tc_launch(const bf16* qkv, const bf16* o, const float* lse, cons
 
 cudaError_t attention_fwd(const bf16* qkv, bf16* o, float* lse, int B, int T, int H, int dh, unsigned* err,
                           cudaStream_t s) {
-  if (((uintptr_t)qkv % 16) || ((uintptr_t)o % 16)) return cudaErrorInvalidValue;
+  if (((uintptr_t)qkv % 16) || ((uintptr_t)o % 16) || ((uintptr_t)lse % 4)) return cudaErrorInvalidValue;
   switch (dh) {
     case 32: return fwd_tc_launch<32>(qkv, o, lse, B, T, H, err, s);
     case 64: return fwd_tc_launch<64>(qkv, o, lse, B, T, H, err, s);
@@ -887,7 +887,10 @@ cudaError_t attention_fwd(const bf16* qkv, bf16* o, float* lse, int B, int T, in
 
 cudaError_t attention_bwd(const bf16* qkv, const bf16* o, const float* lse, const bf16* dout, bf16* dqkv, float* delta,
                              int NB, int B, int T, int H, int dh, unsigned* err, cudaStream_t s) {
-  if (((uintptr_t)qkv % 16) || ((uintptr_t)dout % 16) || ((uintptr_t)dqkv % 16)) return cudaErrorInvalidValue;
+  // o is read with 16-byte loads by the delta kernel, qkv / dout / dqkv by TMA and 16-byte stores
+  if (((uintptr_t)qkv % 16) || ((uintptr_t)o % 16) || ((uintptr_t)dout % 16) || ((uintptr_t)dqkv % 16) ||
+      ((uintptr_t)lse % 4) || ((uintptr_t)delta % 4))
+    return cudaErrorInvalidValue;
   switch (dh) {
     case 32: return bwd_tc_launch<32>(qkv, o, lse, dout, dqkv, delta, NB, B, T, H, err, s);
     case 64: return bwd_tc_launch<64>(qkv, o, lse, dout, dqkv, delta, NB, B, T, H, err, s);

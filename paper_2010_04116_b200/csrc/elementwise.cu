@@ -35,15 +35,103 @@ cudaError_t embed_fwd(const int* tok, const float* wte, const float* wpe, float*
   return cudaGetLastError();
 }
 
-__global__ void embed_bwd_wte_kernel(const int* __restrict__ tok, const float* __restrict__ dx,
-                                     float* __restrict__ dwte, int ntok, int d, int V) {
-  const size_t total = (size_t)ntok * d;
-  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
-    const int row = (int)(i / d);
-    const int c = (int)(i % d);
-    int t = tok[row];
-    t = t < 0 ? 0 : (t >= V ? V - 1 : t);
-    atomicAdd(dwte + (size_t)t * d + c, dx[i]);
+// Deterministic scatter-add of the embedding gradient.  Floating-point atomics would add the rows of a hot token
+// (under a Zipf law the most frequent id holds about a tenth of all positions) in whatever order the hardware
+// serves them; instead the positions are sorted by token id once per batch, and every token's rows are then
+// summed in position order.
+//
+// embed_sort: chunks of SORT_CHUNK positions; a block builds the keys (token << 13 | position in chunk) of its
+// chunk in shared memory and sorts them with a bitonic network (keys are distinct, so the order is total).
+constexpr int SORT_CHUNK = 8192;
+constexpr int SORT_POS_BITS = 13;
+
+__global__ void __launch_bounds__(1024) embed_sort_kernel(const int* __restrict__ tok, unsigned* __restrict__ keys, int ntok,
+                                                          int V) {
+  __shared__ unsigned sk[SORT_CHUNK];
+  const int base = blockIdx.x * SORT_CHUNK;
+  for (int i = threadIdx.x; i < SORT_CHUNK; i += 1024) {
+    unsigned key = 0xFFFFFFFFu;                       // padding sorts to the end
+    if (base + i < ntok) {
+      int t = tok[base + i];
+      t = t < 0 ? 0 : (t >= V ? V - 1 : t);
+      key = ((unsigned)t << SORT_POS_BITS) | (unsigned)i;
+    }
+    sk[i] = key;
+  }
+  __syncthreads();
+  for (int size = 2; size <= SORT_CHUNK; size <<= 1)
+    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+      for (int t = threadIdx.x; t < SORT_CHUNK / 2; t += 1024) {
+        const int lo = 2 * t - (t & (stride - 1));    // index of the lower element of pair t at this stride
+        const int hi = lo + stride;
+        const bool up = (lo & size) == 0;
+        const unsigned a = sk[lo], b = sk[hi];
+        if ((a > b) == up) { sk[lo] = b; sk[hi] = a; }
+      }
+      __syncthreads();
+    }
+  for (int i = threadIdx.x; i < SORT_CHUNK; i += 1024) keys[base + i] = sk[i];
+}
+
+cudaError_t embed_sort(const int* tok, unsigned* keys, int ntok, int V, cudaStream_t s) {
+  if (V > (1 << (32 - SORT_POS_BITS)) - 1) return cudaErrorInvalidValue;
+  embed_sort_kernel<<<ceil_div(ntok, SORT_CHUNK), 1024, 0, s>>>(tok, keys, ntok, V);
+  return cudaGetLastError();
+}
+
+// One block per sorted key of a chunk; the block whose key starts a token's run sums the run.  1024 threads =
+// 4 row groups x 256 column lanes (float4): group g adds rows g, g+4, ... of the run in order and the four
+// partial sums are combined in a fixed order, so the result does not depend on scheduling.
+__global__ void __launch_bounds__(1024) embed_bwd_wte_kernel(const unsigned* __restrict__ keys, const float* __restrict__ dx,
+                                                             float* __restrict__ dwte, int chunk_base, int ntok, int d,
+                                                             int accumulate) {
+  __shared__ float4 part[3][256];
+  const int i = blockIdx.x;                            // index within the chunk
+  const unsigned key = keys[chunk_base + i];
+  if (key == 0xFFFFFFFFu) return;
+  const unsigned tokid = key >> SORT_POS_BITS;
+  if (i > 0 && (keys[chunk_base + i - 1] >> SORT_POS_BITS) == tokid) return;     // not the start of a run
+  int len = 1;
+  const int limit = min(SORT_CHUNK, ntok - chunk_base);
+  while (i + len < limit && (keys[chunk_base + i + len] >> SORT_POS_BITS) == tokid) ++len;
+  const int g = threadIdx.x >> 8, lane = threadIdx.x & 255;
+  const int d4 = d >> 2;
+  constexpr unsigned POS_MASK = (1u << SORT_POS_BITS) - 1u;
+  for (int c0 = 0; c0 < d4; c0 += 256) {
+    const int c = c0 + lane;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (c < d4) {
+      int r = g;
+      for (; r + 12 < len; r += 16) {                  // four rows of this group in flight
+        float4 v[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const int pos = chunk_base + (int)(keys[chunk_base + i + r + 4 * q] & POS_MASK);
+          v[q] = reinterpret_cast<const float4*>(dx + (size_t)pos * d)[c];
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) { acc.x += v[q].x; acc.y += v[q].y; acc.z += v[q].z; acc.w += v[q].w; }
+      }
+      for (; r < len; r += 4) {
+        const int pos = chunk_base + (int)(keys[chunk_base + i + r] & POS_MASK);
+        const float4 v = reinterpret_cast<const float4*>(dx + (size_t)pos * d)[c];
+        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+      }
+    }
+    if (g > 0) part[g - 1][lane] = acc;
+    __syncthreads();
+    if (g == 0 && c < d4) {
+      const float4 p1 = part[0][lane], p2 = part[1][lane], p3 = part[2][lane];
+      acc.x = (acc.x + p1.x) + (p2.x + p3.x); acc.y = (acc.y + p1.y) + (p2.y + p3.y);
+      acc.z = (acc.z + p1.z) + (p2.z + p3.z); acc.w = (acc.w + p1.w) + (p2.w + p3.w);
+      float4* out = reinterpret_cast<float4*>(dwte + (size_t)tokid * d) + c;
+      if (accumulate) {
+        const float4 o = *out;
+        acc.x += o.x; acc.y += o.y; acc.z += o.z; acc.w += o.w;
+      }
+      *out = acc;
+    }
+    __syncthreads();
   }
 }
 __global__ void embed_bwd_wpe_kernel(const float* __restrict__ dx, float* __restrict__ dwpe, int B, int T, int d,
@@ -60,11 +148,13 @@ __global__ void embed_bwd_wpe_kernel(const float* __restrict__ dx, float* __rest
   }
 }
 
-cudaError_t embed_bwd(const int* tok, const float* dx, float* dwte, float* dwpe, int ntok, int T, int d, int V,
-                      int accumulate, cudaStream_t s) {
-  int blocks = ceil_div((size_t)ntok * d, 256);
-  if (blocks > 148 * 16) blocks = 148 * 16;
-  embed_bwd_wte_kernel<<<blocks, 256, 0, s>>>(tok, dx, dwte, ntok, d, V);
+cudaError_t embed_bwd(const int* tok, const unsigned* keys, const float* dx, float* dwte, float* dwpe, int ntok, int T,
+                      int d, int V, int accumulate, cudaStream_t s) {
+  (void)tok; (void)V;
+  // chunk after chunk on the one stream: a token that occurs in several chunks is added to in chunk order
+  for (int base = 0; base < ntok; base += SORT_CHUNK)
+    embed_bwd_wte_kernel<<<min(SORT_CHUNK, ntok - base), 1024, 0, s>>>(keys, dx, dwte, base, ntok, d,
+                                                                        (accumulate || base > 0) ? 1 : 0);
   int blocks2 = ceil_div((size_t)T * (d / 4), 256);
   embed_bwd_wpe_kernel<<<blocks2, 256, 0, s>>>(dx, dwpe, ntok / T, T, d, accumulate);
   return cudaGetLastError();
@@ -553,41 +643,49 @@ cudaError_t f32_to_bf16(const float* in, bf16* out, size_t n, cudaStream_t s) {
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) lse_finalize_kernel(const float* __restrict__ pm, const float* __restrict__ ps,
                                                            int part_ld, int ntiles, const float* __restrict__ tgt_logit,
-                                                           float* __restrict__ lse, float* loss_out, int rows,
-                                                           float inv_rows) {
-  __shared__ float sm[8];
+                                                           float* __restrict__ lse, float* __restrict__ nll, int rows) {
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const int row = blockIdx.x * 8 + w;
-  float contrib = 0.f;
-  if (row < rows) {
-    float m = -INFINITY;
-    for (int t = lane; t < ntiles; t += 32) m = fmaxf(m, pm[(size_t)row * part_ld + t]);
-    m = warp_max(m);
-    float sum = 0.f;
-    for (int t = lane; t < ntiles; t += 32) {
-      const float tm = pm[(size_t)row * part_ld + t];
-      if (tm > -INFINITY) sum += ps[(size_t)row * part_ld + t] * __expf(tm - m);
-    }
-    sum = warp_sum(sum);
-    const float l = m + logf(sum);
-    if (lane == 0) {
-      lse[row] = l;
-      contrib = l - tgt_logit[row];
-    }
+  if (row >= rows) return;
+  float m = -INFINITY;
+  for (int t = lane; t < ntiles; t += 32) m = fmaxf(m, pm[(size_t)row * part_ld + t]);
+  m = warp_max(m);
+  float sum = 0.f;
+  for (int t = lane; t < ntiles; t += 32) {
+    const float tm = pm[(size_t)row * part_ld + t];
+    if (tm > -INFINITY) sum += ps[(size_t)row * part_ld + t] * __expf(tm - m);
   }
-  if (lane == 0) sm[w] = contrib;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    float t = 0.f;
-    for (int i = 0; i < 8; ++i) t += sm[i];
-    atomicAdd(loss_out, t * inv_rows);
+  sum = warp_sum(sum);
+  const float l = m + logf(sum);
+  if (lane == 0) {
+    lse[row] = l;
+    nll[row] = l - tgt_logit[row];
   }
 }
 
 cudaError_t lse_finalize(const float* part_max, const float* part_sum, int part_ld, int ntiles, const float* tgt_logit,
-                         float* lse, float* loss_out, int rows, cudaStream_t s) {
-  lse_finalize_kernel<<<ceil_div(rows, 8), 256, 0, s>>>(part_max, part_sum, part_ld, ntiles, tgt_logit, lse, loss_out,
-                                                         rows, 1.0f / rows);
+                         float* lse, float* nll, int rows, cudaStream_t s) {
+  lse_finalize_kernel<<<ceil_div(rows, 8), 256, 0, s>>>(part_max, part_sum, part_ld, ntiles, tgt_logit, lse, nll, rows);
+  return cudaGetLastError();
+}
+
+// out[0] = mean of x[0..n) with a fixed summation order (one block: strided per-thread sums, then a tree), so the
+// value does not depend on scheduling.
+__global__ void __launch_bounds__(1024) mean_f32_kernel(const float* __restrict__ x, int n, float* __restrict__ out) {
+  __shared__ float sm[1024];
+  float a = 0.f;
+  for (int i = threadIdx.x; i < n; i += 1024) a += x[i];
+  sm[threadIdx.x] = a;
+  __syncthreads();
+  for (int o = 512; o > 0; o >>= 1) {
+    if (threadIdx.x < o) sm[threadIdx.x] += sm[threadIdx.x + o];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) out[0] = sm[0] / (float)n;
+}
+
+cudaError_t mean_f32(const float* x, int n, float* out, cudaStream_t s) {
+  mean_f32_kernel<<<1, 1024, 0, s>>>(x, n, out);
   return cudaGetLastError();
 }
 
@@ -646,7 +744,11 @@ cudaError_t head_backward_prepare(bf16* e, int ld, const float* lse, const int* 
 __global__ void __launch_bounds__(256) adamw_kernel(float4* __restrict__ p, float4* __restrict__ m, float4* __restrict__ v,
                                                     const float4* __restrict__ g, uint2* __restrict__ pb, size_t n4,
                                                     size_t n4_decay, float lr, float b1, float b2, float eps, float wd,
-                                                    float ibc1, float ibc2) {
+                                                    float ibc1, float ibc2, const unsigned* __restrict__ err,
+                                                    unsigned* applied) {
+  // a step whose kernels reported an error must not reach the parameters: leave everything as it is
+  if (err && *reinterpret_cast<const volatile unsigned*>(err) != 0u) return;
+  if (applied && blockIdx.x == 0 && threadIdx.x == 0) *applied += 1u;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
     const float w = i < n4_decay ? wd : 0.f;
     float4 pv = p[i], mv = m[i], vv = v[i];
@@ -666,7 +768,8 @@ __global__ void __launch_bounds__(256) adamw_kernel(float4* __restrict__ p, floa
 }
 
 cudaError_t adamw(float* p, float* m, float* v, const float* g, bf16* p_bf16, size_t n, size_t n_decay, float lr,
-                  float beta1, float beta2, float eps, float wd, float bc1, float bc2, cudaStream_t s) {
+                  float beta1, float beta2, float eps, float wd, float bc1, float bc2, const unsigned* err, unsigned* applied,
+                  cudaStream_t s) {
   const size_t n4 = n / 4;
   if (n4 == 0) return cudaSuccess;
   int blocks = ceil_div(n4, 256);
@@ -674,7 +777,28 @@ cudaError_t adamw(float* p, float* m, float* v, const float* g, bf16* p_bf16, si
   adamw_kernel<<<blocks, 256, 0, s>>>(reinterpret_cast<float4*>(p), reinterpret_cast<float4*>(m),
                                       reinterpret_cast<float4*>(v), reinterpret_cast<const float4*>(g),
                                       reinterpret_cast<uint2*>(p_bf16), n4, n_decay / 4, lr, beta1, beta2, eps, wd,
-                                      1.0f / bc1, 1.0f / bc2);
+                                      1.0f / bc1, 1.0f / bc2, err, applied);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// A wait that cannot succeed: one thread waits, with the given limit, on an mbarrier nobody arrives at, and
+// reports the expiry the way the pipelined kernels do.  It exercises the error path (error word -> host status)
+// without any kernel having to go wrong.
+// ---------------------------------------------------------------------------------------------
+__global__ void wait_probe_kernel(unsigned* err, unsigned long long limit_ns) {
+  __shared__ unsigned long long bar;
+  __shared__ int never;
+  if (threadIdx.x == 0) {
+    never = 0;
+    mbar_init(smem_u32(&bar), 1);
+    fence_mbar_init();
+    if (!mbar_wait(smem_u32(&bar), 0, &never, limit_ns)) atomicExch(err, DEV_TIMEOUT_EPILOGUE);
+  }
+}
+
+cudaError_t wait_probe(unsigned* err, unsigned long long limit_ns, cudaStream_t s) {
+  wait_probe_kernel<<<1, 32, 0, s>>>(err, limit_ns);
   return cudaGetLastError();
 }
 

@@ -5,7 +5,7 @@
 // (32 KB per 64-wide k-slab instead of the 48 KB a lone CTA needs for 128 x 256), the leader issues one
 // tcgen05.mma.cta_group::2 (M256 N256 K16) that reads both CTAs' shared memory and accumulates rows 0-127
 // in its own TMEM and rows 128-255 in the peer's.  Warp roles in each CTA:
-//   warp 0    : TMA producer — one thread streams the slabs into a 5-stage ring (128-byte swizzle); the byte
+//   warp 0    : TMA producer — one thread streams the slabs into a ring of 6 stages (256 x 256 tiles) or 4 (256 x 512), 128-byte swizzle; the byte
 //               counts of both CTAs are credited to the leader's "full" mbarrier.
 //   warp 1    : allocates 512 TMEM columns (two 128 x 256 fp32 accumulators per CTA); in the leader one thread
 //               issues the MMAs and commits (multicast to both CTAs) to the slab's "empty" barriers and,
@@ -155,7 +155,7 @@ __device__ __forceinline__ void epilogue_rowwise(const GemmDev& p, int col, floa
     const float l = st.m;   // lse of this row
     const int tj = st.tgt - (p.col0 + col);
 #pragma unroll
-    for (int j = 0; j < 32; ++j) v[j] = (__expf(v[j] - l) - (j == tj ? 1.0f : 0.0f)) * p.scale;
+    for (int j = 0; j < 32; ++j) v[j] = (ex2_fast((v[j] - l) * 1.4426950408889634f) - (j == tj ? 1.0f : 0.0f)) * p.scale;
   }
 }
 
@@ -721,6 +721,11 @@ static KernelFn pick_kernel(int a_mn, int b_mn, int epi, int nt) {
   return nt == 2 ? pick_kernel_nt<2>(a_mn, b_mn, epi) : pick_kernel_nt<1>(a_mn, b_mn, epi);
 }
 
+// The driver entry point is looked up once per process; the shared-memory opt-in of the kernels is a per-device
+// function attribute and is set once for every device the library is used on (with that device current).
+static std::mutex g_attr_mu;
+static bool g_attr_done[64] = {};
+
 cudaError_t gemm_init() {
   std::call_once(g_once, []() {
     void* fn = nullptr;
@@ -731,19 +736,26 @@ cudaError_t gemm_init() {
       return;
     }
     g_encode = reinterpret_cast<EncodeTiledFn>(fn);
-    for (int a = 0; a < 2; ++a)
-      for (int b = 0; b < 2; ++b)
-        for (int epi = 0; epi < EPI_COUNT; ++epi) {
-          for (int nt = 1; nt <= 2; ++nt) {
-            KernelFn k = pick_kernel(a, b, epi, nt);
-            if (!k) continue;
-            e = cudaFuncSetAttribute(reinterpret_cast<const void*>(k), cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     nt == 2 ? smem_bytes<2>() : smem_bytes<1>());
-            if (e != cudaSuccess) { g_init_err = e; return; }
-          }
-        }
   });
-  return g_init_err;
+  if (g_init_err != cudaSuccess) return g_init_err;
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_attr_mu);
+  if (g_attr_done[dev]) return cudaSuccess;
+  for (int a = 0; a < 2; ++a)
+    for (int b = 0; b < 2; ++b)
+      for (int epi = 0; epi < EPI_COUNT; ++epi)
+        for (int nt = 1; nt <= 2; ++nt) {
+          KernelFn k = pick_kernel(a, b, epi, nt);
+          if (!k) continue;
+          e = cudaFuncSetAttribute(reinterpret_cast<const void*>(k), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   nt == 2 ? smem_bytes<2>() : smem_bytes<1>());
+          if (e != cudaSuccess) return e;
+        }
+  g_attr_done[dev] = true;
+  return cudaSuccess;
 }
 
 bool tma_encode_bf16(CUtensorMap* tm, const void* ptr, int rank, const unsigned long long* dims,

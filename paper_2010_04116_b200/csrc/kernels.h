@@ -10,10 +10,13 @@ namespace il {
 // a_0[i,:] = wte[clamp(tok[i]),:] + wpe[i % T,:]  (fp32 residual stream)
 cudaError_t embed_fwd(const int* tok, const float* wte, const float* wpe, float* x, int ntok, int T, int d, int V,
                       cudaStream_t s);
-// dwte[tok[i],:] += dx[i,:] (atomic), dwpe[t,:] = (accumulate ? dwpe[t,:] : 0) + sum_b dx[b*T+t,:];  dwte must be
-// zeroed by the caller (or hold the sum it is to be added to).
-cudaError_t embed_bwd(const int* tok, const float* dx, float* dwte, float* dwpe, int ntok, int T, int d, int V,
-                      int accumulate, cudaStream_t s);
+// keys [ntok rounded up to 8192] = the batch's (token, position) pairs in sorted order, for embed_bwd.  V < 2^19.
+cudaError_t embed_sort(const int* tok, unsigned* keys, int ntok, int V, cudaStream_t s);
+// dwte[t,:] = (accumulate ? dwte[t,:] : 0) + sum over the positions i with tok[i] = t of dx[i,:], summed in position
+// order (deterministic; rows of tokens that do not occur are left as they are: zero them first unless accumulating);
+// dwpe[t,:] = (accumulate ? dwpe[t,:] : 0) + sum_b dx[b*T+t,:].
+cudaError_t embed_bwd(const int* tok, const unsigned* keys, const float* dx, float* dwte, float* dwpe, int ntok, int T,
+                      int d, int V, int accumulate, cudaStream_t s);
 
 // y(bf16) = gamma * (x - mean) * rstd + beta per row; mean/rstd saved in fp32.
 cudaError_t layernorm_fwd(const float* x, const float* gamma, const float* beta, __nv_bfloat16* y, float* mean,
@@ -47,19 +50,24 @@ cudaError_t lincomb_convert(const float* const* x, const float* w, int count, in
                             __nv_bfloat16* out_bf16, size_t n, cudaStream_t s);
 cudaError_t f32_to_bf16(const float* in, __nv_bfloat16* out, size_t n, cudaStream_t s);
 
-// Merge per-tile online-softmax partials: lse[r] = log sum_t exp(pm[r,t]) * ps[r,t];
-// loss_out += (1/rows) * sum_r (lse[r] - tgt_logit[r])   (loss_out zeroed by the caller).
+// Merge per-tile online-softmax partials: lse[r] = log sum_t exp(pm[r,t]) * ps[r,t]; nll[r] = lse[r] - tgt_logit[r].
+cudaError_t lse_finalize(const float* part_max, const float* part_sum, int part_ld, int ntiles, const float* tgt_logit,
+                         float* lse, float* nll, int rows, cudaStream_t s);
+// out[0] = mean of x[0..n), summed in a fixed order.
+cudaError_t mean_f32(const float* x, int n, float* out, cudaStream_t s);
+// Launches one thread that waits `limit_ns` on a barrier nobody arrives at and then sets *err = DEV_TIMEOUT_EPILOGUE.
+cudaError_t wait_probe(unsigned* err, unsigned long long limit_ns, cudaStream_t s);
 // Head backward set-up on E = exp(logits) (bf16 [rows, ld]): E[r, target_r] -= exp(lse_r); rowscale[r] =
 // scale * exp(-lse_r) / rows; u_scaled[r, :] = rowscale[r] * u[r, :].  Sets *err when an lse lies outside [-80, 80].
 cudaError_t head_backward_prepare(__nv_bfloat16* e, int ld, const float* lse, const int* targets, const __nv_bfloat16* u,
                                   __nv_bfloat16* u_scaled, float* rowscale, int rows, int d, float scale, unsigned* err,
                                   cudaStream_t s);
-cudaError_t lse_finalize(const float* part_max, const float* part_sum, int part_ld, int ntiles, const float* tgt_logit,
-                         float* lse, float* loss_out, int rows, cudaStream_t s);
 
 // AdamW over a flat range: the first n_decay elements get decoupled weight decay.  Writes the bf16 shadow.
+// err (may be NULL): when *err != 0 the kernel changes nothing; applied (may be NULL): += 1 when it does update.
 cudaError_t adamw(float* p, float* m, float* v, const float* g, __nv_bfloat16* p_bf16, size_t n, size_t n_decay,
-                  float lr, float beta1, float beta2, float eps, float wd, float bc1, float bc2, cudaStream_t s);
+                  float lr, float beta1, float beta2, float eps, float wd, float bc1, float bc2, const unsigned* err,
+                  unsigned* applied, cudaStream_t s);
 
 // Causal attention on packed qkv [B*T, 3d] (Q | K | V, head h at columns h*dh) on the tcgen05 tensor cores.
 // dh in {32, 64, 80, 128, 256}; pointers 16-byte aligned.

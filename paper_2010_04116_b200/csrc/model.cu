@@ -18,6 +18,7 @@
 #include <cstdio>
 #include <cstring>
 #include <string>
+#include <utility>
 #include <vector>
 
 #include "../../include/il.h"
@@ -50,10 +51,11 @@ struct CompScratch {     // backward scratch of one component, rows = s_cap * nt
   float* dx; bf16* dxb; bf16* dbig; bf16* dln; bf16* dattn; bf16* dqkv; float* delta;
 };
 struct HeadScratch {
-  bf16* u; float *mean, *rstd, *pmax, *psum, *tgt_logit, *lse, *du, *ghead;
-  bf16* z;   // [Ntok, ldz]: exp(logits) kept by the loss pass; the backward patches the target column in place
-  bf16* us;  // [Ntok, d]: rows of u scaled by exp(-lse) / Ntok
-  float* rs; // [Ntok]: exp(-lse) / Ntok
+  bf16* u; float *mean, *rstd, *pmax, *psum, *tgt_logit, *lse, *nll, *du, *ghead;
+  bf16* z;   // stored mode: [Ntok, ldz] exp(logits) kept by the loss pass, the backward patches the target column in
+             // place; recompute mode: [Ntok, chunk] dZ of one vocabulary chunk
+  bf16* us;  // [Ntok, d]: rows of u scaled by exp(-lse) / Ntok (stored mode)
+  float* rs; // [Ntok]: exp(-lse) / Ntok (stored mode)
 };
 
 struct ProfRec { cudaEvent_t a, b; double flops; };
@@ -65,6 +67,11 @@ struct il_model {
   int Lh;                             // Transformer blocks inside every auxiliary head (0 = LayerNorm + linear)
   int micro, micro_done;              // micro-batches per update, backward passes since the last update
   int rule;                           // IL_RULE_*: which heads update a component's parameters
+  int head_mode;                      // IL_HEAD_STORED / IL_HEAD_RECOMPUTE
+  int placement;                      // IL_PLACE_SINGLE / IL_PLACE_PIPELINE
+  std::vector<int> dev;               // device of component k (all equal to `device` unless placed as a pipeline)
+  std::vector<int> dev_list;          // the distinct devices in use
+  std::vector<int> sms;               // SM count of component k's device
   int device, num_sms;
   int max_batch, max_seq, ntok_max;
   float ln_eps;
@@ -80,18 +87,30 @@ struct il_model {
   size_t off_wte, off_wpe;
   std::vector<size_t> comp_begin, comp_mat_end, comp_end;   // flat ranges per component
   size_t total;
-  float *P, *G, *M1, *M2;
-  bf16* Pb;
+  // Per-component views of the parameter, gradient, Adam and bf16-shadow storage, biased so that view[k] + off is
+  // the element at flat offset `off` for every off in [comp_begin[k], comp_end[k]).  One flat buffer on a single
+  // device (all views equal); one buffer per component, on that component's device, in the pipeline placement.
+  std::vector<float*> P, G, M1, M2;
+  std::vector<bf16*> Pb;
   long long step;
+  int adamw_issued;                   // il_adamw_step calls since the last il_sync
   // activations
   std::vector<float*> a;             // K+1 boundaries; a[k+1] aliases the last layer's x_out
   std::vector<LayerActs> acts;       // same indexing as layer_off
   std::vector<CompScratch> cs;
   std::vector<HeadScratch> hs;
   int s_cap;
-  int *tokens, *targets;
-  float* losses;                     // device [K]
-  unsigned* err_word;
+  std::vector<int*> tokens, targets;  // per component: the batch on that component's device (shared on one device)
+  std::vector<float*> losses;         // per component: device [K] array holding losses[k] at index k
+  // Error words, per component (shared on one device): word 0 = DEV_* code of the first failure, words 1..K =
+  // number of AdamW updates component k-1 applied since the last il_sync (an update is skipped while word 0 is set).
+  std::vector<unsigned*> err_word;
+  // pipeline placement: receive buffers owned by the component's device
+  std::vector<float*> a_in;           // a_{k}: input of component k (k >= 1), copied from component k-1's output
+  std::vector<float*> g_in;           // [s_cap, Ntok, d]: gradient streams passed down from component k+1
+  std::vector<cudaEvent_t> ev_copy;   // per component: last copy into its receive buffers
+  std::vector<int> xfer_log;          // pipeline placement: (direction, boundary, id) of every copy of the current step
+  std::vector<unsigned*> sort_keys;   // [0]: scratch of the deterministic embedding backward on component 0's device
   int part_ld;
   int ldz;                            // row stride of the saved logits (vocabulary rounded up to 64)
   // step state
@@ -99,7 +118,8 @@ struct il_model {
   bool batch_set, bwd_done;
   std::vector<char> fwd_done, loss_done;
   // allocations
-  std::vector<void*> allocs;
+  std::vector<std::pair<void*, int>> allocs;   // (pointer, device it was obtained on)
+  std::vector<size_t> alloc_bytes;
   long long bytes, launches;
   // profiling
   int prof;                           // 0 off, 1 events around each GEMM, 2 the same with the GEMM alone on the GPU
@@ -132,6 +152,19 @@ il_status fail(il_model* m, il_status s, const char* fmt, ...) {
     if (s__ != IL_OK) return s__;         \
   } while (0)
 
+// Nothing may throw across the C boundary: every exported function runs its body through this.  Host containers
+// (the tensor registry, stream bookkeeping, the error string) can raise std::bad_alloc.
+template <class F>
+il_status guarded(F&& body) noexcept {
+  try {
+    return body();
+  } catch (const std::bad_alloc&) {
+    return IL_ERR_OOM;
+  } catch (...) {
+    return IL_ERR_CUDA;
+  }
+}
+
 il_status dev_alloc(il_model* m, void** out, size_t bytes) {
   bytes = (bytes + 255) & ~size_t(255);
   if (bytes == 0) bytes = 256;
@@ -143,10 +176,27 @@ il_status dev_alloc(il_model* m, void** out, size_t bytes) {
   }
   if (!p) return fail(m, IL_ERR_OOM, "device allocation of %zu bytes failed", bytes);
   if ((uintptr_t)p % 256) return fail(m, IL_ERR_INVALID_ARG, "allocator returned a pointer that is not 256-byte aligned");
-  m->allocs.push_back(p);
+  int cur = 0;
+  cudaGetDevice(&cur);
+  m->allocs.push_back(std::make_pair(p, cur));
+  m->alloc_bytes.push_back(bytes);
   m->bytes += (long long)bytes;
   *out = p;
   return IL_OK;
+}
+// Hand one allocation back (the device it came from is made current for the hook).
+void dev_free(il_model* m, void* p) {
+  if (!p) return;
+  for (size_t i = 0; i < m->allocs.size(); ++i)
+    if (m->allocs[i].first == p) {
+      cudaSetDevice(m->allocs[i].second);
+      if (m->opt.free_) m->opt.free_(p, m->opt.alloc_ctx);
+      else cudaFree(p);
+      m->bytes -= (long long)m->alloc_bytes[i];
+      m->allocs.erase(m->allocs.begin() + i);
+      m->alloc_bytes.erase(m->alloc_bytes.begin() + i);
+      return;
+    }
 }
 template <typename T>
 il_status dev_alloc_t(il_model* m, T** out, size_t count) {
@@ -157,6 +207,9 @@ il_status dev_alloc_t(il_model* m, T** out, size_t count) {
 }
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Vocabulary columns per chunk of the recompute head mode (a multiple of the 256-column output tile).
+constexpr int HEAD_CHUNK = 8192;
 
 // termination level of head h under the n-wise rule
 inline int term_of(int h, int n) { return h - n + 1 > 0 ? h - n + 1 : 0; }
@@ -190,7 +243,8 @@ il_status gemm(il_model* m, int k, const GemmArgs& g) {
   if (m->prof) {
     for (int i = 0; i < 2; ++i) {
       cudaEvent_t e;
-      if (!m->prof_pool.empty()) { e = m->prof_pool.back(); m->prof_pool.pop_back(); }
+      // (events belong to the device they were created on: the pool is only drawn from on a single device)
+      if (!m->prof_pool.empty() && m->dev_list.size() == 1) { e = m->prof_pool.back(); m->prof_pool.pop_back(); }
       else IL_CUDA(m, cudaEventCreate(&e));
       (i == 0 ? rec.a : rec.b) = e;
     }
@@ -206,7 +260,7 @@ il_status gemm(il_model* m, int k, const GemmArgs& g) {
     }
     IL_CUDA(m, cudaEventRecord(rec.a, st));
   }
-  cudaError_t e = gemm_launch(g, m->err_word, m->num_sms, st);
+  cudaError_t e = gemm_launch(g, m->err_word[k], m->sms[k], st);
   if (e != cudaSuccess)
     return fail(m, e == cudaErrorInvalidValue ? IL_ERR_INVALID_ARG : IL_ERR_CUDA, "gemm launch (M=%d N=%d K=%d epi=%d): %s",
                 g.M, g.N, g.K, g.epilogue, cudaGetErrorString(e));
@@ -247,7 +301,7 @@ GemmArgs gemm_args(int M, int N, int K, const void* A, int lda, int a_mn, const 
 // 256-wide one) plus the unit's exposed prologue / epilogue.
 il_status wgrad(il_model* m, int k, int M, int N, int K, const bf16* dY, int ld_dy, const bf16* X, int ld_x, float* dW,
                 bool acc) {
-  const int pairs = m->num_sms / 2;
+  const int pairs = m->sms[k] / 2;
   const int slabs = (K + 63) / 64;
   int best_nt = 1, best_s = 1;
   double best_cost = 1e300;
@@ -276,12 +330,21 @@ il_status wgrad(il_model* m, int k, int M, int N, int K, const bf16* dY, int ld_
 }
 
 il_status alloc_scratch(il_model* m, int s_cap) {
-  // grow-only: backward scratch for s_cap stacked gradient streams per component
+  // Backward scratch for s_cap stacked gradient streams per component.  It only grows; a superseded set is handed
+  // back before the larger one is obtained (the callers have synchronised the devices).
   if (s_cap <= m->s_cap) return IL_OK;
   const size_t R = (size_t)s_cap * m->ntok_max;
   const int d = m->d, F = m->F;
+  for (auto& c : m->cs) {
+    dev_free(m, c.dx); dev_free(m, c.dxb); dev_free(m, c.dbig); dev_free(m, c.dln); dev_free(m, c.dattn);
+    dev_free(m, c.dqkv); dev_free(m, c.delta);
+  }
+  for (float* g : m->g_in) dev_free(m, g);
   m->cs.assign(m->K, CompScratch{});
+  m->g_in.assign(m->K, nullptr);
+  m->s_cap = 0;
   for (int k = 0; k < m->K; ++k) {
+    IL_CUDA(m, cudaSetDevice(m->dev[k]));
     CompScratch& c = m->cs[k];
     IL_TRY(dev_alloc_t(m, &c.dx, R * d));
     IL_TRY(dev_alloc_t(m, &c.dxb, R * d));
@@ -290,6 +353,8 @@ il_status alloc_scratch(il_model* m, int s_cap) {
     IL_TRY(dev_alloc_t(m, &c.dattn, R * d));
     IL_TRY(dev_alloc_t(m, &c.dqkv, R * 3 * d));
     IL_TRY(dev_alloc_t(m, &c.delta, R * m->H));
+    // pipeline placement: the gradient streams component k+1 passes down land here, in memory of k's device
+    if (m->placement == IL_PLACE_PIPELINE && k + 1 < m->K) IL_TRY(dev_alloc_t(m, &m->g_in[k], R * d));
   }
   m->s_cap = s_cap;
   return IL_OK;
@@ -312,11 +377,27 @@ const float* head_input(const il_model* m, int k) {
 
 il_status check_model(const il_model* m) { return m ? IL_OK : IL_ERR_INVALID_ARG; }
 
-// Stream-ordered copy on stream 0 followed by a wait: the data is in place when this returns.
-il_status copy_sync(il_model* m, void* dst, const void* src, size_t bytes, cudaMemcpyKind kind) {
-  IL_CUDA(m, cudaMemcpyAsync(dst, src, bytes, kind, m->streams[0]));
-  IL_CUDA(m, cudaStreamSynchronize(m->streams[0]));
+// Stream-ordered copy on component k's stream followed by a wait: the data is in place when this returns.
+il_status copy_sync(il_model* m, int k, void* dst, const void* src, size_t bytes, cudaMemcpyKind kind) {
+  IL_CUDA(m, cudaSetDevice(m->dev[k]));
+  IL_CUDA(m, cudaMemcpyAsync(dst, src, bytes, kind, m->streams[k]));
+  IL_CUDA(m, cudaStreamSynchronize(m->streams[k]));
   return IL_OK;
+}
+
+// Wait for everything enqueued on every device the model uses.
+il_status sync_devices(il_model* m) {
+  for (int dv : m->dev_list) {
+    IL_CUDA(m, cudaSetDevice(dv));
+    IL_CUDA(m, cudaDeviceSynchronize());
+  }
+  return IL_OK;
+}
+
+// input of component k: the embeddings (k = 0), the output of component k-1 read in place (single device), or
+// this device's copy of it (pipeline placement)
+const float* comp_input(const il_model* m, int k) {
+  return (m->placement == IL_PLACE_PIPELINE && k > 0) ? m->a_in[k] : m->a[k];
 }
 
 }  // namespace
@@ -325,43 +406,70 @@ il_status copy_sync(il_model* m, void* dst, const void* src, size_t bytes, cudaM
 // creation / destruction
 // =================================================================================================
 extern "C" il_status il_create(int K, int Lc, int d, int H, int F, int V, int n, const il_options* opt, il_model** out) {
+  return guarded([&]() -> il_status {
   if (!out) return IL_ERR_INVALID_ARG;
   *out = nullptr;
-  if (!opt || K < 1 || Lc < 1 || d < 8 || H < 1 || F < 8 || V < 2 || n < 1 || n > K) return IL_ERR_INVALID_ARG;
+  if (!opt || K < 1 || K > 64 || Lc < 1 || d < 8 || H < 1 || F < 8 || V < 2 || n < 1 || n > K) return IL_ERR_INVALID_ARG;
   if (opt->head_layers < 0 || opt->head_layers > 64) return IL_ERR_INVALID_ARG;
   if (d % H || d % 8 || F % 8 || opt->max_batch < 1 || opt->max_seq < 1) return IL_ERR_INVALID_ARG;
   const int dh = d / H;
   if (!(dh == 32 || dh == 64 || dh == 80 || dh == 128 || dh == 256)) return IL_ERR_INVALID_ARG;
   if (opt->streams && opt->n_streams < K) return IL_ERR_INVALID_ARG;
   if ((opt->alloc == nullptr) != (opt->free_ == nullptr)) return IL_ERR_INVALID_ARG;
+  if (opt->use_bias != 1) return IL_ERR_INVALID_ARG;             // only the GPT-2 form with biases is built
+  if (opt->head_mode != IL_HEAD_STORED && opt->head_mode != IL_HEAD_RECOMPUTE) return IL_ERR_INVALID_ARG;
+  if (opt->placement != IL_PLACE_SINGLE && opt->placement != IL_PLACE_PIPELINE) return IL_ERR_INVALID_ARG;
+  if (opt->devices && (opt->placement != IL_PLACE_PIPELINE || opt->n_devices != K)) return IL_ERR_INVALID_ARG;
 
   il_model* m = new (std::nothrow) il_model();
   if (!m) return IL_ERR_OOM;
   m->K = K; m->Lc = Lc; m->d = d; m->H = H; m->F = F; m->V = V; m->n = n; m->dh = dh;
   m->Lh = opt->head_layers; m->micro = 1; m->micro_done = 0;
   m->opt = *opt;
+  m->opt.devices = nullptr;            // the caller's array is not kept
   m->device = opt->device;
+  m->head_mode = opt->head_mode; m->placement = opt->placement;
   m->max_batch = opt->max_batch; m->max_seq = opt->max_seq;
   m->ntok_max = opt->max_batch * opt->max_seq;
   m->ln_eps = opt->ln_eps > 0 ? opt->ln_eps : 1e-5f;
-  m->rule = IL_RULE_SUM; m->step = 0; m->bytes = 0; m->launches = 0; m->s_cap = 0;
+  m->rule = IL_RULE_SUM; m->step = 0; m->adamw_issued = 0; m->bytes = 0; m->launches = 0; m->s_cap = 0;
   m->prof = 0; m->batch_set = false; m->bwd_done = false;
   m->B = m->T = m->ntok = 0;
-  m->P = m->G = m->M1 = m->M2 = nullptr; m->Pb = nullptr;
+  m->ev_batch = nullptr;
   *out = m;   // returned even on failure below so that il_last_error/il_destroy work
 
   auto bail = [&](il_status s) { return s; };
-  {
-    cudaError_t e = cudaSetDevice(m->device);
-    if (e != cudaSuccess) return bail(fail(m, IL_ERR_CUDA, "cudaSetDevice(%d): %s", m->device, cudaGetErrorString(e)));
+  m->dev.assign(K, opt->device);
+  if (opt->devices)
+    for (int k = 0; k < K; ++k) m->dev[k] = opt->devices[k];
+  m->sms.assign(K, 0);
+  for (int k = 0; k < K; ++k) {
+    if (std::find(m->dev_list.begin(), m->dev_list.end(), m->dev[k]) == m->dev_list.end()) m->dev_list.push_back(m->dev[k]);
+    cudaError_t e = cudaSetDevice(m->dev[k]);
+    if (e != cudaSuccess) return bail(fail(m, IL_ERR_CUDA, "cudaSetDevice(%d): %s", m->dev[k], cudaGetErrorString(e)));
     cudaDeviceProp prop;
-    e = cudaGetDeviceProperties(&prop, m->device);
+    e = cudaGetDeviceProperties(&prop, m->dev[k]);
     if (e != cudaSuccess) return bail(fail(m, IL_ERR_CUDA, "cudaGetDeviceProperties: %s", cudaGetErrorString(e)));
-    if (prop.major != 10) return bail(fail(m, IL_ERR_CUDA, "device %d is sm_%d%d; this library is built for sm_100a only", m->device, prop.major, prop.minor));
-    m->num_sms = prop.multiProcessorCount;
+    if (prop.major != 10) return bail(fail(m, IL_ERR_CUDA, "device %d is sm_%d%d; this library is built for sm_100a only", m->dev[k], prop.major, prop.minor));
+    m->sms[k] = prop.multiProcessorCount;
     e = gemm_init();
     if (e != cudaSuccess) return bail(fail(m, IL_ERR_CUDA, "gemm_init: %s", cudaGetErrorString(e)));
   }
+  m->num_sms = m->sms[0];
+  // Neighbouring devices of the pipeline exchange boundary tensors with cudaMemcpyPeerAsync; with peer access
+  // enabled those copies go over NVLink directly instead of through host memory.  Failure to enable it is not an
+  // error (the copies still work).
+  for (int k = 0; k + 1 < K; ++k)
+    if (m->dev[k] != m->dev[k + 1])
+      for (int dir = 0; dir < 2; ++dir) {
+        const int a = m->dev[k + dir], b = m->dev[k + 1 - dir];
+        int can = 0;
+        if (cudaDeviceCanAccessPeer(&can, a, b) == cudaSuccess && can) {
+          cudaSetDevice(a);
+          cudaDeviceEnablePeerAccess(b, 0);
+          cudaGetLastError();            // "already enabled" is fine
+        }
+      }
 
   // ---- parameter registry and flat layout (per component: matrices first, then vectors)
   auto add = [&](const std::string& name, int comp, int is_head, int rank, long long s0, long long s1) {
@@ -432,10 +540,11 @@ extern "C" il_status il_create(int K, int Lc, int d, int H, int F, int V, int n,
     }
   }
 
-  // ---- streams and events
+  // ---- streams and events (each on its component's device)
   m->own_streams = (opt->streams == nullptr);
   m->streams.resize(K);
   for (int k = 0; k < K; ++k) {
+    IL_CUDA(m, cudaSetDevice(m->dev[k]));
     if (m->own_streams) {
       cudaError_t e = cudaStreamCreateWithFlags(&m->streams[k], cudaStreamNonBlocking);
       if (e != cudaSuccess) { m->streams.resize(k); return bail(fail(m, IL_ERR_CUDA, "cudaStreamCreate: %s", cudaGetErrorString(e))); }
@@ -446,6 +555,7 @@ extern "C" il_status il_create(int K, int Lc, int d, int H, int F, int V, int n,
   auto mk_events = [&](std::vector<cudaEvent_t>& v) -> il_status {
     v.resize(K);
     for (int k = 0; k < K; ++k) {
+      IL_CUDA(m, cudaSetDevice(m->dev[k]));
       cudaError_t e = cudaEventCreateWithFlags(&v[k], cudaEventDisableTiming);
       if (e != cudaSuccess) { v.resize(k); return fail(m, IL_ERR_CUDA, "cudaEventCreate: %s", cudaGetErrorString(e)); }
     }
@@ -454,39 +564,56 @@ extern "C" il_status il_create(int K, int Lc, int d, int H, int F, int V, int n,
   IL_TRY(mk_events(m->ev_fwd));
   IL_TRY(mk_events(m->ev_bwd));
   IL_TRY(mk_events(m->ev_join));
+  IL_TRY(mk_events(m->ev_copy));
+  IL_CUDA(m, cudaSetDevice(m->dev[0]));
   IL_CUDA(m, cudaEventCreateWithFlags(&m->ev_batch, cudaEventDisableTiming));
 
   // ---- parameter, gradient and optimiser storage
-  IL_TRY(dev_alloc_t(m, &m->P, m->total));
-  IL_TRY(dev_alloc_t(m, &m->G, m->total));
-  IL_TRY(dev_alloc_t(m, &m->M1, m->total));
-  IL_TRY(dev_alloc_t(m, &m->M2, m->total));
-  IL_TRY(dev_alloc_t(m, &m->Pb, m->total));
-  // All host<->device copies of the library are stream-ordered on stream 0 (a synchronous cudaMemcpy from
-  // pageable memory may return before its DMA has landed, and the legacy stream does not order against
-  // the non-blocking streams used here).
-  cudaStream_t s0 = m->streams[0];
-  IL_CUDA(m, cudaMemsetAsync(m->P, 0, m->total * 4, s0));
-  IL_CUDA(m, cudaMemsetAsync(m->G, 0, m->total * 4, s0));
-  IL_CUDA(m, cudaMemsetAsync(m->M1, 0, m->total * 4, s0));
-  IL_CUDA(m, cudaMemsetAsync(m->M2, 0, m->total * 4, s0));
-  IL_CUDA(m, cudaMemsetAsync(m->Pb, 0, m->total * 2, s0));
+  // All host<->device copies of the library are stream-ordered on the owning component's stream (a synchronous
+  // cudaMemcpy from pageable memory may return before its DMA has landed, and the legacy stream does not order
+  // against the non-blocking streams used here).
+  const bool pipe = m->placement == IL_PLACE_PIPELINE;
+  m->P.assign(K, nullptr); m->G.assign(K, nullptr); m->M1.assign(K, nullptr); m->M2.assign(K, nullptr);
+  m->Pb.assign(K, nullptr);
+  for (int k = 0; k < K; ++k) {
+    if (!pipe && k > 0) {   // one flat buffer: every component's view is the same pointer
+      m->P[k] = m->P[0]; m->G[k] = m->G[0]; m->M1[k] = m->M1[0]; m->M2[k] = m->M2[0]; m->Pb[k] = m->Pb[0];
+      continue;
+    }
+    IL_CUDA(m, cudaSetDevice(m->dev[k]));
+    const size_t lo = pipe ? m->comp_begin[k] : 0, cnt = pipe ? m->comp_end[k] - m->comp_begin[k] : m->total;
+    float* f[4];
+    for (int i = 0; i < 4; ++i) {
+      IL_TRY(dev_alloc_t(m, &f[i], cnt));
+      IL_CUDA(m, cudaMemsetAsync(f[i], 0, cnt * 4, m->streams[k]));
+    }
+    bf16* pb;
+    IL_TRY(dev_alloc_t(m, &pb, cnt));
+    IL_CUDA(m, cudaMemsetAsync(pb, 0, cnt * 2, m->streams[k]));
+    m->P[k] = f[0] - lo; m->G[k] = f[1] - lo; m->M1[k] = f[2] - lo; m->M2[k] = f[3] - lo; m->Pb[k] = pb - lo;
+  }
   {  // LayerNorm gains start at one
     std::vector<float> ones(d, 1.0f);
     for (auto& t : m->tensors)
       if (t.name.size() >= 2 && t.name.compare(t.name.size() - 2, 2, ".g") == 0) {
-        IL_CUDA(m, cudaMemcpyAsync(m->P + t.off, ones.data(), d * 4, cudaMemcpyHostToDevice, s0));
+        const int k = t.component;
+        IL_CUDA(m, cudaSetDevice(m->dev[k]));
+        IL_CUDA(m, cudaMemcpyAsync(m->P[k] + t.off, ones.data(), d * 4, cudaMemcpyHostToDevice, m->streams[k]));
+        IL_K(m, f32_to_bf16(m->P[k] + t.off, m->Pb[k] + t.off, d, m->streams[k]));
+        IL_CUDA(m, cudaStreamSynchronize(m->streams[k]));   // `ones` is pageable host memory
       }
-    IL_K(m, f32_to_bf16(m->P, m->Pb, m->total, s0));
-    IL_CUDA(m, cudaStreamSynchronize(s0));
   }
 
-  // ---- activations
+  // ---- activations, on the device of the component that produces them
   const size_t N = m->ntok_max;
   m->a.assign(K + 1, nullptr);
+  m->a_in.assign(K, nullptr);
+  IL_CUDA(m, cudaSetDevice(m->dev[0]));
   IL_TRY(dev_alloc_t(m, &m->a[0], N * d));
   m->acts.resize((size_t)K * (Lc + Lh));
-  for (int k = 0; k < K; ++k)
+  for (int k = 0; k < K; ++k) {
+    IL_CUDA(m, cudaSetDevice(m->dev[k]));
+    if (pipe && k > 0) IL_TRY(dev_alloc_t(m, &m->a_in[k], N * d));
     for (int l = 0; l < Lc + Lh; ++l) {
       LayerActs& A = l < Lc ? m->acts[(size_t)k * Lc + l] : m->acts[(size_t)K * Lc + (size_t)k * Lh + (l - Lc)];
       IL_TRY(dev_alloc_t(m, &A.ln1, N * d));
@@ -504,10 +631,14 @@ extern "C" il_status il_create(int K, int Lc, int d, int H, int F, int V, int n,
       IL_TRY(dev_alloc_t(m, &A.x_out, N * d));
       if (l == Lc - 1) m->a[k + 1] = A.x_out;   // the component's output; head blocks (l >= Lc) follow it
     }
+  }
   m->part_ld = (V + 127) / 128;
-  m->ldz = (V + 63) / 64 * 64;
+  // stored mode: row stride of exp(logits) = the vocabulary rounded up to 64; recompute mode: the width of one
+  // vocabulary chunk of dZ (a multiple of the 256-column tile)
+  m->ldz = m->head_mode == IL_HEAD_STORED ? (V + 63) / 64 * 64 : std::min(HEAD_CHUNK, (V + 255) / 256 * 256);
   m->hs.assign(K, HeadScratch{});
   for (int k = 0; k < K; ++k) {
+    IL_CUDA(m, cudaSetDevice(m->dev[k]));
     HeadScratch& h = m->hs[k];
     IL_TRY(dev_alloc_t(m, &h.u, N * d));
     IL_TRY(dev_alloc_t(m, &h.mean, N));
@@ -516,36 +647,61 @@ extern "C" il_status il_create(int K, int Lc, int d, int H, int F, int V, int n,
     IL_TRY(dev_alloc_t(m, &h.psum, N * m->part_ld));
     IL_TRY(dev_alloc_t(m, &h.tgt_logit, N));
     IL_TRY(dev_alloc_t(m, &h.lse, N));
+    IL_TRY(dev_alloc_t(m, &h.nll, N));
     IL_TRY(dev_alloc_t(m, &h.du, N * d));
     IL_TRY(dev_alloc_t(m, &h.ghead, N * d));
     IL_TRY(dev_alloc_t(m, &h.z, N * (size_t)m->ldz));
-    IL_TRY(dev_alloc_t(m, &h.us, N * d));
-    IL_TRY(dev_alloc_t(m, &h.rs, N));
+    if (m->head_mode == IL_HEAD_STORED) {
+      IL_TRY(dev_alloc_t(m, &h.us, N * d));
+      IL_TRY(dev_alloc_t(m, &h.rs, N));
+    }
   }
   IL_TRY(alloc_scratch(m, s_cap_for(K, n)));
-  IL_TRY(dev_alloc_t(m, &m->tokens, N));
-  IL_TRY(dev_alloc_t(m, &m->targets, N));
-  IL_TRY(dev_alloc_t(m, &m->losses, (size_t)K));
-  IL_TRY(dev_alloc_t(m, &m->err_word, (size_t)1));
-  IL_CUDA(m, cudaMemsetAsync(m->err_word, 0, 4, s0));
-  IL_CUDA(m, cudaMemsetAsync(m->losses, 0, K * 4, s0));
+  // batch, losses and error words: one set shared by all components on a single device, one per component otherwise
+  m->tokens.assign(K, nullptr); m->targets.assign(K, nullptr); m->losses.assign(K, nullptr);
+  m->err_word.assign(K, nullptr); m->sort_keys.assign(K, nullptr);
+  for (int k = 0; k < K; ++k) {
+    if (!pipe && k > 0) {
+      m->tokens[k] = m->tokens[0]; m->targets[k] = m->targets[0]; m->losses[k] = m->losses[0];
+      m->err_word[k] = m->err_word[0];
+      continue;
+    }
+    IL_CUDA(m, cudaSetDevice(m->dev[k]));
+    IL_TRY(dev_alloc_t(m, &m->tokens[k], N));
+    IL_TRY(dev_alloc_t(m, &m->targets[k], N));
+    IL_TRY(dev_alloc_t(m, &m->losses[k], (size_t)K));
+    IL_TRY(dev_alloc_t(m, &m->err_word[k], (size_t)(1 + K)));
+    IL_CUDA(m, cudaMemsetAsync(m->err_word[k], 0, 4 * (1 + K), m->streams[k]));
+    IL_CUDA(m, cudaMemsetAsync(m->losses[k], 0, K * 4, m->streams[k]));
+  }
+  IL_CUDA(m, cudaSetDevice(m->dev[0]));
+  IL_TRY(dev_alloc_t(m, &m->sort_keys[0], (N + 8191) / 8192 * 8192));     // embedding backward: sorted (token, position) keys
   m->fwd_done.assign(K, 0);
   m->loss_done.assign(K, 0);
-  IL_CUDA(m, cudaDeviceSynchronize());
+  for (int dv : m->dev_list) {
+    IL_CUDA(m, cudaSetDevice(dv));
+    IL_CUDA(m, cudaDeviceSynchronize());
+  }
   return IL_OK;
+  });
 }
 
 extern "C" il_status il_destroy(il_model* m) {
+  return guarded([&]() -> il_status {
   if (!m) return IL_ERR_INVALID_ARG;
-  cudaSetDevice(m->device);
-  cudaDeviceSynchronize();
-  for (void* p : m->allocs) {
-    if (m->opt.free_) m->opt.free_(p, m->opt.alloc_ctx);
-    else cudaFree(p);
+  for (int dv : m->dev_list) {
+    cudaSetDevice(dv);
+    cudaDeviceSynchronize();
+  }
+  for (auto& pr : m->allocs) {
+    cudaSetDevice(pr.second);
+    if (m->opt.free_) m->opt.free_(pr.first, m->opt.alloc_ctx);
+    else cudaFree(pr.first);
   }
   for (auto e : m->ev_fwd) cudaEventDestroy(e);
   for (auto e : m->ev_bwd) cudaEventDestroy(e);
   for (auto e : m->ev_join) cudaEventDestroy(e);
+  for (auto e : m->ev_copy) cudaEventDestroy(e);
   if (m->ev_batch) cudaEventDestroy(m->ev_batch);
   for (auto e : m->prof_pool) cudaEventDestroy(e);
   for (auto& r : m->prof_recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
@@ -553,27 +709,30 @@ extern "C" il_status il_destroy(il_model* m) {
     for (auto s : m->streams) cudaStreamDestroy(s);
   delete m;
   return IL_OK;
+  });
 }
 
 extern "C" il_status il_set_n(il_model* m, int n) {
+  return guarded([&]() -> il_status {
   IL_TRY(check_model(m));
   if (n < 1 || n > m->K) return fail(m, IL_ERR_INVALID_ARG, "n=%d outside [1, %d]", n, m->K);
-  IL_CUDA(m, cudaSetDevice(m->device));
-  IL_CUDA(m, cudaDeviceSynchronize());
+  IL_TRY(sync_devices(m));
   IL_TRY(alloc_scratch(m, m->rule == IL_RULE_SUM ? s_cap_for(m->K, n) : n));
   m->n = n;
   return IL_OK;
+  });
 }
 
 extern "C" il_status il_set_rule(il_model* m, int rule) {
+  return guarded([&]() -> il_status {
   IL_TRY(check_model(m));
   if (rule != IL_RULE_SUM && rule != IL_RULE_FAR && rule != IL_RULE_MEAN) return fail(m, IL_ERR_INVALID_ARG, "unknown rule %d", rule);
   if (m->n > 8 && rule != IL_RULE_SUM) return fail(m, IL_ERR_INVALID_ARG, "weighted rules support n <= 8");
-  IL_CUDA(m, cudaSetDevice(m->device));
-  IL_CUDA(m, cudaDeviceSynchronize());
+  IL_TRY(sync_devices(m));
   IL_TRY(alloc_scratch(m, rule == IL_RULE_SUM ? s_cap_for(m->K, m->n) : m->n));
   m->rule = rule;
   return IL_OK;
+  });
 }
 
 // =================================================================================================
@@ -583,6 +742,7 @@ extern "C" int il_num_tensors(const il_model* m) { return m ? (int)m->tensors.si
 
 extern "C" il_status il_tensor_info(const il_model* m, int idx, const char** name, int* component, int* is_head, int* rank,
                                     long long shape[2]) {
+  return guarded([&]() -> il_status {
   if (!m || idx < 0 || idx >= (int)m->tensors.size()) return IL_ERR_INVALID_ARG;
   const TensorRec& t = m->tensors[idx];
   if (name) *name = t.name.c_str();
@@ -591,6 +751,7 @@ extern "C" il_status il_tensor_info(const il_model* m, int idx, const char** nam
   if (rank) *rank = t.rank;
   if (shape) { shape[0] = t.shape[0]; shape[1] = t.shape[1]; }
   return IL_OK;
+  });
 }
 
 static il_status tensor_io(il_model* m, int idx, size_t count, const TensorRec** t) {
@@ -598,82 +759,108 @@ static il_status tensor_io(il_model* m, int idx, size_t count, const TensorRec**
   if (idx < 0 || idx >= (int)m->tensors.size()) return fail(m, IL_ERR_INVALID_ARG, "tensor index %d out of range", idx);
   *t = &m->tensors[idx];
   if (count != (*t)->count) return fail(m, IL_ERR_INVALID_ARG, "tensor %s has %zu elements, got %zu", (*t)->name.c_str(), (*t)->count, count);
-  IL_CUDA(m, cudaSetDevice(m->device));
-  IL_CUDA(m, cudaDeviceSynchronize());
+  IL_TRY(sync_devices(m));
   return IL_OK;
 }
 
 extern "C" il_status il_set_param(il_model* m, int idx, const float* host, size_t count) {
+  return guarded([&]() -> il_status {
   const TensorRec* t;
   if (!host) return IL_ERR_INVALID_ARG;
   IL_TRY(tensor_io(m, idx, count, &t));
-  IL_CUDA(m, cudaMemcpyAsync(m->P + t->off, host, count * 4, cudaMemcpyHostToDevice, m->streams[0]));
-  IL_K(m, f32_to_bf16(m->P + t->off, m->Pb + t->off, align_up(count, 4), m->streams[0]));
-  IL_CUDA(m, cudaStreamSynchronize(m->streams[0]));
+  const int k = t->component;
+  IL_CUDA(m, cudaSetDevice(m->dev[k]));
+  IL_CUDA(m, cudaMemcpyAsync(m->P[k] + t->off, host, count * 4, cudaMemcpyHostToDevice, m->streams[k]));
+  IL_K(m, f32_to_bf16(m->P[k] + t->off, m->Pb[k] + t->off, align_up(count, 4), m->streams[k]));
+  IL_CUDA(m, cudaStreamSynchronize(m->streams[k]));
   return IL_OK;
+  });
 }
 extern "C" il_status il_get_param(il_model* m, int idx, float* host, size_t count) {
+  return guarded([&]() -> il_status {
   const TensorRec* t;
   if (!host) return IL_ERR_INVALID_ARG;
   IL_TRY(tensor_io(m, idx, count, &t));
-  IL_TRY(copy_sync(m, host, m->P + t->off, count * 4, cudaMemcpyDeviceToHost));
+  IL_TRY(copy_sync(m, t->component, host, m->P[t->component] + t->off, count * 4, cudaMemcpyDeviceToHost));
   return IL_OK;
+  });
 }
 extern "C" il_status il_get_grad(il_model* m, int idx, float* host, size_t count) {
+  return guarded([&]() -> il_status {
   const TensorRec* t;
   if (!host) return IL_ERR_INVALID_ARG;
   IL_TRY(tensor_io(m, idx, count, &t));
   if (!m->bwd_done) return fail(m, IL_ERR_STATE, "il_get_grad before il_backward_nwise");
-  IL_TRY(copy_sync(m, host, m->G + t->off, count * 4, cudaMemcpyDeviceToHost));
+  IL_TRY(copy_sync(m, t->component, host, m->G[t->component] + t->off, count * 4, cudaMemcpyDeviceToHost));
   return IL_OK;
+  });
 }
 extern "C" il_status il_get_opt_state(il_model* m, int idx, float* mh, float* vh, long long* step) {
+  return guarded([&]() -> il_status {
   IL_TRY(check_model(m));
   if (idx < 0 || idx >= (int)m->tensors.size()) return fail(m, IL_ERR_INVALID_ARG, "tensor index %d out of range", idx);
   const TensorRec* t;
   IL_TRY(tensor_io(m, idx, m->tensors[idx].count, &t));
-  if (mh) IL_TRY(copy_sync(m, mh, m->M1 + t->off, t->count * 4, cudaMemcpyDeviceToHost));
-  if (vh) IL_TRY(copy_sync(m, vh, m->M2 + t->off, t->count * 4, cudaMemcpyDeviceToHost));
+  const int k = t->component;
+  if (mh) IL_TRY(copy_sync(m, k, mh, m->M1[k] + t->off, t->count * 4, cudaMemcpyDeviceToHost));
+  if (vh) IL_TRY(copy_sync(m, k, vh, m->M2[k] + t->off, t->count * 4, cudaMemcpyDeviceToHost));
   if (step) *step = m->step;
   return IL_OK;
+  });
 }
 extern "C" il_status il_set_opt_state(il_model* m, int idx, const float* mh, const float* vh, long long step) {
+  return guarded([&]() -> il_status {
   IL_TRY(check_model(m));
   if (idx < 0 || idx >= (int)m->tensors.size()) return fail(m, IL_ERR_INVALID_ARG, "tensor index %d out of range", idx);
   if (step < 0) return fail(m, IL_ERR_INVALID_ARG, "negative step");
   const TensorRec* t;
   IL_TRY(tensor_io(m, idx, m->tensors[idx].count, &t));
-  if (mh) IL_TRY(copy_sync(m, m->M1 + t->off, mh, t->count * 4, cudaMemcpyHostToDevice));
-  if (vh) IL_TRY(copy_sync(m, m->M2 + t->off, vh, t->count * 4, cudaMemcpyHostToDevice));
+  const int k = t->component;
+  if (mh) IL_TRY(copy_sync(m, k, m->M1[k] + t->off, mh, t->count * 4, cudaMemcpyHostToDevice));
+  if (vh) IL_TRY(copy_sync(m, k, m->M2[k] + t->off, vh, t->count * 4, cudaMemcpyHostToDevice));
   m->step = step;
   return IL_OK;
+  });
 }
 
 // =================================================================================================
 // the step
 // =================================================================================================
 extern "C" il_status il_set_batch(il_model* m, const int* tokens, const int* targets, int B, int T, int on_device) {
+  return guarded([&]() -> il_status {
   IL_TRY(check_model(m));
   if (!tokens || !targets) return fail(m, IL_ERR_INVALID_ARG, "NULL tokens/targets");
   if (B < 1 || T < 1 || B > m->max_batch || T > m->max_seq || (size_t)B * T > (size_t)m->ntok_max)
     return fail(m, IL_ERR_INVALID_ARG, "batch %dx%d exceeds max_batch=%d, max_seq=%d", B, T, m->max_batch, m->max_seq);
-  IL_CUDA(m, cudaSetDevice(m->device));
+  IL_CUDA(m, cudaSetDevice(m->dev[0]));
   // every stream's previous work must be finished before buffers of the last step are overwritten
   IL_TRY(join_all(m));
   cudaStream_t s0 = m->streams[0];
   const size_t bytes = (size_t)B * T * sizeof(int);
-  const cudaMemcpyKind kind = on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
-  IL_CUDA(m, cudaMemcpyAsync(m->tokens, tokens, bytes, kind, s0));
-  IL_CUDA(m, cudaMemcpyAsync(m->targets, targets, bytes, kind, s0));
-  IL_CUDA(m, cudaMemsetAsync(m->losses, 0, m->K * sizeof(float), s0));
+  const cudaMemcpyKind kind = on_device ? cudaMemcpyDefault : cudaMemcpyHostToDevice;
   IL_CUDA(m, cudaEventRecord(m->ev_batch, s0));
-  for (int k = 1; k < m->K; ++k) IL_CUDA(m, cudaStreamWaitEvent(m->streams[k], m->ev_batch, 0));
+  for (int k = 0; k < m->K; ++k) {
+    if (k > 0) IL_CUDA(m, cudaStreamWaitEvent(m->streams[k], m->ev_batch, 0));
+    if (k > 0 && m->tokens[k] == m->tokens[0]) continue;       // one shared copy on a single device
+    IL_CUDA(m, cudaSetDevice(m->dev[k]));
+    IL_CUDA(m, cudaMemcpyAsync(m->tokens[k], tokens, bytes, kind, m->streams[k]));
+    IL_CUDA(m, cudaMemcpyAsync(m->targets[k], targets, bytes, kind, m->streams[k]));
+  }
+  IL_CUDA(m, cudaSetDevice(m->dev[0]));
+  // (token, position) keys in sorted order for the embedding backward: known as soon as the batch is
+  IL_K(m, embed_sort(m->tokens[0], m->sort_keys[0], B * T, m->V, s0));
+  if (m->tokens[1 % m->K] == m->tokens[0]) {     // shared buffers: the other streams start after the copies
+    IL_CUDA(m, cudaEventRecord(m->ev_batch, s0));
+    for (int k = 1; k < m->K; ++k) IL_CUDA(m, cudaStreamWaitEvent(m->streams[k], m->ev_batch, 0));
+  }
   m->B = B; m->T = T; m->ntok = B * T;
+  m->xfer_log.clear();
   m->batch_set = true;
   m->bwd_done = false;
   std::fill(m->fwd_done.begin(), m->fwd_done.end(), 0);
   std::fill(m->loss_done.begin(), m->loss_done.end(), 0);
   return IL_OK;
+  });
 }
 
 namespace {
@@ -685,29 +872,29 @@ il_status layers_forward(il_model* m, int k, size_t base, int count, const float
   for (int l = 0; l < count; ++l) {
     const LayerOff& o = m->layer_off[base + l];
     LayerActs& A = m->acts[base + l];
-    IL_K(m, layernorm_fwd(x_in, m->P + o.ln1g, m->P + o.ln1b, A.ln1, A.mean1, A.rstd1, N, d, m->ln_eps, st));
+    IL_K(m, layernorm_fwd(x_in, m->P[k] + o.ln1g, m->P[k] + o.ln1b, A.ln1, A.mean1, A.rstd1, N, d, m->ln_eps, st));
     {
-      GemmArgs g = gemm_args(N, 3 * d, d, A.ln1, d, 0, m->Pb + o.wqkv, d, 0, EPI_BF16, A.qkv, 3 * d);
-      g.bias = m->P + o.bqkv;
+      GemmArgs g = gemm_args(N, 3 * d, d, A.ln1, d, 0, m->Pb[k] + o.wqkv, d, 0, EPI_BF16, A.qkv, 3 * d);
+      g.bias = m->P[k] + o.bqkv;
       IL_TRY(gemm(m, k, g));
     }
-    IL_K(m, attention_fwd(A.qkv, A.attn_o, A.lse, m->B, m->T, m->H, m->dh, m->err_word, st));
+    IL_K(m, attention_fwd(A.qkv, A.attn_o, A.lse, m->B, m->T, m->H, m->dh, m->err_word[k], st));
     {
-      GemmArgs g = gemm_args(N, d, d, A.attn_o, d, 0, m->Pb + o.wo, d, 0, EPI_F32_RESID, A.x_mid, d);
-      g.bias = m->P + o.bo;
+      GemmArgs g = gemm_args(N, d, d, A.attn_o, d, 0, m->Pb[k] + o.wo, d, 0, EPI_F32_RESID, A.x_mid, d);
+      g.bias = m->P[k] + o.bo;
       g.resid = x_in;
       IL_TRY(gemm(m, k, g));
     }
-    IL_K(m, layernorm_fwd(A.x_mid, m->P + o.ln2g, m->P + o.ln2b, A.ln2, A.mean2, A.rstd2, N, d, m->ln_eps, st));
+    IL_K(m, layernorm_fwd(A.x_mid, m->P[k] + o.ln2g, m->P[k] + o.ln2b, A.ln2, A.mean2, A.rstd2, N, d, m->ln_eps, st));
     {
-      GemmArgs g = gemm_args(N, F, d, A.ln2, d, 0, m->Pb + o.w1, d, 0, EPI_BF16_GELU, A.hgrad, F);
+      GemmArgs g = gemm_args(N, F, d, A.ln2, d, 0, m->Pb[k] + o.w1, d, 0, EPI_BF16_GELU, A.hgrad, F);
       g.C2 = A.hact;
-      g.bias = m->P + o.b1;
+      g.bias = m->P[k] + o.b1;
       IL_TRY(gemm(m, k, g));
     }
     {
-      GemmArgs g = gemm_args(N, d, F, A.hact, F, 0, m->Pb + o.w2, F, 0, EPI_F32_RESID, A.x_out, d);
-      g.bias = m->P + o.b2;
+      GemmArgs g = gemm_args(N, d, F, A.hact, F, 0, m->Pb[k] + o.w2, F, 0, EPI_F32_RESID, A.x_out, d);
+      g.bias = m->P[k] + o.b2;
       g.resid = A.x_mid;
       IL_TRY(gemm(m, k, g));
     }
@@ -719,30 +906,39 @@ il_status layers_forward(il_model* m, int k, size_t base, int count, const float
 }  // namespace
 
 extern "C" il_status il_forward_component(il_model* m, int k) {
+  return guarded([&]() -> il_status {
   IL_TRY(check_model(m));
   if (k < 0 || k >= m->K) return fail(m, IL_ERR_INVALID_ARG, "component %d out of range", k);
   if (!m->batch_set) return fail(m, IL_ERR_STATE, "il_forward_component before il_set_batch");
   if (k > 0 && !m->fwd_done[k - 1]) return fail(m, IL_ERR_STATE, "component %d forward needs component %d first", k, k - 1);
   if (m->fwd_done[k]) return fail(m, IL_ERR_STATE, "component %d already forwarded in this step", k);
-  IL_CUDA(m, cudaSetDevice(m->device));
+  IL_CUDA(m, cudaSetDevice(m->dev[k]));
   cudaStream_t st = m->streams[k];
   const int N = m->ntok, d = m->d;
   if (k == 0) {
-    IL_K(m, embed_fwd(m->tokens, m->P + m->off_wte, m->P + m->off_wpe, m->a[0], N, m->T, d, m->V, st));
+    IL_K(m, embed_fwd(m->tokens[k], m->P[k] + m->off_wte, m->P[k] + m->off_wpe, m->a[0], N, m->T, d, m->V, st));
   } else {
     IL_CUDA(m, cudaStreamWaitEvent(st, m->ev_fwd[k - 1], 0));
+    // pipeline placement (Sec. 3: the module's output is sent to the next accelerator): a_k is copied into a
+    // buffer this component's device owns; every kernel of the component then reads local memory only
+    if (m->placement == IL_PLACE_PIPELINE) {
+      IL_CUDA(m, cudaMemcpyPeerAsync(m->a_in[k], m->dev[k], m->a[k], m->dev[k - 1], (size_t)N * d * sizeof(float), st));
+      m->xfer_log.push_back(0); m->xfer_log.push_back(k - 1); m->xfer_log.push_back(-1);
+    }
   }
-  IL_TRY(layers_forward(m, k, (size_t)k * m->Lc, m->Lc, m->a[k]));
+  IL_TRY(layers_forward(m, k, (size_t)k * m->Lc, m->Lc, comp_input(m, k)));
   IL_CUDA(m, cudaEventRecord(m->ev_fwd[k], st));
   m->fwd_done[k] = 1;
   return IL_OK;
+  });
 }
 
 extern "C" il_status il_aux_head_loss(il_model* m, int k, float* loss_host) {
+  return guarded([&]() -> il_status {
   IL_TRY(check_model(m));
   if (k < 0 || k >= m->K) return fail(m, IL_ERR_INVALID_ARG, "head %d out of range", k);
   if (!m->batch_set || !m->fwd_done[k]) return fail(m, IL_ERR_STATE, "il_aux_head_loss(%d) needs il_forward_component(%d)", k, k);
-  IL_CUDA(m, cudaSetDevice(m->device));
+  IL_CUDA(m, cudaSetDevice(m->dev[k]));
   cudaStream_t st = m->streams[k];
   if (!m->loss_done[k]) {
     const int N = m->ntok, d = m->d, V = m->V;
@@ -751,48 +947,57 @@ extern "C" il_status il_aux_head_loss(il_model* m, int k, float* loss_host) {
     const size_t hbase = (size_t)m->K * m->Lc + (size_t)k * m->Lh;
     if (m->Lh > 0) IL_TRY(layers_forward(m, k, hbase, m->Lh, m->a[k + 1]));
     const float* hx = head_input(m, k);
-    IL_K(m, layernorm_fwd(hx, m->P + o.lng, m->P + o.lnb, h.u, h.mean, h.rstd, N, d, m->ln_eps, st));
-    GemmArgs g = gemm_args(N, V, d, h.u, d, 0, m->Pb + o.w, d, 0, EPI_LSE, h.z, m->ldz);
-    g.targets = m->targets;
+    IL_K(m, layernorm_fwd(hx, m->P[k] + o.lng, m->P[k] + o.lnb, h.u, h.mean, h.rstd, N, d, m->ln_eps, st));
+    // One GEMM over the whole vocabulary whose epilogue keeps per-(row, 128-column block) softmax partials and the
+    // target logit.  Stored mode: it also writes exp(logit) in bf16 for the backward.  Recompute mode: nothing of
+    // the [Ntok, V] matrix is written; the backward forms it again chunk by chunk.
+    const bool stored = m->head_mode == IL_HEAD_STORED;
+    GemmArgs g = gemm_args(N, V, d, h.u, d, 0, m->Pb[k] + o.w, d, 0, EPI_LSE, stored ? h.z : nullptr, stored ? m->ldz : 0);
+    g.targets = m->targets[k];
     g.part_max = h.pmax; g.part_sum = h.psum; g.part_ld = m->part_ld;
     g.tgt_logit = h.tgt_logit;
     g.col0 = 0;
-    g.store_exp = 1;
+    g.store_exp = stored ? 1 : 0;
     IL_TRY(gemm(m, k, g));
-    IL_K(m, lse_finalize(h.pmax, h.psum, m->part_ld, m->part_ld, h.tgt_logit, h.lse, m->losses + k, N, st));
+    // per-row log-sum-exp and negative log-likelihood, then the mean of the latter in a fixed summation order
+    IL_K(m, lse_finalize(h.pmax, h.psum, m->part_ld, m->part_ld, h.tgt_logit, h.lse, h.nll, N, st));
+    IL_K(m, mean_f32(h.nll, N, m->losses[k] + k, st));
     m->loss_done[k] = 1;
   }
   if (loss_host) {
-    IL_CUDA(m, cudaMemcpyAsync(loss_host, m->losses + k, sizeof(float), cudaMemcpyDeviceToHost, st));
+    IL_CUDA(m, cudaMemcpyAsync(loss_host, m->losses[k] + k, sizeof(float), cudaMemcpyDeviceToHost, st));
     IL_CUDA(m, cudaStreamSynchronize(st));
   }
   return IL_OK;
+  });
 }
 
 extern "C" il_status il_get_token_losses(il_model* m, int k, float* host, size_t count) {
+  return guarded([&]() -> il_status {
   IL_TRY(check_model(m));
   if (k < 0 || k >= m->K || !host) return fail(m, IL_ERR_INVALID_ARG, "head %d out of range or NULL output", k);
   if (!m->batch_set || !m->loss_done[k]) return fail(m, IL_ERR_STATE, "head %d has no loss in this step", k);
   if (count != (size_t)m->ntok) return fail(m, IL_ERR_INVALID_ARG, "expected %d values, got %zu", m->ntok, count);
-  IL_CUDA(m, cudaSetDevice(m->device));
-  IL_CUDA(m, cudaStreamSynchronize(m->streams[k]));
-  std::vector<float> tl(count);
-  IL_CUDA(m, cudaMemcpyAsync(host, m->hs[k].lse, count * 4, cudaMemcpyDeviceToHost, m->streams[k]));
-  IL_CUDA(m, cudaMemcpyAsync(tl.data(), m->hs[k].tgt_logit, count * 4, cudaMemcpyDeviceToHost, m->streams[k]));
-  IL_CUDA(m, cudaStreamSynchronize(m->streams[k]));
-  for (size_t i = 0; i < count; ++i) host[i] -= tl[i];
+  IL_TRY(copy_sync(m, k, host, m->hs[k].nll, count * 4, cudaMemcpyDeviceToHost));
   return IL_OK;
+  });
 }
 
 extern "C" il_status il_get_losses(il_model* m, float* losses_host) {
+  return guarded([&]() -> il_status {
   IL_TRY(check_model(m));
   if (!losses_host) return fail(m, IL_ERR_INVALID_ARG, "NULL output");
   for (int k = 0; k < m->K; ++k)
     if (!m->loss_done[k]) return fail(m, IL_ERR_STATE, "head %d has no loss in this step", k);
-  IL_CUDA(m, cudaSetDevice(m->device));
-  for (int k = 0; k < m->K; ++k) IL_CUDA(m, cudaStreamSynchronize(m->streams[k]));
-  IL_TRY(copy_sync(m, losses_host, m->losses, m->K * sizeof(float), cudaMemcpyDeviceToHost));
+  if (m->losses[m->K - 1] == m->losses[0]) {        // one shared array
+    IL_CUDA(m, cudaSetDevice(m->dev[0]));
+    for (int k = 1; k < m->K; ++k) IL_CUDA(m, cudaStreamSynchronize(m->streams[k]));
+    IL_TRY(copy_sync(m, 0, losses_host, m->losses[0], m->K * sizeof(float), cudaMemcpyDeviceToHost));
+  } else {
+    for (int k = 0; k < m->K; ++k) IL_TRY(copy_sync(m, k, losses_host + k, m->losses[k] + k, sizeof(float), cudaMemcpyDeviceToHost));
+  }
   return IL_OK;
+  });
 }
 
 namespace {
@@ -813,39 +1018,39 @@ il_status layers_backward(il_model* m, int k, int s, size_t base, int count, con
     // ---- MLP: x_out = x_mid + W2 gelu(W1 ln2 + b1) + b2
     // bias gradient of FC2: column sums of the incoming gradient (first stream).  Below the top block they come
     // out of the LayerNorm backward that produced this gradient.
-    if (l == count - 1 || !fused_ln) IL_K(m, colsum_f32(c.dx, d, m->G + o.b2, N, d, st));
-    IL_TRY(wgrad(m, k, d, F, N, c.dxb, d, A.hact, F, m->G + o.w2, acc));
+    if (l == count - 1 || !fused_ln) IL_K(m, colsum_f32(c.dx, d, m->G[k] + o.b2, N, d, st));
+    IL_TRY(wgrad(m, k, d, F, N, c.dxb, d, A.hact, F, m->G[k] + o.w2, acc));
     {
-      GemmArgs g = gemm_args(R, F, d, c.dxb, d, 0, m->Pb + o.w2, F, 1, EPI_BF16_DGELU, c.dbig, F);
+      GemmArgs g = gemm_args(R, F, d, c.dxb, d, 0, m->Pb[k] + o.w2, F, 1, EPI_BF16_DGELU, c.dbig, F);
       g.aux = A.hgrad; g.ld_aux = F; g.aux_rows = N;
-      g.colsum = m->G + o.b1;                 // FC1 bias gradient: column sums of the first gradient stream
+      g.colsum = m->G[k] + o.b1;                 // FC1 bias gradient: column sums of the first gradient stream
       IL_TRY(gemm(m, k, g));
     }
-    IL_TRY(wgrad(m, k, F, d, N, c.dbig, F, A.ln2, d, m->G + o.w1, acc));
-    IL_TRY(gemm(m, k, gemm_args(R, d, F, c.dbig, F, 0, m->Pb + o.w1, d, 1, EPI_BF16, c.dln, d)));
+    IL_TRY(wgrad(m, k, F, d, N, c.dbig, F, A.ln2, d, m->G[k] + o.w1, acc));
+    IL_TRY(gemm(m, k, gemm_args(R, d, F, c.dbig, F, 0, m->Pb[k] + o.w1, d, 1, EPI_BF16, c.dln, d)));
     if (fused_ln) {   // LayerNorm backward with its parameter gradients and the bias gradient of Wo in one pass
-      IL_K(m, layernorm_bwd_fused(c.dln, A.x_mid, A.mean2, A.rstd2, m->P + o.ln2g, c.dx, c.dx, c.dxb, m->G + o.ln2g,
-                                  m->G + o.ln2b, m->G + o.bo, R, N, d, st));
+      IL_K(m, layernorm_bwd_fused(c.dln, A.x_mid, A.mean2, A.rstd2, m->P[k] + o.ln2g, c.dx, c.dx, c.dxb, m->G[k] + o.ln2g,
+                                  m->G[k] + o.ln2b, m->G[k] + o.bo, R, N, d, st));
     } else {
-      IL_K(m, layernorm_bwd_params(c.dln, 0, A.x_mid, A.mean2, A.rstd2, m->G + o.ln2g, m->G + o.ln2b, N, d, st));
-      IL_K(m, layernorm_bwd_rows(c.dln, 0, A.x_mid, A.mean2, A.rstd2, m->P + o.ln2g, c.dx, c.dx, c.dxb, R, N, d, st));
+      IL_K(m, layernorm_bwd_params(c.dln, 0, A.x_mid, A.mean2, A.rstd2, m->G[k] + o.ln2g, m->G[k] + o.ln2b, N, d, st));
+      IL_K(m, layernorm_bwd_rows(c.dln, 0, A.x_mid, A.mean2, A.rstd2, m->P[k] + o.ln2g, c.dx, c.dx, c.dxb, R, N, d, st));
       // ---- attention: x_mid = x_in + Wo attn(Wqkv ln1 + bqkv) + bo
-      IL_K(m, colsum_f32(c.dx, d, m->G + o.bo, N, d, st));
+      IL_K(m, colsum_f32(c.dx, d, m->G[k] + o.bo, N, d, st));
     }
-    IL_TRY(wgrad(m, k, d, d, N, c.dxb, d, A.attn_o, d, m->G + o.wo, acc));
-    IL_TRY(gemm(m, k, gemm_args(R, d, d, c.dxb, d, 0, m->Pb + o.wo, d, 1, EPI_BF16, c.dattn, d)));
-    IL_K(m, attention_bwd(A.qkv, A.attn_o, A.lse, c.dattn, c.dqkv, c.delta, s * m->B, m->B, m->T, m->H, m->dh, m->err_word, st));
+    IL_TRY(wgrad(m, k, d, d, N, c.dxb, d, A.attn_o, d, m->G[k] + o.wo, acc));
+    IL_TRY(gemm(m, k, gemm_args(R, d, d, c.dxb, d, 0, m->Pb[k] + o.wo, d, 1, EPI_BF16, c.dattn, d)));
+    IL_K(m, attention_bwd(A.qkv, A.attn_o, A.lse, c.dattn, c.dqkv, c.delta, s * m->B, m->B, m->T, m->H, m->dh, m->err_word[k], st));
     m->launches += 2;
-    IL_K(m, colsum_bf16(c.dqkv, 3 * d, m->G + o.bqkv, N, 3 * d, st));
-    IL_TRY(wgrad(m, k, 3 * d, d, N, c.dqkv, 3 * d, A.ln1, d, m->G + o.wqkv, acc));
-    IL_TRY(gemm(m, k, gemm_args(R, d, 3 * d, c.dqkv, 3 * d, 0, m->Pb + o.wqkv, d, 1, EPI_BF16, c.dln, d)));
+    IL_K(m, colsum_bf16(c.dqkv, 3 * d, m->G[k] + o.bqkv, N, 3 * d, st));
+    IL_TRY(wgrad(m, k, 3 * d, d, N, c.dqkv, 3 * d, A.ln1, d, m->G[k] + o.wqkv, acc));
+    IL_TRY(gemm(m, k, gemm_args(R, d, 3 * d, c.dqkv, 3 * d, 0, m->Pb[k] + o.wqkv, d, 1, EPI_BF16, c.dln, d)));
     if (fused_ln) {   // ... and the FC2 bias gradient of the block below
-      float* b2_below = l > 0 ? m->G + m->layer_off[base + l - 1].b2 : nullptr;
-      IL_K(m, layernorm_bwd_fused(c.dln, x_in, A.mean1, A.rstd1, m->P + o.ln1g, c.dx, c.dx, c.dxb, m->G + o.ln1g,
-                                  m->G + o.ln1b, b2_below, R, N, d, st));
+      float* b2_below = l > 0 ? m->G[k] + m->layer_off[base + l - 1].b2 : nullptr;
+      IL_K(m, layernorm_bwd_fused(c.dln, x_in, A.mean1, A.rstd1, m->P[k] + o.ln1g, c.dx, c.dx, c.dxb, m->G[k] + o.ln1g,
+                                  m->G[k] + o.ln1b, b2_below, R, N, d, st));
     } else {
-      IL_K(m, layernorm_bwd_params(c.dln, 0, x_in, A.mean1, A.rstd1, m->G + o.ln1g, m->G + o.ln1b, N, d, st));
-      IL_K(m, layernorm_bwd_rows(c.dln, 0, x_in, A.mean1, A.rstd1, m->P + o.ln1g, c.dx, c.dx, c.dxb, R, N, d, st));
+      IL_K(m, layernorm_bwd_params(c.dln, 0, x_in, A.mean1, A.rstd1, m->G[k] + o.ln1g, m->G[k] + o.ln1b, N, d, st));
+      IL_K(m, layernorm_bwd_rows(c.dln, 0, x_in, A.mean1, A.rstd1, m->P[k] + o.ln1g, c.dx, c.dx, c.dxb, R, N, d, st));
     }
   }
   return IL_OK;
@@ -863,38 +1068,68 @@ il_status head_backward(il_model* m, int k, bool acc, float scale) {
   const int N = m->ntok, d = m->d, V = m->V;
   const HeadOff& o = m->head_off[k];
   HeadScratch& h = m->hs[k];
-  IL_K(m, head_backward_prepare(h.z, m->ldz, h.lse, m->targets, h.u, h.us, h.rs, N, d, scale, m->err_word, st));
-  {  // dU = diag(s) (E' W).  Not split over the contraction: atomically added partial sums would make dU, and
-     // with it every gradient below this head, depend on the order the work units finish in.
-    GemmArgs g = gemm_args(N, d, V, h.z, m->ldz, 0, m->Pb + o.w, d, 1, EPI_F32, h.du, d);
-    g.rowscale = h.rs;
-    IL_TRY(gemm(m, k, g));
-  }
-  {  // dW = E'^T (diag(s) U)
-    GemmArgs g = gemm_args(V, d, N, h.z, m->ldz, 1, h.us, d, 1, EPI_F32, m->G + o.w, d);
-    g.accumulate = acc ? 1 : 0;
-    IL_TRY(gemm(m, k, g));
+  if (m->head_mode == IL_HEAD_STORED) {
+    IL_K(m, head_backward_prepare(h.z, m->ldz, h.lse, m->targets[k], h.u, h.us, h.rs, N, d, scale, m->err_word[k], st));
+    {  // dU = diag(s) (E' W).  Not split over the contraction: atomically added partial sums would make dU, and
+       // with it every gradient below this head, depend on the order the work units finish in.
+      GemmArgs g = gemm_args(N, d, V, h.z, m->ldz, 0, m->Pb[k] + o.w, d, 1, EPI_F32, h.du, d);
+      g.rowscale = h.rs;
+      IL_TRY(gemm(m, k, g));
+    }
+    {  // dW = E'^T (diag(s) U)
+      GemmArgs g = gemm_args(V, d, N, h.z, m->ldz, 1, h.us, d, 1, EPI_F32, m->G[k] + o.w, d);
+      g.accumulate = acc ? 1 : 0;
+      IL_TRY(gemm(m, k, g));
+    }
+  } else {
+    // Recompute mode: nothing of the [Ntok, V] matrix was kept.  The vocabulary is walked in chunks of HEAD_CHUNK
+    // columns; per chunk the logits are formed again and turned into dZ = (softmax - onehot) * scale / Ntok in the
+    // GEMM's epilogue (bf16, [Ntok, chunk]), then dU += dZ W_chunk and dW_chunk = dZ^T U.  The chunks follow each
+    // other on this head's stream, so dU is summed in a fixed order.
+    const int chunk = m->ldz;
+    for (int c0 = 0; c0 < V; c0 += chunk) {
+      const int w = std::min(chunk, V - c0);
+      {
+        GemmArgs g = gemm_args(N, w, d, h.u, d, 0, m->Pb[k] + o.w + (size_t)c0 * d, d, 0, EPI_DZ, h.z, chunk);
+        g.targets = m->targets[k];
+        g.lse = h.lse;
+        g.scale = scale / (float)N;
+        g.col0 = c0;
+        IL_TRY(gemm(m, k, g));
+      }
+      {
+        GemmArgs g = gemm_args(N, d, w, h.z, chunk, 0, m->Pb[k] + o.w + (size_t)c0 * d, d, 1, EPI_F32, h.du, d);
+        g.accumulate = c0 > 0 ? 1 : 0;
+        IL_TRY(gemm(m, k, g));
+      }
+      {
+        GemmArgs g = gemm_args(w, d, N, h.z, chunk, 1, h.u, d, 1, EPI_F32, m->G[k] + o.w + (size_t)c0 * d, d);
+        g.accumulate = acc ? 1 : 0;
+        IL_TRY(gemm(m, k, g));
+      }
+    }
   }
   const float* hx = head_input(m, k);
-  IL_K(m, layernorm_bwd_params(h.du, 1, hx, h.mean, h.rstd, m->G + o.lng, m->G + o.lnb, N, d, st));
+  IL_K(m, layernorm_bwd_params(h.du, 1, hx, h.mean, h.rstd, m->G[k] + o.lng, m->G[k] + o.lnb, N, d, st));
   if (m->Lh == 0) {
-    IL_K(m, layernorm_bwd_rows(h.du, 1, hx, h.mean, h.rstd, m->P + o.lng, nullptr, h.ghead, nullptr, N, N, d, st));
+    IL_K(m, layernorm_bwd_rows(h.du, 1, hx, h.mean, h.rstd, m->P[k] + o.lng, nullptr, h.ghead, nullptr, N, N, d, st));
     return IL_OK;
   }
   CompScratch& c = m->cs[k];
-  IL_K(m, layernorm_bwd_rows(h.du, 1, hx, h.mean, h.rstd, m->P + o.lng, nullptr, c.dx, c.dxb, N, N, d, st));
+  IL_K(m, layernorm_bwd_rows(h.du, 1, hx, h.mean, h.rstd, m->P[k] + o.lng, nullptr, c.dx, c.dxb, N, N, d, st));
   IL_TRY(layers_backward(m, k, 1, (size_t)m->K * m->Lc + (size_t)k * m->Lh, m->Lh, m->a[k + 1], acc));
   IL_CUDA(m, cudaMemcpyAsync(h.ghead, c.dx, (size_t)N * d * sizeof(float), cudaMemcpyDeviceToDevice, st));
   return IL_OK;
 }
 
 il_status component_backward(il_model* m, int k, int s, bool acc) {
-  return layers_backward(m, k, s, (size_t)k * m->Lc, m->Lc, m->a[k], acc);
+  return layers_backward(m, k, s, (size_t)k * m->Lc, m->Lc, comp_input(m, k), acc);
 }
 
 }  // namespace
 
 extern "C" il_status il_backward_nwise(il_model* m) {
+  return guarded([&]() -> il_status {
   IL_TRY(check_model(m));
   if (!m->batch_set) return fail(m, IL_ERR_STATE, "il_backward_nwise before il_set_batch");
   for (int k = 0; k < m->K; ++k)
@@ -903,9 +1138,25 @@ extern "C" il_status il_backward_nwise(il_model* m) {
   if (m->bwd_done) return fail(m, IL_ERR_STATE, "il_backward_nwise already called in this step");
   if (m->micro > 1 && m->micro_done >= m->micro)
     return fail(m, IL_ERR_STATE, "all %d micro-batches of this update have been back-propagated; call il_adamw_step", m->micro);
-  IL_CUDA(m, cudaSetDevice(m->device));
   const int K = m->K, n = m->n, N = m->ntok, d = m->d;
   const size_t slice = (size_t)N * d;
+  // Gradient stream `slot` of component k+1 as component k reads it: in place on a single device; in the pipeline
+  // placement (Sec. 3: gradients are sent back to the previous accelerator) copied, once, on stream k into the
+  // receive buffer that k's device owns.  Stream k has already waited for component k+1's backward.
+  std::vector<char> fetched;
+  cudaError_t fetch_err = cudaSuccess;
+  auto from_above = [&](int k, int slot, int id) -> const float* {
+    const float* src = m->cs[k + 1].dx + (size_t)slot * slice;
+    if (m->placement != IL_PLACE_PIPELINE) return src;
+    float* dst = m->g_in[k] + (size_t)slot * slice;
+    if (!fetched[slot]) {
+      cudaError_t e = cudaMemcpyPeerAsync(dst, m->dev[k], src, m->dev[k + 1], slice * sizeof(float), m->streams[k]);
+      if (e != cudaSuccess) fetch_err = e;
+      fetched[slot] = 1;
+      m->xfer_log.push_back(1); m->xfer_log.push_back(k); m->xfer_log.push_back(id);
+    }
+    return dst;
+  };
   // Micro-batching (Sec. 3.1): the first backward pass of an update overwrites the gradients, the later ones add
   // to them; each pass is scaled by 1 / micro-batches so that the buffers end up holding the mini-batch mean.
   const bool acc = m->micro > 1 && m->micro_done > 0;
@@ -914,12 +1165,13 @@ extern "C" il_status il_backward_nwise(il_model* m) {
   // every head's own backward is independent of the others: enqueue all of them first
   for (int k = 0; k < K; ++k) {
     cudaStream_t st = m->streams[k];
-    if (!acc) {   // vectors and embeddings are summed into atomically
-      IL_CUDA(m, cudaMemsetAsync(m->G + m->comp_mat_end[k], 0, (m->comp_end[k] - m->comp_mat_end[k]) * 4, st));
+    IL_CUDA(m, cudaSetDevice(m->dev[k]));
+    if (!acc) {   // vectors are summed into atomically; embedding rows no token selects must read zero
+      IL_CUDA(m, cudaMemsetAsync(m->G[k] + m->comp_mat_end[k], 0, (m->comp_end[k] - m->comp_mat_end[k]) * 4, st));
       if (k == 0) {
         const size_t emb = (size_t)m->V * d;
-        IL_CUDA(m, cudaMemsetAsync(m->G + m->off_wte, 0, emb * 4, st));
-        IL_CUDA(m, cudaMemsetAsync(m->G + m->off_wpe, 0, (size_t)m->max_seq * d * 4, st));
+        IL_CUDA(m, cudaMemsetAsync(m->G[k] + m->off_wte, 0, emb * 4, st));
+        IL_CUDA(m, cudaMemsetAsync(m->G[k] + m->off_wpe, 0, (size_t)m->max_seq * d * 4, st));
       }
     }
     IL_TRY(head_backward(m, k, acc, gscale));
@@ -929,6 +1181,8 @@ extern "C" il_status il_backward_nwise(il_model* m) {
     std::vector<int> above;   // termination levels of the streams of component k+1
     for (int k = K - 1; k >= 0; --k) {
       cudaStream_t st = m->streams[k];
+      IL_CUDA(m, cudaSetDevice(m->dev[k]));
+      fetched.assign((size_t)m->s_cap + 1, 0);
       const std::vector<int> terms = terms_of(k, K, n);
       const int s = (int)terms.size();
       bool needs_above = false;
@@ -940,12 +1194,13 @@ extern "C" il_status il_backward_nwise(il_model* m) {
           IL_CUDA(m, cudaStreamWaitEvent(st, m->ev_bwd[k + 1], 0));
           needs_above = true;
         }
-        const float* passed = src >= 0 ? m->cs[k + 1].dx + (size_t)src * slice : nullptr;
+        const float* passed = src >= 0 ? from_above(k, src, terms[j]) : nullptr;
+        if (fetch_err != cudaSuccess) return fail(m, IL_ERR_CUDA, "cudaMemcpyPeerAsync: %s", cudaGetErrorString(fetch_err));
         IL_K(m, add_convert(m->hs[k].ghead, passed, m->cs[k].dx + (size_t)j * slice, m->cs[k].dxb + (size_t)j * slice, slice, st));
       }
       IL_TRY(component_backward(m, k, s, acc));
       if (k == 0) {
-        IL_K(m, embed_bwd(m->tokens, m->cs[0].dx, m->G + m->off_wte, m->G + m->off_wpe, N, m->T, d, m->V, acc ? 1 : 0, st));
+        IL_K(m, embed_bwd(m->tokens[k], m->sort_keys[0], m->cs[0].dx, m->G[k] + m->off_wte, m->G[k] + m->off_wpe, N, m->T, d, m->V, acc ? 1 : 0, st));
         m->launches++;
       }
       IL_CUDA(m, cudaEventRecord(m->ev_bwd[k], st));
@@ -960,11 +1215,13 @@ extern "C" il_status il_backward_nwise(il_model* m) {
     std::vector<int> above_slots;     // ... and the slot each of them occupies there
     for (int k = K - 1; k >= 0; --k) {
       cudaStream_t st = m->streams[k];
+      IL_CUDA(m, cudaSetDevice(m->dev[k]));
+      fetched.assign((size_t)m->s_cap + 1, 0);
       const int hi = k + n - 1 < K - 1 ? k + n - 1 : K - 1;
       auto grad_of = [&](int h) -> const float* {      // gradient of head h at the output of component k
         if (h == k) return m->hs[k].ghead;
         for (size_t q = 0; q < above_heads.size(); ++q)
-          if (above_heads[q] == h) return m->cs[k + 1].dx + (size_t)above_slots[q] * slice;
+          if (above_heads[q] == h) return from_above(k, above_slots[q], h);
         return nullptr;
       };
       if (hi > k) IL_CUDA(m, cudaStreamWaitEvent(st, m->ev_bwd[k + 1], 0));
@@ -1000,9 +1257,10 @@ extern "C" il_status il_backward_nwise(il_model* m) {
             IL_K(m, add_convert(src, nullptr, m->cs[k].dx + (size_t)used * slice, m->cs[k].dxb + (size_t)used * slice, slice, st));
             mine_slots.push_back(used++);
           }
+      if (fetch_err != cudaSuccess) return fail(m, IL_ERR_CUDA, "cudaMemcpyPeerAsync: %s", cudaGetErrorString(fetch_err));
       IL_TRY(component_backward(m, k, used, acc));
       if (k == 0) {
-        IL_K(m, embed_bwd(m->tokens, m->cs[0].dx, m->G + m->off_wte, m->G + m->off_wpe, N, m->T, d, m->V, acc ? 1 : 0, st));
+        IL_K(m, embed_bwd(m->tokens[k], m->sort_keys[0], m->cs[0].dx, m->G[k] + m->off_wte, m->G[k] + m->off_wpe, N, m->T, d, m->V, acc ? 1 : 0, st));
         m->launches++;
       }
       IL_CUDA(m, cudaEventRecord(m->ev_bwd[k], st));
@@ -1013,32 +1271,38 @@ extern "C" il_status il_backward_nwise(il_model* m) {
   m->bwd_done = true;
   m->micro_done = m->micro > 1 ? m->micro_done + 1 : 1;
   return IL_OK;
+  });
 }
 
 extern "C" il_status il_set_micro_batches(il_model* m, int micro_batches) {
+  return guarded([&]() -> il_status {
   IL_TRY(check_model(m));
   if (micro_batches < 1) return fail(m, IL_ERR_INVALID_ARG, "micro_batches must be >= 1");
   m->micro = micro_batches;
   m->micro_done = 0;      // gradients accumulated so far are abandoned: the next backward pass overwrites them
   return IL_OK;
+  });
 }
 
 extern "C" il_status il_lr_schedule(long long step, int d_model, int warmup_steps, double* lr) {
+  return guarded([&]() -> il_status {
   if (step < 1 || d_model < 1 || warmup_steps < 1 || !lr) return IL_ERR_INVALID_ARG;
   const double s = (double)step, w = (double)warmup_steps;
   const double a = 1.0 / sqrt(s), b = s / (w * sqrt(w));
   *lr = (a < b ? a : b) / sqrt((double)d_model);
   return IL_OK;
+  });
 }
 
 extern "C" il_status il_adamw_step(il_model* m, float lr, float beta1, float beta2, float eps, float wd) {
+  return guarded([&]() -> il_status {
   IL_TRY(check_model(m));
   if (!m->bwd_done || !m->batch_set) return fail(m, IL_ERR_STATE, "il_adamw_step needs il_backward_nwise of the current step");
   if (m->micro_done != m->micro)
     return fail(m, IL_ERR_STATE, "il_adamw_step after %d of %d micro-batches", m->micro_done, m->micro);
   if (!(beta1 >= 0 && beta1 < 1 && beta2 >= 0 && beta2 < 1 && eps >= 0)) return fail(m, IL_ERR_INVALID_ARG, "bad AdamW hyper-parameters");
-  IL_CUDA(m, cudaSetDevice(m->device));
   m->step += 1;
+  m->adamw_issued += 1;
   const double bc1 = 1.0 - pow((double)beta1, (double)m->step);
   const double bc2 = 1.0 - pow((double)beta2, (double)m->step);
   // Parameters, gradients and bf16 shadows of component k (its head and, for k = 0, the embeddings included)
@@ -1046,62 +1310,94 @@ extern "C" il_status il_adamw_step(il_model* m, float lr, float beta1, float bet
   // gradients are final (the last backward pass through a module triggers its update, App. C).
   for (int k = 0; k < m->K; ++k) {
     const size_t b = m->comp_begin[k], e = m->comp_end[k], me = m->comp_mat_end[k];
-    IL_K(m, adamw(m->P + b, m->M1 + b, m->M2 + b, m->G + b, m->Pb + b, e - b, me - b, lr, beta1, beta2, eps, wd, (float)bc1,
-                  (float)bc2, m->streams[k]));
+    IL_CUDA(m, cudaSetDevice(m->dev[k]));
+    // the kernel leaves everything untouched while the error word is set (the gradients of a failed step are not
+    // applied) and otherwise counts the update in word 1 + k
+    IL_K(m, adamw(m->P[k] + b, m->M1[k] + b, m->M2[k] + b, m->G[k] + b, m->Pb[k] + b, e - b, me - b, lr, beta1, beta2, eps, wd,
+                  (float)bc1, (float)bc2, m->err_word[k], m->err_word[k] + 1 + k, m->streams[k]));
   }
   m->batch_set = false;   // a new batch is required for the next step
   m->micro_done = 0;
   return IL_OK;
+  });
 }
 
 extern "C" il_status il_sync(il_model* m) {
+  return guarded([&]() -> il_status {
   IL_TRY(check_model(m));
-  IL_CUDA(m, cudaSetDevice(m->device));
-  for (int k = 0; k < m->K; ++k) IL_CUDA(m, cudaStreamSynchronize(m->streams[k]));
-  unsigned w = 0;
-  IL_TRY(copy_sync(m, &w, m->err_word, 4, cudaMemcpyDeviceToHost));
-  if (w) {
-    IL_CUDA(m, cudaMemsetAsync(m->err_word, 0, 4, m->streams[0]));
-    IL_CUDA(m, cudaStreamSynchronize(m->streams[0]));
-    if (w == DEV_LOGIT_RANGE)
-      return fail(m, IL_ERR_NONFINITE, "a head's log-sum-exp left [-80, 80]: exp(logit) is not representable");
-    return fail(m, IL_ERR_TIMEOUT, "a bounded device-side wait expired (code %u)", w);
+  for (int k = 0; k < m->K; ++k) {
+    IL_CUDA(m, cudaSetDevice(m->dev[k]));
+    IL_CUDA(m, cudaStreamSynchronize(m->streams[k]));
+  }
+  // error word and per-component update counters of every distinct buffer
+  unsigned first = 0;
+  int applied_min = m->adamw_issued, applied_max = 0;
+  unsigned words[1 + 64];                 // K <= 64 (il_create)
+  const bool shared = m->err_word[m->K - 1] == m->err_word[0];
+  for (int k = 0; k < m->K; ++k) {
+    if (shared && k > 0) break;
+    IL_TRY(copy_sync(m, k, words, m->err_word[k], 4 * (size_t)(1 + m->K), cudaMemcpyDeviceToHost));
+    if (words[0] && !first) first = words[0];
+    for (int j = shared ? 0 : k; j <= (shared ? m->K - 1 : k); ++j) {
+      applied_min = std::min(applied_min, (int)words[1 + j]);
+      applied_max = std::max(applied_max, (int)words[1 + j]);
+    }
+    IL_CUDA(m, cudaMemsetAsync(m->err_word[k], 0, 4 * (size_t)(1 + m->K), m->streams[k]));
+    IL_CUDA(m, cudaStreamSynchronize(m->streams[k]));
+  }
+  const int issued = m->adamw_issued;
+  m->adamw_issued = 0;
+  if (first) {
+    // Updates enqueued after the failure were skipped on the device: the step counter goes back to the number of
+    // updates that were applied.  A component whose update ran before another component raised the error keeps it.
+    m->step -= (issued - applied_max);
+    const char* partial = applied_min != applied_max ? "; some components applied an update that others skipped" : "";
+    if (first == DEV_LOGIT_RANGE)
+      return fail(m, IL_ERR_NONFINITE, "a head's log-sum-exp left [-80, 80]: exp(logit) is not representable; "
+                  "%d of %d optimiser updates since the last il_sync were applied%s", applied_max, issued, partial);
+    return fail(m, IL_ERR_TIMEOUT, "a bounded device-side wait expired (code %u); %d of %d optimiser updates since the "
+                "last il_sync were applied%s", first, applied_max, issued, partial);
   }
   return IL_OK;
+  });
 }
 
 extern "C" il_status il_get_boundary(il_model* m, int k, float* host, size_t count) {
+  return guarded([&]() -> il_status {
   IL_TRY(check_model(m));
   if (k < 0 || k > m->K || !host) return fail(m, IL_ERR_INVALID_ARG, "boundary %d out of range", k);
   if (!m->batch_set || (k > 0 && !m->fwd_done[k - 1]) || (k == 0 && !m->fwd_done[0])) return fail(m, IL_ERR_STATE, "boundary %d not computed in this step", k);
   if (count != (size_t)m->ntok * m->d) return fail(m, IL_ERR_INVALID_ARG, "boundary has %zu elements, got %zu", (size_t)m->ntok * m->d, count);
-  IL_CUDA(m, cudaSetDevice(m->device));
-  IL_CUDA(m, cudaDeviceSynchronize());
-  IL_TRY(copy_sync(m, host, m->a[k], count * 4, cudaMemcpyDeviceToHost));
+  IL_TRY(sync_devices(m));
+  IL_TRY(copy_sync(m, k > 0 ? k - 1 : 0, host, m->a[k], count * 4, cudaMemcpyDeviceToHost));
   return IL_OK;
+  });
 }
 
 extern "C" il_status il_stats(const il_model* m, long long* device_bytes, long long* kernel_launches) {
+  return guarded([&]() -> il_status {
   if (!m) return IL_ERR_INVALID_ARG;
   if (device_bytes) *device_bytes = m->bytes;
   if (kernel_launches) *kernel_launches = m->launches;
   return IL_OK;
+  });
 }
 
 extern "C" il_status il_profile(il_model* m, int enable) {
+  return guarded([&]() -> il_status {
   IL_TRY(check_model(m));
-  IL_CUDA(m, cudaSetDevice(m->device));
-  IL_CUDA(m, cudaDeviceSynchronize());
+  IL_TRY(sync_devices(m));
   for (auto& r : m->prof_recs) { m->prof_pool.push_back(r.a); m->prof_pool.push_back(r.b); }
   m->prof_recs.clear();
   m->prof = enable == 2 ? 2 : (enable != 0 ? 1 : 0);
   return IL_OK;
+  });
 }
 
 extern "C" il_status il_profile_read(il_model* m, double* gemm_ms, long long* gemm_launches, double* gemm_flops) {
+  return guarded([&]() -> il_status {
   IL_TRY(check_model(m));
-  IL_CUDA(m, cudaSetDevice(m->device));
-  IL_CUDA(m, cudaDeviceSynchronize());
+  IL_TRY(sync_devices(m));
   double ms = 0, fl = 0;
   for (auto& r : m->prof_recs) {
     float t = 0;
@@ -1115,15 +1411,74 @@ extern "C" il_status il_profile_read(il_model* m, double* gemm_ms, long long* ge
   for (auto& r : m->prof_recs) { m->prof_pool.push_back(r.a); m->prof_pool.push_back(r.b); }
   m->prof_recs.clear();
   return IL_OK;
+  });
 }
 
 extern "C" il_status il_nwise_streams(int K, int n, int k, int* terms, int* count) {
+  return guarded([&]() -> il_status {
   if (K < 1 || n < 1 || n > K || k < 0 || k >= K || !count) return IL_ERR_INVALID_ARG;
   const std::vector<int> t = terms_of(k, K, n);
   *count = (int)t.size();
   if (terms)
     for (size_t i = 0; i < t.size(); ++i) terms[i] = t[i];
   return IL_OK;
+  });
+}
+
+// The tensors that cross component boundaries in one step, in the order the step issues them.
+static void plan_transfers(int K, int n, int rule, std::vector<int>& out) {
+  for (int b = 0; b + 1 < K; ++b) { out.push_back(0); out.push_back(b); out.push_back(-1); }
+  for (int k = K - 2; k >= 0; --k) {
+    if (rule == IL_RULE_SUM) {
+      // stream j of component k continues the stream of component k+1 with the same termination level
+      const std::vector<int> mine = terms_of(k, K, n), above = terms_of(k + 1, K, n);
+      for (int t : mine)
+        if (std::find(above.begin(), above.end(), t) != above.end()) { out.push_back(1); out.push_back(k); out.push_back(t); }
+    } else {
+      // one tensor per head above k that component k uses: the farthest head of its window (the one that updates
+      // its parameters) and, unless k is the lowest component, the heads it relays further down
+      const int hi = k + n - 1 < K - 1 ? k + n - 1 : K - 1;
+      if (hi > k) { out.push_back(1); out.push_back(k); out.push_back(hi); }
+      if (k > 0)
+        for (int h = k + 1; h <= hi; ++h)
+          if (h != hi && h < k + n - 1) { out.push_back(1); out.push_back(k); out.push_back(h); }
+    }
+  }
+}
+
+extern "C" il_status il_pipeline_transfers(int K, int n, int rule, int* records, int capacity, int* count) {
+  return guarded([&]() -> il_status {
+  if (K < 1 || n < 1 || n > K || !count || capacity < 0) return IL_ERR_INVALID_ARG;
+  if (rule != IL_RULE_SUM && rule != IL_RULE_FAR && rule != IL_RULE_MEAN) return IL_ERR_INVALID_ARG;
+  std::vector<int> plan;
+  plan_transfers(K, n, rule, plan);
+  *count = (int)plan.size() / 3;
+  if (records)
+    for (int i = 0; i < *count && i < capacity; ++i)
+      for (int j = 0; j < 3; ++j) records[3 * i + j] = plan[3 * i + j];
+  return IL_OK;
+  });
+}
+
+extern "C" il_status il_pipeline_last_transfers(il_model* m, int* records, int capacity, int* count) {
+  return guarded([&]() -> il_status {
+  IL_TRY(check_model(m));
+  if (!count || capacity < 0) return fail(m, IL_ERR_INVALID_ARG, "NULL count");
+  *count = (int)m->xfer_log.size() / 3;
+  if (records)
+    for (int i = 0; i < *count && i < capacity; ++i)
+      for (int j = 0; j < 3; ++j) records[3 * i + j] = m->xfer_log[3 * i + j];
+  return IL_OK;
+  });
+}
+
+extern "C" il_status il_error_word(il_model* m, int k, void** device_ptr) {
+  return guarded([&]() -> il_status {
+  IL_TRY(check_model(m));
+  if (k < 0 || k >= m->K || !device_ptr) return fail(m, IL_ERR_INVALID_ARG, "component %d out of range or NULL output", k);
+  *device_ptr = m->err_word[k];
+  return IL_OK;
+  });
 }
 
 extern "C" const char* il_last_error(const il_model* m) { return m ? m->err.c_str() : "null model"; }
@@ -1150,6 +1505,7 @@ static il_status op_status(cudaError_t e) {
 }
 
 extern "C" il_status il_op_gemm(const il_gemm_desc* q, unsigned* err_word, void* stream) {
+  return guarded([&]() -> il_status {
   if (!q || !err_word) return IL_ERR_INVALID_ARG;
   GemmArgs g = gemm_args(q->M, q->N, q->K, q->A, q->lda, q->a_mn_major, q->B, q->ldb, q->b_mn_major, q->epilogue, q->C, q->ldc);
   g.C2 = q->C2; g.bias = q->bias; g.resid = q->resid; g.aux = q->aux; g.ld_aux = q->ld_aux; g.aux_rows = q->aux_rows; g.colsum = q->colsum;
@@ -1160,29 +1516,44 @@ extern "C" il_status il_op_gemm(const il_gemm_desc* q, unsigned* err_word, void*
   if (cudaGetDevice(&dev) != cudaSuccess) return IL_ERR_CUDA;
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return IL_ERR_CUDA;
   return op_status(gemm_launch(g, err_word, sms, reinterpret_cast<cudaStream_t>(stream)));
+  });
 }
 
 extern "C" il_status il_op_attention_fwd(const void* qkv, void* o, float* lse, int B, int T, int H, int dh, void* stream) {
+  return guarded([&]() -> il_status {
   if (!qkv || !o || !lse || B < 1 || T < 1 || H < 1) return IL_ERR_INVALID_ARG;
   return op_status(attention_fwd((const bf16*)qkv, (bf16*)o, lse, B, T, H, dh, nullptr, reinterpret_cast<cudaStream_t>(stream)));
+  });
 }
 
 extern "C" il_status il_op_attention_bwd(const void* qkv, const void* o, const float* lse, const void* dout, void* dqkv,
                                          float* delta, int NB, int B, int T, int H, int dh, void* stream) {
+  return guarded([&]() -> il_status {
   if (!qkv || !o || !lse || !dout || !dqkv || !delta || B < 1 || NB < 1 || T < 1 || H < 1) return IL_ERR_INVALID_ARG;
   return op_status(attention_bwd((const bf16*)qkv, (const bf16*)o, lse, (const bf16*)dout, (bf16*)dqkv, delta, NB, B, T, H, dh,
                                  nullptr, reinterpret_cast<cudaStream_t>(stream)));
+  });
+}
+
+extern "C" il_status il_op_wait_probe(unsigned* err_word, unsigned limit_us, void* stream) {
+  return guarded([&]() -> il_status {
+  if (!err_word || limit_us < 1 || limit_us > 1000000u) return IL_ERR_INVALID_ARG;
+  return op_status(wait_probe(err_word, 1000ull * limit_us, reinterpret_cast<cudaStream_t>(stream)));
+  });
 }
 
 extern "C" il_status il_op_layernorm_fwd(const float* x, const float* gamma, const float* beta, void* y, float* mean,
                                          float* rstd, int rows, int d, float eps, void* stream) {
+  return guarded([&]() -> il_status {
   if (!x || !gamma || !beta || !y || !mean || !rstd || rows < 1 || d < 8 || d % 8) return IL_ERR_INVALID_ARG;
   return op_status(layernorm_fwd(x, gamma, beta, (bf16*)y, mean, rstd, rows, d, eps, reinterpret_cast<cudaStream_t>(stream)));
+  });
 }
 
 extern "C" il_status il_op_layernorm_bwd(const void* dy, int dy_is_f32, const float* x, const float* mean, const float* rstd,
                                          const float* gamma, const float* resid, float* dx, void* dx_bf16, float* dgamma,
                                          float* dbeta, int rows, int x_rows, int d, void* stream) {
+  return guarded([&]() -> il_status {
   if (!dy || !x || !mean || !rstd || !gamma || !dx || rows < 1 || x_rows < 1 || d < 8 || d % 8) return IL_ERR_INVALID_ARG;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   if (dgamma && dbeta) {
@@ -1190,14 +1561,17 @@ extern "C" il_status il_op_layernorm_bwd(const void* dy, int dy_is_f32, const fl
     if (e != cudaSuccess) return op_status(e);
   }
   return op_status(layernorm_bwd_rows(dy, dy_is_f32, x, mean, rstd, gamma, resid, dx, (bf16*)dx_bf16, rows, x_rows, d, st));
+  });
 }
 
 extern "C" il_status il_op_layernorm_bwd_fused(const void* dy, const float* x, const float* mean, const float* rstd,
                                                const float* gamma, const float* resid, float* dx, void* dx_bf16,
                                                float* dgamma, float* dbeta, float* colsum, int rows, int x_rows, int d,
                                                void* stream) {
+  return guarded([&]() -> il_status {
   if (!dy || !x || !mean || !rstd || !gamma || !dx || !dgamma || !dbeta || rows < 1 || x_rows < 1) return IL_ERR_INVALID_ARG;
   if (d < 128 || d > 1024 || d % 128) return IL_ERR_INVALID_ARG;
   return op_status(layernorm_bwd_fused((const bf16*)dy, x, mean, rstd, gamma, resid, dx, (bf16*)dx_bf16, dgamma, dbeta, colsum,
                                        rows, x_rows, d, reinterpret_cast<cudaStream_t>(stream)));
+  });
 }

@@ -3,9 +3,6 @@ through the C ABI: useful for comparing kernel changes and as a small case for p
 
     python -m paper_2010_04116_b200.opbench <op> [iterations] [gradient batches]
 
-The environment variable IL_OPBENCH_TILE (1 or 2) forces the GEMM tile width (256 or 512 columns) where the op
-takes one; unset, the library chooses.
-
 ops: logits (auxiliary head: vocabulary projection with the softmax / exp(logit) epilogue), plain (the same
 contraction with a plain bf16 output), fc1 (first MLP projection with the GELU epilogue and its two outputs),
 fc1_plain (the same contraction, bias and bf16 output only), dgelu (gradient through the second MLP projection,
@@ -15,7 +12,6 @@ gradient streams x 8).
 """
 from __future__ import annotations
 
-import os
 import sys
 
 import torch
@@ -23,7 +19,7 @@ import torch
 from . import binding as il
 
 DEV = "cuda:0"
-TILE = int(os.environ.get("IL_OPBENCH_TILE", "0"))
+TILE = 0          # output tile width of the GEMMs: chosen by the library from the shape
 
 
 def _timeit(name, fn, flops, iters, err):

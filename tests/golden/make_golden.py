@@ -4,10 +4,13 @@
     python tests/golden/make_golden.py cfg2 2        # -> tests/golden/cfg2_n2.json
 
 It runs the fp64 CPU oracle (oracle/il_oracle.py) — and nothing else — on the seeded synthetic workload
-of workloads.py at the configuration's full size, and stores a compact summary of the result: the K head
-losses and, for every parameter tensor, the L2 norm of its n-wise gradient, its values at seeded sample
-positions and its inner products with seeded +-1 vectors.  Takes minutes (GPT-2-small shape) to tens of
-minutes (GPT-2-medium shape) on 8 cores and up to ~45 GB of host memory.
+of workloads.py at the configuration's full size, and stores a compact summary of the result.
+<cfg>_n<n>.json: the K head losses, the oracle's run time and core count and, per parameter tensor, the L2 norm
+of its n-wise gradient and its values at seeded sample positions.  <cfg>_n<n>.npz (float32 / float64 arrays,
+see tests/golden/sketch.py): per tensor a 64-bucket count sketch (64 seeded +-1 projections with disjoint
+supports, whose squared distance estimates the squared L2 distance), the whole gradient of every rank-1 tensor
+and four full rows of every matrix.  Takes minutes (GPT-2-small shape) to tens of minutes (GPT-2-medium
+shape) on 8 cores and up to ~45 GB of host memory.
 """
 from __future__ import annotations
 
@@ -23,19 +26,19 @@ sys.path.insert(0, ROOT)
 
 import workloads as wl  # noqa: E402
 from oracle import il_oracle as orc  # noqa: E402
+sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
+import sketch  # noqa: E402
 
 N_SAMPLES = 8
-N_SKETCH = 2
 
 
-def summarize(name: str, index: int, g: np.ndarray) -> dict:
+def summarize(name: str, index: int, g: np.ndarray, arrays: dict) -> dict:
     flat = g.reshape(-1)
     idx = wl.sample_indices(name, index, flat.size, N_SAMPLES)
-    return {
-        "norm": float(np.linalg.norm(flat)),
-        "samples": [float(flat[i]) for i in idx],
-        "sketch": [float(np.dot(flat, wl.rademacher(index, flat.size, j).astype(np.float64))) for j in range(N_SKETCH)],
-    }
+    for key, val in sketch.summarize(name, index, g).items():
+        if key != "norm":
+            arrays[f"{index}:{key}"] = val
+    return {"norm": float(np.linalg.norm(flat)), "samples": [float(flat[i]) for i in idx]}
 
 
 def main():
@@ -46,13 +49,15 @@ def main():
     tok, tgt = wl.draw_tokens(w)
     losses, G = orc.nwise_gradients(P, tok, tgt, w.K, w.Lc, w.H, n, rule=w.rule, head_layers=w.Lh)
     out = {"config": cfg, "n": n, "rule": w.rule, "head_layers": w.Lh, "weight_seed": wl.WEIGHT_SEED, "token_seed": wl.TOKEN_SEED,
-           "oracle_seconds": None, "losses": [float(x) for x in losses], "tensors": {}}
-    for i, (name, _, _, _) in enumerate(wl.tensor_specs(w)):
-        out["tensors"][name] = summarize(name, i, G[name])
+           "oracle_seconds": None, "oracle_cores": os.cpu_count(), "losses": [float(x) for x in losses], "tensors": {}}
     out["oracle_seconds"] = round(time.time() - t0, 1)
+    arrays = {}
+    for i, (name, _, _, _) in enumerate(wl.tensor_specs(w)):
+        out["tensors"][name] = summarize(name, i, G[name], arrays)
     path = os.path.join(os.path.dirname(os.path.abspath(__file__)), f"{cfg}_n{n}.json")
     with open(path, "w") as f:
         json.dump(out, f, indent=0)
+    np.savez(path[:-5] + ".npz", **arrays)
     print(path, out["oracle_seconds"], "s", losses)
 
 

@@ -16,10 +16,10 @@ LOSS_RTOL = 1e-3
 GRAD_RTOL = 2e-2
 
 
-def _check_step(w, n, check_boundaries=True, adamw=False, rule="sum"):
+def _check_step(w, n, check_boundaries=True, adamw=False, rule="sum", head_mode="stored", placement="single"):
     P = wl.draw_params(w)
     tok, tgt = wl.draw_tokens(w)
-    m = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, n, w.B, w.T)
+    m = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, n, w.B, w.T, head_mode=head_mode, placement=placement)
     try:
         m.set_params(P)
         if rule != "sum":
@@ -67,16 +67,30 @@ def _check_step(w, n, check_boundaries=True, adamw=False, rule="sum"):
         m.close()
 
 
+HEAD_MODES = ["stored", "recompute"]
+
+
+@pytest.mark.parametrize("head_mode", HEAD_MODES)
 @pytest.mark.parametrize("n", [1, 2])
-def test_cfg1_matches_oracle(n):
-    _check_step(wl.CONFIGS["cfg1"], n, adamw=(n == 2))
+def test_cfg1_matches_oracle(n, head_mode):
+    _check_step(wl.CONFIGS["cfg1"], n, adamw=(n == 2), head_mode=head_mode)
 
 
+@pytest.mark.parametrize("head_mode", HEAD_MODES)
 @pytest.mark.parametrize("n", [1, 2, 3, 4])
-def test_four_components_all_n(n):
+def test_four_components_all_n(n, head_mode):
     """K = 4 exercises every stream pattern: dropped, passed-down and stacked gradient streams."""
     w = wl.Workload("k4", K=4, Lc=1, d=128, H=2, F=256, V=1000, T=96, B=3, n=n, zipf=True)
-    _check_step(w, n)
+    _check_step(w, n, head_mode=head_mode)
+
+
+@pytest.mark.parametrize("rule", ["sum", "mean"])
+@pytest.mark.parametrize("n", [1, 2, 3, 4])
+def test_four_components_pipeline_placement_matches_oracle(n, rule):
+    """The paper's placement (Sec. 3: one module per accelerator) with every component mapped to the one device:
+    boundary activations and passed-down gradients go through the copy path into receive buffers."""
+    w = wl.Workload("k4p", K=4, Lc=1, d=128, H=2, F=256, V=1000, T=96, B=3, n=n, zipf=True)
+    _check_step(w, n, rule=rule, placement="pipeline", check_boundaries=(rule == "sum"))
 
 
 @pytest.mark.parametrize("rule", ["far", "mean"])
@@ -92,6 +106,13 @@ def test_gpt2_small_width_single_sequence():
     GEMM tiles, 13 vocabulary chunks with a ragged last one, 16 attention blocks."""
     w = wl.CONFIGS["cfg2"].with_(B=1, K=2, Lc=1)
     _check_step(w, 2, check_boundaries=False)
+
+
+def test_gpt2_small_width_single_sequence_recompute_head():
+    """The same with the head that keeps nothing of size [tokens, vocabulary]: 7 vocabulary chunks of 8192 columns,
+    the last one 1105 wide."""
+    w = wl.CONFIGS["cfg2"].with_(B=1, K=2, Lc=1)
+    _check_step(w, 2, check_boundaries=False, head_mode="recompute")
 
 
 def test_single_component_is_plain_training():

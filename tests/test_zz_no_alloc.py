@@ -44,6 +44,13 @@ def test_no_alloc_attention_backward_matches_on_two_calls_in_a_row():
         rel = np.linalg.norm(a - b) / np.linalg.norm(b)
         assert rel < 1.5e-2, rel          # tolerance of the attention parity tests; the two paths are in fact identical
         assert np.array_equal(a, b)
+        assert il.op_attention_bwd_noalloc_status() == 0      # no bounded wait expired in that call
+        # and directly against the fp64 oracle's attention backward (first gradient batch)
+        from oracle import il_oracle as orc
+        ref64 = orc.attention_bwd(dout[:B * T].float().cpu().numpy().astype(np.float64),
+                                  qkv.float().cpu().numpy().astype(np.float64), B, T, H)
+        rel64 = np.linalg.norm(a[:B * T] - ref64) / np.linalg.norm(ref64)
+        assert rel64 < 1.5e-2, rel64
 
 
 def test_no_alloc_attention_backward_rejects_sizes_beyond_its_scratch():
