@@ -2,6 +2,7 @@
 """Throughput of one n-wise training step (tokens/s) on synthetic data.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config cfg4] [--n 2] [--impl reference]
+                    [--head-mode stored|recompute] [--placement replicas|pipeline]
 
 A step is the whole hot path on one batch: il_set_batch, K x (il_forward_component, il_aux_head_loss),
 il_backward_nwise and, where the configuration says so, il_adamw_step.  The default workload is the
@@ -9,6 +10,12 @@ GPT-2-medium-shaped configuration (24 layers in 8 components, d 1024, seq 1024, 
 n = 2, AdamW).  With N > 1 (launched under torch.distributed.run) every rank runs an independent
 replica of the same step on its own GPU: the path has no exchange step, so there is no collective on
 the data path and the scaling is weak.  Rank 0 prints one JSON line.
+
+`--placement pipeline` times the paper's own placement instead (Sec. 3: one module per accelerator): one process
+drives all N GPUs, component k lives on GPU k*N//K, boundary activations and passed-down gradients are copied into
+buffers the receiving GPU owns.  Under torch.distributed.run rank 0 does this alone and the other ranks exit.  The
+line then also carries the time per batch of the paper's model (Sec. 3.1) with its slot cost fitted to the measured
+1-wise step of the same placement.
 
 `--impl reference` times the fp64 CPU oracle, as it stands, on the host cores on a bounded sample of
 the same workload (one sequence of the batch).
@@ -32,8 +39,8 @@ import workloads as wl  # noqa: E402
 
 
 # DRAM bytes per algorithmic flop of the GEMM kernel, from one ncu capture (dram__bytes_read.sum +
-# dram__bytes_write.sum over 400 consecutive GEMM launches of the cfg4-2x1 step, whose launch shapes are cfg4's;
-# profiles/gemm_dram_traffic_cfg4_shapes.md).  Traffic grows with the flops of a launch at fixed shapes, so the
+# dram__bytes_write.sum over 400 consecutive GEMM launches of the cfg4-2x1 step, whose launch shapes are cfg4's).
+# Traffic grows with the flops of a launch at fixed shapes, so the
 # per-launch figure of another step mix is this ratio times that mix's flops per launch.  Set to None whenever
 # gemm.cu changes after the capture.
 GEMM_DRAM_BYTES_PER_FLOP = 1.2568e-3
@@ -141,6 +148,28 @@ def oracle_sample(w: wl.Workload, n: int, steps: int, warmup: int, params=None, 
             "sample": f"{len(times)} oracle step(s) (forward, K heads, per-head n-wise backward; no optimiser) on the "
                       f"first {ts} positions of 1 of {w.B} sequences of {w.name} (full model, n={n}); "
                       f"{sec:.2f} s per step"}
+    # The short sample is dominated by costs that do not grow with the tokens (every weight matrix is widened to
+    # fp64 and read once per step whatever the batch), so two more figures are given: the sample scaled to the full
+    # step by the ratio of algorithmic flops, and the oracle's own time for the full-size step where the run that
+    # wrote the stored expected values recorded it.
+    full_flops = model_flops_per_token(w, n) * w.ntok
+    sample_flops = model_flops_per_token(ws, n) * ws.ntok
+    sec_full = sec * full_flops / sample_flops
+    info["live_extrapolation"] = {"value": w.ntok / sec_full, "unit": "tokens/s", "seconds_per_full_step": sec_full,
+                                  "how": "live sample time x (algorithmic flops of the full step / of the sample)"}
+    gold = os.path.join(ROOT, "tests", "golden", f"{w.name}_n{n}.json")
+    info["cached_full_run"] = None
+    if os.path.exists(gold):
+        try:
+            g = json.load(open(gold))
+            if g.get("oracle_seconds"):
+                info["cached_full_run"] = {"value": w.ntok / float(g["oracle_seconds"]), "unit": "tokens/s",
+                                           "seconds_per_full_step": float(g["oracle_seconds"]),
+                                           "cores": g.get("oracle_cores", 8),
+                                           "how": "wall time of the oracle's full-size step (with the summaries it "
+                                                  "stores) on the machine that wrote tests/golden"}
+        except Exception:
+            pass
     return ws.ntok / sec, sec, info
 
 
@@ -159,6 +188,93 @@ def job_tokens_per_s(tokens_per_rank_step: int, steps: int, world: int, ms: floa
     return tokens_per_rank_step * steps * max(world, 1) / (ms * 1e-3)
 
 
+def bench_pipeline(args, w, n, metric, cfg_desc):
+    """One process, N GPUs, component k on GPU k*N//K (Sec. 3: one module per accelerator; several modules on one
+    accelerator are merged).  Times the requested n and n = 1 and sets them beside the paper's time-per-batch
+    model T(A, 1, N) = 2 N c (Sec. 3.1) with the slot cost c taken from the measured 1-wise step."""
+    import torch
+    from paper_2010_04116_b200 import Model, time_per_batch
+
+    ngpu = max(1, min(args.gpus, torch.cuda.device_count(), w.K))
+    devices = [k * ngpu // w.K for k in range(w.K)]
+    use_adamw = bool(w.adamw and not args.no_adamw)
+    hp = dict(lr=1e-4, beta1=0.9, beta2=0.98, eps=1e-9, weight_decay=w.weight_decay) if use_adamw else None
+    m = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, n, w.B // w.M, w.T, device=0, head_layers=w.Lh, head_mode=args.head_mode,
+              placement="pipeline", devices=devices)
+    if w.rule != "sum":
+        m.set_rule(w.rule)
+    if w.M > 1:
+        m.set_micro_batches(w.M)
+    params = wl.draw_params(w)
+    m.set_params(params)
+    dev0 = torch.device("cuda", 0)
+    nb = 4
+    batches = [tuple(torch.tensor(x, device=dev0) for x in wl.draw_tokens(w, step=s)) for s in range(nb)]
+
+    def run(count):
+        for i in range(count):
+            tok, tgt = batches[i % nb]
+            if w.M > 1:
+                if hp is None:
+                    m.set_micro_batches(w.M)
+                m.train_minibatch(tok, tgt, w.M, adamw=hp)
+            else:
+                m.train_step(tok, tgt, adamw=hp)
+
+    def timed(count):
+        m.sync()
+        s0 = m.streams[0]
+        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.device(0):
+            start.record(s0)
+            run(count)
+            for s in m.streams[1:]:
+                s0.wait_stream(s)
+            end.record(s0)
+        m.sync()
+        return start.elapsed_time(end)
+
+    results = {}
+    sampler = ClockSampler(0)
+    for nn in sorted({1, n}):
+        m.set_n(nn)
+        run(max(args.warmup, 3))
+        if nn == n:
+            sampler.start()
+        results[nn] = timed(args.steps) / args.steps
+    clocks = sampler.stop()
+    launches_per_step = None
+    l0 = m.stats()[1]
+    run(1)
+    m.sync()
+    launches_per_step = m.stats()[1] - l0
+    transfers = m.last_transfers()
+    c = results[1] / 2.0
+    model_ms = time_per_batch(w.K, 1, n, c, 0.0)
+    flops_tok = model_flops_per_token(w, n)
+    value = w.ntok / (results[n] * 1e-3)
+    out = {"metric": metric, "value": value, "unit": "tokens/s", "n_gpus": ngpu, "steps": args.steps,
+           "warmup": max(args.warmup, 3), "ms_per_step": results[n], "higher_is_better": True, "scaling": "strong",
+           "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+           "config": dict(cfg_desc, parallelism=f"pipeline placement: {w.K} components on {ngpu} GPU(s), map {devices}",
+                          global_batch=w.B),
+           "clocks": clocks, "gpu_launches": int(launches_per_step * args.steps),
+           "placement": {"devices": devices,
+                         "copies_per_step": {"forward": sum(1 for t in transfers if t[0] == 0),
+                                             "backward": sum(1 for t in transfers if t[0] == 1)},
+                         "bytes_per_copy": int(w.ntok // w.M * w.d * 4),
+                         "ms_per_step_1wise": results[1]},
+           "timing_model": {"A": w.K, "M": 1, "N": n, "slot_cost_ms": c, "time_per_batch_ms": model_ms,
+                            "measured_ms": results[n],
+                            "note": ("Sec. 3.1: T = 2 N c for M = 1, c fitted as half the measured 1-wise step of this "
+                                     "placement; the model describes one accelerator per module, so it applies when "
+                                     f"n_gpus = {w.K}" + ("" if ngpu == w.K else f" (this run: {ngpu})"))},
+           "model_flops": {"per_token_mflop": flops_tok / 1e6, "tflops_whole_job": value * flops_tok / 1e12},
+           "e2e": None, "roofline": None, "cpu_baseline": None}
+    m.close()
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -169,6 +285,9 @@ def main():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-adamw", action="store_true")
+    ap.add_argument("--head-mode", default="stored", choices=["stored", "recompute"])
+    ap.add_argument("--placement", default="replicas", choices=["replicas", "pipeline"])
+    ap.add_argument("--no-head-mode-comparison", action="store_true")
     args = ap.parse_args()
 
     w = wl.CONFIGS[args.config]
@@ -180,7 +299,7 @@ def main():
     extra = (f", {w.Lh} blocks per auxiliary head, rule={w.rule}, {w.M} micro-batches per update"
              if (w.Lh or w.M > 1 or w.rule != "sum") else "")
     cfg_desc = {"workload": f"{w.name}: {w.K}x{w.Lc} layers, d={w.d}, H={w.H}, F={w.F}, T={w.T}, B={w.B}, V={w.V}, "
-                            f"n={n}, adamw={bool(w.adamw and not args.no_adamw)}{extra}",
+                            f"n={n}, adamw={bool(w.adamw and not args.no_adamw)}{extra}, head_mode={args.head_mode}",
                 "global_batch": w.B * max(world, 1), "seq_len": w.T, "parallelism": f"replicas x{max(world, 1)}",
                 "l2": "inputs larger than L2 (each step streams several GB of weights and activations)"}
 
@@ -202,6 +321,10 @@ def main():
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback for the product path")
+    if args.placement == "pipeline":
+        if rank == 0:
+            bench_pipeline(args, w, n, metric, cfg_desc)
+        return
     torch.cuda.set_device(local_rank)
     dist = None
     if world > 1:
@@ -210,7 +333,8 @@ def main():
 
     use_adamw = bool(w.adamw and not args.no_adamw)
     hp = dict(lr=1e-4, beta1=0.9, beta2=0.98, eps=1e-9, weight_decay=w.weight_decay) if use_adamw else None
-    m = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, n, w.B // w.M, w.T, device=local_rank, head_layers=w.Lh)
+    m = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, n, w.B // w.M, w.T, device=local_rank, head_layers=w.Lh,
+              head_mode=args.head_mode)
     if w.rule != "sum":
         m.set_rule(w.rule)
     if w.M > 1:
@@ -319,12 +443,31 @@ def main():
     }
     if losses is not None:
         out["last_losses"] = [float(x) for x in losses]
+    dev_bytes = m.stats()[0]
+    out["head_mode"] = {"mode": args.head_mode, "ms_per_step": ms / args.steps, "device_bytes": int(dev_bytes)}
+    m.close()
+    if world == 1 and not args.no_head_mode_comparison:
+        # the other head mode on the same workload: step time and device memory side by side
+        other = "recompute" if args.head_mode == "stored" else "stored"
+        torch.cuda.empty_cache()
+        m = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, n, w.B // w.M, w.T, device=local_rank, head_layers=w.Lh, head_mode=other)
+        if w.rule != "sum":
+            m.set_rule(w.rule)
+        if w.M > 1:
+            m.set_micro_batches(w.M)
+        m.set_params(params)
+        s0 = m.streams[0]
+        run_steps(max(args.warmup, 3), False)
+        m.sync()
+        ms_other = timed(args.steps, False)
+        out["head_mode"]["other"] = {"mode": other, "ms_per_step": ms_other / args.steps,
+                                     "device_bytes": int(m.stats()[0])}
+        m.close()
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         _, _, info = oracle_sample(w, n, 1, 0, params=params)
         out["cpu_baseline"] = info
     elif rank == 0:
         out["cpu_baseline"] = None
-    m.close()
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()

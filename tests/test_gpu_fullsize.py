@@ -37,29 +37,31 @@ def _golden(cfg, n):
 _models = {}
 
 
-def _model(cfg):
+def _model(cfg, head_mode="stored"):
     """One model per configuration, reused across n (parameters are copied once)."""
-    if cfg not in _models:
+    key = cfg
+    cfg = cfg.split("/")[0]
+    if key not in _models:
         for m in _models.values():
             m.close()
         _models.clear()
         torch.cuda.empty_cache()
         w = wl.CONFIGS[cfg]
-        m = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, 1, w.B // w.M, w.T, head_layers=w.Lh)
+        m = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, 1, w.B // w.M, w.T, head_layers=w.Lh, head_mode=head_mode)
         for i, (name, _, _, shape) in enumerate(wl.tensor_specs(w)):
             m.set_param(name, wl.draw_tensor(name, i, shape))
         if w.rule != "sum":
             m.set_rule(w.rule)
         if w.M > 1:
             m.set_micro_batches(w.M)
-        _models[cfg] = m
-    return _models[cfg]
+        _models[key] = m
+    return _models[key]
 
 
-def _check_against_golden(cfg, n):
+def _check_against_golden(cfg, n, head_mode="stored"):
     gold = _golden(cfg, n)
     w = wl.CONFIGS[cfg]
-    m = _model(cfg)
+    m = _model(cfg if head_mode == "stored" else f"{cfg}/{head_mode}", head_mode)
     m.set_n(n)
     tok, tgt = wl.draw_tokens(w)
     dt, dg = torch.tensor(tok, device="cuda:0"), torch.tensor(tgt, device="cuda:0")
@@ -113,6 +115,11 @@ def test_gpt2_small_shape_full_size(n):
 @pytest.mark.parametrize("n", [2, 3])
 def test_gpt2_medium_shape_full_size(n):
     _check_against_golden("cfg4", n)
+
+
+def test_gpt2_medium_shape_full_size_recompute_head():
+    """The same step with the head that never holds a [tokens, vocabulary] matrix (7 vocabulary chunks per head)."""
+    _check_against_golden("cfg4", 2, head_mode="recompute")
 
 
 def test_paper_shape_full_model_reduced_batch():
