@@ -72,6 +72,12 @@ typedef struct {
                                     /* parameters, optimiser state and activations; a_k travels forward and at most    */
                                     /* n-1 gradient tensors travel backward per boundary, each copied into a buffer    */
                                     /* the receiving device owns (see il_pipeline_transfers)                           */
+  int attn_bwd;                     /* IL_ATTN_BWD_ONE_SWEEP (0, default): attention backward in one sweep that         */
+                                    /* recomputes the scores once; dQ is summed over key tiles with fp32 atomics, so    */
+                                    /* its last bit (and that of everything computed from it) may differ between runs.  */
+                                    /* IL_ATTN_BWD_TWO_KERNELS (1): dK/dV and dQ in two kernels that each recompute the */
+                                    /* scores; slower, every sum in a fixed order.  Head dims other than 32 / 64 always */
+                                    /* take the two-kernel form                                                         */
   const int* devices;               /* IL_PLACE_PIPELINE: K device ordinals (n_devices == K), or NULL: every component */
   int n_devices;                    /* on `device`, still exchanged through the copy path.  Caller-owned streams[k]    */
                                     /* must belong to devices[k]; the alloc hook is called with that device current    */
@@ -79,6 +85,7 @@ typedef struct {
 
 enum { IL_HEAD_STORED = 0, IL_HEAD_RECOMPUTE = 1 };
 enum { IL_PLACE_SINGLE = 0, IL_PLACE_PIPELINE = 1 };
+enum { IL_ATTN_BWD_ONE_SWEEP = 0, IL_ATTN_BWD_TWO_KERNELS = 1 };
 
 /* Build a model: K components x layers_per_component blocks, d_model, n_heads, d_ff, vocab, and the
  * n of the n-wise rule (Sec. 3: N in [1, number of modules]).  Requires d_model % n_heads == 0,

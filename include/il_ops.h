@@ -73,6 +73,15 @@ il_status il_op_attention_fwd(const void* qkv, void* o, float* lse, int B, int T
 il_status il_op_attention_bwd(const void* qkv, const void* o, const float* lse, const void* dout, void* dqkv,
                               float* delta, int NB, int B, int T, int H, int dh, void* stream);
 
+/* The same gradients from one sweep over the scores (head dimensions 32 and 64): dK, dV and dQ come from a single
+ * recomputation of S and dP (five products instead of the seven of the two-kernel form above).  dq_acc: scratch
+ * [NB*T, H*dh] fp32, 16-byte aligned; every key tile adds its share of dQ into it with floating-point atomics
+ * (the order of that sum, and so the last bit of dQ, may differ between runs), and a final pass writes it to dqkv
+ * as bf16.  err_word: device word set non-zero if a bounded wait expired (may be NULL). */
+il_status il_op_attention_bwd_one_sweep(const void* qkv, const void* o, const float* lse, const void* dout, void* dqkv,
+                                        float* delta, float* dq_acc, int NB, int B, int T, int H, int dh,
+                                        unsigned* err_word, void* stream);
+
 /* The same backward for callers that cannot allocate device memory (no counterpart in the paper: it exists
  * for code embedded where cudaMalloc is not allowed — inside another framework's memory pool, in a
  * real-time loop that bans driver allocations after start-up, or under a fixed device-memory budget).  The

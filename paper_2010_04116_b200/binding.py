@@ -32,7 +32,7 @@ class il_options(C.Structure):
                 ("alloc", ALLOC_FN), ("free_", FREE_FN), ("alloc_ctx", C.c_void_p),
                 ("streams", C.POINTER(C.c_void_p)), ("n_streams", C.c_int),
                 ("use_bias", C.c_int), ("ln_eps", C.c_float), ("head_layers", C.c_int),
-                ("head_mode", C.c_int), ("placement", C.c_int),
+                ("head_mode", C.c_int), ("placement", C.c_int), ("attn_bwd", C.c_int),
                 ("devices", C.POINTER(C.c_int)), ("n_devices", C.c_int)]
 
 
@@ -96,6 +96,7 @@ def lib() -> C.CDLL:
         "il_op_attention_fwd": [vp, vp, vp, i, i, i, i, vp],
         "il_op_attention_bwd": [vp, vp, vp, vp, vp, vp, i, i, i, i, i, vp],
         "il_op_attention_bwd_noalloc": [vp, vp, vp, vp, vp, i, i, i, i, i, vp],
+        "il_op_attention_bwd_one_sweep": [vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, vp, vp],
         "il_op_layernorm_fwd": [vp, vp, vp, vp, vp, vp, i, i, f, vp],
         "il_op_layernorm_bwd": [vp, i, vp, vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, vp],
         "il_op_layernorm_bwd_fused": [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, vp],
@@ -179,7 +180,7 @@ class Model:
     def __init__(self, K: int, Lc: int, d: int, H: int, F: int, V: int, n: int, max_batch: int, max_seq: int,
                  device: int = 0, torch_alloc: bool = True, torch_streams: bool = True, head_layers: int = 0,
                  head_mode: str = "stored", placement: str = "single", devices: Optional[Sequence[int]] = None,
-                 alloc_fail_at: Optional[int] = None):
+                 alloc_fail_at: Optional[int] = None, attn_bwd: str = "one_sweep"):
         """head_mode: 'stored' (exp(logits) kept for the backward) or 'recompute' (vocabulary-chunked backward that
         forms the logits again).  placement: 'single', or 'pipeline' = one component per entry of `devices`
         (default: all on `device`, still exchanged through the copy path).  alloc_fail_at: make the allocator
@@ -199,6 +200,7 @@ class Model:
         opt.head_layers = head_layers
         opt.head_mode = {"stored": 0, "recompute": 1}[head_mode]
         opt.placement = {"single": 0, "pipeline": 1}[placement]
+        opt.attn_bwd = {"one_sweep": 0, "two_kernels": 1}[attn_bwd]
         self.head_mode, self.placement = head_mode, placement
         self.devices = list(devices) if devices is not None else [device] * K
         if devices is not None:
@@ -457,6 +459,13 @@ def op_attention_bwd(qkv, o, lse, dout, dqkv, delta, NB, B, T, H, dh, stream=Non
                                    dh, stream)
     if st != IL_OK:
         raise ILError(st, "il_op_attention_bwd")
+
+
+def op_attention_bwd_one_sweep(qkv, o, lse, dout, dqkv, delta, dq_acc, NB, B, T, H, dh, err_word=None, stream=None):
+    st = lib().il_op_attention_bwd_one_sweep(_ptr(qkv), _ptr(o), _ptr(lse), _ptr(dout), _ptr(dqkv), _ptr(delta),
+                                             _ptr(dq_acc), NB, B, T, H, dh, _ptr(err_word), stream)
+    if st != IL_OK:
+        raise ILError(st, "il_op_attention_bwd_one_sweep")
 
 
 def op_wait_probe(err_word_ptr: int, limit_us: int, stream=None):

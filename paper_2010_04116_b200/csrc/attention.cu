@@ -791,11 +791,387 @@ __global__ void __launch_bounds__(256) attn_bwd_dq_tc_kernel(const __grid_consta
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Backward in one sweep (head dimensions up to 64).  The two-kernel form above recomputes the scores twice (seven
+// products for five); here a CTA owns 128 keys, sweeps the queries in blocks of 128 and produces dV, dK and its
+// share of dQ from one recomputation of S^T and dP^T:
+//   S^T, dP^T   tcgen05.mma M128 (keys) N64 per 64-query half -> TMEM, two halves per step
+//   P^T, dS^T   threads (two per key row, 32 columns each) recompute the probabilities from the saved
+//               log-sum-exp, round to bf16 and store the packed pairs back over the score columns
+//   dV += P^T dO, dK += dS^T Q      A operand read from those TMEM columns, accumulated over the whole sweep
+//   dQ_blk = dS K                   needs dS with the queries as rows: the same threads also write their dS values
+//                                   to shared memory in the layout of an MN-major A operand (swizzled 128-byte
+//                                   rows, one row per key); the product lands in one of two TMEM buffers and is
+//                                   added to an fp32 [rows, d] accumulator in global memory with red.add (every
+//                                   key tile of a (sequence, head) contributes to the same query rows)
+// Roles: warps 0-7 recompute / convert / flush dQ, warp 8 issues every MMA, warp 9 feeds the Q / dO ring by TMA
+// and the per-query lse / delta vectors by plain loads.  The halves give the pipeline its overlap: while the
+// threads work on one half of the step, the tensor pipe runs the other half's products and the next step's
+// scores for the half just finished.  One CTA per SM (all 512 TMEM columns, ~195 KB of shared memory).
+// The sum over key tiles in dQ is made by floating-point atomics: its order, and with it the last bit of dQ,
+// depends on scheduling.  Every wait is bounded.
+// ------------------------------------------------------------------------------------------------
+template <int DH>
+struct FusedCfg {
+  static constexpr int NST = 3;                          // Q / dO ring depth
+  static constexpr int ROW_BYTES = TQ * 128;             // a 128-row operand (one 64-column chunk)
+  static constexpr int DS_BYTES = 2 * TQ * 128;          // dS of one step: two 64-query chunks x 128 key rows x 128 B
+  static constexpr int VEC_BYTES = 2 * TQ * 4;           // lse (log2 units) and delta of the step's 128 queries
+  static constexpr int SMEM = 2 * ROW_BYTES + NST * (2 * ROW_BYTES + VEC_BYTES) + 2 * DS_BYTES + 256 + 1024;
+  // TMEM columns: S^T [0,128) (two halves), dP^T [128,256), dV [256,256+DH), dK [320,320+DH), dQ [384,384+DH) / [448,448+DH)
+  static constexpr int C_S = 0, C_DP = 128, C_DV = 256, C_DK = 320, C_DQ = 384;
+};
+
+template <int DH>
+__global__ void __launch_bounds__(320, 1) attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmRow,     // qkv, 128-row box
+                                                                const __grid_constant__ CUtensorMap tmdO,      // dout, 128-row box
+                                                                const float* __restrict__ lse, const float* __restrict__ delta,
+                                                                bf16* __restrict__ dqkv, float* __restrict__ dq_acc, int B,
+                                                                int T, int H, float scale, unsigned* err) {
+  using C = FusedCfg<DH>;
+  constexpr int NST = C::NST;
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ int abort_flag;
+  __shared__ uint32_t tmem_base_smem;
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t sK = base, sV = sK + C::ROW_BYTES;
+  const uint32_t sQ0 = sV + C::ROW_BYTES;                                  // stage st: Q at sQ0 + st * STAGE, dO after it
+  constexpr uint32_t STAGE = 2 * C::ROW_BYTES;
+  const uint32_t sDS = sQ0 + NST * STAGE;                                  // two dS buffers
+  const uint32_t sVec = sDS + 2 * C::DS_BYTES;                             // NST x (lse2[128], delta[128])
+  const uint32_t bars = sVec + NST * C::VEC_BYTES;
+  // barriers (8 bytes each)
+  const uint32_t bar_kv = bars, bar_acc = bars + 8, bar_drain = bars + 16;
+  auto bar_full = [&](int st) { return bars + 24 + 8 * st; };
+  auto bar_empty = [&](int st) { return bars + 24 + 8 * (NST + st); };
+  auto bar_s = [&](int x) { return bars + 24 + 8 * (2 * NST + x); };          // scores of half x ready
+  auto bar_p = [&](int x) { return bars + 24 + 8 * (2 * NST + 2 + x); };      // P^T / dS^T of half x written
+  auto bar_dq = [&](int b) { return bars + 24 + 8 * (2 * NST + 4 + b); };     // dQ buffer b complete
+  auto bar_dqfree = [&](int b) { return bars + 24 + 8 * (2 * NST + 6 + b); }; // dQ buffer b flushed
+  uint8_t* gen = smem_raw + (base - smem_u32(smem_raw));
+  float* s_vec = reinterpret_cast<float*>(gen + (sVec - base));
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int kb = blockIdx.x;                                       // key tile; tile 0 has the longest sweep and runs first
+  const int nb = blockIdx.y / H, h = blockIdx.y % H;
+  const int bs = nb % B;
+  const int d = H * DH;
+  const int nq = (T + TQ - 1) / TQ;
+  const int nit = nq - kb;                                         // query blocks kb .. nq-1 see these keys
+  volatile int* abortp = &abort_flag;
+
+  if (tid == 0) {
+    abort_flag = 0;
+    mbar_init(bar_kv, 1);
+    mbar_init(bar_acc, 1);
+    mbar_init(bar_drain, 1);
+    for (int st = 0; st < NST; ++st) { mbar_init(bar_full(st), 1); mbar_init(bar_empty(st), 1); }
+    for (int x = 0; x < 2; ++x) {
+      mbar_init(bar_s(x), 1);
+      mbar_init(bar_p(x), 8);            // one arrival per recompute warp
+      mbar_init(bar_dq(x), 1);
+      mbar_init(bar_dqfree(x), 8);
+    }
+    fence_mbar_init();
+    tma_prefetch_desc(&tmRow);
+    tma_prefetch_desc(&tmdO);
+  }
+  if (warp == 8) {
+    tmem_alloc(smem_u32(&tmem_base_smem), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_smem;
+  const float c2 = scale * IL_LOG2E;
+  int fail = 0;
+
+  if (warp == 9) {
+    // ---------------------------------------------------------------- loads
+    if (lane == 0) {
+      mbar_expect_tx(bar_kv, 2 * C::ROW_BYTES);
+      tma_load_4d(sK, &tmRow, 0, H + h, kb * TQ, bs, bar_kv);
+      tma_load_4d(sV, &tmRow, 0, 2 * H + h, kb * TQ, bs, bar_kv);
+    }
+    const float* lse_b = lse + ((size_t)bs * H + h) * T;
+    const float* del_b = delta + ((size_t)nb * H + h) * T;
+    for (int it = 0; it < nit; ++it) {
+      const int st = it % NST, j = kb + it;
+      int ok = 1;
+      if (lane == 0 && it >= NST) ok = mbar_wait(bar_empty(st), (uint32_t)(it / NST - 1) & 1u, abortp) ? 1 : 0;
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) { fail = 1; abort_flag = 1; break; }
+      float* vec = s_vec + st * (2 * TQ);
+#pragma unroll
+      for (int q4 = 0; q4 < 4; ++q4) {
+        const int q = j * TQ + q4 * 32 + lane;
+        vec[q4 * 32 + lane] = q < T ? lse_b[q] * IL_LOG2E : 0.f;
+        vec[TQ + q4 * 32 + lane] = q < T ? del_b[q] : 0.f;
+      }
+      __syncwarp();
+      if (lane == 0) {
+        mbar_expect_tx(bar_full(st), 2 * C::ROW_BYTES);          // its release also publishes the warp's vector stores
+        tma_load_4d(sQ0 + st * STAGE, &tmRow, 0, h, j * TQ, bs, bar_full(st));
+        tma_load_4d(sQ0 + st * STAGE + C::ROW_BYTES, &tmdO, 0, h, j * TQ, nb, bar_full(st));
+      }
+    }
+  } else if (warp == 8) {
+    // ---------------------------------------------------------------- MMA issue
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = make_idesc_bf16(TQ, TK, 0, 0);          // S^T / dP^T half: M128 N64, both K-major
+      constexpr uint32_t idesc_g = make_idesc_bf16(TQ, DH, 0, 1);          // dV / dK: A from TMEM, B MN-major
+      constexpr uint32_t idesc_q = make_idesc_bf16(TQ, DH, 1, 1);          // dQ: A = dS (MN-major), B = K (MN-major)
+      const SmemDescBase dk_k = make_smem_desc_base(sK, 16, 1024), dv_k = make_smem_desc_base(sV, 16, 1024);
+      const SmemDescBase dk_mn = make_smem_desc_base(sK, TQ * 128, 1024);
+      const SmemDescBase dq_k = make_smem_desc_base(sQ0, 16, 1024), ddo_k = make_smem_desc_base(sQ0 + C::ROW_BYTES, 16, 1024);
+      const SmemDescBase dq_mn = make_smem_desc_base(sQ0, TQ * 128, 1024), ddo_mn = make_smem_desc_base(sQ0 + C::ROW_BYTES, TQ * 128, 1024);
+      const SmemDescBase dds_mn = make_smem_desc_base(sDS, TQ * 128, 1024);
+      bool ok = true;
+      // scores of half x of the step held in stage st: rows 64x .. 64x+63 of the Q / dO tiles (8 KB further)
+      auto issue_scores = [&](int st, int x) {
+        const uint32_t so = (uint32_t)st * STAGE + (uint32_t)x * (TK * 128);
+#pragma unroll
+        for (int ks = 0; ks < DH / 16; ++ks) {
+          umma_bf16(tmem_base + C::C_S + 64 * x, desc_at(dk_k, ks * 32), desc_at(dq_k, so + ks * 32), idesc_s, ks ? 1u : 0u);
+          umma_bf16(tmem_base + C::C_DP + 64 * x, desc_at(dv_k, ks * 32), desc_at(ddo_k, so + ks * 32), idesc_s, ks ? 1u : 0u);
+        }
+        umma_commit(bar_s(x));
+      };
+      if (!mbar_wait(bar_kv, 0, abortp)) ok = false;
+      if (ok && !mbar_wait(bar_full(0), 0, abortp)) ok = false;
+      if (ok) {
+        tc_fence_after();
+        issue_scores(0, 0);
+        issue_scores(0, 1);
+      }
+      for (int it = 0; it < nit && ok; ++it) {
+        const int st = it % NST, b = it & 1;
+        const uint32_t ph = (uint32_t)it & 1u;
+        for (int x = 0; x < 2 && ok; ++x) {
+          if (!mbar_wait(bar_p(x), ph, abortp)) { ok = false; break; }
+          tc_fence_after();
+          // dV += P^T(x) dO(x), dK += dS^T(x) Q(x): contraction over the half's 64 queries (MN-major B: 16 queries = 2048 B)
+          const uint32_t so = (uint32_t)st * STAGE + (uint32_t)x * (TK * 128);
+#pragma unroll
+          for (int ks = 0; ks < TK / 16; ++ks) {
+            const uint32_t acc = (it | x | ks) ? 1u : 0u;
+            umma_bf16_ts(tmem_base + C::C_DV, tmem_base + C::C_S + 64 * x + packed_col(ks), desc_at(ddo_mn, so + ks * 2048), idesc_g, acc);
+            umma_bf16_ts(tmem_base + C::C_DK, tmem_base + C::C_DP + 64 * x + packed_col(ks), desc_at(dq_mn, so + ks * 2048), idesc_g, acc);
+          }
+          if (x == 1) {
+            umma_commit(bar_empty(st));                     // the stage's tiles have been read once these retire
+            // dQ(it) = dS K over this tile's 128 keys, into buffer b (free once the flush of step it-2 is done)
+            if (it >= 2 && !mbar_wait(bar_dqfree(b), (uint32_t)((it >> 1) - 1) & 1u, abortp)) { ok = false; break; }
+            tc_fence_after();
+#pragma unroll
+            for (int ks = 0; ks < TQ / 16; ++ks)
+              umma_bf16(tmem_base + C::C_DQ + 64 * b, desc_at(dds_mn, (uint32_t)b * C::DS_BYTES + ks * 2048),
+                        desc_at(dk_mn, ks * 2048), idesc_q, ks ? 1u : 0u);
+            umma_commit(bar_dq(b));
+          }
+          if (it + 1 < nit) {
+            // next step's scores for the half just consumed (the pipe runs them after the products above)
+            const int st1 = (it + 1) % NST;
+            if (x == 0 && !mbar_wait(bar_full(st1), (uint32_t)((it + 1) / NST) & 1u, abortp)) { ok = false; break; }
+            tc_fence_after();
+            issue_scores(st1, x);
+          }
+        }
+      }
+      if (ok) umma_commit(bar_acc);
+      else { fail = 1; abort_flag = 1; }
+    }
+  } else {
+    // ---------------------------------------------------------------- recompute, convert, flush (warps 0-7)
+    const int r = tid & 127, hf = tid >> 7;
+    const int key = kb * TQ + r;
+    const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+    auto flush_dq = [&](int it) -> bool {        // add dQ of step `it` to the global accumulator
+      const int b = it & 1;
+      int got = 1;
+      if (lane == 0) got = mbar_wait(bar_dq(b), (uint32_t)(it >> 1) & 1u, abortp) ? 1 : 0;
+      got = __shfl_sync(0xffffffffu, got, 0);
+      if (!got) return false;
+      tc_fence_after();
+      const int q = (kb + it) * TQ + r;
+      float* dst = dq_acc + ((size_t)nb * T + q) * d + h * DH;
+      if constexpr (DH == 64) {
+        uint32_t rr[32];
+        tmem_ld_32x32(t_lane + C::C_DQ + 64 * b + 32 * hf, rr);
+        tmem_ld_wait();
+        if (q < T) {
+#pragma unroll
+          for (int i = 0; i < 32; i += 4)
+            red_add_f32x4(dst + 32 * hf + i, make_float4(__uint_as_float(rr[i]), __uint_as_float(rr[i + 1]),
+                                                         __uint_as_float(rr[i + 2]), __uint_as_float(rr[i + 3])));
+        }
+      } else {   // DH == 32: 16 columns per thread
+        uint32_t rr[16];
+        tmem_ld_32x16(t_lane + C::C_DQ + 64 * b + 16 * hf, rr);
+        tmem_ld_wait();
+        if (q < T) {
+#pragma unroll
+          for (int i = 0; i < 16; i += 4)
+            red_add_f32x4(dst + 16 * hf + i, make_float4(__uint_as_float(rr[i]), __uint_as_float(rr[i + 1]),
+                                                         __uint_as_float(rr[i + 2]), __uint_as_float(rr[i + 3])));
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_dqfree(b));
+      return true;
+    };
+    for (int it = 0; it < nit && !fail; ++it) {
+      const int st = it % NST, b = it & 1, j = kb + it;
+      const uint32_t ph = (uint32_t)it & 1u;
+      const float* vec = s_vec + st * (2 * TQ);
+      {   // the stage's lse / delta vectors were published with its "full" barrier (long complete by now)
+        int got = 1;
+        if (lane == 0) got = mbar_wait(bar_full(st), (uint32_t)(it / NST) & 1u, abortp) ? 1 : 0;
+        got = __shfl_sync(0xffffffffu, got, 0);
+        if (!got) { fail = 1; abort_flag = 1; break; }
+      }
+      const bool diag = (j == kb);                       // some queries of this block precede some keys of this CTA
+      const bool tail = (j * TQ + TQ > T);
+      for (int x = 0; x < 2; ++x) {
+        {
+          int got = 1;
+          if (lane == 0) got = mbar_wait(bar_s(x), ph, abortp) ? 1 : 0;
+          got = __shfl_sync(0xffffffffu, got, 0);
+          if (!got) { fail = 1; abort_flag = 1; break; }
+        }
+        tc_fence_after();
+        uint32_t r0[32], r1[32];
+        tmem_ld_32x32(t_lane + C::C_S + 64 * x + 32 * hf, r0);
+        tmem_ld_32x32(t_lane + C::C_DP + 64 * x + 32 * hf, r1);
+        tmem_ld_wait();
+        float p[32], ds[32];
+        const float4* lv = reinterpret_cast<const float4*>(vec + 64 * x + 32 * hf);
+        const float4* dv_ = reinterpret_cast<const float4*>(vec + TQ + 64 * x + 32 * hf);
+        const int qbase = j * TQ + 64 * x + 32 * hf;
+#pragma unroll
+        for (int i4 = 0; i4 < 8; ++i4) {
+          const float4 l4 = lv[i4], d4 = dv_[i4];
+          const float ll[4] = {l4.x, l4.y, l4.z, l4.w}, dd[4] = {d4.x, d4.y, d4.z, d4.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int i = 4 * i4 + e;
+            p[i] = ex2_fast(fmaf(__uint_as_float(r0[i]), c2, -ll[e]));
+            ds[i] = __uint_as_float(r1[i]) - dd[e];
+          }
+        }
+        if (diag || tail) {                              // uniform across the CTA
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if (qbase + i < key || qbase + i >= T) p[i] = 0.f;
+        }
+#pragma unroll
+        for (int i = 0; i < 32; ++i) ds[i] *= p[i];
+        uint32_t pw[16], dw[16];
+        pack_row32(p, pw);
+        pack_row32(ds, dw);
+        tmem_st_32x16(t_lane + C::C_S + 64 * x + 32 * hf, pw);      // P^T over the first half of the columns this thread read
+        tmem_st_32x16(t_lane + C::C_DP + 64 * x + 32 * hf, dw);     // dS^T likewise
+        // dS as the A operand of dQ = dS K: row = key, 64 queries of half x = one swizzled 128-byte row of chunk x
+        {
+          const uint32_t rowaddr = sDS + (uint32_t)b * C::DS_BYTES + (uint32_t)x * (TQ * 128) + (uint32_t)r * 128;
+#pragma unroll
+          for (int t = 0; t < 4; ++t) {
+            const uint32_t unit = (uint32_t)(4 * hf + t) ^ (uint32_t)(r & 7);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(rowaddr + unit * 16), "r"(dw[4 * t]), "r"(dw[4 * t + 1]),
+                         "r"(dw[4 * t + 2]), "r"(dw[4 * t + 3])
+                         : "memory");
+          }
+        }
+        tmem_st_wait();
+        fence_proxy_async();                               // the dS rows are read by the tensor pipe (async proxy)
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_p(x));
+        // between the halves: the previous step's dQ has long been complete
+        if (x == 0 && it > 0) {
+          if (!flush_dq(it - 1)) { fail = 1; abort_flag = 1; break; }
+        }
+      }
+    }
+    if (!fail && nit > 0) {
+      if (!flush_dq(nit - 1)) { fail = 1; abort_flag = 1; }
+    }
+    if (!fail) {
+      int got = 1;
+      if (lane == 0) got = mbar_wait(bar_acc, 0, abortp) ? 1 : 0;
+      got = __shfl_sync(0xffffffffu, got, 0);
+      if (!got) { fail = 1; abort_flag = 1; }
+      tc_fence_after();
+    }
+    if (!fail) {
+      // dV (first half of the threads) and dK (second half) of this CTA's 128 keys
+      bf16* rowp = dqkv + ((size_t)nb * T + key) * (3 * d) + h * DH;
+      bf16* dst = rowp + (hf == 0 ? 2 * d : d);
+      const float f = hf == 0 ? 1.0f : scale;
+      const uint32_t tcol = t_lane + (hf == 0 ? C::C_DV : C::C_DK);
+#pragma unroll
+      for (int c0 = 0; c0 < DH; c0 += 32) {
+        uint32_t rr[32];
+        tmem_ld_32x32(tcol + c0, rr);
+        tmem_ld_wait();
+        if (key < T) {
+#pragma unroll
+          for (int i = 0; i < 32; i += 8) {
+            uint4 pk;
+            pk.x = pack_bf16x2(__uint_as_float(rr[i]) * f, __uint_as_float(rr[i + 1]) * f);
+            pk.y = pack_bf16x2(__uint_as_float(rr[i + 2]) * f, __uint_as_float(rr[i + 3]) * f);
+            pk.z = pack_bf16x2(__uint_as_float(rr[i + 4]) * f, __uint_as_float(rr[i + 5]) * f);
+            pk.w = pack_bf16x2(__uint_as_float(rr[i + 6]) * f, __uint_as_float(rr[i + 7]) * f);
+            *reinterpret_cast<uint4*>(dst + c0 + i) = pk;
+          }
+        }
+      }
+    }
+  }
+  fail = __syncthreads_or(fail);
+  if (tid == 8 * 32) {
+    if (fail && err) atomicExch(err, DEV_TIMEOUT_MMA);
+    umma_commit(bar_drain);                      // every MMA issued by this CTA has retired before TMEM goes
+    int never = 0;
+    mbar_wait(bar_drain, 0, &never);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 8) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// dqkv[row, h*dh + c] (the Q third) = bf16(scale * dq_acc[row, h*dh + c]): the accumulated dQ leaves fp32 here.
+__global__ void __launch_bounds__(256) attn_dq_convert_kernel(const float* __restrict__ acc, bf16* __restrict__ dqkv, size_t rows,
+                                                              int d, float scale) {
+  const int d8 = d >> 3;
+  const size_t total = rows * (size_t)d8;
+  for (size_t i = (size_t)blockIdx.x * 256 + threadIdx.x; i < total; i += (size_t)gridDim.x * 256) {
+    const size_t row = i / d8;
+    const int c = (int)(i % d8) * 8;
+    const float4 a = *reinterpret_cast<const float4*>(acc + row * d + c);
+    const float4 b = *reinterpret_cast<const float4*>(acc + row * d + c + 4);
+    uint4 o;
+    o.x = pack_bf16x2(a.x * scale, a.y * scale);
+    o.y = pack_bf16x2(a.z * scale, a.w * scale);
+    o.z = pack_bf16x2(b.x * scale, b.y * scale);
+    o.w = pack_bf16x2(b.z * scale, b.w * scale);
+    *reinterpret_cast<uint4*>(dqkv + row * (size_t)(3 * d) + c) = o;
+  }
+}
+
 // delta[nb, h, t] = sum_c dO[nb*T+t, h*dh+c] * O[(nb%B)*T+t, h*dh+c].  A thread takes 8 consecutive columns
 // (16 bytes of each operand); the dh/8 threads of a (row, head) sit in one warp and combine by shuffles.
+// With dq_zero != NULL the same threads also clear their 8 columns of the fp32 dQ accumulator [NB*T, H*dh] that the
+// one-sweep backward adds into.
 template <int DH>
 __global__ void __launch_bounds__(256) attn_delta_tc_kernel(const bf16* __restrict__ dout, const bf16* __restrict__ o,
-                                                            float* __restrict__ delta, int NB, int B, int T, int H) {
+                                                            float* __restrict__ delta, float* __restrict__ dq_zero, int NB,
+                                                            int B, int T, int H) {
   constexpr int TPR = (DH == 80) ? 16 : DH / 8;      // threads per (row, head): a power of two (dh 80: 10 of 16 active)
   const long long gid = (long long)blockIdx.x * 256 + threadIdx.x;
   const long long item = gid / TPR;                  // (row, head) index
@@ -810,6 +1186,11 @@ __global__ void __launch_bounds__(256) attn_delta_tc_kernel(const bf16* __restri
     const int nb = (int)(row / T), t = (int)(row % T);
     if (part * 8 < DH) {
       const int d = H * DH;
+      if (dq_zero) {
+        float4* z = reinterpret_cast<float4*>(dq_zero + (size_t)row * d + h * DH + part * 8);
+        z[0] = make_float4(0.f, 0.f, 0.f, 0.f);
+        z[1] = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
       const uint4 a = *reinterpret_cast<const uint4*>(dout + (size_t)row * d + h * DH + part * 8);
       const uint4 c = *reinterpret_cast<const uint4*>(o + ((size_t)(nb % B) * T + t) * d + h * DH + part * 8);
       const __nv_bfloat162* a2 = reinterpret_cast<const __nv_bfloat162*>(&a);
@@ -857,7 +1238,7 @@ cudaError_t bwd_tc_launch(const bf16* qkv, const bf16* o, const float* lse, cons
   if (e != cudaSuccess) return e;
   constexpr int TPR = (DH == 80) ? 16 : DH / 8;
   const long long nthreads = (long long)NB * T * H * TPR;
-  attn_delta_tc_kernel<DH><<<(unsigned)((nthreads + 255) / 256), 256, 0, s>>>(dout, o, delta, NB, B, T, H);
+  attn_delta_tc_kernel<DH><<<(unsigned)((nthreads + 255) / 256), 256, 0, s>>>(dout, o, delta, nullptr, NB, B, T, H);
   dim3 grid((T + TQ - 1) / TQ, NB * H);
   const float scale = rsqrtf((float)DH);
   if constexpr (SPLIT) {
@@ -867,6 +1248,35 @@ cudaError_t bwd_tc_launch(const bf16* qkv, const bf16* o, const float* lse, cons
     attn_bwd_dkv_tc_kernel<DH, 0><<<grid, 256, C::SMEM_KV, s>>>(tmRow, tmBlk, tmdO64, lse, delta, dqkv, B, T, H, scale, err);
   }
   attn_bwd_dq_tc_kernel<DH><<<grid, 256, C::SMEM_Q, s>>>(tmRow, tmBlk, tmdO128, lse, delta, dqkv, B, T, H, scale, err);
+  return cudaGetLastError();
+}
+
+// One-sweep backward: delta (+ clearing the accumulator), the sweep, then dQ from fp32 to bf16.
+template <int DH>
+cudaError_t bwd_fused_launch(const bf16* qkv, const bf16* o, const float* lse, const bf16* dout, bf16* dqkv, float* delta,
+                             float* dq_acc, int NB, int B, int T, int H, unsigned* err, cudaStream_t s) {
+  using C = FusedCfg<DH>;
+  const unsigned long long d3 = 3ull * H * DH, d1 = (unsigned long long)H * DH;
+  const unsigned long long dims[4] = {(unsigned long long)DH, 3ull * H, (unsigned long long)T, (unsigned long long)B};
+  const unsigned long long strides[3] = {(unsigned long long)DH * 2, d3 * 2, (unsigned long long)T * d3 * 2};
+  const unsigned long long ddims[4] = {(unsigned long long)DH, (unsigned long long)H, (unsigned long long)T, (unsigned long long)NB};
+  const unsigned long long dstrides[3] = {(unsigned long long)DH * 2, d1 * 2, (unsigned long long)T * d1 * 2};
+  const unsigned box128[4] = {64, 1, TQ, 1};
+  CUtensorMap tmRow, tmdO;
+  if (!tma_encode_bf16(&tmRow, qkv, 4, dims, strides, box128) || !tma_encode_bf16(&tmdO, dout, 4, ddims, dstrides, box128))
+    return cudaErrorInvalidValue;
+  cudaError_t e = cudaFuncSetAttribute(attn_bwd_fused_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
+  if (e != cudaSuccess) return e;
+  constexpr int TPR = DH / 8;
+  const long long nthreads = (long long)NB * T * H * TPR;
+  attn_delta_tc_kernel<DH><<<(unsigned)((nthreads + 255) / 256), 256, 0, s>>>(dout, o, delta, dq_acc, NB, B, T, H);
+  dim3 grid((T + TQ - 1) / TQ, NB * H);
+  const float scale = rsqrtf((float)DH);
+  attn_bwd_fused_kernel<DH><<<grid, 320, C::SMEM, s>>>(tmRow, tmdO, lse, delta, dqkv, dq_acc, B, T, H, scale, err);
+  const size_t rows = (size_t)NB * T;
+  size_t blocks = (rows * (size_t)(H * DH / 8) + 255) / 256;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  attn_dq_convert_kernel<<<(unsigned)blocks, 256, 0, s>>>(dq_acc, dqkv, rows, H * DH, scale);
   return cudaGetLastError();
 }
 
@@ -886,11 +1296,16 @@ cudaError_t attention_fwd(const bf16* qkv, bf16* o, float* lse, int B, int T, in
 }
 
 cudaError_t attention_bwd(const bf16* qkv, const bf16* o, const float* lse, const bf16* dout, bf16* dqkv, float* delta,
-                             int NB, int B, int T, int H, int dh, unsigned* err, cudaStream_t s) {
+                          float* dq_acc, int NB, int B, int T, int H, int dh, unsigned* err, cudaStream_t s) {
   // o is read with 16-byte loads by the delta kernel, qkv / dout / dqkv by TMA and 16-byte stores
   if (((uintptr_t)qkv % 16) || ((uintptr_t)o % 16) || ((uintptr_t)dout % 16) || ((uintptr_t)dqkv % 16) ||
       ((uintptr_t)lse % 4) || ((uintptr_t)delta % 4))
     return cudaErrorInvalidValue;
+  if (dq_acc && (dh == 32 || dh == 64)) {        // one sweep, dQ summed over key tiles in the fp32 accumulator
+    if ((uintptr_t)dq_acc % 16) return cudaErrorInvalidValue;
+    return dh == 32 ? bwd_fused_launch<32>(qkv, o, lse, dout, dqkv, delta, dq_acc, NB, B, T, H, err, s)
+                    : bwd_fused_launch<64>(qkv, o, lse, dout, dqkv, delta, dq_acc, NB, B, T, H, err, s);
+  }
   switch (dh) {
     case 32: return bwd_tc_launch<32>(qkv, o, lse, dout, dqkv, delta, NB, B, T, H, err, s);
     case 64: return bwd_tc_launch<64>(qkv, o, lse, dout, dqkv, delta, NB, B, T, H, err, s);

@@ -77,8 +77,11 @@ cudaError_t attention_fwd(const __nv_bfloat16* qkv, __nv_bfloat16* o, float* lse
                           unsigned* err, cudaStream_t s);
 // Backward.  NB batches of gradients share one saved forward of B sequences: gradient batch b uses saved
 // sequence (b % B).  dqkv [NB*T, 3d] bf16; delta is scratch [NB, H, T] fp32.
+// dq_acc: NULL = two kernels (dK/dV, then dQ; each recomputes the scores; every sum has a fixed order); otherwise
+// scratch [NB*T, d] fp32 (16-byte aligned) for the one-sweep form (head dimensions 32 and 64; other sizes fall back
+// to two kernels): one recomputation of the scores, dQ summed over key tiles with floating-point atomics.
 cudaError_t attention_bwd(const __nv_bfloat16* qkv, const __nv_bfloat16* o, const float* lse, const __nv_bfloat16* dout,
-                          __nv_bfloat16* dqkv, float* delta, int NB, int B, int T, int H, int dh, unsigned* err,
-                          cudaStream_t s);
+                          __nv_bfloat16* dqkv, float* delta, float* dq_acc, int NB, int B, int T, int H, int dh,
+                          unsigned* err, cudaStream_t s);
 
 }  // namespace il

@@ -68,6 +68,7 @@ struct il_model {
   int micro, micro_done;              // micro-batches per update, backward passes since the last update
   int rule;                           // IL_RULE_*: which heads update a component's parameters
   int head_mode;                      // IL_HEAD_STORED / IL_HEAD_RECOMPUTE
+  int attn_bwd;                       // IL_ATTN_BWD_ONE_SWEEP / IL_ATTN_BWD_TWO_KERNELS
   int placement;                      // IL_PLACE_SINGLE / IL_PLACE_PIPELINE
   std::vector<int> dev;               // device of component k (all equal to `device` unless placed as a pipeline)
   std::vector<int> dev_list;          // the distinct devices in use
@@ -419,6 +420,7 @@ extern "C" il_status il_create(int K, int Lc, int d, int H, int F, int V, int n,
   if (opt->use_bias != 1) return IL_ERR_INVALID_ARG;             // only the GPT-2 form with biases is built
   if (opt->head_mode != IL_HEAD_STORED && opt->head_mode != IL_HEAD_RECOMPUTE) return IL_ERR_INVALID_ARG;
   if (opt->placement != IL_PLACE_SINGLE && opt->placement != IL_PLACE_PIPELINE) return IL_ERR_INVALID_ARG;
+  if (opt->attn_bwd != IL_ATTN_BWD_ONE_SWEEP && opt->attn_bwd != IL_ATTN_BWD_TWO_KERNELS) return IL_ERR_INVALID_ARG;
   if (opt->devices && (opt->placement != IL_PLACE_PIPELINE || opt->n_devices != K)) return IL_ERR_INVALID_ARG;
 
   il_model* m = new (std::nothrow) il_model();
@@ -428,7 +430,7 @@ extern "C" il_status il_create(int K, int Lc, int d, int H, int F, int V, int n,
   m->opt = *opt;
   m->opt.devices = nullptr;            // the caller's array is not kept
   m->device = opt->device;
-  m->head_mode = opt->head_mode; m->placement = opt->placement;
+  m->head_mode = opt->head_mode; m->placement = opt->placement; m->attn_bwd = opt->attn_bwd;
   m->max_batch = opt->max_batch; m->max_seq = opt->max_seq;
   m->ntok_max = opt->max_batch * opt->max_seq;
   m->ln_eps = opt->ln_eps > 0 ? opt->ln_eps : 1e-5f;
@@ -1039,7 +1041,11 @@ il_status layers_backward(il_model* m, int k, int s, size_t base, int count, con
     }
     IL_TRY(wgrad(m, k, d, d, N, c.dxb, d, A.attn_o, d, m->G[k] + o.wo, acc));
     IL_TRY(gemm(m, k, gemm_args(R, d, d, c.dxb, d, 0, m->Pb[k] + o.wo, d, 1, EPI_BF16, c.dattn, d)));
-    IL_K(m, attention_bwd(A.qkv, A.attn_o, A.lse, c.dattn, c.dqkv, c.delta, s * m->B, m->B, m->T, m->H, m->dh, m->err_word[k], st));
+    // dQ accumulator of the one-sweep attention backward: the FC1 gradient buffer (bf16 [R, F], at least the
+    // [R, d] fp32 needed whenever F >= 2 d) is free between the MLP's and the attention's backward
+    float* dq_acc = (m->attn_bwd == IL_ATTN_BWD_ONE_SWEEP && F >= 2 * d) ? reinterpret_cast<float*>(c.dbig) : nullptr;
+    IL_K(m, attention_bwd(A.qkv, A.attn_o, A.lse, c.dattn, c.dqkv, c.delta, dq_acc, s * m->B, m->B, m->T, m->H, m->dh,
+                          m->err_word[k], st));
     m->launches += 2;
     IL_K(m, colsum_bf16(c.dqkv, 3 * d, m->G[k] + o.bqkv, N, 3 * d, st));
     IL_TRY(wgrad(m, k, 3 * d, d, N, c.dqkv, 3 * d, A.ln1, d, m->G[k] + o.wqkv, acc));
@@ -1530,8 +1536,19 @@ extern "C" il_status il_op_attention_bwd(const void* qkv, const void* o, const f
                                          float* delta, int NB, int B, int T, int H, int dh, void* stream) {
   return guarded([&]() -> il_status {
   if (!qkv || !o || !lse || !dout || !dqkv || !delta || B < 1 || NB < 1 || T < 1 || H < 1) return IL_ERR_INVALID_ARG;
-  return op_status(attention_bwd((const bf16*)qkv, (const bf16*)o, lse, (const bf16*)dout, (bf16*)dqkv, delta, NB, B, T, H, dh,
-                                 nullptr, reinterpret_cast<cudaStream_t>(stream)));
+  return op_status(attention_bwd((const bf16*)qkv, (const bf16*)o, lse, (const bf16*)dout, (bf16*)dqkv, delta, nullptr, NB, B, T,
+                                 H, dh, nullptr, reinterpret_cast<cudaStream_t>(stream)));
+  });
+}
+
+extern "C" il_status il_op_attention_bwd_one_sweep(const void* qkv, const void* o, const float* lse, const void* dout,
+                                                   void* dqkv, float* delta, float* dq_acc, int NB, int B, int T, int H,
+                                                   int dh, unsigned* err_word, void* stream) {
+  return guarded([&]() -> il_status {
+  if (!qkv || !o || !lse || !dout || !dqkv || !delta || !dq_acc || B < 1 || NB < 1 || T < 1 || H < 1) return IL_ERR_INVALID_ARG;
+  if (dh != 32 && dh != 64) return IL_ERR_INVALID_ARG;
+  return op_status(attention_bwd((const bf16*)qkv, (const bf16*)o, lse, (const bf16*)dout, (bf16*)dqkv, delta, dq_acc, NB, B, T,
+                                 H, dh, err_word, reinterpret_cast<cudaStream_t>(stream)));
   });
 }
 

@@ -61,7 +61,7 @@ extern "C" il_status il_op_attention_bwd_noalloc(const void* qkv, const void* o,
   // Every element of delta that the kernels read is written by the same call first, so nothing has to be cleared.
   cudaError_t e = il::attention_bwd(reinterpret_cast<const __nv_bfloat16*>(qkv), reinterpret_cast<const __nv_bfloat16*>(o),
                                     lse, reinterpret_cast<const __nv_bfloat16*>(dout),
-                                    reinterpret_cast<__nv_bfloat16*>(dqkv), delta, NB, B, T, H, dh, err,
+                                    reinterpret_cast<__nv_bfloat16*>(dqkv), delta, nullptr, NB, B, T, H, dh, err,
                                     reinterpret_cast<cudaStream_t>(stream));
   if (e == cudaSuccess) return IL_OK;
   return e == cudaErrorInvalidValue ? IL_ERR_INVALID_ARG : IL_ERR_CUDA;

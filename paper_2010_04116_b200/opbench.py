@@ -7,7 +7,7 @@ ops: logits (auxiliary head: vocabulary projection with the softmax / exp(logit)
 contraction with a plain bf16 output), fc1 (first MLP projection with the GELU epilogue and its two outputs),
 fc1_plain (the same contraction, bias and bf16 output only), dgelu (gradient through the second MLP projection,
 multiplied by the saved GELU derivative, with the bias-gradient column sums; dgelu_nosum without them; dgelu_plain
-the bare contraction), attn_fwd, attn_bwd (gradient batches = stacked
+the bare contraction), attn_fwd, attn_bwd (two kernels), attn_bwd_one (one sweep; gradient batches = stacked
 gradient streams x 8).
 """
 from __future__ import annotations
@@ -80,7 +80,7 @@ def main(argv):
             fn = lambda: il.op_gemm(R, N, K, dY, K, 0, W2, N, 1, 3, err, C_=out, ldc=N, aux=aux, ld_aux=N,
                                     aux_rows=R // 2, colsum=cs if which == "dgelu" else None, tile_blocks=TILE)
         _timeit(which, fn, 2.0 * R * N * K, iters, err)
-    elif which in ("attn_fwd", "attn_bwd"):
+    elif which in ("attn_fwd", "attn_bwd", "attn_bwd_one"):
         B, T, H, dh = 8, 1024, 16, 64
         NB = int(argv[3]) if len(argv) > 3 else B
         d = H * dh
@@ -95,8 +95,12 @@ def main(argv):
             do = torch.randn(NB * T, d, device=DEV).to(torch.bfloat16)
             dqkv = torch.empty(NB * T, 3 * d, dtype=torch.bfloat16, device=DEV)
             delta = torch.empty(NB * H * T, device=DEV)
-            _timeit(which, lambda: il.op_attention_bwd(qkv, o, lse, do, dqkv, delta, NB, B, T, H, dh),
-                    2.5 * causal * NB / B, iters, err)
+            if which == "attn_bwd":
+                fn = lambda: il.op_attention_bwd(qkv, o, lse, do, dqkv, delta, NB, B, T, H, dh)
+            else:
+                acc = torch.empty(NB * T, d, device=DEV)
+                fn = lambda: il.op_attention_bwd_one_sweep(qkv, o, lse, do, dqkv, delta, acc, NB, B, T, H, dh, err_word=err)
+            _timeit(which, fn, 2.5 * causal * NB / B, iters, err)
     else:
         raise SystemExit(__doc__)
 

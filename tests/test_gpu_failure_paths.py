@@ -139,13 +139,13 @@ def test_growing_n_hands_back_the_superseded_scratch():
 def test_checkpoint_resume_gives_the_identical_next_update():
     """Parameters, Adam moments and the step counter moved to a fresh model give the same second update
     (compared on tensors whose gradients are summed in a fixed order; the others within 1e-6)."""
-    w, m, P, tok, tgt = _small()
+    w, m, P, tok, tgt = _small(attn_bwd="two_kernels")
     tok2, tgt2 = wl.draw_tokens(w, step=1)
     m2 = None
     try:
         m.train_step(tok, tgt, adamw=HP)
         m.sync()
-        m2 = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, 2, w.B, w.T)
+        m2 = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, 2, w.B, w.T, attn_bwd="two_kernels")
         for nm in m.names:
             m2.set_param(nm, m.get_param(nm))
             mm, vv, step = m.get_opt_state(nm)
@@ -174,7 +174,7 @@ def test_two_runs_of_a_step_are_bit_identical_where_sums_have_a_fixed_order():
     w = wl.Workload("det", K=3, Lc=1, d=128, H=2, F=256, V=64, T=128, B=6, n=2, zipf=True)   # few ids: long runs per token
     P = wl.draw_params(w)
     tok, tgt = wl.draw_tokens(w)
-    m = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, 2, w.B, w.T)
+    m = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, 2, w.B, w.T, attn_bwd="two_kernels")   # the one-sweep form sums dQ atomically
     try:
         m.set_params(P)
         runs = []
@@ -211,7 +211,7 @@ def test_pipeline_placement_on_one_device_reproduces_the_single_device_step(n, r
     tok, tgt = wl.draw_tokens(w)
     res = {}
     for placement in ("single", "pipeline"):
-        m = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, n, w.B, w.T, placement=placement)
+        m = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, n, w.B, w.T, placement=placement, attn_bwd="two_kernels")
         try:
             m.set_params(P)
             if rule != "sum":

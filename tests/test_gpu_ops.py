@@ -218,6 +218,45 @@ def test_attention_forward_backward(B, T, H, dh):
             assert _rel(gj[:, sl], refj[:, sl]) < 1.5e-2, (j, name)
 
 
+@pytest.mark.parametrize("B,T,H,dh,NB", [(2, 64, 2, 32, 2), (1, 200, 2, 64, 2), (2, 256, 3, 64, 4), (1, 1, 1, 64, 1),
+                                         (1, 129, 2, 64, 1), (2, 1024, 2, 64, 2), (1, 700, 1, 32, 3)])
+def test_attention_backward_one_sweep(B, T, H, dh, NB):
+    """dK, dV and dQ from a single recomputation of the scores (dQ summed over key tiles in an fp32 accumulator):
+    against the oracle, and against the two-kernel form (dK / dV take the same arithmetic path in both: equal bits)."""
+    rng = np.random.default_rng(7 * B + T + dh + NB)
+    d = H * dh
+    qkv_t, qkv = _bf16(rng.standard_normal((B * T, 3 * d)))
+    o = torch.zeros((B * T, d), dtype=torch.bfloat16, device=DEV)
+    lse = torch.zeros((B, H, T), dtype=torch.float32, device=DEV)
+    il.op_attention_fwd(qkv_t, o, lse, B, T, H, dh)
+    do_t, do = _bf16(rng.standard_normal((NB * T, d)))
+    two = torch.zeros((NB * T, 3 * d), dtype=torch.bfloat16, device=DEV)
+    delta = torch.zeros(NB * H * T, dtype=torch.float32, device=DEV)
+    il.op_attention_bwd(qkv_t, o, lse, do_t, two, delta, NB, B, T, H, dh)
+    err = torch.zeros(1, dtype=torch.int32, device=DEV)
+    for attempt in range(2):                      # twice: the accumulator holds the first call's values at the second
+        one = torch.full((NB * T, 3 * d), 3.0, dtype=torch.bfloat16, device=DEV)
+        acc = torch.full((NB * T, d), 5.0, dtype=torch.float32, device=DEV) if attempt == 0 else acc
+        il.op_attention_bwd_one_sweep(qkv_t, o, lse, do_t, one, delta, acc, NB, B, T, H, dh, err_word=err)
+        torch.cuda.synchronize()
+        assert int(err.item()) == 0
+        got = one.float().cpu().numpy()
+        assert np.isfinite(got).all()
+        for j in range(NB):
+            refj = orc.attention_bwd(do[j * T:(j + 1) * T], qkv[(j % B) * T:(j % B + 1) * T], 1, T, H)
+            gj = got[j * T:(j + 1) * T]
+            for part, name in enumerate(["dq", "dk", "dv"]):
+                sl = slice(part * d, (part + 1) * d)
+                if np.linalg.norm(refj[:, sl]) < 1e-9:             # a single token: dQ and dK vanish identically
+                    assert np.max(np.abs(gj[:, sl])) < 1e-5, (attempt, j, name)
+                else:
+                    assert _rel(gj[:, sl], refj[:, sl]) < 1.5e-2, (attempt, j, name)
+        ref2 = two.float().cpu().numpy()
+        assert np.array_equal(got[:, d:], ref2[:, d:])                 # dK, dV
+        if T > 1:
+            assert _rel(got[:, :d], ref2[:, :d]) < 4e-3                # dQ: the same values up to the order of the sum
+
+
 @pytest.mark.parametrize("rows,d", [(64, 128), (1000, 768), (333, 2560)])
 def test_layernorm_forward_backward(rows, d):
     rng = np.random.default_rng(rows + d)
