@@ -200,7 +200,7 @@ def bench_pipeline(args, w, n, metric, cfg_desc):
     use_adamw = bool(w.adamw and not args.no_adamw)
     hp = dict(lr=1e-4, beta1=0.9, beta2=0.98, eps=1e-9, weight_decay=w.weight_decay) if use_adamw else None
     m = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, n, w.B // w.M, w.T, device=0, head_layers=w.Lh, head_mode=args.head_mode,
-              placement="pipeline", devices=devices)
+              placement="pipeline", devices=devices, attn_bwd=args.attn_bwd)
     if w.rule != "sum":
         m.set_rule(w.rule)
     if w.M > 1:
@@ -287,6 +287,7 @@ def main():
     ap.add_argument("--no-adamw", action="store_true")
     ap.add_argument("--head-mode", default="stored", choices=["stored", "recompute"])
     ap.add_argument("--placement", default="replicas", choices=["replicas", "pipeline"])
+    ap.add_argument("--attn-bwd", default="one_sweep", choices=["one_sweep", "two_kernels"])
     ap.add_argument("--no-head-mode-comparison", action="store_true")
     args = ap.parse_args()
 
@@ -299,7 +300,7 @@ def main():
     extra = (f", {w.Lh} blocks per auxiliary head, rule={w.rule}, {w.M} micro-batches per update"
              if (w.Lh or w.M > 1 or w.rule != "sum") else "")
     cfg_desc = {"workload": f"{w.name}: {w.K}x{w.Lc} layers, d={w.d}, H={w.H}, F={w.F}, T={w.T}, B={w.B}, V={w.V}, "
-                            f"n={n}, adamw={bool(w.adamw and not args.no_adamw)}{extra}, head_mode={args.head_mode}",
+                            f"n={n}, adamw={bool(w.adamw and not args.no_adamw)}{extra}, head_mode={args.head_mode}, attn_bwd={args.attn_bwd}",
                 "global_batch": w.B * max(world, 1), "seq_len": w.T, "parallelism": f"replicas x{max(world, 1)}",
                 "l2": "inputs larger than L2 (each step streams several GB of weights and activations)"}
 
@@ -334,7 +335,7 @@ def main():
     use_adamw = bool(w.adamw and not args.no_adamw)
     hp = dict(lr=1e-4, beta1=0.9, beta2=0.98, eps=1e-9, weight_decay=w.weight_decay) if use_adamw else None
     m = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, n, w.B // w.M, w.T, device=local_rank, head_layers=w.Lh,
-              head_mode=args.head_mode)
+              head_mode=args.head_mode, attn_bwd=args.attn_bwd)
     if w.rule != "sum":
         m.set_rule(w.rule)
     if w.M > 1:
@@ -450,7 +451,8 @@ def main():
         # the other head mode on the same workload: step time and device memory side by side
         other = "recompute" if args.head_mode == "stored" else "stored"
         torch.cuda.empty_cache()
-        m = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, n, w.B // w.M, w.T, device=local_rank, head_layers=w.Lh, head_mode=other)
+        m = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, n, w.B // w.M, w.T, device=local_rank, head_layers=w.Lh, head_mode=other,
+                  attn_bwd=args.attn_bwd)
         if w.rule != "sum":
             m.set_rule(w.rule)
         if w.M > 1:

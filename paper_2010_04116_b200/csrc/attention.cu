@@ -796,7 +796,7 @@ __global__ void __launch_bounds__(256) attn_bwd_dq_tc_kernel(const __grid_consta
 // products for five); here a CTA owns 128 keys, sweeps the queries in blocks of 128 and produces dV, dK and its
 // share of dQ from one recomputation of S^T and dP^T:
 //   S^T, dP^T   tcgen05.mma M128 (keys) N64 per 64-query half -> TMEM, two halves per step
-//   P^T, dS^T   threads (two per key row, 32 columns each) recompute the probabilities from the saved
+//   P^T, dS^T   threads (four per key row, 16 columns of a half each) recompute the probabilities from the saved
 //               log-sum-exp, round to bf16 and store the packed pairs back over the score columns
 //   dV += P^T dO, dK += dS^T Q      A operand read from those TMEM columns, accumulated over the whole sweep
 //   dQ_blk = dS K                   needs dS with the queries as rows: the same threads also write their dS values
@@ -804,10 +804,14 @@ __global__ void __launch_bounds__(256) attn_bwd_dq_tc_kernel(const __grid_consta
 //                                   rows, one row per key); the product lands in one of two TMEM buffers and is
 //                                   added to an fp32 [rows, d] accumulator in global memory with red.add (every
 //                                   key tile of a (sequence, head) contributes to the same query rows)
-// Roles: warps 0-7 recompute / convert / flush dQ, warp 8 issues every MMA, warp 9 feeds the Q / dO ring by TMA
-// and the per-query lse / delta vectors by plain loads.  The halves give the pipeline its overlap: while the
-// threads work on one half of the step, the tensor pipe runs the other half's products and the next step's
-// scores for the half just finished.  One CTA per SM (all 512 TMEM columns, ~195 KB of shared memory).
+// Roles: warps 0-15 recompute and convert (four threads per key row), warps 16-19 add finished dQ blocks to the
+// global accumulator and store an item's dV / dK, warps 20 and 21 issue the MMAs (scores and dQ / dV and dK: a
+// single thread issues small MMAs no faster than one per ~54 cycles), warp 22 feeds the Q / dO ring by TMA and the
+// per-query lse / delta vectors by plain loads.  The halves
+// give the pipeline its overlap: while the threads work on one half of the step, the tensor pipe runs the other
+// half's products and the next step's scores for the half just finished.  One CTA per SM (all 512 TMEM columns,
+// ~195 KB of shared memory), persistent: a CTA walks a list of (key tile, sequence, head) items, and the loads and
+// scores of an item start while the previous item's dV / dK are still being written out.
 // The sum over key tiles in dQ is made by floating-point atomics: its order, and with it the last bit of dQ,
 // depends on scheduling.  Every wait is bounded.
 // ------------------------------------------------------------------------------------------------
@@ -822,12 +826,30 @@ struct FusedCfg {
   static constexpr int C_S = 0, C_DP = 128, C_DV = 256, C_DK = 320, C_DQ = 384;
 };
 
+constexpr int FUSED_THREADS = 768;   // warps 0-15 recompute, 16-19 flush dQ and store dV / dK, 20-22 issue MMAs, 23 loads
+constexpr int FUSED_RW = 16;         // recompute warps: four threads per key row, 16 query columns of a half each
+
+// Work item = (key tile, gradient sequence, head).  Items are numbered key tile first, so the long sweeps (key tile
+// 0 sees every query block) come first; CTA c takes items c, c + gridDim.x, ...  Every role walks the same list and
+// counts the same global step number g, from which ring stages and barrier parities follow.
+struct FusedItem { int kb, nb, h, bs, nit; };
+__device__ __forceinline__ FusedItem fused_item(int item, int nbh, int H, int B, int nq) {
+  FusedItem w;
+  w.kb = item / nbh;
+  const int r = item - w.kb * nbh;
+  w.nb = r / H;
+  w.h = r - w.nb * H;
+  w.bs = w.nb % B;
+  w.nit = nq - w.kb;                    // query blocks kb .. nq-1 see these keys
+  return w;
+}
+
 template <int DH>
-__global__ void __launch_bounds__(320, 1) attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmRow,     // qkv, 128-row box
-                                                                const __grid_constant__ CUtensorMap tmdO,      // dout, 128-row box
-                                                                const float* __restrict__ lse, const float* __restrict__ delta,
-                                                                bf16* __restrict__ dqkv, float* __restrict__ dq_acc, int B,
-                                                                int T, int H, float scale, unsigned* err) {
+__global__ void __launch_bounds__(FUSED_THREADS, 1) attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmRow,     // qkv, 128-row box
+                                                                          const __grid_constant__ CUtensorMap tmdO,      // dout, 128-row box
+                                                                          const float* __restrict__ lse, const float* __restrict__ delta,
+                                                                          bf16* __restrict__ dqkv, float* __restrict__ dq_acc, int NB,
+                                                                          int B, int T, int H, float scale, unsigned* err) {
   using C = FusedCfg<DH>;
   constexpr int NST = C::NST;
   extern __shared__ uint8_t smem_raw[];
@@ -841,42 +863,48 @@ __global__ void __launch_bounds__(320, 1) attn_bwd_fused_kernel(const __grid_con
   const uint32_t sVec = sDS + 2 * C::DS_BYTES;                             // NST x (lse2[128], delta[128])
   const uint32_t bars = sVec + NST * C::VEC_BYTES;
   // barriers (8 bytes each)
-  const uint32_t bar_kv = bars, bar_acc = bars + 8, bar_drain = bars + 16;
-  auto bar_full = [&](int st) { return bars + 24 + 8 * st; };
-  auto bar_empty = [&](int st) { return bars + 24 + 8 * (NST + st); };
-  auto bar_s = [&](int x) { return bars + 24 + 8 * (2 * NST + x); };          // scores of half x ready
-  auto bar_p = [&](int x) { return bars + 24 + 8 * (2 * NST + 2 + x); };      // P^T / dS^T of half x written
-  auto bar_dq = [&](int b) { return bars + 24 + 8 * (2 * NST + 4 + b); };     // dQ buffer b complete
-  auto bar_dqfree = [&](int b) { return bars + 24 + 8 * (2 * NST + 6 + b); }; // dQ buffer b flushed
+  const uint32_t bar_kv = bars, bar_kvfree = bars + 8, bar_acc = bars + 16, bar_accfree = bars + 24, bar_ds = bars + 32, bar_init = bars + 40;
+  auto bar_drain = [&](int t) { return bars + 48 + 8 * t; };                   // one per issuing thread
+  auto bar_full = [&](int st) { return bars + 72 + 8 * st; };
+  auto bar_empty = [&](int st) { return bars + 72 + 8 * (NST + st); };
+  auto bar_s = [&](int x) { return bars + 72 + 8 * (2 * NST + x); };           // scores of half x ready
+  auto bar_p = [&](int x) { return bars + 72 + 8 * (2 * NST + 2 + x); };       // P^T / dS^T of half x in tensor memory
+  auto bar_dq = [&](int b) { return bars + 72 + 8 * (2 * NST + 4 + b); };      // dQ buffer b complete
+  auto bar_dqfree = [&](int b) { return bars + 72 + 8 * (2 * NST + 6 + b); };  // dQ buffer b flushed
+  auto bar_vec = [&](int st) { return bars + 72 + 8 * (2 * NST + 8 + st); };   // lse / delta vectors of stage st written
   uint8_t* gen = smem_raw + (base - smem_u32(smem_raw));
   float* s_vec = reinterpret_cast<float*>(gen + (sVec - base));
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int kb = blockIdx.x;                                       // key tile; tile 0 has the longest sweep and runs first
-  const int nb = blockIdx.y / H, h = blockIdx.y % H;
-  const int bs = nb % B;
   const int d = H * DH;
   const int nq = (T + TQ - 1) / TQ;
-  const int nit = nq - kb;                                         // query blocks kb .. nq-1 see these keys
+  const int nbh = NB * H;
+  const int nitems = nq * nbh;
   volatile int* abortp = &abort_flag;
 
   if (tid == 0) {
     abort_flag = 0;
     mbar_init(bar_kv, 1);
-    mbar_init(bar_acc, 1);
-    mbar_init(bar_drain, 1);
-    for (int st = 0; st < NST; ++st) { mbar_init(bar_full(st), 1); mbar_init(bar_empty(st), 1); }
+    mbar_init(bar_kvfree, 3);            // the three issuing threads
+    mbar_init(bar_acc, 2);               // the two half threads
+    mbar_init(bar_init, 1);
+    mbar_init(bar_accfree, 4);           // one arrival per flush warp
+    mbar_init(bar_ds, FUSED_RW);         // one arrival per recompute warp
+    mbar_init(bar_drain(0), 1);
+    mbar_init(bar_drain(1), 1);
+    mbar_init(bar_drain(2), 1);
+    for (int st = 0; st < NST; ++st) { mbar_init(bar_full(st), 1); mbar_init(bar_empty(st), 2); mbar_init(bar_vec(st), 1); }
     for (int x = 0; x < 2; ++x) {
       mbar_init(bar_s(x), 1);
-      mbar_init(bar_p(x), 8);            // one arrival per recompute warp
+      mbar_init(bar_p(x), FUSED_RW);
       mbar_init(bar_dq(x), 1);
-      mbar_init(bar_dqfree(x), 8);
+      mbar_init(bar_dqfree(x), 4);       // one arrival per flush warp
     }
     fence_mbar_init();
     tma_prefetch_desc(&tmRow);
     tma_prefetch_desc(&tmdO);
   }
-  if (warp == 8) {
+  if (warp == 20) {
     tmem_alloc(smem_u32(&tmem_base_smem), 512);
     tmem_relinquish();
   }
@@ -887,49 +915,69 @@ __global__ void __launch_bounds__(320, 1) attn_bwd_fused_kernel(const __grid_con
   const float c2 = scale * IL_LOG2E;
   int fail = 0;
 
-  if (warp == 9) {
+  if (warp == 23) {
     // ---------------------------------------------------------------- loads
-    if (lane == 0) {
-      mbar_expect_tx(bar_kv, 2 * C::ROW_BYTES);
-      tma_load_4d(sK, &tmRow, 0, H + h, kb * TQ, bs, bar_kv);
-      tma_load_4d(sV, &tmRow, 0, 2 * H + h, kb * TQ, bs, bar_kv);
-    }
-    const float* lse_b = lse + ((size_t)bs * H + h) * T;
-    const float* del_b = delta + ((size_t)nb * H + h) * T;
-    for (int it = 0; it < nit; ++it) {
-      const int st = it % NST, j = kb + it;
-      int ok = 1;
-      if (lane == 0 && it >= NST) ok = mbar_wait(bar_empty(st), (uint32_t)(it / NST - 1) & 1u, abortp) ? 1 : 0;
-      ok = __shfl_sync(0xffffffffu, ok, 0);
-      if (!ok) { fail = 1; abort_flag = 1; break; }
-      float* vec = s_vec + st * (2 * TQ);
+    int g = 0, n_item = 0;
+    for (int item = blockIdx.x; item < nitems && !fail; item += gridDim.x, ++n_item) {
+      const FusedItem w = fused_item(item, nbh, H, B, nq);
+      const float* lse_b = lse + ((size_t)w.bs * H + w.h) * T;
+      const float* del_b = delta + ((size_t)w.nb * H + w.h) * T;
+      for (int it = 0; it < w.nit; ++it) {
+        const int gs = g + it, st = gs % NST, j = w.kb + it;
+        int ok = 1;
+        if (lane == 0 && gs >= NST) ok = mbar_wait(bar_empty(st), (uint32_t)(gs / NST - 1) & 1u, abortp) ? 1 : 0;
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) { fail = 1; abort_flag = 1; break; }
+        // the tiles first (their latency is the longer one), then the step's lse / delta vectors by plain loads,
+        // published on a barrier of their own
+        if (lane == 0) {
+          mbar_expect_tx(bar_full(st), 2 * C::ROW_BYTES);
+          tma_load_4d(sQ0 + st * STAGE, &tmRow, 0, w.h, j * TQ, w.bs, bar_full(st));
+          tma_load_4d(sQ0 + st * STAGE + C::ROW_BYTES, &tmdO, 0, w.h, j * TQ, w.nb, bar_full(st));
+        }
+        float* vec = s_vec + st * (2 * TQ);
 #pragma unroll
-      for (int q4 = 0; q4 < 4; ++q4) {
-        const int q = j * TQ + q4 * 32 + lane;
-        vec[q4 * 32 + lane] = q < T ? lse_b[q] * IL_LOG2E : 0.f;
-        vec[TQ + q4 * 32 + lane] = q < T ? del_b[q] : 0.f;
+        for (int q4 = 0; q4 < 4; ++q4) {
+          const int q = j * TQ + q4 * 32 + lane;
+          vec[q4 * 32 + lane] = q < T ? lse_b[q] * IL_LOG2E : 0.f;
+          vec[TQ + q4 * 32 + lane] = q < T ? del_b[q] : 0.f;
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_vec(st));                   // its release publishes the warp's stores
+        if (it == 0) {
+          // the item's K and V (after its first query block, which does not depend on the previous item): their
+          // buffers are free once the previous item's last products that read them have retired
+          int ok2 = 1;
+          if (lane == 0 && n_item > 0) ok2 = mbar_wait(bar_kvfree, (uint32_t)(n_item - 1) & 1u, abortp) ? 1 : 0;
+          ok2 = __shfl_sync(0xffffffffu, ok2, 0);
+          if (!ok2) { fail = 1; abort_flag = 1; break; }
+          if (lane == 0) {
+            mbar_expect_tx(bar_kv, 2 * C::ROW_BYTES);
+            tma_load_4d(sK, &tmRow, 0, H + w.h, w.kb * TQ, w.bs, bar_kv);
+            tma_load_4d(sV, &tmRow, 0, 2 * H + w.h, w.kb * TQ, w.bs, bar_kv);
+          }
+        }
       }
-      __syncwarp();
-      if (lane == 0) {
-        mbar_expect_tx(bar_full(st), 2 * C::ROW_BYTES);          // its release also publishes the warp's vector stores
-        tma_load_4d(sQ0 + st * STAGE, &tmRow, 0, h, j * TQ, bs, bar_full(st));
-        tma_load_4d(sQ0 + st * STAGE + C::ROW_BYTES, &tmdO, 0, h, j * TQ, nb, bar_full(st));
-      }
+      g += w.nit;
     }
-  } else if (warp == 8) {
-    // ---------------------------------------------------------------- MMA issue
+  } else if (warp == 20 || warp == 21) {
+    // ---------------------------------------------------------------- MMA issue, one thread per half x of the query block
+    // A thread issues small MMAs no faster than one per ~54 cycles, and every hand-over between threads costs a
+    // commit / barrier round trip of several hundred cycles.  So each half has its own issuing thread that does, in
+    // program order (the tensor pipe keeps one thread's MMAs in order), dV += P^T(x) dO(x), dK += dS^T(x) Q(x) and
+    // then the next step's S^T(x), dP^T(x) into the score columns those products have just read.  Both threads add
+    // into the same dV / dK accumulators (the pipe executes one MMA at a time; the order in which the two halves are
+    // added is not fixed).
     if (lane == 0) {
+      const int x = warp - 20;
       constexpr uint32_t idesc_s = make_idesc_bf16(TQ, TK, 0, 0);          // S^T / dP^T half: M128 N64, both K-major
       constexpr uint32_t idesc_g = make_idesc_bf16(TQ, DH, 0, 1);          // dV / dK: A from TMEM, B MN-major
-      constexpr uint32_t idesc_q = make_idesc_bf16(TQ, DH, 1, 1);          // dQ: A = dS (MN-major), B = K (MN-major)
       const SmemDescBase dk_k = make_smem_desc_base(sK, 16, 1024), dv_k = make_smem_desc_base(sV, 16, 1024);
-      const SmemDescBase dk_mn = make_smem_desc_base(sK, TQ * 128, 1024);
       const SmemDescBase dq_k = make_smem_desc_base(sQ0, 16, 1024), ddo_k = make_smem_desc_base(sQ0 + C::ROW_BYTES, 16, 1024);
       const SmemDescBase dq_mn = make_smem_desc_base(sQ0, TQ * 128, 1024), ddo_mn = make_smem_desc_base(sQ0 + C::ROW_BYTES, TQ * 128, 1024);
-      const SmemDescBase dds_mn = make_smem_desc_base(sDS, TQ * 128, 1024);
       bool ok = true;
-      // scores of half x of the step held in stage st: rows 64x .. 64x+63 of the Q / dO tiles (8 KB further)
-      auto issue_scores = [&](int st, int x) {
+      // scores of this half of the step held in stage st: rows 64x .. 64x+63 of the Q / dO tiles (8 KB further)
+      auto issue_scores = [&](int st) {
         const uint32_t so = (uint32_t)st * STAGE + (uint32_t)x * (TK * 128);
 #pragma unroll
         for (int ks = 0; ks < DH / 16; ++ks) {
@@ -938,17 +986,23 @@ __global__ void __launch_bounds__(320, 1) attn_bwd_fused_kernel(const __grid_con
         }
         umma_commit(bar_s(x));
       };
-      if (!mbar_wait(bar_kv, 0, abortp)) ok = false;
-      if (ok && !mbar_wait(bar_full(0), 0, abortp)) ok = false;
-      if (ok) {
+      int g = 0, n_item = 0;
+      for (int item = blockIdx.x; item < nitems && ok; item += gridDim.x, ++n_item) {
+        const FusedItem w = fused_item(item, nbh, H, B, nq);
+        // first step of the item: its scores need the item's K / V and the step's Q / dO (the score columns are free:
+        // this thread's own last products of the previous item come before them in the pipe)
+        if (!mbar_wait(bar_kv, (uint32_t)n_item & 1u, abortp)) { ok = false; break; }
+        if (!mbar_wait(bar_full(g % NST), (uint32_t)(g / NST) & 1u, abortp)) { ok = false; break; }
         tc_fence_after();
-        issue_scores(0, 0);
-        issue_scores(0, 1);
-      }
-      for (int it = 0; it < nit && ok; ++it) {
-        const int st = it % NST, b = it & 1;
-        const uint32_t ph = (uint32_t)it & 1u;
-        for (int x = 0; x < 2 && ok; ++x) {
+        issue_scores(g % NST);
+        // the accumulators still hold the previous item's dV / dK until they have been stored; the half-1 thread also
+        // lets the half-0 thread's first products (which overwrite instead of adding) go first
+        if (n_item > 0 && !mbar_wait(bar_accfree, (uint32_t)(n_item - 1) & 1u, abortp)) { ok = false; break; }
+        if (x == 1 && !mbar_wait(bar_init, (uint32_t)n_item & 1u, abortp)) { ok = false; break; }
+        for (int it = 0; it < w.nit && ok; ++it) {
+          const int gs = g + it, st = gs % NST, st1 = (gs + 1) % NST;
+          const uint32_t ph = (uint32_t)gs & 1u;
+          const bool more = it + 1 < w.nit;
           if (!mbar_wait(bar_p(x), ph, abortp)) { ok = false; break; }
           tc_fence_after();
           // dV += P^T(x) dO(x), dK += dS^T(x) Q(x): contraction over the half's 64 queries (MN-major B: 16 queries = 2048 B)
@@ -956,190 +1010,221 @@ __global__ void __launch_bounds__(320, 1) attn_bwd_fused_kernel(const __grid_con
 #pragma unroll
           for (int ks = 0; ks < TK / 16; ++ks) {
             const uint32_t acc = (it | x | ks) ? 1u : 0u;
-            umma_bf16_ts(tmem_base + C::C_DV, tmem_base + C::C_S + 64 * x + packed_col(ks), desc_at(ddo_mn, so + ks * 2048), idesc_g, acc);
-            umma_bf16_ts(tmem_base + C::C_DK, tmem_base + C::C_DP + 64 * x + packed_col(ks), desc_at(dq_mn, so + ks * 2048), idesc_g, acc);
+            umma_bf16_ts(tmem_base + C::C_DV, tmem_base + C::C_S + 64 * x + 16 * ks, desc_at(ddo_mn, so + ks * 2048), idesc_g, acc);
+            umma_bf16_ts(tmem_base + C::C_DK, tmem_base + C::C_DP + 64 * x + 16 * ks, desc_at(dq_mn, so + ks * 2048), idesc_g, acc);
           }
-          if (x == 1) {
-            umma_commit(bar_empty(st));                     // the stage's tiles have been read once these retire
-            // dQ(it) = dS K over this tile's 128 keys, into buffer b (free once the flush of step it-2 is done)
-            if (it >= 2 && !mbar_wait(bar_dqfree(b), (uint32_t)((it >> 1) - 1) & 1u, abortp)) { ok = false; break; }
+          if (x == 0 && it == 0) umma_commit(bar_init);
+          umma_commit(bar_empty(st));                       // (one of two arrivals) the stage's tiles have been read by this half
+          if (more) {
+            if (!mbar_wait(bar_full(st1), (uint32_t)((gs + 1) / NST) & 1u, abortp)) { ok = false; break; }
             tc_fence_after();
-#pragma unroll
-            for (int ks = 0; ks < TQ / 16; ++ks)
-              umma_bf16(tmem_base + C::C_DQ + 64 * b, desc_at(dds_mn, (uint32_t)b * C::DS_BYTES + ks * 2048),
-                        desc_at(dk_mn, ks * 2048), idesc_q, ks ? 1u : 0u);
-            umma_commit(bar_dq(b));
-          }
-          if (it + 1 < nit) {
-            // next step's scores for the half just consumed (the pipe runs them after the products above)
-            const int st1 = (it + 1) % NST;
-            if (x == 0 && !mbar_wait(bar_full(st1), (uint32_t)((it + 1) / NST) & 1u, abortp)) { ok = false; break; }
-            tc_fence_after();
-            issue_scores(st1, x);
+            issue_scores(st1);
+          } else {
+            umma_commit(bar_kvfree);                        // (one of three) nothing of this item reads K / V from this thread any more
+            umma_commit(bar_acc);                           // (one of two) this half's share of dV / dK is complete
           }
         }
+        g += w.nit;
       }
-      if (ok) umma_commit(bar_acc);
-      else { fail = 1; abort_flag = 1; }
+      if (!ok) { fail = 1; abort_flag = 1; }
+      umma_commit(bar_drain(x));                   // every MMA this thread issued has retired before TMEM goes
+      int never = 0;
+      mbar_wait(bar_drain(x), 0, &never);
     }
-  } else {
-    // ---------------------------------------------------------------- recompute, convert, flush (warps 0-7)
-    const int r = tid & 127, hf = tid >> 7;
-    const int key = kb * TQ + r;
-    const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
-    auto flush_dq = [&](int it) -> bool {        // add dQ of step `it` to the global accumulator
-      const int b = it & 1;
-      int got = 1;
-      if (lane == 0) got = mbar_wait(bar_dq(b), (uint32_t)(it >> 1) & 1u, abortp) ? 1 : 0;
-      got = __shfl_sync(0xffffffffu, got, 0);
-      if (!got) return false;
-      tc_fence_after();
-      const int q = (kb + it) * TQ + r;
-      float* dst = dq_acc + ((size_t)nb * T + q) * d + h * DH;
-      if constexpr (DH == 64) {
-        uint32_t rr[32];
-        tmem_ld_32x32(t_lane + C::C_DQ + 64 * b + 32 * hf, rr);
-        tmem_ld_wait();
-        if (q < T) {
+  } else if (warp == 22) {
+    // ---------------------------------------------------------------- MMA issue, third thread: dQ
+    if (lane == 0) {
+      constexpr uint32_t idesc_q = make_idesc_bf16(TQ, DH, 1, 1);          // A = dS (MN-major), B = K (MN-major)
+      const SmemDescBase dk_mn = make_smem_desc_base(sK, TQ * 128, 1024);
+      const SmemDescBase dds_mn = make_smem_desc_base(sDS, TQ * 128, 1024);
+      bool ok = true;
+      int g = 0, n_item = 0;
+      for (int item = blockIdx.x; item < nitems && ok; item += gridDim.x, ++n_item) {
+        const FusedItem w = fused_item(item, nbh, H, B, nq);
+        if (!mbar_wait(bar_kv, (uint32_t)n_item & 1u, abortp)) { ok = false; break; }     // this item's K is in place
+        for (int it = 0; it < w.nit && ok; ++it) {
+          const int gs = g + it, b = gs & 1;
+          // dQ(step) = dS K over this tile's 128 keys: both halves of dS are in shared memory (bar_ds; the item's K
+          // arrived before the scores that dS came from), buffer b of the accumulator is free once the flush of
+          // step gs-2 is done
+          if (!mbar_wait(bar_ds, (uint32_t)gs & 1u, abortp)) { ok = false; break; }
+          if (gs >= 2 && !mbar_wait(bar_dqfree(b), (uint32_t)((gs >> 1) - 1) & 1u, abortp)) { ok = false; break; }
+          tc_fence_after();
 #pragma unroll
-          for (int i = 0; i < 32; i += 4)
-            red_add_f32x4(dst + 32 * hf + i, make_float4(__uint_as_float(rr[i]), __uint_as_float(rr[i + 1]),
-                                                         __uint_as_float(rr[i + 2]), __uint_as_float(rr[i + 3])));
+          for (int ks = 0; ks < TQ / 16; ++ks)
+            umma_bf16(tmem_base + C::C_DQ + 64 * b, desc_at(dds_mn, (uint32_t)b * C::DS_BYTES + ks * 2048), desc_at(dk_mn, ks * 2048),
+                      idesc_q, ks ? 1u : 0u);
+          umma_commit(bar_dq(b));
+          if (it + 1 == w.nit) umma_commit(bar_kvfree);      // (one of three)
         }
-      } else {   // DH == 32: 16 columns per thread
-        uint32_t rr[16];
-        tmem_ld_32x16(t_lane + C::C_DQ + 64 * b + 16 * hf, rr);
-        tmem_ld_wait();
-        if (q < T) {
+        g += w.nit;
+      }
+      if (!ok) { fail = 1; abort_flag = 1; }
+      umma_commit(bar_drain(2));
+      int never = 0;
+      mbar_wait(bar_drain(2), 0, &never);
+    }
+  } else if (warp >= 16 && warp < 20) {
+    // ---------------------------------------------------------------- dQ flush and dV / dK store (warps 16-19: thread = row)
+    const int r = tid - 512;
+    const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+    int g = 0, n_item = 0;
+    for (int item = blockIdx.x; item < nitems && !fail; item += gridDim.x, ++n_item) {
+      const FusedItem w = fused_item(item, nbh, H, B, nq);
+      for (int it = 0; it < w.nit; ++it) {
+        const int gs = g + it, b = gs & 1;
+        int got = 1;
+        if (lane == 0) got = mbar_wait(bar_dq(b), (uint32_t)(gs >> 1) & 1u, abortp) ? 1 : 0;
+        got = __shfl_sync(0xffffffffu, got, 0);
+        if (!got) { fail = 1; abort_flag = 1; break; }
+        tc_fence_after();
+        const int q = (w.kb + it) * TQ + r;
+        float* dst = dq_acc + ((size_t)w.nb * T + q) * d + w.h * DH;
 #pragma unroll
-          for (int i = 0; i < 16; i += 4)
-            red_add_f32x4(dst + 16 * hf + i, make_float4(__uint_as_float(rr[i]), __uint_as_float(rr[i + 1]),
-                                                         __uint_as_float(rr[i + 2]), __uint_as_float(rr[i + 3])));
+        for (int c0 = 0; c0 < DH; c0 += 32) {
+          uint32_t rr[32];
+          tmem_ld_32x32(t_lane + C::C_DQ + 64 * b + c0, rr);
+          tmem_ld_wait();
+          if (q < T) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 4)
+              red_add_f32x4(dst + c0 + i, make_float4(__uint_as_float(rr[i]), __uint_as_float(rr[i + 1]), __uint_as_float(rr[i + 2]),
+                                                      __uint_as_float(rr[i + 3])));
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_dqfree(b));
+      }
+      if (fail) break;
+      g += w.nit;
+      // the item's dV and dK: this thread's key row, scaled and rounded to bf16
+      {
+        int got = 1;
+        if (lane == 0) got = mbar_wait(bar_acc, (uint32_t)n_item & 1u, abortp) ? 1 : 0;
+        got = __shfl_sync(0xffffffffu, got, 0);
+        if (!got) { fail = 1; abort_flag = 1; break; }
+      }
+      tc_fence_after();
+      const int key = w.kb * TQ + r;
+      bf16* rowp = dqkv + ((size_t)w.nb * T + key) * (3 * d) + w.h * DH;
+#pragma unroll
+      for (int which = 0; which < 2; ++which) {
+        bf16* dst = rowp + (which == 0 ? 2 * d : d);
+        const float f = which == 0 ? 1.0f : scale;
+        const uint32_t tcol = t_lane + (which == 0 ? C::C_DV : C::C_DK);
+#pragma unroll
+        for (int c0 = 0; c0 < DH; c0 += 32) {
+          uint32_t rr[32];
+          tmem_ld_32x32(tcol + c0, rr);
+          tmem_ld_wait();
+          if (key < T) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 8) {
+              uint4 pk;
+              pk.x = pack_bf16x2(__uint_as_float(rr[i]) * f, __uint_as_float(rr[i + 1]) * f);
+              pk.y = pack_bf16x2(__uint_as_float(rr[i + 2]) * f, __uint_as_float(rr[i + 3]) * f);
+              pk.z = pack_bf16x2(__uint_as_float(rr[i + 4]) * f, __uint_as_float(rr[i + 5]) * f);
+              pk.w = pack_bf16x2(__uint_as_float(rr[i + 6]) * f, __uint_as_float(rr[i + 7]) * f);
+              *reinterpret_cast<uint4*>(dst + c0 + i) = pk;
+            }
+          }
         }
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_dqfree(b));
-      return true;
-    };
-    for (int it = 0; it < nit && !fail; ++it) {
-      const int st = it % NST, b = it & 1, j = kb + it;
-      const uint32_t ph = (uint32_t)it & 1u;
-      const float* vec = s_vec + st * (2 * TQ);
-      {   // the stage's lse / delta vectors were published with its "full" barrier (long complete by now)
-        int got = 1;
-        if (lane == 0) got = mbar_wait(bar_full(st), (uint32_t)(it / NST) & 1u, abortp) ? 1 : 0;
-        got = __shfl_sync(0xffffffffu, got, 0);
-        if (!got) { fail = 1; abort_flag = 1; break; }
-      }
-      const bool diag = (j == kb);                       // some queries of this block precede some keys of this CTA
-      const bool tail = (j * TQ + TQ > T);
-      for (int x = 0; x < 2; ++x) {
-        {
-          int got = 1;
-          if (lane == 0) got = mbar_wait(bar_s(x), ph, abortp) ? 1 : 0;
-          got = __shfl_sync(0xffffffffu, got, 0);
-          if (!got) { fail = 1; abort_flag = 1; break; }
-        }
-        tc_fence_after();
-        uint32_t r0[32], r1[32];
-        tmem_ld_32x32(t_lane + C::C_S + 64 * x + 32 * hf, r0);
-        tmem_ld_32x32(t_lane + C::C_DP + 64 * x + 32 * hf, r1);
-        tmem_ld_wait();
-        float p[32], ds[32];
-        const float4* lv = reinterpret_cast<const float4*>(vec + 64 * x + 32 * hf);
-        const float4* dv_ = reinterpret_cast<const float4*>(vec + TQ + 64 * x + 32 * hf);
-        const int qbase = j * TQ + 64 * x + 32 * hf;
-#pragma unroll
-        for (int i4 = 0; i4 < 8; ++i4) {
-          const float4 l4 = lv[i4], d4 = dv_[i4];
-          const float ll[4] = {l4.x, l4.y, l4.z, l4.w}, dd[4] = {d4.x, d4.y, d4.z, d4.w};
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const int i = 4 * i4 + e;
-            p[i] = ex2_fast(fmaf(__uint_as_float(r0[i]), c2, -ll[e]));
-            ds[i] = __uint_as_float(r1[i]) - dd[e];
-          }
-        }
-        if (diag || tail) {                              // uniform across the CTA
-#pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if (qbase + i < key || qbase + i >= T) p[i] = 0.f;
-        }
-#pragma unroll
-        for (int i = 0; i < 32; ++i) ds[i] *= p[i];
-        uint32_t pw[16], dw[16];
-        pack_row32(p, pw);
-        pack_row32(ds, dw);
-        tmem_st_32x16(t_lane + C::C_S + 64 * x + 32 * hf, pw);      // P^T over the first half of the columns this thread read
-        tmem_st_32x16(t_lane + C::C_DP + 64 * x + 32 * hf, dw);     // dS^T likewise
-        // dS as the A operand of dQ = dS K: row = key, 64 queries of half x = one swizzled 128-byte row of chunk x
-        {
-          const uint32_t rowaddr = sDS + (uint32_t)b * C::DS_BYTES + (uint32_t)x * (TQ * 128) + (uint32_t)r * 128;
-#pragma unroll
-          for (int t = 0; t < 4; ++t) {
-            const uint32_t unit = (uint32_t)(4 * hf + t) ^ (uint32_t)(r & 7);
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(rowaddr + unit * 16), "r"(dw[4 * t]), "r"(dw[4 * t + 1]),
-                         "r"(dw[4 * t + 2]), "r"(dw[4 * t + 3])
-                         : "memory");
-          }
-        }
-        tmem_st_wait();
-        fence_proxy_async();                               // the dS rows are read by the tensor pipe (async proxy)
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_p(x));
-        // between the halves: the previous step's dQ has long been complete
-        if (x == 0 && it > 0) {
-          if (!flush_dq(it - 1)) { fail = 1; abort_flag = 1; break; }
-        }
-      }
+      if (lane == 0) mbar_arrive(bar_accfree);               // the accumulators may be overwritten by the next item
     }
-    if (!fail && nit > 0) {
-      if (!flush_dq(nit - 1)) { fail = 1; abort_flag = 1; }
-    }
-    if (!fail) {
+  } else if (warp < FUSED_RW) {
+    // ---------------------------------------------------------------- recompute and convert (warps 0-15)
+    // thread (r, sub): key row r, query columns [16 sub, 16 sub + 16) of each 64-column half
+    const int r = tid & 127, sub = tid >> 7;
+    const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+    auto wait = [&](uint32_t bar, uint32_t parity) -> bool {     // lane 0 polls, the warp learns the outcome
       int got = 1;
-      if (lane == 0) got = mbar_wait(bar_acc, 0, abortp) ? 1 : 0;
-      got = __shfl_sync(0xffffffffu, got, 0);
-      if (!got) { fail = 1; abort_flag = 1; }
-      tc_fence_after();
-    }
-    if (!fail) {
-      // dV (first half of the threads) and dK (second half) of this CTA's 128 keys
-      bf16* rowp = dqkv + ((size_t)nb * T + key) * (3 * d) + h * DH;
-      bf16* dst = rowp + (hf == 0 ? 2 * d : d);
-      const float f = hf == 0 ? 1.0f : scale;
-      const uint32_t tcol = t_lane + (hf == 0 ? C::C_DV : C::C_DK);
+      if (lane == 0) got = mbar_wait(bar, parity, abortp) ? 1 : 0;
+      return __shfl_sync(0xffffffffu, got, 0) != 0;
+    };
+    int g = 0;
+    for (int item = blockIdx.x; item < nitems && !fail; item += gridDim.x) {
+      const FusedItem w = fused_item(item, nbh, H, B, nq);
+      const int key = w.kb * TQ + r;
+      for (int it = 0; it < w.nit && !fail; ++it) {
+        const int gs = g + it, st = gs % NST, b = gs & 1, j = w.kb + it;
+        const uint32_t ph = (uint32_t)gs & 1u;
+        const float* vec = s_vec + st * (2 * TQ);
+        // the stage's lse / delta vectors have their own barrier; the dS buffer of this step is free
+        // once the dQ product of step gs-2 has read it (both long complete by now)
+        if (!wait(bar_vec(st), (uint32_t)(gs / NST) & 1u)) { fail = 1; abort_flag = 1; break; }
+        if (gs >= 2 && !wait(bar_dq(b), (uint32_t)((gs >> 1) - 1) & 1u)) { fail = 1; abort_flag = 1; break; }
+        const bool diag = (it == 0);                       // some queries of this block precede some keys of this tile
+        const bool tail = (j * TQ + TQ > T);
+        for (int x = 0; x < 2; ++x) {
+          if (!wait(bar_s(x), ph)) { fail = 1; abort_flag = 1; break; }
+          tc_fence_after();
+          uint32_t r0[16], r1[16];
+          tmem_ld_32x16(t_lane + C::C_S + 64 * x + 16 * sub, r0);
+          tmem_ld_32x16(t_lane + C::C_DP + 64 * x + 16 * sub, r1);
+          tmem_ld_wait();
+          float p[16], ds[16];
+          const float4* lv = reinterpret_cast<const float4*>(vec + 64 * x + 16 * sub);
+          const float4* dv_ = reinterpret_cast<const float4*>(vec + TQ + 64 * x + 16 * sub);
+          const int qbase = j * TQ + 64 * x + 16 * sub;
 #pragma unroll
-      for (int c0 = 0; c0 < DH; c0 += 32) {
-        uint32_t rr[32];
-        tmem_ld_32x32(tcol + c0, rr);
-        tmem_ld_wait();
-        if (key < T) {
+          for (int i4 = 0; i4 < 4; ++i4) {
+            const float4 l4 = lv[i4], d4 = dv_[i4];
+            const float ll[4] = {l4.x, l4.y, l4.z, l4.w}, dd[4] = {d4.x, d4.y, d4.z, d4.w};
 #pragma unroll
-          for (int i = 0; i < 32; i += 8) {
-            uint4 pk;
-            pk.x = pack_bf16x2(__uint_as_float(rr[i]) * f, __uint_as_float(rr[i + 1]) * f);
-            pk.y = pack_bf16x2(__uint_as_float(rr[i + 2]) * f, __uint_as_float(rr[i + 3]) * f);
-            pk.z = pack_bf16x2(__uint_as_float(rr[i + 4]) * f, __uint_as_float(rr[i + 5]) * f);
-            pk.w = pack_bf16x2(__uint_as_float(rr[i + 6]) * f, __uint_as_float(rr[i + 7]) * f);
-            *reinterpret_cast<uint4*>(dst + c0 + i) = pk;
+            for (int e = 0; e < 4; ++e) {
+              const int i = 4 * i4 + e;
+              p[i] = ex2_fast(fmaf(__uint_as_float(r0[i]), c2, -ll[e]));
+              ds[i] = __uint_as_float(r1[i]) - dd[e];
+            }
+          }
+          if (diag || tail) {                              // uniform across the CTA
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+              if (qbase + i < key || qbase + i >= T) p[i] = 0.f;
+          }
+          uint32_t pw[8], dw[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            pw[i] = pack_bf16x2(p[2 * i], p[2 * i + 1]);
+            dw[i] = pack_bf16x2(ds[2 * i] * p[2 * i], ds[2 * i + 1] * p[2 * i + 1]);
+          }
+          tmem_st_32x8(t_lane + C::C_S + 64 * x + 16 * sub, pw);      // P^T over the first half of the columns this thread read
+          tmem_st_32x8(t_lane + C::C_DP + 64 * x + 16 * sub, dw);     // dS^T likewise
+          tmem_st_wait();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_p(x));                       // dV / dK of this half can go
+          // dS as the A operand of dQ = dS K: row = key, 64 queries of half x = one swizzled 128-byte row of chunk x
+          {
+            const uint32_t rowaddr = sDS + (uint32_t)b * C::DS_BYTES + (uint32_t)x * (TQ * 128) + (uint32_t)r * 128;
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+              const uint32_t unit = (uint32_t)(2 * sub + t) ^ (uint32_t)(r & 7);
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(rowaddr + unit * 16), "r"(dw[4 * t]), "r"(dw[4 * t + 1]),
+                           "r"(dw[4 * t + 2]), "r"(dw[4 * t + 3])
+                           : "memory");
+            }
+          }
+          if (x == 1) {
+            fence_proxy_async();                             // both halves' dS rows are read by the tensor pipe (async proxy)
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_ds);
           }
         }
       }
+      if (fail) break;
+      g += w.nit;
     }
   }
   fail = __syncthreads_or(fail);
-  if (tid == 8 * 32) {
-    if (fail && err) atomicExch(err, DEV_TIMEOUT_MMA);
-    umma_commit(bar_drain);                      // every MMA issued by this CTA has retired before TMEM goes
-    int never = 0;
-    mbar_wait(bar_drain, 0, &never);
-  }
+  if (tid == 0 && fail && err) atomicExch(err, DEV_TIMEOUT_MMA);
   tc_fence_before();
   __syncthreads();
-  if (warp == 8) {
+  if (warp == 20) {
     tc_fence_after();
     tmem_dealloc(tmem_base, 512);
   }
@@ -1270,9 +1355,14 @@ cudaError_t bwd_fused_launch(const bf16* qkv, const bf16* o, const float* lse, c
   constexpr int TPR = DH / 8;
   const long long nthreads = (long long)NB * T * H * TPR;
   attn_delta_tc_kernel<DH><<<(unsigned)((nthreads + 255) / 256), 256, 0, s>>>(dout, o, delta, dq_acc, NB, B, T, H);
-  dim3 grid((T + TQ - 1) / TQ, NB * H);
+  // persistent CTAs, one per SM, each walking its share of the (key tile, sequence, head) items
+  int dev = 0, sms = 0;
+  if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+  if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+  const long long nitems = (long long)((T + TQ - 1) / TQ) * NB * H;
+  const int grid = (int)(nitems < sms ? nitems : sms);
   const float scale = rsqrtf((float)DH);
-  attn_bwd_fused_kernel<DH><<<grid, 320, C::SMEM, s>>>(tmRow, tmdO, lse, delta, dqkv, dq_acc, B, T, H, scale, err);
+  attn_bwd_fused_kernel<DH><<<grid, FUSED_THREADS, C::SMEM, s>>>(tmRow, tmdO, lse, delta, dqkv, dq_acc, NB, B, T, H, scale, err);
   const size_t rows = (size_t)NB * T;
   size_t blocks = (rows * (size_t)(H * DH / 8) + 255) / 256;
   if (blocks > 148 * 16) blocks = 148 * 16;
