@@ -139,27 +139,35 @@ def test_2p7b_shape_full_size():
 
 def test_sweep_invariants_on_device_full_size():
     """Head gradients do not depend on n; the top component's gradient does not depend on n; with n = 1
-    component k's gradient is that of its own head only, so n = 2 differs from it for every k < K-1."""
-    w = wl.CONFIGS["cfg2"]
-    m = _model("cfg2")
-    tok, tgt = wl.draw_tokens(w)
-    dt, dg = torch.tensor(tok, device="cuda:0"), torch.tensor(tgt, device="cuda:0")
-    probes = ["head0.w", "head3.ln.g", f"c{w.K - 1}.l0.mlp.w1", "c0.l1.attn.wqkv", "c1.l0.mlp.w2"]
-    res = {}
-    for n in (1, 2, 4):
-        m.set_n(n)
-        m.train_step(dt, dg)
-        m.sync()
-        res[n] = {p: m.get_grad(p) for p in probes}
-    for p in probes[:3]:
-        for n in (2, 4):
-            den = np.linalg.norm(res[1][p])
-            assert np.linalg.norm(res[n][p] - res[1][p]) / den < 1e-5, (p, n)
-    for p in probes[3:]:
-        assert np.linalg.norm(res[2][p] - res[1][p]) / np.linalg.norm(res[1][p]) > 1e-2, p
+    component k's gradient is that of its own head only, so n = 2 differs from it for every k < K-1.
+    Run with the two-kernel attention backward, whose sums have a fixed order: the one-sweep form adds dQ over key
+    tiles with floating-point atomics, so two runs of the same gradient agree only to rounding (about 2e-5 here)."""
     for m_ in _models.values():
         m_.close()
     _models.clear()
+    torch.cuda.empty_cache()
+    w = wl.CONFIGS["cfg2"]
+    m = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, 1, w.B, w.T, attn_bwd="two_kernels")
+    try:
+        for i, (name, _, _, shape) in enumerate(wl.tensor_specs(w)):
+            m.set_param(name, wl.draw_tensor(name, i, shape))
+        tok, tgt = wl.draw_tokens(w)
+        dt, dg = torch.tensor(tok, device="cuda:0"), torch.tensor(tgt, device="cuda:0")
+        probes = ["head0.w", "head3.ln.g", f"c{w.K - 1}.l0.mlp.w1", "c0.l1.attn.wqkv", "c1.l0.mlp.w2"]
+        res = {}
+        for n in (1, 2, 4):
+            m.set_n(n)
+            m.train_step(dt, dg)
+            m.sync()
+            res[n] = {p: m.get_grad(p) for p in probes}
+        for p in probes[:3]:
+            for n in (2, 4):
+                den = np.linalg.norm(res[1][p])
+                assert np.linalg.norm(res[n][p] - res[1][p]) / den < 1e-5, (p, n)
+        for p in probes[3:]:
+            assert np.linalg.norm(res[2][p] - res[1][p]) / np.linalg.norm(res[1][p]) > 1e-2, p
+    finally:
+        m.close()
 
 
 def test_cfg5_width_reduced_depth_matches_oracle():
