@@ -745,11 +745,12 @@ __global__ void __launch_bounds__(256) adamw_kernel(float4* __restrict__ p, floa
                                                     const float4* __restrict__ g, uint2* __restrict__ pb, size_t n4,
                                                     size_t n4_decay, float lr, float b1, float b2, float eps, float wd,
                                                     float ibc1, float ibc2, const unsigned* __restrict__ err,
-                                                    unsigned* applied) {
+                                                    unsigned* applied, size_t skip0, size_t skip1) {
   // a step whose kernels reported an error must not reach the parameters: leave everything as it is
   if (err && *reinterpret_cast<const volatile unsigned*>(err) != 0u) return;
   if (applied && blockIdx.x == 0 && threadIdx.x == 0) *applied += 1u;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+    if (i >= skip0 && i < skip1) continue;          // a sub-range updated by another launch
     const float w = i < n4_decay ? wd : 0.f;
     float4 pv = p[i], mv = m[i], vv = v[i];
     const float4 gv = g[i];
@@ -769,7 +770,7 @@ __global__ void __launch_bounds__(256) adamw_kernel(float4* __restrict__ p, floa
 
 cudaError_t adamw(float* p, float* m, float* v, const float* g, bf16* p_bf16, size_t n, size_t n_decay, float lr,
                   float beta1, float beta2, float eps, float wd, float bc1, float bc2, const unsigned* err, unsigned* applied,
-                  cudaStream_t s) {
+                  size_t skip_begin, size_t skip_end, cudaStream_t s) {
   const size_t n4 = n / 4;
   if (n4 == 0) return cudaSuccess;
   int blocks = ceil_div(n4, 256);
@@ -777,7 +778,7 @@ cudaError_t adamw(float* p, float* m, float* v, const float* g, bf16* p_bf16, si
   adamw_kernel<<<blocks, 256, 0, s>>>(reinterpret_cast<float4*>(p), reinterpret_cast<float4*>(m),
                                       reinterpret_cast<float4*>(v), reinterpret_cast<const float4*>(g),
                                       reinterpret_cast<uint2*>(p_bf16), n4, n_decay / 4, lr, beta1, beta2, eps, wd,
-                                      1.0f / bc1, 1.0f / bc2, err, applied);
+                                      1.0f / bc1, 1.0f / bc2, err, applied, skip_begin / 4, skip_end / 4);
   return cudaGetLastError();
 }
 

@@ -65,9 +65,10 @@ cudaError_t head_backward_prepare(__nv_bfloat16* e, int ld, const float* lse, co
 
 // AdamW over a flat range: the first n_decay elements get decoupled weight decay.  Writes the bf16 shadow.
 // err (may be NULL): when *err != 0 the kernel changes nothing; applied (may be NULL): += 1 when it does update.
+// Elements [skip_begin, skip_end) (multiples of 4) are left alone: another launch updates them.
 cudaError_t adamw(float* p, float* m, float* v, const float* g, __nv_bfloat16* p_bf16, size_t n, size_t n_decay,
                   float lr, float beta1, float beta2, float eps, float wd, float bc1, float bc2, const unsigned* err,
-                  unsigned* applied, cudaStream_t s);
+                  unsigned* applied, size_t skip_begin, size_t skip_end, cudaStream_t s);
 
 // Causal attention on packed qkv [B*T, 3d] (Q | K | V, head h at columns h*dh) on the tcgen05 tensor cores.
 // dh in {32, 64, 80, 128, 256}; pointers 16-byte aligned.

@@ -80,6 +80,10 @@ struct il_model {
   bool own_streams;
   std::vector<cudaStream_t> streams;
   std::vector<cudaEvent_t> ev_fwd, ev_bwd, ev_join;
+  // The vocabulary matrix of head k is final as soon as the head's own backward is: its optimiser update runs on a
+  // side stream that waits for that point only (ev_head), beside the component's backward.
+  std::vector<cudaStream_t> side;
+  std::vector<cudaEvent_t> ev_head, ev_side;
   cudaEvent_t ev_batch;
   // parameters
   std::vector<TensorRec> tensors;
@@ -567,6 +571,14 @@ extern "C" il_status il_create(int K, int Lc, int d, int H, int F, int V, int n,
   IL_TRY(mk_events(m->ev_bwd));
   IL_TRY(mk_events(m->ev_join));
   IL_TRY(mk_events(m->ev_copy));
+  IL_TRY(mk_events(m->ev_head));
+  IL_TRY(mk_events(m->ev_side));
+  m->side.resize(K);
+  for (int k = 0; k < K; ++k) {
+    IL_CUDA(m, cudaSetDevice(m->dev[k]));
+    cudaError_t e = cudaStreamCreateWithFlags(&m->side[k], cudaStreamNonBlocking);
+    if (e != cudaSuccess) { m->side.resize(k); return bail(fail(m, IL_ERR_CUDA, "cudaStreamCreate: %s", cudaGetErrorString(e))); }
+  }
   IL_CUDA(m, cudaSetDevice(m->dev[0]));
   IL_CUDA(m, cudaEventCreateWithFlags(&m->ev_batch, cudaEventDisableTiming));
 
@@ -704,6 +716,9 @@ extern "C" il_status il_destroy(il_model* m) {
   for (auto e : m->ev_bwd) cudaEventDestroy(e);
   for (auto e : m->ev_join) cudaEventDestroy(e);
   for (auto e : m->ev_copy) cudaEventDestroy(e);
+  for (auto e : m->ev_head) cudaEventDestroy(e);
+  for (auto e : m->ev_side) cudaEventDestroy(e);
+  for (auto st : m->side) cudaStreamDestroy(st);
   if (m->ev_batch) cudaEventDestroy(m->ev_batch);
   for (auto e : m->prof_pool) cudaEventDestroy(e);
   for (auto& r : m->prof_recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
@@ -1181,6 +1196,7 @@ extern "C" il_status il_backward_nwise(il_model* m) {
       }
     }
     IL_TRY(head_backward(m, k, acc, gscale));
+    IL_CUDA(m, cudaEventRecord(m->ev_head[k], st));      // head k's parameter gradients are final from here on
   }
   if (m->rule == IL_RULE_SUM) {
     // components from the top down; component k needs the pass-down of component k+1 when any stream crosses
@@ -1317,10 +1333,20 @@ extern "C" il_status il_adamw_step(il_model* m, float lr, float beta1, float bet
   for (int k = 0; k < m->K; ++k) {
     const size_t b = m->comp_begin[k], e = m->comp_end[k], me = m->comp_mat_end[k];
     IL_CUDA(m, cudaSetDevice(m->dev[k]));
-    // the kernel leaves everything untouched while the error word is set (the gradients of a failed step are not
-    // applied) and otherwise counts the update in word 1 + k
+    // The kernels leave everything untouched while the error word is set (the gradients of a failed step are not
+    // applied); the main launch counts the update in word 1 + k.  The head's vocabulary matrix (the last matrix of
+    // the component's range, more than half of its parameters) is updated on the side stream as soon as the head's
+    // own backward is done, so that this HBM-bound pass runs beside the component's tensor-bound backward.
+    const size_t hw0 = m->head_off[k].w, hw1 = me;
+    const bool aside = m->prof != 2;        // (the exclusive GEMM timing mode keeps everything on the component streams)
+    cudaStream_t hs = aside ? m->side[k] : m->streams[k];
+    if (aside) IL_CUDA(m, cudaStreamWaitEvent(hs, m->ev_head[k], 0));
+    IL_K(m, adamw(m->P[k] + hw0, m->M1[k] + hw0, m->M2[k] + hw0, m->G[k] + hw0, m->Pb[k] + hw0, hw1 - hw0, hw1 - hw0, lr, beta1, beta2,
+                  eps, wd, (float)bc1, (float)bc2, m->err_word[k], nullptr, 0, 0, hs));
+    if (aside) IL_CUDA(m, cudaEventRecord(m->ev_side[k], hs));
     IL_K(m, adamw(m->P[k] + b, m->M1[k] + b, m->M2[k] + b, m->G[k] + b, m->Pb[k] + b, e - b, me - b, lr, beta1, beta2, eps, wd,
-                  (float)bc1, (float)bc2, m->err_word[k], m->err_word[k] + 1 + k, m->streams[k]));
+                  (float)bc1, (float)bc2, m->err_word[k], m->err_word[k] + 1 + k, hw0 - b, hw1 - b, m->streams[k]));
+    if (aside) IL_CUDA(m, cudaStreamWaitEvent(m->streams[k], m->ev_side[k], 0));   // stream k's tail covers the side stream
   }
   m->batch_set = false;   // a new batch is required for the next step
   m->micro_done = 0;
