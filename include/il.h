@@ -169,7 +169,8 @@ il_status il_set_micro_batches(il_model* m, int micro_batches);
  * the exp(logit) range) a component's parameters, Adam moments and bf16 copies are left untouched, and the next
  * il_sync reports the error and takes the skipped updates back off the step counter.  The check is per component
  * and per launch: a component whose update ran before another component raised the error keeps that update
- * (il_last_error then says so). */
+ * (il_last_error then says so); the same holds for a head's vocabulary matrix, whose update is enqueued on a side
+ * stream right behind the head's own backward and may therefore run before an error raised later in the step. */
 il_status il_adamw_step(il_model* m, float lr, float beta1, float beta2, float eps, float weight_decay);
 /* Wait for all enqueued work; reports device-side timeouts as IL_ERR_TIMEOUT and a head whose
  * log-sum-exp left [-80, 80] in il_backward_nwise as IL_ERR_NONFINITE (that step's gradients are invalid).
