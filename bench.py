@@ -43,7 +43,7 @@ import workloads as wl  # noqa: E402
 # Traffic grows with the flops of a launch at fixed shapes, so the
 # per-launch figure of another step mix is this ratio times that mix's flops per launch.  Set to None whenever
 # gemm.cu changes after the capture.
-GEMM_DRAM_BYTES_PER_FLOP = 1.2568e-3
+GEMM_DRAM_BYTES_PER_FLOP = 1.2556e-3
 
 
 def model_flops_per_token(w: wl.Workload, n: int) -> float:
