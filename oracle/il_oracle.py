@@ -379,6 +379,70 @@ def nwise_gradients(P, tokens: np.ndarray, targets: np.ndarray, K: int, Lc: int,
     return losses, G
 
 
+def nwise_gradients_bounded(P, tokens: np.ndarray, targets: np.ndarray, K: int, Lc: int, H: int, n: int, emit,
+                            rule: str = "sum", head_layers: int = 0) -> List[float]:
+    """The step of nwise_gradients with bounded memory, for configurations whose intermediate values do not fit
+    the host (the arithmetic of every pass is the same; only what is kept, and for how long, differs).
+
+    * The forward pass keeps the K+1 boundary activations only; the blocks' intermediate values of a component are
+      recomputed (component_fwd from its stored input) each time a head's backward pass reaches it.
+    * Heads are taken from the top down.  Component k receives gradient from heads k .. k+n-1 (Sec. 3), so once head k
+      has been processed its parameter gradients are final: they are handed to emit(name, gradient) and dropped.
+      Head parameters are final right after their own pass.  Tensors that never received a gradient are emitted
+      as zeros.
+    Returns the K head losses.  A test pins it to nwise_gradients on small nets for every n and rule.
+    """
+    if not (1 <= n <= K):
+        raise ValueError("n must be in [1, K]")
+    B, T = tokens.shape
+    a = [embed_fwd(tokens, P)]
+    for k in range(K):
+        x, _ = component_fwd(a[-1], P, k, Lc, B, T, H)
+        a.append(x)
+    losses: List[float] = [0.0] * K
+    G: Dict[str, np.ndarray] = {}
+    emitted = set()
+
+    def flush(prefixes):
+        for name in list(G.keys()):
+            if any(name == p or name.startswith(p) for p in prefixes):
+                emit(name, G.pop(name))
+                emitted.add(name)
+
+    for h in reversed(range(K)):
+        loss, da, hg = head_loss(a[h + 1], targets, P, h, True, head_layers=head_layers, B=B, T=T, H=H)
+        losses[h] = loss
+        for name, val in hg.items():
+            emit(name, val)
+            emitted.add(name)
+        del hg
+        dx = da
+        lowest = max(h - n + 1, 0)
+        for k in range(h, lowest - 1, -1):
+            _, caches_k = component_fwd(a[k], P, k, Lc, B, T, H)
+            wk = head_weight(k, h, n, K, rule)
+            if wk == 1.0:
+                dx = component_bwd(dx, caches_k, P, k, B, T, H, G)
+                if k == 0:
+                    embed_bwd(dx, tokens, P, G)
+            else:
+                Gk: Dict[str, np.ndarray] = {}
+                dx = component_bwd(dx, caches_k, P, k, B, T, H, Gk)
+                if k == 0:
+                    embed_bwd(dx, tokens, P, Gk)
+                if wk != 0.0:
+                    for name, val in Gk.items():
+                        G[name] = G[name] + wk * val if name in G else wk * val
+                del Gk
+            del caches_k
+        # every head whose window covers component h has now been processed
+        flush([f"c{h}."] + (["wte", "wpe"] if h == 0 else []))
+    for name in P:
+        if name not in emitted:
+            emit(name, np.zeros(P[name].shape, dtype=F64))
+    return [float(x) for x in losses]
+
+
 def nwise_gradients_microbatched(P, tokens: np.ndarray, targets: np.ndarray, K: int, Lc: int, H: int, n: int,
                                  micro_batches: int, rule: str = "sum", head_layers: int = 0):
     """The same step with the mini-batch split into `micro_batches` equal groups of sequences (Sec. 3.1:

@@ -847,13 +847,15 @@ __device__ __forceinline__ FusedItem fused_item(int item, int nbh, int H, int B,
 template <int DH>
 __global__ void __launch_bounds__(FUSED_THREADS, 1) attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tmRow,     // qkv, 128-row box
                                                                           const __grid_constant__ CUtensorMap tmdO,      // dout, 128-row box
+                                                                          const __grid_constant__ CUtensorMap tmAcc,     // dQ accumulator (fp32), 32 x 128 box
                                                                           const float* __restrict__ lse, const float* __restrict__ delta,
-                                                                          bf16* __restrict__ dqkv, float* __restrict__ dq_acc, int NB,
+                                                                          bf16* __restrict__ dqkv, int NB,
                                                                           int B, int T, int H, float scale, unsigned* err) {
   using C = FusedCfg<DH>;
   constexpr int NST = C::NST;
   extern __shared__ uint8_t smem_raw[];
   __shared__ int abort_flag;
+  __shared__ volatile int flush_fail;
   __shared__ uint32_t tmem_base_smem;
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t sK = base, sV = sK + C::ROW_BYTES;
@@ -872,6 +874,7 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) attn_bwd_fused_kernel(const 
   auto bar_dq = [&](int b) { return bars + 72 + 8 * (2 * NST + 4 + b); };      // dQ buffer b complete
   auto bar_dqfree = [&](int b) { return bars + 72 + 8 * (2 * NST + 6 + b); };  // dQ buffer b flushed
   auto bar_vec = [&](int st) { return bars + 72 + 8 * (2 * NST + 8 + st); };   // lse / delta vectors of stage st written
+  auto bar_dsfree = [&](int b) { return bars + 72 + 8 * (3 * NST + 8 + b); };  // dS buffer b (also the staging of its dQ block) free again
   uint8_t* gen = smem_raw + (base - smem_u32(smem_raw));
   float* s_vec = reinterpret_cast<float*>(gen + (sVec - base));
 
@@ -884,6 +887,7 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) attn_bwd_fused_kernel(const 
 
   if (tid == 0) {
     abort_flag = 0;
+    flush_fail = 0;
     mbar_init(bar_kv, 1);
     mbar_init(bar_kvfree, 3);            // the three issuing threads
     mbar_init(bar_acc, 2);               // the two half threads
@@ -899,10 +903,12 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) attn_bwd_fused_kernel(const 
       mbar_init(bar_p(x), FUSED_RW);
       mbar_init(bar_dq(x), 1);
       mbar_init(bar_dqfree(x), 4);       // one arrival per flush warp
+      mbar_init(bar_dsfree(x), 1);
     }
     fence_mbar_init();
     tma_prefetch_desc(&tmRow);
     tma_prefetch_desc(&tmdO);
+    tma_prefetch_desc(&tmAcc);
   }
   if (warp == 20) {
     tmem_alloc(smem_u32(&tmem_base_smem), 512);
@@ -1068,6 +1074,13 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) attn_bwd_fused_kernel(const 
     // ---------------------------------------------------------------- dQ flush and dV / dK store (warps 16-19: thread = row)
     const int r = tid - 512;
     const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+    // The four flush warps meet at a named barrier inside every step, so they must leave the loops together: the
+    // outcome of a wait is agreed on (through a shared flag and that barrier) before anyone acts on it.
+    auto all_ok = [&](int got) -> bool {
+      if (!got) flush_fail = 1;
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      return flush_fail == 0;
+    };
     int g = 0, n_item = 0;
     for (int item = blockIdx.x; item < nitems && !fail; item += gridDim.x, ++n_item) {
       const FusedItem w = fused_item(item, nbh, H, B, nq);
@@ -1076,25 +1089,38 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) attn_bwd_fused_kernel(const 
         int got = 1;
         if (lane == 0) got = mbar_wait(bar_dq(b), (uint32_t)(gs >> 1) & 1u, abortp) ? 1 : 0;
         got = __shfl_sync(0xffffffffu, got, 0);
-        if (!got) { fail = 1; abort_flag = 1; break; }
+        if (!all_ok(got)) { fail = 1; abort_flag = 1; break; }
         tc_fence_after();
-        const int q = (w.kb + it) * TQ + r;
-        float* dst = dq_acc + ((size_t)w.nb * T + q) * d + w.h * DH;
+        // The block goes to the global accumulator as one bulk reduction per 32 columns: the rows are staged in the
+        // dS buffer of this step (its dQ product, the only reader, has retired) in the 128-byte-swizzled layout of
+        // the tensor map, and one thread issues cp.reduce.async.bulk.tensor (rows past the sequence end are dropped
+        // by the map's bounds).
+        const uint32_t stage = sDS + (uint32_t)b * C::DS_BYTES;
 #pragma unroll
         for (int c0 = 0; c0 < DH; c0 += 32) {
           uint32_t rr[32];
           tmem_ld_32x32(t_lane + C::C_DQ + 64 * b + c0, rr);
           tmem_ld_wait();
-          if (q < T) {
+          const uint32_t rowaddr = stage + (uint32_t)(c0 / 32) * (TQ * 128) + (uint32_t)r * 128;
 #pragma unroll
-            for (int i = 0; i < 32; i += 4)
-              red_add_f32x4(dst + c0 + i, make_float4(__uint_as_float(rr[i]), __uint_as_float(rr[i + 1]), __uint_as_float(rr[i + 2]),
-                                                      __uint_as_float(rr[i + 3])));
-          }
+          for (int t = 0; t < 8; ++t)
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(rowaddr + (((uint32_t)t ^ (uint32_t)(r & 7)) * 16)), "r"(rr[4 * t]),
+                         "r"(rr[4 * t + 1]), "r"(rr[4 * t + 2]), "r"(rr[4 * t + 3])
+                         : "memory");
         }
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(bar_dqfree(b));
+        if (lane == 0) mbar_arrive(bar_dqfree(b));               // the TMEM buffer has been read
+        fence_proxy_async();
+        asm volatile("bar.sync 1, 128;" ::: "memory");           // the four flush warps: the block is staged
+        if (r == 0) {
+#pragma unroll
+          for (int c0 = 0; c0 < DH; c0 += 32)
+            tma_reduce_add_3d(&tmAcc, stage + (uint32_t)(c0 / 32) * (TQ * 128), w.h * DH + c0, (w.kb + it) * TQ, w.nb);
+          bulk_commit_group();
+          bulk_wait_group_read0();                               // the staging has been read: the buffer may be rewritten
+          mbar_arrive(bar_dsfree(b));
+        }
       }
       if (fail) break;
       g += w.nit;
@@ -1103,7 +1129,7 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) attn_bwd_fused_kernel(const 
         int got = 1;
         if (lane == 0) got = mbar_wait(bar_acc, (uint32_t)n_item & 1u, abortp) ? 1 : 0;
         got = __shfl_sync(0xffffffffu, got, 0);
-        if (!got) { fail = 1; abort_flag = 1; break; }
+        if (!all_ok(got)) { fail = 1; abort_flag = 1; break; }
       }
       tc_fence_after();
       const int key = w.kb * TQ + r;
@@ -1135,6 +1161,7 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) attn_bwd_fused_kernel(const 
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_accfree);               // the accumulators may be overwritten by the next item
     }
+    if (r == 0) bulk_wait_group0();                            // every reduction this thread issued has reached memory
   } else if (warp < FUSED_RW) {
     // ---------------------------------------------------------------- recompute and convert (warps 0-15)
     // thread (r, sub): key row r, query columns [16 sub, 16 sub + 16) of each 64-column half
@@ -1153,10 +1180,10 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) attn_bwd_fused_kernel(const 
         const int gs = g + it, st = gs % NST, b = gs & 1, j = w.kb + it;
         const uint32_t ph = (uint32_t)gs & 1u;
         const float* vec = s_vec + st * (2 * TQ);
-        // the stage's lse / delta vectors have their own barrier; the dS buffer of this step is free
-        // once the dQ product of step gs-2 has read it (both long complete by now)
+        // the stage's lse / delta vectors have their own barrier; the dS buffer of this step is free once the dQ
+        // block of step gs-2, staged in it after its product, has been handed to the bulk reduction
         if (!wait(bar_vec(st), (uint32_t)(gs / NST) & 1u)) { fail = 1; abort_flag = 1; break; }
-        if (gs >= 2 && !wait(bar_dq(b), (uint32_t)((gs >> 1) - 1) & 1u)) { fail = 1; abort_flag = 1; break; }
+        if (gs >= 2 && !wait(bar_dsfree(b), (uint32_t)((gs >> 1) - 1) & 1u)) { fail = 1; abort_flag = 1; break; }
         const bool diag = (it == 0);                       // some queries of this block precede some keys of this tile
         const bool tail = (j * TQ + TQ > T);
         for (int x = 0; x < 2; ++x) {
@@ -1347,9 +1374,14 @@ cudaError_t bwd_fused_launch(const bf16* qkv, const bf16* o, const float* lse, c
   const unsigned long long ddims[4] = {(unsigned long long)DH, (unsigned long long)H, (unsigned long long)T, (unsigned long long)NB};
   const unsigned long long dstrides[3] = {(unsigned long long)DH * 2, d1 * 2, (unsigned long long)T * d1 * 2};
   const unsigned box128[4] = {64, 1, TQ, 1};
-  CUtensorMap tmRow, tmdO;
+  CUtensorMap tmRow, tmdO, tmAcc;
   if (!tma_encode_bf16(&tmRow, qkv, 4, dims, strides, box128) || !tma_encode_bf16(&tmdO, dout, 4, ddims, dstrides, box128))
     return cudaErrorInvalidValue;
+  // the fp32 dQ accumulator [NB, T, d] as the target of the bulk reductions: boxes of 32 columns x 128 rows of one sequence
+  const unsigned long long adims[3] = {d1, (unsigned long long)T, (unsigned long long)NB};
+  const unsigned long long astrides[2] = {d1 * 4, (unsigned long long)T * d1 * 4};
+  const unsigned abox[3] = {32, TQ, 1};
+  if (!tma_encode_f32(&tmAcc, dq_acc, 3, adims, astrides, abox)) return cudaErrorInvalidValue;
   cudaError_t e = cudaFuncSetAttribute(attn_bwd_fused_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
   if (e != cudaSuccess) return e;
   constexpr int TPR = DH / 8;
@@ -1362,7 +1394,7 @@ cudaError_t bwd_fused_launch(const bf16* qkv, const bf16* o, const float* lse, c
   const long long nitems = (long long)((T + TQ - 1) / TQ) * NB * H;
   const int grid = (int)(nitems < sms ? nitems : sms);
   const float scale = rsqrtf((float)DH);
-  attn_bwd_fused_kernel<DH><<<grid, FUSED_THREADS, C::SMEM, s>>>(tmRow, tmdO, lse, delta, dqkv, dq_acc, NB, B, T, H, scale, err);
+  attn_bwd_fused_kernel<DH><<<grid, FUSED_THREADS, C::SMEM, s>>>(tmRow, tmdO, tmAcc, lse, delta, dqkv, NB, B, T, H, scale, err);
   const size_t rows = (size_t)NB * T;
   size_t blocks = (rows * (size_t)(H * DH / 8) + 255) / 256;
   if (blocks > 148 * 16) blocks = 148 * 16;

@@ -758,16 +758,25 @@ cudaError_t gemm_init() {
   return cudaSuccess;
 }
 
-bool tma_encode_bf16(CUtensorMap* tm, const void* ptr, int rank, const unsigned long long* dims,
-                     const unsigned long long* strides_bytes, const unsigned* box) {
+static bool tma_encode_any(CUtensorMap* tm, CUtensorMapDataType dt, const void* ptr, int rank, const unsigned long long* dims,
+                           const unsigned long long* strides_bytes, const unsigned* box) {
   if (gemm_init() != cudaSuccess || rank < 2 || rank > 5) return false;
   cuuint64_t d[5], st[4];
   cuuint32_t b[5], es[5] = {1, 1, 1, 1, 1};
   for (int i = 0; i < rank; ++i) { d[i] = dims[i]; b[i] = box[i]; }
   for (int i = 0; i < rank - 1; ++i) st[i] = strides_bytes[i];
-  return g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(ptr), d, st, b, es,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return g_encode(tm, dt, (cuuint32_t)rank, const_cast<void*>(ptr), d, st, b, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool tma_encode_bf16(CUtensorMap* tm, const void* ptr, int rank, const unsigned long long* dims,
+                     const unsigned long long* strides_bytes, const unsigned* box) {
+  return tma_encode_any(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, ptr, rank, dims, strides_bytes, box);
+}
+
+bool tma_encode_f32(CUtensorMap* tm, const void* ptr, int rank, const unsigned long long* dims,
+                    const unsigned long long* strides_bytes, const unsigned* box) {
+  return tma_encode_any(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, ptr, rank, dims, strides_bytes, box);
 }
 
 // rows = extent of the operand's own index (M or N), kdim = contraction extent, box_rows = tile rows.

@@ -10,4 +10,8 @@ namespace il {
 bool tma_encode_bf16(CUtensorMap* tm, const void* ptr, int rank, const unsigned long long* dims,
                      const unsigned long long* strides_bytes, const unsigned* box);
 
+// The same for fp32 tensors (inner box extent at most 32 elements = 128 bytes).
+bool tma_encode_f32(CUtensorMap* tm, const void* ptr, int rank, const unsigned long long* dims,
+                    const unsigned long long* strides_bytes, const unsigned* box);
+
 }  // namespace il

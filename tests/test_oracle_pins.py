@@ -474,3 +474,31 @@ def test_paper_rules_relations():
     for name, comp, is_head, _ in specs:
         if not is_head:
             assert np.allclose(G[("far", w.K)][name], Pt[name].grad.numpy(), rtol=1e-9, atol=1e-13), name
+
+
+@pytest.mark.parametrize("rule", ["sum", "far", "mean"])
+@pytest.mark.parametrize("head_layers", [0, 1])
+def test_bounded_memory_step_equals_the_plain_one(rule, head_layers):
+    """nwise_gradients_bounded (boundaries kept, blocks recomputed, gradients emitted when final, heads from the
+    top down) gives the losses and gradients of nwise_gradients for every n: same passes, other bookkeeping."""
+    import workloads as wl
+    w = wl.Workload("bnd", K=3, Lc=2, d=8, H=2, F=16, V=11, T=5, B=2, n=1, zipf=False, Lh=head_layers)
+    P = wl.draw_params(w)
+    tok, tgt = wl.draw_tokens(w)
+    for n in (1, 2, 3):
+        l0, G0 = orc.nwise_gradients(P, tok, tgt, w.K, w.Lc, w.H, n, rule=rule, head_layers=head_layers)
+        got = {}
+        order = []
+
+        def emit(name, g):
+            assert name not in got
+            got[name] = np.array(g, dtype=np.float64, copy=True)
+            order.append(name)
+
+        l1 = orc.nwise_gradients_bounded(P, tok, tgt, w.K, w.Lc, w.H, n, emit, rule=rule, head_layers=head_layers)
+        assert np.allclose(l0, l1, rtol=1e-13, atol=0)
+        assert set(got) == set(G0)
+        for name in G0:
+            assert np.allclose(got[name], G0[name], rtol=1e-10, atol=1e-15), (n, name)
+        # a component's tensors are emitted only after its own head has been processed, i.e. after every head above
+        assert order.index("head2.w") < order.index("c2.l0.mlp.w1") < order.index("head1.w") < order.index("c1.l0.mlp.w1")
