@@ -444,6 +444,30 @@ def main():
     }
     if losses is not None:
         out["last_losses"] = [float(x) for x in losses]
+    # Per-phase times (a diagnostic beside the step time, not part of it): three more steps with a device
+    # synchronisation between the phases, so nothing of one phase overlaps the next; host clock around the syncs.
+    if w.M == 1:
+        ph = np.zeros(3)
+        for i in range(3):
+            tok, tgt = dev_batches[i % nb]
+            m.sync()
+            t0 = time.perf_counter()
+            m.set_batch(tok, tgt)
+            for k in range(w.K):
+                m.forward_component(k)
+                m.aux_head_loss(k)
+            m.sync()
+            t1 = time.perf_counter()
+            m.backward_nwise()
+            m.sync()
+            t2 = time.perf_counter()
+            if hp is not None:
+                m.adamw_step(**hp)
+                m.sync()
+            t3 = time.perf_counter()
+            ph += np.array([t1 - t0, t2 - t1, t3 - t2]) * 1e3 / 3
+        out["phases_ms"] = {"forward_and_head_losses": float(ph[0]), "backward_nwise": float(ph[1]), "adamw": float(ph[2]),
+                            "note": "each phase alone on the GPU (synchronised between phases); in the timed step they overlap"}
     dev_bytes = m.stats()[0]
     out["head_mode"] = {"mode": args.head_mode, "ms_per_step": ms / args.steps, "device_bytes": int(dev_bytes)}
     m.close()
