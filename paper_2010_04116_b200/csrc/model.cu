@@ -21,6 +21,8 @@
 #include <utility>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "../../include/il.h"
 #include "../../include/il_ops.h"
 #include "common.cuh"
@@ -59,6 +61,18 @@ struct HeadScratch {
 };
 
 struct ProfRec { cudaEvent_t a, b; double flops; };
+
+// Named range on the host timeline of a profiler (NVTX; costs nothing when no tool is attached): one per call of
+// the step and, inside the backward, one per component, so that a trace shows which launches belong to which
+// component and phase.
+struct Range {
+  explicit Range(const char* fmt, int k = -1) {
+    char buf[64];
+    snprintf(buf, sizeof buf, fmt, k);
+    nvtxRangePushA(buf);
+  }
+  ~Range() { nvtxRangePop(); }
+};
 
 }  // namespace
 
@@ -846,6 +860,7 @@ extern "C" il_status il_set_opt_state(il_model* m, int idx, const float* mh, con
 extern "C" il_status il_set_batch(il_model* m, const int* tokens, const int* targets, int B, int T, int on_device) {
   return guarded([&]() -> il_status {
   IL_TRY(check_model(m));
+  Range range("il_set_batch");
   if (!tokens || !targets) return fail(m, IL_ERR_INVALID_ARG, "NULL tokens/targets");
   if (B < 1 || T < 1 || B > m->max_batch || T > m->max_seq || (size_t)B * T > (size_t)m->ntok_max)
     return fail(m, IL_ERR_INVALID_ARG, "batch %dx%d exceeds max_batch=%d, max_seq=%d", B, T, m->max_batch, m->max_seq);
@@ -925,6 +940,7 @@ il_status layers_forward(il_model* m, int k, size_t base, int count, const float
 extern "C" il_status il_forward_component(il_model* m, int k) {
   return guarded([&]() -> il_status {
   IL_TRY(check_model(m));
+  Range range("il_forward_component %d", k);
   if (k < 0 || k >= m->K) return fail(m, IL_ERR_INVALID_ARG, "component %d out of range", k);
   if (!m->batch_set) return fail(m, IL_ERR_STATE, "il_forward_component before il_set_batch");
   if (k > 0 && !m->fwd_done[k - 1]) return fail(m, IL_ERR_STATE, "component %d forward needs component %d first", k, k - 1);
@@ -953,6 +969,7 @@ extern "C" il_status il_forward_component(il_model* m, int k) {
 extern "C" il_status il_aux_head_loss(il_model* m, int k, float* loss_host) {
   return guarded([&]() -> il_status {
   IL_TRY(check_model(m));
+  Range range("il_aux_head_loss %d", k);
   if (k < 0 || k >= m->K) return fail(m, IL_ERR_INVALID_ARG, "head %d out of range", k);
   if (!m->batch_set || !m->fwd_done[k]) return fail(m, IL_ERR_STATE, "il_aux_head_loss(%d) needs il_forward_component(%d)", k, k);
   IL_CUDA(m, cudaSetDevice(m->dev[k]));
@@ -1152,6 +1169,7 @@ il_status component_backward(il_model* m, int k, int s, bool acc) {
 extern "C" il_status il_backward_nwise(il_model* m) {
   return guarded([&]() -> il_status {
   IL_TRY(check_model(m));
+  Range range("il_backward_nwise");
   if (!m->batch_set) return fail(m, IL_ERR_STATE, "il_backward_nwise before il_set_batch");
   for (int k = 0; k < m->K; ++k)
     if (!m->fwd_done[k] || !m->loss_done[k])
@@ -1195,7 +1213,10 @@ extern "C" il_status il_backward_nwise(il_model* m) {
         IL_CUDA(m, cudaMemsetAsync(m->G[k] + m->off_wpe, 0, (size_t)m->max_seq * d * 4, st));
       }
     }
-    IL_TRY(head_backward(m, k, acc, gscale));
+    {
+      Range r2("head backward %d", k);
+      IL_TRY(head_backward(m, k, acc, gscale));
+    }
     IL_CUDA(m, cudaEventRecord(m->ev_head[k], st));      // head k's parameter gradients are final from here on
   }
   if (m->rule == IL_RULE_SUM) {
@@ -1220,7 +1241,10 @@ extern "C" il_status il_backward_nwise(il_model* m) {
         if (fetch_err != cudaSuccess) return fail(m, IL_ERR_CUDA, "cudaMemcpyPeerAsync: %s", cudaGetErrorString(fetch_err));
         IL_K(m, add_convert(m->hs[k].ghead, passed, m->cs[k].dx + (size_t)j * slice, m->cs[k].dxb + (size_t)j * slice, slice, st));
       }
-      IL_TRY(component_backward(m, k, s, acc));
+      {
+        Range r2("component backward %d", k);
+        IL_TRY(component_backward(m, k, s, acc));
+      }
       if (k == 0) {
         IL_K(m, embed_bwd(m->tokens[k], m->sort_keys[0], m->cs[0].dx, m->G[k] + m->off_wte, m->G[k] + m->off_wpe, N, m->T, d, m->V, acc ? 1 : 0, st));
         m->launches++;
@@ -1280,7 +1304,10 @@ extern "C" il_status il_backward_nwise(il_model* m) {
             mine_slots.push_back(used++);
           }
       if (fetch_err != cudaSuccess) return fail(m, IL_ERR_CUDA, "cudaMemcpyPeerAsync: %s", cudaGetErrorString(fetch_err));
-      IL_TRY(component_backward(m, k, used, acc));
+      {
+        Range r2("component backward %d", k);
+        IL_TRY(component_backward(m, k, used, acc));
+      }
       if (k == 0) {
         IL_K(m, embed_bwd(m->tokens[k], m->sort_keys[0], m->cs[0].dx, m->G[k] + m->off_wte, m->G[k] + m->off_wpe, N, m->T, d, m->V, acc ? 1 : 0, st));
         m->launches++;
@@ -1319,6 +1346,7 @@ extern "C" il_status il_lr_schedule(long long step, int d_model, int warmup_step
 extern "C" il_status il_adamw_step(il_model* m, float lr, float beta1, float beta2, float eps, float wd) {
   return guarded([&]() -> il_status {
   IL_TRY(check_model(m));
+  Range range("il_adamw_step");
   if (!m->bwd_done || !m->batch_set) return fail(m, IL_ERR_STATE, "il_adamw_step needs il_backward_nwise of the current step");
   if (m->micro_done != m->micro)
     return fail(m, IL_ERR_STATE, "il_adamw_step after %d of %d micro-batches", m->micro_done, m->micro);
