@@ -25,6 +25,10 @@
  *  - Components, heads and tensors are 0-based.  Matrices are row-major [out, in].
  *  - Work is issued on K CUDA streams (component k on stream k); calls return once the
  *    work is enqueued unless stated otherwise.  One host thread per model.
+ *  - Kernels are launched with programmatic stream serialization: a kernel may become
+ *    resident while its predecessor in the stream drains, and waits (griddepcontrol.wait)
+ *    before it touches global memory.  Stream order as seen by the caller is unchanged.
+ *    IL_NO_DEPENDENT_LAUNCH=1 in the environment (read once) launches the ordinary way.
  *  - Arithmetic: bf16 tensor-core operands, fp32 accumulation, fp32 residual stream,
  *    fp32 master weights, gradients and optimiser state.
  */

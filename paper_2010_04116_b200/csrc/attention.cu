@@ -80,6 +80,7 @@ __global__ void __launch_bounds__(128) attn_fwd_tc_kernel(const __grid_constant_
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  grid_dep_sync();
   const uint32_t tmem_base = tmem_base_smem;                  // scores at columns [0, 64) (then P packed in [0, 32)), O at [64, 64 + dh)
   const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
   volatile int* abortp = &abort_flag;
@@ -287,7 +288,7 @@ cudaError_t fwd_tc_launch(const bf16* qkv, bf16* o, float* lse, int B, int T, in
   cudaError_t e = cudaFuncSetAttribute(attn_fwd_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
   if (e != cudaSuccess) return e;
   dim3 grid((T + TQ - 1) / TQ, B * H);
-  attn_fwd_tc_kernel<DH><<<grid, 128, C::SMEM, s>>>(tmQ, tmKV, o, lse, T, H, rsqrtf((float)DH), err);
+  launch_dep(attn_fwd_tc_kernel<DH>, dim3(grid), dim3(128), C::SMEM, s, tmQ, tmKV, o, lse, T, H, rsqrtf((float)DH), err);
   return cudaGetLastError();
 }
 
@@ -379,6 +380,9 @@ __global__ void __launch_bounds__(256) attn_bwd_dkv_tc_kernel(const __grid_const
     tmem_alloc(smem_u32(&tmem_base_smem), C::TCOLS_KV);
     tmem_relinquish();
   }
+  tc_fence_before();
+  __syncthreads();          // tensor memory is held by this CTA before the next kernel may become resident
+  grid_dep_sync();
   // lse (in log2 units) and delta of a query block: fetched from global memory into a register one sweep
   // step before they are put into shared memory (buffer j&1), two steps before they are used, so that no
   // step waits on that load
@@ -642,6 +646,7 @@ __global__ void __launch_bounds__(256) attn_bwd_dq_tc_kernel(const __grid_consta
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  grid_dep_sync();
   const uint32_t tmem_base = tmem_base_smem;     // S [0,64), dP [64,128) (later in part the packed dS), dQ [128,128+dh)
   const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
   volatile int* abortp = &abort_flag;
@@ -917,6 +922,7 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) attn_bwd_fused_kernel(const 
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  grid_dep_sync();
   const uint32_t tmem_base = tmem_base_smem;
   const float c2 = scale * IL_LOG2E;
   int fail = 0;
@@ -1260,6 +1266,7 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) attn_bwd_fused_kernel(const 
 // dqkv[row, h*dh + c] (the Q third) = bf16(scale * dq_acc[row, h*dh + c]): the accumulated dQ leaves fp32 here.
 __global__ void __launch_bounds__(256) attn_dq_convert_kernel(const float* __restrict__ acc, bf16* __restrict__ dqkv, size_t rows,
                                                               int d, float scale) {
+  grid_dep_sync();
   const int d8 = d >> 3;
   const size_t total = rows * (size_t)d8;
   for (size_t i = (size_t)blockIdx.x * 256 + threadIdx.x; i < total; i += (size_t)gridDim.x * 256) {
@@ -1284,6 +1291,7 @@ template <int DH>
 __global__ void __launch_bounds__(256) attn_delta_tc_kernel(const bf16* __restrict__ dout, const bf16* __restrict__ o,
                                                             float* __restrict__ delta, float* __restrict__ dq_zero, int NB,
                                                             int B, int T, int H) {
+  grid_dep_sync();
   constexpr int TPR = (DH == 80) ? 16 : DH / 8;      // threads per (row, head): a power of two (dh 80: 10 of 16 active)
   const long long gid = (long long)blockIdx.x * 256 + threadIdx.x;
   const long long item = gid / TPR;                  // (row, head) index
@@ -1350,16 +1358,16 @@ cudaError_t bwd_tc_launch(const bf16* qkv, const bf16* o, const float* lse, cons
   if (e != cudaSuccess) return e;
   constexpr int TPR = (DH == 80) ? 16 : DH / 8;
   const long long nthreads = (long long)NB * T * H * TPR;
-  attn_delta_tc_kernel<DH><<<(unsigned)((nthreads + 255) / 256), 256, 0, s>>>(dout, o, delta, nullptr, NB, B, T, H);
+  launch_dep(attn_delta_tc_kernel<DH>, dim3((unsigned)((nthreads + 255) / 256)), dim3(256), 0, s, dout, o, delta, nullptr, NB, B, T, H);
   dim3 grid((T + TQ - 1) / TQ, NB * H);
   const float scale = rsqrtf((float)DH);
   if constexpr (SPLIT) {
-    attn_bwd_dkv_tc_kernel<DH, 1><<<grid, 256, C::SMEM_KV, s>>>(tmRow, tmBlk, tmdO64, lse, delta, dqkv, B, T, H, scale, err);
-    attn_bwd_dkv_tc_kernel<DH, 2><<<grid, 256, C::SMEM_KV, s>>>(tmRow, tmBlk, tmdO64, lse, delta, dqkv, B, T, H, scale, err);
+    launch_dep(attn_bwd_dkv_tc_kernel<DH, 1>, dim3(grid), dim3(256), C::SMEM_KV, s, tmRow, tmBlk, tmdO64, lse, delta, dqkv, B, T, H, scale, err);
+    launch_dep(attn_bwd_dkv_tc_kernel<DH, 2>, dim3(grid), dim3(256), C::SMEM_KV, s, tmRow, tmBlk, tmdO64, lse, delta, dqkv, B, T, H, scale, err);
   } else {
-    attn_bwd_dkv_tc_kernel<DH, 0><<<grid, 256, C::SMEM_KV, s>>>(tmRow, tmBlk, tmdO64, lse, delta, dqkv, B, T, H, scale, err);
+    launch_dep(attn_bwd_dkv_tc_kernel<DH, 0>, dim3(grid), dim3(256), C::SMEM_KV, s, tmRow, tmBlk, tmdO64, lse, delta, dqkv, B, T, H, scale, err);
   }
-  attn_bwd_dq_tc_kernel<DH><<<grid, 256, C::SMEM_Q, s>>>(tmRow, tmBlk, tmdO128, lse, delta, dqkv, B, T, H, scale, err);
+  launch_dep(attn_bwd_dq_tc_kernel<DH>, dim3(grid), dim3(256), C::SMEM_Q, s, tmRow, tmBlk, tmdO128, lse, delta, dqkv, B, T, H, scale, err);
   return cudaGetLastError();
 }
 
@@ -1386,7 +1394,7 @@ cudaError_t bwd_fused_launch(const bf16* qkv, const bf16* o, const float* lse, c
   if (e != cudaSuccess) return e;
   constexpr int TPR = DH / 8;
   const long long nthreads = (long long)NB * T * H * TPR;
-  attn_delta_tc_kernel<DH><<<(unsigned)((nthreads + 255) / 256), 256, 0, s>>>(dout, o, delta, dq_acc, NB, B, T, H);
+  launch_dep(attn_delta_tc_kernel<DH>, dim3((unsigned)((nthreads + 255) / 256)), dim3(256), 0, s, dout, o, delta, dq_acc, NB, B, T, H);
   // persistent CTAs, one per SM, each walking its share of the (key tile, sequence, head) items
   int dev = 0, sms = 0;
   if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
@@ -1394,11 +1402,11 @@ cudaError_t bwd_fused_launch(const bf16* qkv, const bf16* o, const float* lse, c
   const long long nitems = (long long)((T + TQ - 1) / TQ) * NB * H;
   const int grid = (int)(nitems < sms ? nitems : sms);
   const float scale = rsqrtf((float)DH);
-  attn_bwd_fused_kernel<DH><<<grid, FUSED_THREADS, C::SMEM, s>>>(tmRow, tmdO, tmAcc, lse, delta, dqkv, NB, B, T, H, scale, err);
+  launch_dep(attn_bwd_fused_kernel<DH>, dim3(grid), dim3(FUSED_THREADS), C::SMEM, s, tmRow, tmdO, tmAcc, lse, delta, dqkv, NB, B, T, H, scale, err);
   const size_t rows = (size_t)NB * T;
   size_t blocks = (rows * (size_t)(H * DH / 8) + 255) / 256;
   if (blocks > 148 * 16) blocks = 148 * 16;
-  attn_dq_convert_kernel<<<(unsigned)blocks, 256, 0, s>>>(dq_acc, dqkv, rows, H * DH, scale);
+  launch_dep(attn_dq_convert_kernel, dim3((unsigned)blocks), dim3(256), 0, s, dq_acc, dqkv, rows, H * DH, scale);
   return cudaGetLastError();
 }
 

@@ -5,6 +5,10 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <cstdlib>
+#include <cstring>
+#include <utility>
+
 namespace il {
 
 typedef __nv_bfloat16 bf16;
@@ -379,6 +383,47 @@ __device__ __forceinline__ void red_add_f32x4(float* addr, float4 v) {
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// ---- programmatic dependent launch ----------------------------------------------------------------
+// A step is several hundred short kernels, each depending on the one before it in its stream.  Launched with
+// launch_dep() a kernel may become resident while its predecessor is still draining: its CTAs take the SMs the
+// predecessor's CTAs leave, set themselves up (barriers, tensor memory, descriptor prefetch) and then stop in
+// grid_dep_sync() until the predecessor has completed and its memory is visible.  Rules every kernel follows:
+//   * nothing in global memory is read or written before grid_dep_sync(), and every thread executes it;
+//   * a CTA calls grid_dep_sync() only after it holds all the resources it will ever take (tensor memory above
+//     all): the successor's CTAs may then take what is left without this kernel ever waiting for them;
+//   * the same call lets the successor become resident (the successor of a kernel is therefore launched only
+//     after the kernel's own predecessor has completed: at most two kernels of a stream are on the GPU).
+// On a kernel launched the ordinary way, or first in its stream, both instructions do nothing.
+__device__ __forceinline__ void grid_dep_sync() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+// IL_NO_DEPENDENT_LAUNCH=1 in the environment turns the launch attribute off (ordinary stream order).
+inline bool dependent_launch_enabled() {
+  static const bool on = [] {
+    const char* e = getenv("IL_NO_DEPENDENT_LAUNCH");
+    return !(e && e[0] == '1');
+  }();
+  return on;
+}
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dep(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof cfg);
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = dependent_launch_enabled() ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, KArgs(std::forward<Args>(args))...);
 }
 
 }  // namespace il

@@ -13,6 +13,7 @@ static inline int ceil_div(long long a, long long b) { return (int)((a + b - 1) 
 // ---------------------------------------------------------------------------------------------
 __global__ void embed_fwd_kernel(const int* __restrict__ tok, const float* __restrict__ wte,
                                  const float* __restrict__ wpe, float* __restrict__ x, int ntok, int T, int d, int V) {
+  grid_dep_sync();
   const int d4 = d >> 2;
   const size_t total = (size_t)ntok * d4;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
@@ -31,7 +32,7 @@ cudaError_t embed_fwd(const int* tok, const float* wte, const float* wpe, float*
   const size_t total = (size_t)ntok * (d / 4);
   int blocks = ceil_div(total, 256);
   if (blocks > 148 * 16) blocks = 148 * 16;
-  embed_fwd_kernel<<<blocks, 256, 0, s>>>(tok, wte, wpe, x, ntok, T, d, V);
+  launch_dep(embed_fwd_kernel, dim3(blocks), dim3(256), 0, s, tok, wte, wpe, x, ntok, T, d, V);
   return cudaGetLastError();
 }
 
@@ -47,6 +48,7 @@ constexpr int SORT_POS_BITS = 13;
 
 __global__ void __launch_bounds__(1024) embed_sort_kernel(const int* __restrict__ tok, unsigned* __restrict__ keys, int ntok,
                                                           int V) {
+  grid_dep_sync();
   __shared__ unsigned sk[SORT_CHUNK];
   const int base = blockIdx.x * SORT_CHUNK;
   for (int i = threadIdx.x; i < SORT_CHUNK; i += 1024) {
@@ -75,7 +77,7 @@ __global__ void __launch_bounds__(1024) embed_sort_kernel(const int* __restrict_
 
 cudaError_t embed_sort(const int* tok, unsigned* keys, int ntok, int V, cudaStream_t s) {
   if (V > (1 << (32 - SORT_POS_BITS)) - 1) return cudaErrorInvalidValue;
-  embed_sort_kernel<<<ceil_div(ntok, SORT_CHUNK), 1024, 0, s>>>(tok, keys, ntok, V);
+  launch_dep(embed_sort_kernel, dim3(ceil_div(ntok, SORT_CHUNK)), dim3(1024), 0, s, tok, keys, ntok, V);
   return cudaGetLastError();
 }
 
@@ -85,6 +87,7 @@ cudaError_t embed_sort(const int* tok, unsigned* keys, int ntok, int V, cudaStre
 __global__ void __launch_bounds__(1024) embed_bwd_wte_kernel(const unsigned* __restrict__ keys, const float* __restrict__ dx,
                                                              float* __restrict__ dwte, int chunk_base, int ntok, int d,
                                                              int accumulate) {
+  grid_dep_sync();
   __shared__ float4 part[3][256];
   const int i = blockIdx.x;                            // index within the chunk
   const unsigned key = keys[chunk_base + i];
@@ -136,6 +139,7 @@ __global__ void __launch_bounds__(1024) embed_bwd_wte_kernel(const unsigned* __r
 }
 __global__ void embed_bwd_wpe_kernel(const float* __restrict__ dx, float* __restrict__ dwpe, int B, int T, int d,
                                      int accumulate) {
+  grid_dep_sync();
   const int d4 = d >> 2;
   const size_t total = (size_t)T * d4;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
@@ -153,10 +157,10 @@ cudaError_t embed_bwd(const int* tok, const unsigned* keys, const float* dx, flo
   (void)tok; (void)V;
   // chunk after chunk on the one stream: a token that occurs in several chunks is added to in chunk order
   for (int base = 0; base < ntok; base += SORT_CHUNK)
-    embed_bwd_wte_kernel<<<min(SORT_CHUNK, ntok - base), 1024, 0, s>>>(keys, dx, dwte, base, ntok, d,
+    launch_dep(embed_bwd_wte_kernel, dim3(min(SORT_CHUNK, ntok - base)), dim3(1024), 0, s, keys, dx, dwte, base, ntok, d,
                                                                         (accumulate || base > 0) ? 1 : 0);
   int blocks2 = ceil_div((size_t)T * (d / 4), 256);
-  embed_bwd_wpe_kernel<<<blocks2, 256, 0, s>>>(dx, dwpe, ntok / T, T, d, accumulate);
+  launch_dep(embed_bwd_wpe_kernel, dim3(blocks2), dim3(256), 0, s, dx, dwpe, ntok / T, T, d, accumulate);
   return cudaGetLastError();
 }
 
@@ -167,6 +171,7 @@ __global__ void __launch_bounds__(256) layernorm_fwd_kernel(const float* __restr
                                                             const float* __restrict__ beta, bf16* __restrict__ y,
                                                             float* __restrict__ mean, float* __restrict__ rstd,
                                                             int rows, int d, float eps) {
+  grid_dep_sync();
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (row >= rows) return;
@@ -204,6 +209,7 @@ __global__ void __launch_bounds__(256) layernorm_fwd_reg_kernel(const float* __r
                                                                 const float* __restrict__ beta, bf16* __restrict__ y,
                                                                 float* __restrict__ mean, float* __restrict__ rstd,
                                                                 int rows, float eps) {
+  grid_dep_sync();
   constexpr int d = NV * 128;
   const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
@@ -240,11 +246,11 @@ cudaError_t layernorm_fwd(const float* x, const float* gamma, const float* beta,
                           int rows, int d, float eps, cudaStream_t s) {
   const int blocks = ceil_div(rows, 8);
 #define IL_LNR(NV) \
-  case NV: layernorm_fwd_reg_kernel<NV><<<blocks, 256, 0, s>>>(x, gamma, beta, y, mean, rstd, rows, eps); break;
+  case NV: launch_dep(layernorm_fwd_reg_kernel<NV>, dim3(blocks), dim3(256), 0, s, x, gamma, beta, y, mean, rstd, rows, eps); break;
   if (d % 128 == 0 && d <= 1024) {
     switch (d / 128) { IL_LNR(1) IL_LNR(2) IL_LNR(3) IL_LNR(4) IL_LNR(5) IL_LNR(6) IL_LNR(7) IL_LNR(8) }
   } else {
-    layernorm_fwd_kernel<<<blocks, 256, 0, s>>>(x, gamma, beta, y, mean, rstd, rows, d, eps);
+    launch_dep(layernorm_fwd_kernel, dim3(blocks), dim3(256), 0, s, x, gamma, beta, y, mean, rstd, rows, d, eps);
   }
 #undef IL_LNR
   return cudaGetLastError();
@@ -272,6 +278,7 @@ __global__ void __launch_bounds__(256) layernorm_bwd_rows_kernel(const void* __r
                                                                  const float* __restrict__ gamma, const float* resid,
                                                                  float* dx_out, bf16* __restrict__ dx_bf16, int rows,
                                                                  int x_rows, int d) {
+  grid_dep_sync();
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (row >= rows) return;
@@ -320,10 +327,10 @@ cudaError_t layernorm_bwd_rows(const void* dy, int dy_is_f32, const float* x, co
                                const float* gamma, const float* resid, float* dx_out, bf16* dx_bf16, int rows, int x_rows,
                                int d, cudaStream_t s) {
   if (dy_is_f32)
-    layernorm_bwd_rows_kernel<true><<<ceil_div(rows, 8), 256, 0, s>>>(dy, x, mean, rstd, gamma, resid, dx_out, dx_bf16,
+    launch_dep(layernorm_bwd_rows_kernel<true>, dim3(ceil_div(rows, 8)), dim3(256), 0, s, dy, x, mean, rstd, gamma, resid, dx_out, dx_bf16,
                                                                        rows, x_rows, d);
   else
-    layernorm_bwd_rows_kernel<false><<<ceil_div(rows, 8), 256, 0, s>>>(dy, x, mean, rstd, gamma, resid, dx_out, dx_bf16,
+    launch_dep(layernorm_bwd_rows_kernel<false>, dim3(ceil_div(rows, 8)), dim3(256), 0, s, dy, x, mean, rstd, gamma, resid, dx_out, dx_bf16,
                                                                         rows, x_rows, d);
   return cudaGetLastError();
 }
@@ -345,6 +352,7 @@ __global__ void __launch_bounds__(256, 1) layernorm_bwd_fused_kernel(const bf16*
                                                                      float* dx_out, bf16* __restrict__ dx_bf16,
                                                                      float* __restrict__ dgamma, float* __restrict__ dbeta,
                                                                      float* __restrict__ colsum, int rows, int x_rows) {
+  grid_dep_sync();
   constexpr int d = NV * 128;
   __shared__ float4 red[8][NV * 32];
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
@@ -438,7 +446,7 @@ cudaError_t layernorm_bwd_fused(const bf16* dy, const float* x, const float* mea
   if (blocks > 148) blocks = 148;
 #define IL_LNF(NV)                                                                                                        \
   case NV:                                                                                                                \
-    layernorm_bwd_fused_kernel<NV><<<blocks, 256, 0, s>>>(dy, x, mean, rstd, gamma, resid, dx_out, dx_bf16, dgamma, dbeta, \
+    launch_dep(layernorm_bwd_fused_kernel<NV>, dim3(blocks), dim3(256), 0, s, dy, x, mean, rstd, gamma, resid, dx_out, dx_bf16, dgamma, dbeta, \
                                                           colsum, rows, x_rows);                                          \
     break;
   switch (d / 128) {
@@ -459,6 +467,7 @@ __global__ void __launch_bounds__(256) layernorm_bwd_params_kernel(const void* _
                                                                    const float* __restrict__ rstd,
                                                                    float* __restrict__ dgamma, float* __restrict__ dbeta,
                                                                    int rows, int d, int rows_per_block) {
+  grid_dep_sync();
   __shared__ float4 sg[8][32], sb[8][32];
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const int c4 = blockIdx.x * 32 + lane;       // float4 column index
@@ -508,15 +517,16 @@ cudaError_t layernorm_bwd_params(const void* dy, int dy_is_f32, const float* x, 
   int rpb;
   colreduce_grid(rows, 128, d, &grid, &rpb);
   if (dy_is_f32)
-    layernorm_bwd_params_kernel<true><<<grid, 256, 0, s>>>(dy, x, mean, rstd, dgamma, dbeta, rows, d, rpb);
+    launch_dep(layernorm_bwd_params_kernel<true>, dim3(grid), dim3(256), 0, s, dy, x, mean, rstd, dgamma, dbeta, rows, d, rpb);
   else
-    layernorm_bwd_params_kernel<false><<<grid, 256, 0, s>>>(dy, x, mean, rstd, dgamma, dbeta, rows, d, rpb);
+    launch_dep(layernorm_bwd_params_kernel<false>, dim3(grid), dim3(256), 0, s, dy, x, mean, rstd, dgamma, dbeta, rows, d, rpb);
   return cudaGetLastError();
 }
 
 template <bool IN_F32>
 __global__ void __launch_bounds__(256) colsum_kernel(const void* __restrict__ y, int ld, float* __restrict__ out, int rows,
                                                      int cols, int rows_per_block) {
+  grid_dep_sync();
   __shared__ float4 sm[8][32];
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const int c4 = blockIdx.x * 32 + lane;
@@ -553,14 +563,14 @@ cudaError_t colsum_bf16(const bf16* y, int ld, float* out, int rows, int cols, c
   dim3 grid;
   int rpb;
   colreduce_grid(rows, 128, cols, &grid, &rpb);
-  colsum_kernel<false><<<grid, 256, 0, s>>>(y, ld, out, rows, cols, rpb);
+  launch_dep(colsum_kernel<false>, dim3(grid), dim3(256), 0, s, y, ld, out, rows, cols, rpb);
   return cudaGetLastError();
 }
 cudaError_t colsum_f32(const float* y, int ld, float* out, int rows, int cols, cudaStream_t s) {
   dim3 grid;
   int rpb;
   colreduce_grid(rows, 128, cols, &grid, &rpb);
-  colsum_kernel<true><<<grid, 256, 0, s>>>(y, ld, out, rows, cols, rpb);
+  launch_dep(colsum_kernel<true>, dim3(grid), dim3(256), 0, s, y, ld, out, rows, cols, rpb);
   return cudaGetLastError();
 }
 
@@ -569,6 +579,7 @@ cudaError_t colsum_f32(const float* y, int ld, float* out, int rows, int cols, c
 // ---------------------------------------------------------------------------------------------
 __global__ void add_convert_kernel(const float4* __restrict__ a, const float4* __restrict__ b, float4* out_f32,
                                    uint2* __restrict__ out_bf16, size_t n4) {
+  grid_dep_sync();
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
     float4 v = a[i];
     if (b) {
@@ -590,7 +601,7 @@ cudaError_t add_convert(const float* a, const float* b, float* out_f32, bf16* ou
   int blocks = ceil_div(n4, 256);
   if (blocks > 148 * 16) blocks = 148 * 16;
   if (blocks < 1) blocks = 1;
-  add_convert_kernel<<<blocks, 256, 0, s>>>(reinterpret_cast<const float4*>(a), reinterpret_cast<const float4*>(b),
+  launch_dep(add_convert_kernel, dim3(blocks), dim3(256), 0, s, reinterpret_cast<const float4*>(a), reinterpret_cast<const float4*>(b),
                                             reinterpret_cast<float4*>(out_f32), reinterpret_cast<uint2*>(out_bf16), n4);
   return cudaGetLastError();
 }
@@ -598,6 +609,7 @@ cudaError_t add_convert(const float* a, const float* b, float* out_f32, bf16* ou
 struct LinComb { const float4* x[4]; float w[4]; int count; int accumulate; };
 
 __global__ void lincomb_convert_kernel(LinComb c, float4* out_f32, uint2* __restrict__ out_bf16, size_t n4) {
+  grid_dep_sync();
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
     float4 v = c.accumulate ? out_f32[i] : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
@@ -630,7 +642,7 @@ cudaError_t lincomb_convert(const float* const* x, const float* w, int count, in
   int blocks = ceil_div(n4, 256);
   if (blocks > 148 * 16) blocks = 148 * 16;
   if (blocks < 1) blocks = 1;
-  lincomb_convert_kernel<<<blocks, 256, 0, s>>>(c, reinterpret_cast<float4*>(out_f32), reinterpret_cast<uint2*>(out_bf16), n4);
+  launch_dep(lincomb_convert_kernel, dim3(blocks), dim3(256), 0, s, c, reinterpret_cast<float4*>(out_f32), reinterpret_cast<uint2*>(out_bf16), n4);
   return cudaGetLastError();
 }
 
@@ -644,6 +656,7 @@ cudaError_t f32_to_bf16(const float* in, bf16* out, size_t n, cudaStream_t s) {
 __global__ void __launch_bounds__(256) lse_finalize_kernel(const float* __restrict__ pm, const float* __restrict__ ps,
                                                            int part_ld, int ntiles, const float* __restrict__ tgt_logit,
                                                            float* __restrict__ lse, float* __restrict__ nll, int rows) {
+  grid_dep_sync();
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const int row = blockIdx.x * 8 + w;
   if (row >= rows) return;
@@ -665,13 +678,14 @@ __global__ void __launch_bounds__(256) lse_finalize_kernel(const float* __restri
 
 cudaError_t lse_finalize(const float* part_max, const float* part_sum, int part_ld, int ntiles, const float* tgt_logit,
                          float* lse, float* nll, int rows, cudaStream_t s) {
-  lse_finalize_kernel<<<ceil_div(rows, 8), 256, 0, s>>>(part_max, part_sum, part_ld, ntiles, tgt_logit, lse, nll, rows);
+  launch_dep(lse_finalize_kernel, dim3(ceil_div(rows, 8)), dim3(256), 0, s, part_max, part_sum, part_ld, ntiles, tgt_logit, lse, nll, rows);
   return cudaGetLastError();
 }
 
 // out[0] = mean of x[0..n) with a fixed summation order (one block: strided per-thread sums, then a tree), so the
 // value does not depend on scheduling.
 __global__ void __launch_bounds__(1024) mean_f32_kernel(const float* __restrict__ x, int n, float* __restrict__ out) {
+  grid_dep_sync();
   __shared__ float sm[1024];
   float a = 0.f;
   for (int i = threadIdx.x; i < n; i += 1024) a += x[i];
@@ -685,7 +699,7 @@ __global__ void __launch_bounds__(1024) mean_f32_kernel(const float* __restrict_
 }
 
 cudaError_t mean_f32(const float* x, int n, float* out, cudaStream_t s) {
-  mean_f32_kernel<<<1, 1024, 0, s>>>(x, n, out);
+  launch_dep(mean_f32_kernel, dim3(1), dim3(1024), 0, s, x, n, out);
   return cudaGetLastError();
 }
 
@@ -702,6 +716,7 @@ __global__ void __launch_bounds__(256) head_backward_prepare_kernel(bf16* __rest
                                                                     const int* __restrict__ targets, const bf16* __restrict__ u,
                                                                     bf16* __restrict__ u_scaled, float* __restrict__ rowscale,
                                                                     int rows, int d, float inv_rows, unsigned* err) {
+  grid_dep_sync();
   const int lane = threadIdx.x & 31;
   const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
   if (row >= rows) return;
@@ -733,7 +748,7 @@ __global__ void __launch_bounds__(256) head_backward_prepare_kernel(bf16* __rest
 cudaError_t head_backward_prepare(bf16* e, int ld, const float* lse, const int* targets, const bf16* u, bf16* u_scaled,
                                   float* rowscale, int rows, int d, float scale, unsigned* err, cudaStream_t s) {
   if ((d % 8) || ((uintptr_t)u % 16) || ((uintptr_t)u_scaled % 16) || !err) return cudaErrorInvalidValue;
-  head_backward_prepare_kernel<<<ceil_div(rows, 8), 256, 0, s>>>(e, ld, lse, targets, u, u_scaled, rowscale, rows, d,
+  launch_dep(head_backward_prepare_kernel, dim3(ceil_div(rows, 8)), dim3(256), 0, s, e, ld, lse, targets, u, u_scaled, rowscale, rows, d,
                                                                  scale / (float)rows, err);
   return cudaGetLastError();
 }
@@ -746,6 +761,7 @@ __global__ void __launch_bounds__(256) adamw_kernel(float4* __restrict__ p, floa
                                                     size_t n4_decay, float lr, float b1, float b2, float eps, float wd,
                                                     float ibc1, float ibc2, const unsigned* __restrict__ err,
                                                     unsigned* applied, size_t skip0, size_t skip1) {
+  grid_dep_sync();
   // a step whose kernels reported an error must not reach the parameters: leave everything as it is
   if (err && *reinterpret_cast<const volatile unsigned*>(err) != 0u) return;
   if (applied && blockIdx.x == 0 && threadIdx.x == 0) *applied += 1u;
@@ -775,7 +791,7 @@ cudaError_t adamw(float* p, float* m, float* v, const float* g, bf16* p_bf16, si
   if (n4 == 0) return cudaSuccess;
   int blocks = ceil_div(n4, 256);
   if (blocks > 148 * 16) blocks = 148 * 16;
-  adamw_kernel<<<blocks, 256, 0, s>>>(reinterpret_cast<float4*>(p), reinterpret_cast<float4*>(m),
+  launch_dep(adamw_kernel, dim3(blocks), dim3(256), 0, s, reinterpret_cast<float4*>(p), reinterpret_cast<float4*>(m),
                                       reinterpret_cast<float4*>(v), reinterpret_cast<const float4*>(g),
                                       reinterpret_cast<uint2*>(p_bf16), n4, n_decay / 4, lr, beta1, beta2, eps, wd,
                                       1.0f / bc1, 1.0f / bc2, err, applied, skip_begin / 4, skip_end / 4);
@@ -788,6 +804,7 @@ cudaError_t adamw(float* p, float* m, float* v, const float* g, bf16* p_bf16, si
 // without any kernel having to go wrong.
 // ---------------------------------------------------------------------------------------------
 __global__ void wait_probe_kernel(unsigned* err, unsigned long long limit_ns) {
+  grid_dep_sync();
   __shared__ unsigned long long bar;
   __shared__ int never;
   if (threadIdx.x == 0) {
@@ -799,7 +816,7 @@ __global__ void wait_probe_kernel(unsigned* err, unsigned long long limit_ns) {
 }
 
 cudaError_t wait_probe(unsigned* err, unsigned long long limit_ns, cudaStream_t s) {
-  wait_probe_kernel<<<1, 32, 0, s>>>(err, limit_ns);
+  launch_dep(wait_probe_kernel, dim3(1), dim3(32), 0, s, err, limit_ns);
   return cudaGetLastError();
 }
 

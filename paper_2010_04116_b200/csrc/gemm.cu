@@ -319,6 +319,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   __syncthreads();
   cluster_sync_all();       // the peer's barriers are initialised before anything is signalled remotely
   tc_fence_after();
+  grid_dep_sync();          // tensor memory is held, nothing in global memory has been touched yet
   const uint32_t tmem_base = tmem_base_smem;
   volatile int* abortp = &abort_flag;
 
@@ -855,7 +856,7 @@ cudaError_t gemm_launch(const GemmArgs& a, unsigned* err_word, int num_sms, cuda
   const long long tiles = (long long)p.tiles_m * p.tiles_n * p.split_k;
   const int pairs = (int)(tiles < num_sms / 2 ? tiles : num_sms / 2);
   const int grid = 2 * pairs;
-  kern<<<grid, GEMM_THREADS, nt == 2 ? smem_bytes<2>() : smem_bytes<1>(), stream>>>(tmA, tmB, p);
+  launch_dep(kern, dim3(grid), dim3(GEMM_THREADS), nt == 2 ? smem_bytes<2>() : smem_bytes<1>(), stream, tmA, tmB, p);
   return cudaGetLastError();
 }
 

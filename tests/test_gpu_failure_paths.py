@@ -242,3 +242,47 @@ def test_pipeline_placement_on_one_device_reproduces_the_single_device_step(n, r
 
 def test_noalloc_status_reports_no_error():
     assert il.op_attention_bwd_noalloc_status() == 0
+
+
+_STEP_DIGEST = r"""
+import hashlib, sys
+import numpy as np
+import workloads as wl
+from paper_2010_04116_b200 import Model
+w = wl.Workload("det", K=3, Lc=1, d=128, H=2, F=256, V=64, T=128, B=6, n=2, zipf=True)
+P = wl.draw_params(w)
+tok, tgt = wl.draw_tokens(w)
+m = Model(w.K, w.Lc, w.d, w.H, w.F, w.V, 2, w.B, w.T, attn_bwd="two_kernels")
+m.set_params(P)
+m.train_step(tok, tgt)
+losses = m.get_losses()
+m.sync()
+h = hashlib.sha256(np.asarray(losses, dtype=np.float32).tobytes())
+for k in range(w.K + 1):
+    h.update(np.ascontiguousarray(m.get_boundary(k, w.ntok)).tobytes())
+for nm in m.names:
+    g = m.get_grad(nm)
+    if g.ndim == 2:
+        h.update(np.ascontiguousarray(g).tobytes())
+m.close()
+print("DIGEST", h.hexdigest())
+"""
+
+
+def test_dependent_launch_and_ordinary_launch_give_identical_bits():
+    """Kernels launched so that they may become resident while their predecessor drains (the default) wait for
+    it before touching memory: losses, boundary activations and weight-matrix gradients are bit for bit those
+    of the same step launched in ordinary stream order (two fresh processes; the switch is read once)."""
+    import os
+    import subprocess
+    import sys
+
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    digests = []
+    for off in ("0", "1"):
+        env = dict(os.environ, IL_NO_DEPENDENT_LAUNCH=off, PYTHONPATH=root)
+        out = subprocess.run([sys.executable, "-c", _STEP_DIGEST], cwd=root, env=env, capture_output=True, text=True,
+                             timeout=600)
+        assert out.returncode == 0, out.stderr[-2000:]
+        digests.append([l for l in out.stdout.splitlines() if l.startswith("DIGEST")][0])
+    assert digests[0] == digests[1]
