@@ -143,13 +143,18 @@ il_status il_forward_component(il_model* m, int k);
  *                     (vocab * 2 bytes per token and head: 824 MB per head at 8192 tokens and a 50257-word
  *                     vocabulary); the backward runs its two contractions on that matrix without recomputing
  *                     anything.  Price besides the memory: every row's log-sum-exp must lie in [-80, 80]
- *                     (checked; a violation makes il_sync return IL_ERR_NONFINITE and skips the update).
+ *                     (checked; a violation makes il_sync return IL_ERR_NONFINITE, skips the update and
+ *                     switches the model to IL_HEAD_RECOMPUTE for all later steps, reusing the matrix's memory
+ *                     as the chunk buffer: parameters and optimiser state are untouched, so the caller repeats
+ *                     the step; il_head_mode reads the mode in force).
  *   IL_HEAD_RECOMPUTE nothing of size [B*T, vocab] is ever held: the backward walks the vocabulary in chunks of
  *                     8192 columns, forms the chunk's logits again, turns them into dZ in the epilogue and
  *                     feeds dZ to the two gradient contractions (one third more head flops, no range limit).
  * Needs il_forward_component(k).  loss_host != NULL makes the call wait for this head and return its loss;
  * NULL leaves it asynchronous. */
 il_status il_aux_head_loss(il_model* m, int k, float* loss_host);
+/* The head mode in force (IL_HEAD_STORED or IL_HEAD_RECOMPUTE; see above); -1 for a NULL model. */
+int il_head_mode(const il_model* m);
 /* Per-token negative log-likelihood of head k for the current step, fp32 [B*T] to host (their mean is
  * the head's loss).  Needs il_aux_head_loss(k); waits for it. */
 il_status il_get_token_losses(il_model* m, int k, float* host, size_t count);

@@ -88,6 +88,7 @@ def lib() -> C.CDLL:
         "il_pipeline_transfers": [i, i, i, C.POINTER(i), i, C.POINTER(i)],
         "il_pipeline_last_transfers": [vp, C.POINTER(i), i, C.POINTER(i)],
         "il_error_word": [vp, i, C.POINTER(vp)],
+        "il_head_mode": [vp],
         "il_op_wait_probe": [vp, C.c_uint, vp],
         "il_op_attention_bwd_noalloc_status": [vp],
         "il_time_per_batch": [i, i, i, C.c_double, C.c_double, C.POINTER(C.c_double)],
@@ -201,7 +202,7 @@ class Model:
         opt.head_mode = {"stored": 0, "recompute": 1}[head_mode]
         opt.placement = {"single": 0, "pipeline": 1}[placement]
         opt.attn_bwd = {"one_sweep": 0, "two_kernels": 1}[attn_bwd]
-        self.head_mode, self.placement = head_mode, placement
+        self.placement = placement
         self.devices = list(devices) if devices is not None else [device] * K
         if devices is not None:
             self._dev_arr = (C.c_int * K)(*self.devices)
@@ -387,6 +388,11 @@ class Model:
         out = np.empty((ntok, self.d), dtype=np.float32)
         self._ck(self.L.il_get_boundary(self._h, k, out.ctypes.data, out.size))
         return out
+
+    @property
+    def head_mode(self) -> str:
+        """The head mode in force: a stored-mode model switches to "recompute" when a row leaves the stored form's range."""
+        return {0: "stored", 1: "recompute"}[self.L.il_head_mode(self._h)]
 
     def stats(self):
         b, l = C.c_longlong(0), C.c_longlong(0)

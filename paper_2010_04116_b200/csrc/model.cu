@@ -131,7 +131,8 @@ struct il_model {
   std::vector<int> xfer_log;          // pipeline placement: (direction, boundary, id) of every copy of the current step
   std::vector<unsigned*> sort_keys;   // [0]: scratch of the deterministic embedding backward on component 0's device
   int part_ld;
-  int ldz;                            // row stride of the saved logits (vocabulary rounded up to 64)
+  int ldz;                            // stored mode: row stride of exp(logits) (vocabulary rounded up to 64)
+  int head_chunk;                     // recompute mode: columns per vocabulary chunk = row stride of the dZ chunk
   // step state
   int B, T, ntok;
   bool batch_set, bwd_done;
@@ -664,6 +665,10 @@ extern "C" il_status il_create(int K, int Lc, int d, int H, int F, int V, int n,
   // stored mode: row stride of exp(logits) = the vocabulary rounded up to 64; recompute mode: the width of one
   // vocabulary chunk of dZ (a multiple of the 256-column tile)
   m->ldz = m->head_mode == IL_HEAD_STORED ? (V + 63) / 64 * 64 : std::min(HEAD_CHUNK, (V + 255) / 256 * 256);
+  // A stored-mode model can fall back to recomputation (il_sync, after a row left the representable range): its
+  // [Ntok, ldz] buffer then serves as the chunk buffer, so the chunk is the largest multiple of 256 it holds
+  // (the whole vocabulary in one chunk when it is narrower than that).
+  m->head_chunk = m->head_mode != IL_HEAD_STORED ? m->ldz : (m->ldz >= 256 ? std::min(HEAD_CHUNK, m->ldz / 256 * 256) : m->ldz);
   m->hs.assign(K, HeadScratch{});
   for (int k = 0; k < K; ++k) {
     IL_CUDA(m, cudaSetDevice(m->dev[k]));
@@ -1124,7 +1129,7 @@ il_status head_backward(il_model* m, int k, bool acc, float scale) {
     // columns; per chunk the logits are formed again and turned into dZ = (softmax - onehot) * scale / Ntok in the
     // GEMM's epilogue (bf16, [Ntok, chunk]), then dU += dZ W_chunk and dW_chunk = dZ^T U.  The chunks follow each
     // other on this head's stream, so dU is summed in a fixed order.
-    const int chunk = m->ldz;
+    const int chunk = m->head_chunk;
     for (int c0 = 0; c0 < V; c0 += chunk) {
       const int w = std::min(chunk, V - c0);
       {
@@ -1412,9 +1417,14 @@ extern "C" il_status il_sync(il_model* m) {
     // updates that were applied.  A component whose update ran before another component raised the error keeps it.
     m->step -= (issued - applied_max);
     const char* partial = applied_min != applied_max ? "; some components applied an update that others skipped" : "";
-    if (first == DEV_LOGIT_RANGE)
+    if (first == DEV_LOGIT_RANGE) {
+      // Only the stored-exp(logit) head has this limit.  From here on the model recomputes the logits in the head
+      // backward instead (the stored matrix's memory becomes the chunk buffer); the caller repeats the step.
+      m->head_mode = IL_HEAD_RECOMPUTE;
       return fail(m, IL_ERR_NONFINITE, "a head's log-sum-exp left [-80, 80]: exp(logit) is not representable; "
-                  "%d of %d optimiser updates since the last il_sync were applied%s", applied_max, issued, partial);
+                  "%d of %d optimiser updates since the last il_sync were applied%s; the model has switched to "
+                  "IL_HEAD_RECOMPUTE (no range limit): repeat the step", applied_max, issued, partial);
+    }
     return fail(m, IL_ERR_TIMEOUT, "a bounded device-side wait expired (code %u); %d of %d optimiser updates since the "
                 "last il_sync were applied%s", first, applied_max, issued, partial);
   }
@@ -1433,6 +1443,8 @@ extern "C" il_status il_get_boundary(il_model* m, int k, float* host, size_t cou
   return IL_OK;
   });
 }
+
+extern "C" int il_head_mode(const il_model* m) { return m ? m->head_mode : -1; }
 
 extern "C" il_status il_stats(const il_model* m, long long* device_bytes, long long* kernel_launches) {
   return guarded([&]() -> il_status {

@@ -11,7 +11,8 @@ of its n-wise gradient and its values at seeded sample positions.  <cfg>_n<n>.np
 see tests/golden/sketch.py): per tensor a 64-bucket count sketch (64 seeded +-1 projections with disjoint
 supports, whose squared distance estimates the squared L2 distance), the whole gradient of every rank-1 tensor
 and four full rows of every matrix.  Takes minutes (GPT-2-small shape) to tens of minutes (GPT-2-medium
-shape) on 8 cores and up to ~45 GB of host memory.
+shape) on 8 cores and up to ~45 GB of host memory; the 2.7B-parameter shape takes half an hour on 16 cores and more
+than 62 GB in the plain form (the bounded form trades time for memory).
 """
 from __future__ import annotations
 

@@ -100,6 +100,38 @@ def test_recompute_head_has_no_logit_range_limit():
         m.close()
 
 
+def test_stored_head_falls_back_to_recomputation_when_a_row_leaves_its_range():
+    """The stored-exp(logit) head reports a row outside [-80, 80] and the model switches to the recomputing head
+    (which has no such limit) for all later steps: the repeated step succeeds, and gives bit for bit what a model
+    created in recompute mode gives (same chunking, same kernels)."""
+    w, m, P, tok, tgt = _small(n=2, attn_bwd="two_kernels")           # every sum of these sizes in a fixed order
+    _, m2, _, _, _ = _small(n=2, head_mode="recompute", attn_bwd="two_kernels")
+    try:
+        bad = (P["head0.w"] * 4000.0).astype(np.float32)
+        assert m.head_mode == "stored" and m2.head_mode == "recompute"
+        m.set_param("head0.w", bad)
+        m2.set_param("head0.w", bad)
+        with pytest.raises(ILError) as e:
+            m.train_step(tok, tgt, adamw=HP)
+            m.sync()
+        assert e.value.status == 6 and "IL_HEAD_RECOMPUTE" in str(e.value)
+        assert m.head_mode == "recompute"
+        assert m.get_opt_state("head1.w")[2] == 0            # nothing was applied
+        m.train_step(tok, tgt)                                # the same step again, same parameters
+        losses = m.get_losses()
+        m.sync()
+        m2.train_step(tok, tgt)
+        losses2 = m2.get_losses()
+        m2.sync()
+        assert np.array_equal(losses, losses2)
+        for nm in ("head0.w", "head1.w", "c0.l0.mlp.w1", "c1.l1.attn.wqkv"):
+            g = m.get_grad(nm)
+            assert np.all(np.isfinite(g)) and np.array_equal(g, m2.get_grad(nm)), nm
+    finally:
+        m.close()
+        m2.close()
+
+
 def test_allocator_returning_null_gives_oom_and_everything_is_handed_back():
     w = wl.CONFIGS["cfg1"]
     torch.cuda.synchronize()
