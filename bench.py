@@ -39,11 +39,11 @@ import workloads as wl  # noqa: E402
 
 
 # DRAM bytes per algorithmic flop of the GEMM kernel, from one ncu capture (dram__bytes_read.sum +
-# dram__bytes_write.sum over 400 consecutive GEMM launches of the cfg4-2x1 step, whose launch shapes are cfg4's).
+# dram__bytes_write.sum over all 270 GEMM launches of a cfg4-2x1 run, whose launch shapes are cfg4's).
 # Traffic grows with the flops of a launch at fixed shapes, so the
 # per-launch figure of another step mix is this ratio times that mix's flops per launch.  Set to None whenever
 # gemm.cu changes after the capture.
-GEMM_DRAM_BYTES_PER_FLOP = 1.2556e-3
+GEMM_DRAM_BYTES_PER_FLOP = 1.2558e-3
 
 
 def model_flops_per_token(w: wl.Workload, n: int) -> float:
