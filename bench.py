@@ -388,20 +388,21 @@ def main():
     ms = timed(args.steps, False)
     clocks = sampler.stop()
     launches = m.stats()[1] - l0
-    # The same K steps once more with a pair of CUDA events around every GEMM launch (on the launch's own stream):
-    # the GEMM kernel's durations inside a running step.  The events cost time of their own (two records per GEMM,
+    # Two more steps with every GEMM alone on the GPU (a pair of CUDA events around each, all other streams held
+    # back meanwhile) give the kernel's own durations at the step's launch shapes, straight after the timed steps.
+    m.profile(2)
+    run_steps(2, False)
+    m.sync()
+    x_ms, x_launches, x_flops = m.profile_read()
+    m.profile(False)
+    # The K steps once more with a pair of CUDA events around every GEMM launch (on the launch's own stream): the
+    # GEMM kernel's durations inside a running step, where the component streams share the GPU and the intervals
+    # include waiting for SMs.  The events cost time of their own (two records per GEMM,
     # and a kernel between events cannot set itself up while its predecessor drains), so these steps are not the
     # ones the headline value is taken from; their step time is reported beside the figure.
     m.profile(True)
     ms_events = timed(args.steps, False)
     gemm_ms, gemm_launches, gemm_flops = m.profile_read()
-    m.profile(False)
-    # The component streams share the GPU, so the intervals above include waiting for SMs.  Two more steps with
-    # every GEMM alone on the GPU give the kernels' own durations (same launches, same shapes).
-    m.profile(2)
-    run_steps(2, False)
-    m.sync()
-    x_ms, x_launches, x_flops = m.profile_read()
     m.profile(False)
     losses = m.get_losses() if not use_adamw else None
     # end to end: pinned host tokens copied in, losses read back, every step
